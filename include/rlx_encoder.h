@@ -1,0 +1,243 @@
+/*
+ * rlx_encoder.h - C ABI of the B200 (sm_100a) masked transformer-encoder forward.
+ *
+ * The library computes the forward pass of the sentence-embedding encoder that
+ * the paper's inference benchmark times (Section 8.2: a 384-d, 6-layer
+ * MiniLM-style model, "p50 of the encoder forward"):
+ *
+ *   token ids + attention mask + weights  ->  mean-pooled, L2-normalised embeddings
+ *
+ * as a create-once / run-many object with caller-bound buffers, mirroring the
+ * paper's compile-once CompiledGraph executed with bound inputs (Section 3.3).
+ * Every step runs in hand-written CUDA kernels; there is no CPU fallback.
+ *
+ * Conventions common to every entry point
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are host memory.
+ *   - The caller owns every buffer (ids, mask, weights, outputs, workspace) and
+ *     the stream.  The library owns only its host-side object (descriptors,
+ *     captured graphs).  No entry point allocates or frees device memory.
+ *   - Matrices are row-major.  Linear weights are [out_features, in_features]
+ *     (both GEMM operands are contiguous along the contraction axis).
+ *   - Storage types: embedding tables, Linear weights and activations are
+ *     bfloat16; biases and LayerNorm gamma/beta are float32; token ids and
+ *     masks are int32; the embeddings returned are float32.
+ *   - All device pointers must be 16-byte aligned.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*)
+ *     unless stated otherwise.  One encoder object per host thread / stream.
+ *   - Every call returns a status; nothing throws, aborts or traps.  Argument
+ *     errors are detected on the host before any launch.  Conditions only the
+ *     device can see (a token id outside the vocabulary, which is clamped; a
+ *     pipeline wait that ran out of its time budget) set bits in a sticky
+ *     32-bit device status word that rlx_encoder_last_device_status reads.
+ */
+#ifndef RLX_ENCODER_H
+#define RLX_ENCODER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rlx_encoder rlx_encoder_t; /* opaque, library-owned host object */
+
+typedef enum {
+    RLX_OK = 0,
+    RLX_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, non-positive or too large size   */
+    RLX_ERR_UNSUPPORTED = 2,    /* shape the kernels are not built for (see rlx_encoder_create) */
+    RLX_ERR_WORKSPACE = 3,      /* workspace_bytes < rlx_encoder_workspace_bytes(batch, seq)    */
+    RLX_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed                            */
+    RLX_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (results invalid)         */
+    RLX_ERR_TOKEN_RANGE = 6     /* a token id was outside [0, vocab) and was clamped            */
+} rlx_status_t;
+
+/* Bits of the device status word. */
+#define RLX_DEVSTAT_TOKEN_RANGE 0x1u
+#define RLX_DEVSTAT_TIMEOUT 0x2u
+
+/* rlx_encoder_config_t.flags */
+#define RLX_FLAG_NO_GRAPH 0x1u  /* launch kernels one by one instead of replaying a CUDA graph */
+#define RLX_FLAG_GEMM_SIMT 0x2u /* use the plain CUDA-core GEMM (bring-up / cross-check only)  */
+
+typedef struct {
+    uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */
+    int32_t num_layers;
+    int32_t hidden;     /* H; multiple of 128, <= 1024                      */
+    int32_t num_heads;  /* h; head_dim d = H / h must be 32 or 64           */
+    int32_t ffn;        /* F; multiple of 64                                */
+    int32_t vocab;      /* V                                                */
+    int32_t max_pos;    /* rows of the position table; seq <= max_pos       */
+    int32_t type_vocab; /* rows of the token-type table (row 0 is used)     */
+    float ln_eps;       /* LayerNorm epsilon, inside the square root        */
+    int32_t max_batch;  /* upper bounds accepted by forward                 */
+    int32_t max_seq;
+    int32_t device;     /* CUDA device ordinal the object is bound to       */
+    uint32_t flags;     /* RLX_FLAG_*                                       */
+} rlx_encoder_config_t;
+
+/* One encoder layer (post-LayerNorm):  all pointers dev. */
+typedef struct {
+    const void *wqkv;   /* bf16 [3H, H]: rows 0..H = query, H..2H = key, 2H..3H = value;
+                           head j owns output features j*d .. (j+1)*d of each block */
+    const float *bqkv;  /* f32 [3H] */
+    const void *wo;     /* bf16 [H, H]  attention output projection */
+    const float *bo;    /* f32 [H] */
+    const float *ln1_g; /* f32 [H]  LayerNorm after the attention residual */
+    const float *ln1_b;
+    const void *w1;     /* bf16 [F, H]  feed-forward up projection (GELU follows) */
+    const float *b1;    /* f32 [F] */
+    const void *w2;     /* bf16 [H, F]  feed-forward down projection */
+    const float *b2;    /* f32 [H] */
+    const float *ln2_g; /* f32 [H]  LayerNorm after the feed-forward residual */
+    const float *ln2_b;
+} rlx_layer_weights_t;
+
+typedef struct {
+    uint32_t struct_size;   /* sizeof(rlx_encoder_weights_t) */
+    const void *word_emb;   /* dev bf16 [V, H] */
+    const void *pos_emb;    /* dev bf16 [max_pos, H] (absolute positions 0..S-1) */
+    const void *type_emb;   /* dev bf16 [type_vocab, H] (row 0 is added to every token) */
+    const float *emb_ln_g;  /* dev f32 [H] */
+    const float *emb_ln_b;  /* dev f32 [H] */
+    const rlx_layer_weights_t *layers; /* HOST array [num_layers] of dev pointers */
+} rlx_encoder_weights_t;
+
+/*
+ * Create an encoder object for one model shape on config->device.
+ * Host only: validates the shape and precomputes the workspace layout.
+ * Returns RLX_ERR_INVALID_ARG for null/negative fields or a wrong struct_size,
+ * RLX_ERR_UNSUPPORTED when H % 128 != 0, H > 1024, H % h != 0, head_dim not in
+ * {32, 64}, F % 64 != 0, or max_seq > max_pos.
+ */
+rlx_status_t rlx_encoder_create(const rlx_encoder_config_t *config, rlx_encoder_t **out_encoder);
+
+/* Frees the host object and its captured graphs.  Device buffers stay the caller's. */
+void rlx_encoder_destroy(rlx_encoder_t *encoder);
+
+/*
+ * Bytes of device workspace that forward needs for (batch, seq): the packed
+ * activations of one layer (the arena of Section 3.2's memory planning, with
+ * fixed offsets), the status word and the staging area of the host-buffer
+ * entry point.  Returns 0 for sizes outside the configured bounds.
+ */
+size_t rlx_encoder_workspace_bytes(const rlx_encoder_t *encoder, int32_t batch, int32_t seq);
+
+/*
+ * The encoder forward (Section 8.2 workload; masked attention is the
+ * key-padding instance of Section 3.1's mask kinds; q/k/v are strided views of
+ * the packed projection as in Section 3.2):
+ *
+ *   x   = LN(word[ids] + pos[0..S) + type[0])
+ *   per layer:  qkv = x Wqkv^T + bqkv
+ *               ctx = softmax(q k^T / sqrt(d), keys with mask 0 excluded) v   per head
+ *               x1  = LN(ctx Wo^T + bo + x)
+ *               x   = LN(gelu(x1 W1^T + b1) W2^T + b2 + x1)          (erf GELU)
+ *   out[b] = normalise_L2( sum_s mask[b,s] x[b,s] / max(sum_s mask[b,s], 1e-9) )
+ *
+ * token_ids       dev int32 [batch, seq]; ids outside [0, V) are clamped and flagged
+ * attention_mask  dev int32 [batch, seq]; nonzero = valid position (holes allowed)
+ * weights         host struct of dev pointers (see above); read during the call only
+ * out             dev f32 [batch, H]; a sequence with no valid position yields zeros
+ * workspace       dev, 256-byte aligned, >= rlx_encoder_workspace_bytes(batch, seq);
+ *                 scratch: contents are overwritten by every call
+ *
+ * Asynchronous on cuda_stream.  Unless RLX_FLAG_NO_GRAPH is set the kernel
+ * sequence is captured once per distinct (batch, seq, pointer set) into a CUDA
+ * graph and replayed afterwards.  Activations are computed in bf16 storage
+ * with fp32 accumulation and fp32 LayerNorm/softmax/GELU arithmetic.
+ */
+rlx_status_t rlx_encoder_forward(rlx_encoder_t *encoder, const int32_t *token_ids,
+                                 const int32_t *attention_mask, int32_t batch, int32_t seq,
+                                 const rlx_encoder_weights_t *weights, float *out, void *workspace,
+                                 size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Same computation with HOST inputs and output (the end-to-end path): copies
+ * ids and mask host->device into the workspace staging area, runs the forward,
+ * copies the embeddings device->host and synchronises the stream before
+ * returning.  token_ids / attention_mask / out are host pointers (pinned memory
+ * makes the copies asynchronous); weights and workspace are as above.
+ */
+rlx_status_t rlx_encoder_forward_host(rlx_encoder_t *encoder, const int32_t *token_ids_host,
+                                      const int32_t *attention_mask_host, int32_t batch,
+                                      int32_t seq, const rlx_encoder_weights_t *weights,
+                                      float *out_host, void *workspace, size_t workspace_bytes,
+                                      void *cuda_stream);
+
+/*
+ * Synchronises cuda_stream, reads and clears the sticky device status word kept
+ * in `workspace`, and maps it to RLX_OK / RLX_ERR_TOKEN_RANGE /
+ * RLX_ERR_DEVICE_TIMEOUT (timeout wins).
+ */
+rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t *encoder, void *workspace, void *cuda_stream);
+
+/* Number of kernels one forward of (batch, seq) launches (for launch accounting). */
+int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t *encoder);
+
+/* Static string for a status code. */
+const char *rlx_status_string(rlx_status_t status);
+
+/* ------------------------------------------------------------------------- *
+ * Kernel-level entry points (the steps of the forward, one by one).  They are
+ * what the forward launches internally and exist so that each step can be
+ * checked against the oracle in isolation.  All pointers dev; `status` is an
+ * optional dev int32 that receives RLX_DEVSTAT_* bits (may be NULL).
+ * ------------------------------------------------------------------------- */
+
+/* x[t] = LN(word[ids[t]] + pos[t % seq] + type[0]) -> bf16 [tokens, H]. */
+rlx_status_t rlx_embed_layernorm(const int32_t *token_ids, const void *word_emb, const void *pos_emb,
+                                 const void *type_emb, const float *gamma, const float *beta,
+                                 int32_t tokens, int32_t seq, int32_t hidden, int32_t vocab, float eps,
+                                 void *out_bf16, int32_t *status, void *cuda_stream);
+
+/* out = LN(x; gamma, beta), rows of `hidden` bf16 values, fp32 statistics. */
+rlx_status_t rlx_layernorm(const void *x_bf16, const float *gamma, const float *beta, int32_t rows,
+                           int32_t hidden, float eps, void *out_bf16, void *cuda_stream);
+
+typedef enum {
+    RLX_EPI_BIAS = 0,          /* out = A W^T + bias                */
+    RLX_EPI_BIAS_GELU = 1,     /* out = gelu(A W^T + bias)          */
+    RLX_EPI_BIAS_RESIDUAL = 2  /* out = A W^T + bias + residual     */
+} rlx_epilogue_t;
+
+typedef enum {
+    RLX_GEMM_TCGEN05 = 0, /* TMA-fed tcgen05 MMA with TMEM accumulators (the product path) */
+    RLX_GEMM_SIMT = 1     /* plain CUDA-core tiles (bring-up / cross-check)                */
+} rlx_gemm_impl_t;
+
+/*
+ * The "Linear" block (Section 3.1) with a fused epilogue: A bf16 [M,K],
+ * W bf16 [N,K], bias f32 [N], residual bf16 [M,N] (only for
+ * RLX_EPI_BIAS_RESIDUAL), out bf16 [M,N]; fp32 accumulation (the AMP policy of
+ * Section 3.2).  K % 8 == 0 and N % 64 == 0 are required (RLX_ERR_UNSUPPORTED).
+ */
+rlx_status_t rlx_gemm_bf16(const void *A, const void *W, const float *bias, const void *residual,
+                           rlx_epilogue_t epilogue, int32_t M, int32_t N, int32_t K, void *out,
+                           rlx_gemm_impl_t impl, int32_t *status, void *cuda_stream);
+
+/*
+ * Key-padding-masked scaled-dot-product attention over the packed projection
+ * (Section 3.1 mask kinds; Section 3.2 "Narrow x3 -> Attention" views):
+ * qkv [batch*seq, 3H] with q | k | v column blocks, head j = columns j*d..(j+1)*d
+ * of each block; ctx [batch*seq, H].  Rows whose own mask is 0 receive zeros or
+ * finite don't-care values.  head_dim in {32, 64}.
+ *   _bf16: bf16 in / bf16 out, tensor-core products, fp32 online softmax.
+ *   _f32 : fp32 in / fp32 out, shared-memory staged CUDA-core kernel with
+ *          warp-shuffle reductions (the reference-precision mode).
+ */
+rlx_status_t rlx_attention_bf16(const void *qkv_bf16, const int32_t *attention_mask, int32_t batch,
+                                int32_t seq, int32_t num_heads, int32_t head_dim, void *ctx_bf16,
+                                void *cuda_stream);
+rlx_status_t rlx_attention_f32(const float *qkv_f32, const int32_t *attention_mask, int32_t batch,
+                               int32_t seq, int32_t num_heads, int32_t head_dim, float *ctx_f32,
+                               void *cuda_stream);
+
+/* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
+rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,
+                             int32_t seq, int32_t hidden, float *out, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLX_ENCODER_H */

@@ -1,0 +1,20 @@
+"""B200 (sm_100a) masked transformer-encoder forward behind a C ABI.
+
+``binding`` is a thin ctypes layer over ``librlx_encoder.so`` (same names as
+``include/rlx_encoder.h``); it only marshals arguments.  There is no CPU or
+library fallback: if the shared library has not been built, importing the
+binding raises.
+"""
+from .binding import (  # noqa: F401
+    DeviceWeights,
+    Encoder,
+    RlxError,
+    attention_bf16,
+    attention_f32,
+    embed_layernorm,
+    gemm_bf16,
+    layernorm,
+    lib_path,
+    pool_l2norm,
+    upload_weights,
+)

@@ -1,0 +1,247 @@
+"""ctypes binding of ``librlx_encoder.so`` (declared in ``include/rlx_encoder.h``).
+
+Argument marshalling only: every step of the encoder runs inside the CUDA
+library.  PyTorch is used for device memory and streams, nothing else.  The
+library must have been built (``python -m paper_2609_37916_b200.build``);
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "librlx_encoder.so")
+
+RLX_OK = 0
+STATUS_NAMES = {0: "RLX_OK", 1: "RLX_ERR_INVALID_ARG", 2: "RLX_ERR_UNSUPPORTED", 3: "RLX_ERR_WORKSPACE",
+                4: "RLX_ERR_CUDA", 5: "RLX_ERR_DEVICE_TIMEOUT", 6: "RLX_ERR_TOKEN_RANGE"}
+FLAG_NO_GRAPH = 0x1
+FLAG_GEMM_SIMT = 0x2
+EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
+GEMM_TCGEN05, GEMM_SIMT = 0, 1
+
+EXPORTS = (
+    "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
+    "rlx_encoder_forward_host", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward",
+    "rlx_status_string", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
+    "rlx_attention_f32", "rlx_pool_l2norm",
+)
+
+
+class RlxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class _Config(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("num_layers", C.c_int32), ("hidden", C.c_int32),
+                ("num_heads", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32), ("max_pos", C.c_int32),
+                ("type_vocab", C.c_int32), ("ln_eps", C.c_float), ("max_batch", C.c_int32),
+                ("max_seq", C.c_int32), ("device", C.c_int32), ("flags", C.c_uint32)]
+
+
+LAYER_FIELDS = ("wqkv", "bqkv", "wo", "bo", "ln1_g", "ln1_b", "w1", "b1", "w2", "b2", "ln2_g", "ln2_b")
+BF16_FIELDS = {"wqkv", "wo", "w1", "w2", "word_emb", "pos_emb", "type_emb"}
+
+
+class _Layer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in LAYER_FIELDS]
+
+
+class _Weights(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("word_emb", C.c_void_p), ("pos_emb", C.c_void_p),
+                ("type_emb", C.c_void_p), ("emb_ln_g", C.c_void_p), ("emb_ln_b", C.c_void_p),
+                ("layers", C.POINTER(_Layer))]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_37916_b200.build` "
+                              "(there is no fallback path)")
+        _lib = C.CDLL(_LIB_PATH)
+        _lib.rlx_encoder_workspace_bytes.restype = C.c_size_t
+        _lib.rlx_status_string.restype = C.c_char_p
+        _lib.rlx_encoder_destroy.restype = None
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != RLX_OK:
+        raise RlxError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> C.c_void_p:
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+class DeviceWeights:
+    """Device-resident parameter set + the host struct of pointers the ABI takes."""
+
+    def __init__(self, params: Dict[str, torch.Tensor], layers: Sequence[Dict[str, torch.Tensor]]):
+        self.params = params
+        self.layers = list(layers)
+        self._layer_arr = (_Layer * max(len(self.layers), 1))()
+        for i, lw in enumerate(self.layers):
+            for n in LAYER_FIELDS:
+                t = lw[n]
+                want = torch.bfloat16 if n in BF16_FIELDS else torch.float32
+                assert t.is_cuda and t.is_contiguous() and t.dtype == want, (n, t.dtype)
+                setattr(self._layer_arr[i], n, t.data_ptr())
+        self.c = _Weights()
+        self.c.struct_size = C.sizeof(_Weights)
+        for n in ("word_emb", "pos_emb", "type_emb", "emb_ln_g", "emb_ln_b"):
+            t = params[n]
+            want = torch.bfloat16 if n in BF16_FIELDS else torch.float32
+            assert t.is_cuda and t.is_contiguous() and t.dtype == want, (n, t.dtype)
+            setattr(self.c, n, t.data_ptr())
+        self.c.layers = self._layer_arr
+
+
+def upload_weights(params, layers, device="cuda") -> DeviceWeights:
+    """Copy numpy float32 parameters (matrices already on the bf16 grid) to the device in the
+    storage types the ABI expects: bf16 for tables / Linear weights, fp32 for biases and LN."""
+    def put(name, a):
+        t = torch.from_numpy(a).to(device)
+        return t.to(torch.bfloat16).contiguous() if name in BF16_FIELDS else t.float().contiguous()
+
+    p = {n: put(n, params[n]) for n in ("word_emb", "pos_emb", "type_emb", "emb_ln_g", "emb_ln_b")}
+    ls = [{n: put(n, lw[n]) for n in LAYER_FIELDS} for lw in layers]
+    return DeviceWeights(p, ls)
+
+
+class Encoder:
+    """rlx_encoder_create / _forward / _destroy."""
+
+    def __init__(self, num_layers: int, hidden: int, num_heads: int, ffn: int, vocab: int = 30522,
+                 max_pos: int = 512, type_vocab: int = 2, ln_eps: float = 1e-12, max_batch: int = 256,
+                 max_seq: int = 512, device: int = 0, flags: int = 0):
+        self._h = C.c_void_p()
+        self.hidden = hidden
+        self.cfg = _Config(C.sizeof(_Config), num_layers, hidden, num_heads, ffn, vocab, max_pos, type_vocab,
+                           ln_eps, max_batch, max_seq, device, flags)
+        _check(_load().rlx_encoder_create(C.byref(self.cfg), C.byref(self._h)), "rlx_encoder_create")
+
+    @classmethod
+    def from_config(cls, cfg, **kw) -> "Encoder":
+        kw.setdefault("max_batch", max(cfg.batch, 1))
+        kw.setdefault("max_seq", cfg.max_pos)
+        return cls(cfg.num_layers, cfg.hidden, cfg.num_heads, cfg.ffn, cfg.vocab, cfg.max_pos, cfg.type_vocab,
+                   cfg.ln_eps, **kw)
+
+    def close(self) -> None:
+        if self._h:
+            _load().rlx_encoder_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace_bytes(self, batch: int, seq: int) -> int:
+        return int(_load().rlx_encoder_workspace_bytes(self._h, batch, seq))
+
+    def kernels_per_forward(self) -> int:
+        return int(_load().rlx_encoder_kernels_per_forward(self._h))
+
+    def alloc_workspace(self, batch: int, seq: int, device="cuda") -> torch.Tensor:
+        n = self.workspace_bytes(batch, seq)
+        if n == 0:
+            raise RlxError(1, "rlx_encoder_workspace_bytes")
+        return torch.zeros(n, dtype=torch.uint8, device=device)
+
+    def forward(self, ids: torch.Tensor, mask: torch.Tensor, weights: DeviceWeights, out: torch.Tensor,
+                workspace: torch.Tensor, stream=None) -> torch.Tensor:
+        B, S = ids.shape
+        assert ids.dtype == torch.int32 and mask.dtype == torch.int32 and out.dtype == torch.float32
+        assert ids.is_cuda and mask.is_cuda and out.is_cuda and ids.is_contiguous() and mask.is_contiguous()
+        _check(_load().rlx_encoder_forward(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights.c), _ptr(out),
+                                           _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)),
+               "rlx_encoder_forward")
+        return out
+
+    def forward_host(self, ids: torch.Tensor, mask: torch.Tensor, weights: DeviceWeights, out: torch.Tensor,
+                     workspace: torch.Tensor, stream=None) -> torch.Tensor:
+        B, S = ids.shape
+        assert not ids.is_cuda and not mask.is_cuda and not out.is_cuda
+        assert ids.dtype == torch.int32 and mask.dtype == torch.int32 and out.dtype == torch.float32
+        _check(_load().rlx_encoder_forward_host(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights.c),
+                                                _ptr(out), _ptr(workspace), C.c_size_t(workspace.numel()),
+                                                _stream(stream)), "rlx_encoder_forward_host")
+        return out
+
+    def last_device_status(self, workspace: torch.Tensor, stream=None) -> int:
+        return int(_load().rlx_encoder_last_device_status(self._h, _ptr(workspace), _stream(stream)))
+
+
+# ------------------------------------------------------------------ kernel-level entry points
+def embed_layernorm(ids, word, pos, type_, gamma, beta, seq: int, vocab: int, eps: float, status=None, stream=None):
+    T, H = ids.numel(), word.shape[1]
+    out = torch.empty((T, H), dtype=torch.bfloat16, device=ids.device)
+    _check(_load().rlx_embed_layernorm(_ptr(ids), _ptr(word), _ptr(pos), _ptr(type_), _ptr(gamma), _ptr(beta), T, seq,
+                                       H, vocab, C.c_float(eps), _ptr(out), _ptr(status), _stream(stream)),
+           "rlx_embed_layernorm")
+    return out
+
+
+def layernorm(x, gamma, beta, eps: float, stream=None):
+    rows, H = x.shape
+    out = torch.empty_like(x)
+    _check(_load().rlx_layernorm(_ptr(x), _ptr(gamma), _ptr(beta), rows, H, C.c_float(eps), _ptr(out), _stream(stream)),
+           "rlx_layernorm")
+    return out
+
+
+def gemm_bf16(a, w, bias, residual=None, epilogue: int = EPI_BIAS, impl: int = GEMM_TCGEN05, status=None, stream=None):
+    M, K = a.shape
+    N = w.shape[0]
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
+    _check(_load().rlx_gemm_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(residual), epilogue, M, N, K, _ptr(out), impl,
+                                 _ptr(status), _stream(stream)), "rlx_gemm_bf16")
+    return out
+
+
+def attention_bf16(qkv, mask, num_heads: int, stream=None):
+    B, S, H3 = qkv.shape
+    H = H3 // 3
+    ctx = torch.empty((B, S, H), dtype=torch.bfloat16, device=qkv.device)
+    _check(_load().rlx_attention_bf16(_ptr(qkv), _ptr(mask), B, S, num_heads, H // num_heads, _ptr(ctx), _stream(stream)),
+           "rlx_attention_bf16")
+    return ctx
+
+
+def attention_f32(qkv, mask, num_heads: int, stream=None):
+    B, S, H3 = qkv.shape
+    H = H3 // 3
+    ctx = torch.empty((B, S, H), dtype=torch.float32, device=qkv.device)
+    _check(_load().rlx_attention_f32(_ptr(qkv), _ptr(mask), B, S, num_heads, H // num_heads, _ptr(ctx), _stream(stream)),
+           "rlx_attention_f32")
+    return ctx
+
+
+def pool_l2norm(x, mask, stream=None):
+    B, S, H = x.shape
+    out = torch.empty((B, H), dtype=torch.float32, device=x.device)
+    _check(_load().rlx_pool_l2norm(_ptr(x), _ptr(mask), B, S, H, _ptr(out), _stream(stream)), "rlx_pool_l2norm")
+    return out

@@ -1,0 +1,330 @@
+// bf16 "Linear" GEMM for sm_100a: out[M,N] = epilogue(A[M,K] * W[N,K]^T + bias).
+//
+// Structure (one persistent CTA per SM, 192 threads):
+//   warp 0      TMA producer: streams 128x64 A tiles and BLOCK_N x 64 W tiles (128-byte swizzle)
+//               through a STAGES-deep shared-memory ring guarded by full/empty mbarriers
+//   warp 1      allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N=BLOCK_N,
+//               K=16 per instruction) into one of two fp32 accumulator buffers in TMEM and
+//               commits stage releases / accumulator-ready signals to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (one TMEM lane quadrant per warp, one output
+//               row per thread), add bias, apply GELU or add the residual in fp32, round to bf16
+//               and store; the second accumulator buffer lets tile i's epilogue overlap tile
+//               i+1's main loop
+// Every mbarrier wait is bounded by a wall-clock budget; on expiry the CTA raises an abort flag,
+// records RLX_DEVSTAT_TIMEOUT, drains, frees its tensor memory and returns.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+#include "epilogue.cuh"
+
+namespace rlx {
+namespace tc {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;   // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kThreads = 192;
+constexpr int kEpiWarps = 4;
+constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
+
+template <int BLOCK_N>
+struct Cfg {
+    static constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;
+    static constexpr int B_BYTES = BLOCK_N * BLOCK_K * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (220 * 1024 / STAGE_BYTES) > 8 ? 8 : (220 * 1024 / STAGE_BYTES);
+    static constexpr int TMEM_COLS = (2 * BLOCK_N <= 32) ? 32 : (2 * BLOCK_N <= 64) ? 64 : (2 * BLOCK_N <= 128) ? 128
+                                     : (2 * BLOCK_N <= 256) ? 256 : 512;
+    static constexpr int BAR_BYTES = 256;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // +1024: manual alignment
+    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128");
+    static_assert(B_BYTES % 1024 == 0, "stage tiles must stay 1024-byte aligned");
+    static_assert(STAGES >= 2, "ring too shallow");
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the budget ran out or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xff) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitBudgetNs) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap* tmap, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (thread = lane = row)
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows written by TMA with the 128-byte
+// swizzle; 8-row groups are 1024 bytes apart (stride byte offset); the leading byte offset is not
+// used by swizzled K-major layouts (encoded 1); descriptor version 1; swizzle mode 2 = 128 B.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct Params {
+    const float* bias;               // [N]
+    const __nv_bfloat16* residual;   // [M,N] or null
+    __nv_bfloat16* out;              // [M,N]
+    int M, N, K;
+    int32_t* status;                 // device status word (may be null)
+};
+
+template <int BLOCK_N, int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+    using C = Cfg<BLOCK_N>;
+    extern __shared__ unsigned char smem_raw[];
+    // manual 1024-byte alignment (required by the 128-byte swizzle atoms)
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - raw);
+    const uint32_t bars = base + C::STAGES * C::STAGE_BYTES;
+    // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem slot, abort flag
+    const uint32_t full_bar = bars, empty_bar = bars + 8 * C::STAGES;
+    const uint32_t tfull_bar = bars + 16 * C::STAGES, tempty_bar = tfull_bar + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + 16 * C::STAGES + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = p.N / BLOCK_N;
+    const int m_tiles = (p.M + BLOCK_M - 1) / BLOCK_M;
+    const int num_tiles = n_tiles * m_tiles;
+    const int num_kb = (p.K + BLOCK_K - 1) / BLOCK_K;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::STAGES; ++i) {
+            mbar_init(full_bar + 8 * i, 1);
+            mbar_init(empty_bar + 8 * i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(tfull_bar + 8 * i, 1);
+            mbar_init(tempty_bar + 8 * i, kEpiWarps);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap_a);
+        prefetch_tmap(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                    mbar_expect_tx(full_bar + 8 * stage, C::STAGE_BYTES);
+                    tma_load_2d(sa, &tmap_a, kb * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
+                    tma_load_2d(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+                const int as = it & 1;
+                const uint32_t aphase = (it >> 1) & 1;
+                if (!mbar_wait(tempty_bar + 8 * as, aphase ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + as * BLOCK_N;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
+                    const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                        // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
+                        umma_bf16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar + 8 * stage);  // stage reusable once these MMAs have read it
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (ok) umma_commit(tfull_bar + 8 * as);  // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+            const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+            const int as = it & 1;
+            const uint32_t aphase = (it >> 1) & 1;
+            if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int m = m_blk * BLOCK_M + quad * 32 + lane;
+            const bool row_ok = m < p.M;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N;
+            __nv_bfloat16* orow = p.out + (size_t)m * p.N + n_blk * BLOCK_N;
+            const __nv_bfloat16* rrow = p.residual + (size_t)m * p.N + n_blk * BLOCK_N;
+            const float* brow = p.bias + n_blk * BLOCK_N;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + c0, r);
+                tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c0) + i);
+                    v[4 * i + 0] = __uint_as_float(r[4 * i + 0]) + b4.x;
+                    v[4 * i + 1] = __uint_as_float(r[4 * i + 1]) + b4.y;
+                    v[4 * i + 2] = __uint_as_float(r[4 * i + 2]) + b4.z;
+                    v[4 * i + 3] = __uint_as_float(r[4 * i + 3]) + b4.w;
+                }
+                if (EPI == 1) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
+                }
+                if (row_ok) {
+                    if (EPI == 2) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 q = __ldg(reinterpret_cast<const uint4*>(rrow + c0) + i);
+                            v[8 * i + 0] += bf16lo(q.x); v[8 * i + 1] += bf16hi(q.x);
+                            v[8 * i + 2] += bf16lo(q.y); v[8 * i + 3] += bf16hi(q.y);
+                            v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
+                            v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 q;
+                        q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
+                        q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+                        q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+                        q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+                        *(reinterpret_cast<uint4*>(orow + c0) + i) = q;
+                    }
+                }
+            }
+            // release this accumulator buffer to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar + 8 * as);
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, RLX_DEVSTAT_TIMEOUT_BIT);
+        // give copies that may still be in flight time to land before shared memory is released
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+}  // namespace tc
+}  // namespace rlx

@@ -1,0 +1,520 @@
+// C-ABI library of the sm_100a encoder forward: host runtime (validation, workspace arena,
+// tensor-map construction, CUDA-graph cache) and the launchers of every kernel.
+// Single translation unit: all kernels are included below.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "../../include/rlx_encoder.h"
+#include "attention.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tcgen05.cuh"
+#include "rowwise.cuh"
+
+namespace {
+
+using bf16 = __nv_bfloat16;
+
+#define RLX_CUDA_TRY(expr)                      \
+    do {                                        \
+        cudaError_t _e = (expr);                \
+        if (_e != cudaSuccess) {                \
+            g_last_cuda_error = _e;             \
+            return RLX_ERR_CUDA;                \
+        }                                       \
+    } while (0)
+
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ------------------------------------------------------------------ tensor maps
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_fn() {
+    static encode_tiled_fn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(p);
+    });
+    return fn;
+}
+
+// bf16 row-major [rows, cols] matrix, box = box_rows x 64 columns, 128-byte swizzle, zero OOB fill.
+bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * sizeof(bf16)};
+    cuuint32_t box[2] = {(cuuint32_t)rlx::tc::BLOCK_K, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------ one-time kernel attributes
+template <int BN, int EPI>
+cudaError_t set_gemm_attr() {
+    return cudaFuncSetAttribute(rlx::tc::gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                rlx::tc::Cfg<BN>::SMEM_BYTES);
+}
+template <int BN>
+cudaError_t set_gemm_attr_all() {
+    cudaError_t e;
+    if ((e = set_gemm_attr<BN, 0>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr<BN, 1>()) != cudaSuccess) return e;
+    return set_gemm_attr<BN, 2>();
+}
+
+cudaError_t init_kernels_for_current_device() {
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lk(mu);
+    if (dev < 64 && done[dev]) return cudaSuccess;
+    if ((e = set_gemm_attr_all<64>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr_all<128>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr_all<192>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr_all<256>()) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)sizeof(rlx::AttSmem<32>))) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)sizeof(rlx::AttSmem<64>))) != cudaSuccess) return e;
+    if (dev < 64) done[dev] = true;
+    return cudaSuccess;
+}
+
+// ------------------------------------------------------------------ launchers
+rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* pos, const bf16* type,
+                             const float* g, const float* b, int T, int S, int H, int V, float eps, bf16* out,
+                             int32_t* status, cudaStream_t st) {
+    const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
+    switch (H / 128) {
+#define RLX_CASE(NV) case NV: rlx::embed_ln_kernel<NV><<<grid, thr, 0, st>>>(ids, word, pos, type, g, b, out, T, S, V, eps, status); break;
+        RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
+#undef RLX_CASE
+        default: return RLX_ERR_UNSUPPORTED;
+    }
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int T, int H, float eps, bf16* out,
+                              cudaStream_t st) {
+    const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
+    switch (H / 128) {
+#define RLX_CASE(NV) case NV: rlx::layernorm_kernel<NV><<<grid, thr, 0, st>>>(x, g, b, out, T, eps); break;
+        RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
+#undef RLX_CASE
+        default: return RLX_ERR_UNSUPPORTED;
+    }
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H, float* out, cudaStream_t st) {
+    const int vecs = H / 8, G = rlx::kPoolThreads / vecs;
+    const size_t smem = (size_t)G * H * sizeof(float);
+    rlx::pool_l2norm_kernel<<<B, rlx::kPoolThreads, smem, st>>>(x, mask, out, S, H);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, int B, int S, int h, int d, bf16* ctx,
+                                   cudaStream_t st) {
+    const int H = h * d;
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
+    dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
+    if (d == 32)
+        rlx::attention_bf16_kernel<32><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st>>>(qkv, mask, ctx, S, H, scale_log2e);
+    else if (d == 64)
+        rlx::attention_bf16_kernel<64><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st>>>(qkv, mask, ctx, S, H, scale_log2e);
+    else
+        return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+int pick_block_n(int M, int N) {
+    const int m_tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
+    const int cand[4] = {256, 192, 128, 64};
+    // largest tile that still gives every SM work; otherwise the smallest that divides N
+    for (int i = 0; i < 4; ++i)
+        if (N % cand[i] == 0 && m_tiles * (N / cand[i]) >= rlx::kNumSMs) return cand[i];
+    for (int i = 3; i >= 0; --i)
+        if (N % cand[i] == 0) return cand[i];
+    return 0;
+}
+
+template <int BN>
+rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const rlx::tc::Params& p, int epi,
+                               cudaStream_t st) {
+    const int tiles = ((p.M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M) * (p.N / BN);
+    const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
+    const int smem = rlx::tc::Cfg<BN>::SMEM_BYTES;
+    switch (epi) {
+        case 0: rlx::tc::gemm_tcgen05_kernel<BN, 0><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
+        case 1: rlx::tc::gemm_tcgen05_kernel<BN, 1><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
+        case 2: rlx::tc::gemm_tcgen05_kernel<BN, 2><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
+        default: return RLX_ERR_INVALID_ARG;
+    }
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const bf16* residual, int epi, int M, int N,
+                         int K, bf16* out, bool simt, int32_t* status, cudaStream_t st) {
+    if (simt) {
+        dim3 grid((N + rlx::kSimtTile - 1) / rlx::kSimtTile, (M + rlx::kSimtTile - 1) / rlx::kSimtTile);
+        switch (epi) {
+            case 0: rlx::gemm_simt_kernel<0><<<grid, 256, 0, st>>>(A, W, bias, residual, out, M, N, K); break;
+            case 1: rlx::gemm_simt_kernel<1><<<grid, 256, 0, st>>>(A, W, bias, residual, out, M, N, K); break;
+            case 2: rlx::gemm_simt_kernel<2><<<grid, 256, 0, st>>>(A, W, bias, residual, out, M, N, K); break;
+            default: return RLX_ERR_INVALID_ARG;
+        }
+        RLX_CUDA_TRY(cudaGetLastError());
+        return RLX_OK;
+    }
+    const int bn = pick_block_n(M, N);
+    if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
+    CUtensorMap ta, tb;
+    if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
+    if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)bn)) return RLX_ERR_CUDA;
+    rlx::tc::Params p{bias, residual, out, M, N, K, status};
+    switch (bn) {
+        case 64: return launch_gemm_tc_bn<64>(ta, tb, p, epi, st);
+        case 128: return launch_gemm_tc_bn<128>(ta, tb, p, epi, st);
+        case 192: return launch_gemm_tc_bn<192>(ta, tb, p, epi, st);
+        case 256: return launch_gemm_tc_bn<256>(ta, tb, p, epi, st);
+    }
+    return RLX_ERR_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------ workspace arena
+struct Arena {
+    size_t status, ids, mask, out, x, qkv, ctx, y, x1, g, total;
+};
+
+Arena plan_arena(int B, int S, int H, int F) {
+    const size_t T = (size_t)B * S;
+    Arena a{};
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off += round_up(bytes, 256);
+        return o;
+    };
+    a.status = take(256);
+    a.ids = take(T * 4);
+    a.mask = take(T * 4);
+    a.out = take((size_t)B * H * 4);
+    a.x = take(T * H * 2);
+    a.qkv = take(T * 3 * H * 2);
+    a.ctx = take(T * H * 2);
+    a.y = take(T * H * 2);
+    a.x1 = take(T * H * 2);
+    a.g = take(T * F * 2);
+    a.total = off;
+    return a;
+}
+
+struct GraphEntry {
+    int B, S;
+    const void *ids, *mask, *out, *ws;
+    cudaGraphExec_t exec;
+};
+
+}  // namespace
+
+struct rlx_encoder {
+    rlx_encoder_config_t cfg;
+    int head_dim;
+    std::vector<rlx_layer_weights_t> layers;  // last weight set seen (graph-cache key)
+    rlx_encoder_weights_t weights;
+    bool have_weights = false;
+    std::vector<GraphEntry> graphs;
+};
+
+namespace {
+
+bool same_weights(const rlx_encoder* e, const rlx_encoder_weights_t* w) {
+    if (!e->have_weights) return false;
+    if (w->word_emb != e->weights.word_emb || w->pos_emb != e->weights.pos_emb || w->type_emb != e->weights.type_emb ||
+        w->emb_ln_g != e->weights.emb_ln_g || w->emb_ln_b != e->weights.emb_ln_b)
+        return false;
+    return std::memcmp(w->layers, e->layers.data(), sizeof(rlx_layer_weights_t) * e->layers.size()) == 0;
+}
+
+void drop_graphs(rlx_encoder* e) {
+    for (auto& g : e->graphs) cudaGraphExecDestroy(g.exec);
+    e->graphs.clear();
+}
+
+// The kernel sequence of one forward, enqueued on `st` (eagerly or under stream capture).
+rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
+                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
+    const rlx_encoder_config_t& c = e->cfg;
+    const int H = c.hidden, F = c.ffn, T = B * S, h = c.num_heads, d = e->head_dim;
+    const bool simt = (c.flags & RLX_FLAG_GEMM_SIMT) != 0;
+    const Arena a = plan_arena(B, S, H, F);
+    int32_t* status = reinterpret_cast<int32_t*>(ws + a.status);
+    bf16* x = reinterpret_cast<bf16*>(ws + a.x);
+    bf16* qkv = reinterpret_cast<bf16*>(ws + a.qkv);
+    bf16* ctx = reinterpret_cast<bf16*>(ws + a.ctx);
+    bf16* y = reinterpret_cast<bf16*>(ws + a.y);
+    bf16* x1 = reinterpret_cast<bf16*>(ws + a.x1);
+    bf16* g = reinterpret_cast<bf16*>(ws + a.g);
+    rlx_status_t s;
+#define RLX_TRY(call) do { s = (call); if (s != RLX_OK) return s; } while (0)
+    RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
+                            w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st));
+    for (int l = 0; l < c.num_layers; ++l) {
+        const rlx_layer_weights_t& lw = w->layers[l];
+        RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, simt, status, st));
+        RLX_TRY(launch_attention_bf16(qkv, mask, B, S, h, d, ctx, st));
+        RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st));
+        RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st));
+        RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st));
+        RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st));
+        RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st));
+    }
+    RLX_TRY(launch_pool(x, mask, B, S, H, out, st));
+#undef RLX_TRY
+    return RLX_OK;
+}
+
+rlx_status_t check_forward_args(const rlx_encoder* e, const void* ids, const void* mask, int B, int S,
+                                const rlx_encoder_weights_t* w, const void* out, const void* ws, size_t ws_bytes,
+                                bool host_io) {
+    if (!e || !ids || !mask || !w || !out || !ws) return RLX_ERR_INVALID_ARG;
+    if (w->struct_size != sizeof(rlx_encoder_weights_t) || !w->layers) return RLX_ERR_INVALID_ARG;
+    if (B <= 0 || S <= 0 || B > e->cfg.max_batch || S > e->cfg.max_seq) return RLX_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return RLX_ERR_INVALID_ARG;
+    if (!host_io && (!aligned16(ids) || !aligned16(mask) || !aligned16(out))) return RLX_ERR_INVALID_ARG;
+    const void* tabs[5] = {w->word_emb, w->pos_emb, w->type_emb, w->emb_ln_g, w->emb_ln_b};
+    for (const void* p : tabs)
+        if (!p || !aligned16(p)) return RLX_ERR_INVALID_ARG;
+    for (int l = 0; l < e->cfg.num_layers; ++l) {
+        const void* const* ptrs = reinterpret_cast<const void* const*>(&w->layers[l]);
+        for (size_t i = 0; i < sizeof(rlx_layer_weights_t) / sizeof(void*); ++i)
+            if (!ptrs[i] || !aligned16(ptrs[i])) return RLX_ERR_INVALID_ARG;
+    }
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    if (ws_bytes < a.total) return RLX_ERR_WORKSPACE;
+    return RLX_OK;
+}
+
+rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
+                            const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st);
+
+    if (!same_weights(e, w)) {
+        drop_graphs(e);
+        e->weights = *w;
+        e->layers.assign(w->layers, w->layers + e->cfg.num_layers);
+        e->weights.layers = e->layers.data();
+        e->have_weights = true;
+    }
+    for (const auto& g : e->graphs)
+        if (g.B == B && g.S == S && g.ids == ids && g.mask == mask && g.out == out && g.ws == ws) {
+            RLX_CUDA_TRY(cudaGraphLaunch(g.exec, st));
+            return RLX_OK;
+        }
+    // capture once for this (batch, seq, pointer set)
+    cudaGraph_t graph = nullptr;
+    RLX_CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, st);
+    cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (s != RLX_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return s;
+    }
+    RLX_CUDA_TRY(ce);
+    cudaGraphExec_t exec = nullptr;
+    ce = cudaGraphInstantiate(&exec, graph, 0);
+    cudaGraphDestroy(graph);
+    RLX_CUDA_TRY(ce);
+    if (e->graphs.size() >= 16) {  // bound the cache
+        cudaGraphExecDestroy(e->graphs.front().exec);
+        e->graphs.erase(e->graphs.begin());
+    }
+    e->graphs.push_back(GraphEntry{B, S, ids, mask, out, ws, exec});
+    RLX_CUDA_TRY(cudaGraphLaunch(exec, st));
+    return RLX_OK;
+}
+
+}  // namespace
+
+// =================================================================== C ABI
+extern "C" {
+
+rlx_status_t rlx_encoder_create(const rlx_encoder_config_t* c, rlx_encoder_t** out) {
+    if (!c || !out) return RLX_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (c->struct_size != sizeof(rlx_encoder_config_t)) return RLX_ERR_INVALID_ARG;
+    if (c->num_layers <= 0 || c->hidden <= 0 || c->num_heads <= 0 || c->ffn <= 0 || c->vocab <= 0 || c->max_pos <= 0 ||
+        c->type_vocab <= 0 || c->max_batch <= 0 || c->max_seq <= 0 || c->device < 0 || !(c->ln_eps >= 0.f))
+        return RLX_ERR_INVALID_ARG;
+    if (c->hidden % 128 != 0 || c->hidden > 1024 || c->hidden % c->num_heads != 0) return RLX_ERR_UNSUPPORTED;
+    const int d = c->hidden / c->num_heads;
+    if ((d != 32 && d != 64) || c->ffn % 64 != 0 || c->max_seq > c->max_pos || c->max_seq > 512)
+        return RLX_ERR_UNSUPPORTED;
+    if ((long long)c->max_batch * c->max_seq > (1ll << 30)) return RLX_ERR_UNSUPPORTED;
+    rlx_encoder* e = new (std::nothrow) rlx_encoder();
+    if (!e) return RLX_ERR_INVALID_ARG;
+    e->cfg = *c;
+    e->head_dim = d;
+    *out = e;
+    return RLX_OK;
+}
+
+void rlx_encoder_destroy(rlx_encoder_t* e) {
+    if (!e) return;
+    drop_graphs(e);
+    delete e;
+}
+
+size_t rlx_encoder_workspace_bytes(const rlx_encoder_t* e, int32_t batch, int32_t seq) {
+    if (!e || batch <= 0 || seq <= 0 || batch > e->cfg.max_batch || seq > e->cfg.max_seq) return 0;
+    return plan_arena(batch, seq, e->cfg.hidden, e->cfg.ffn).total;
+}
+
+int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e) { return e ? 2 + 7 * e->cfg.num_layers : 0; }
+
+rlx_status_t rlx_encoder_forward(rlx_encoder_t* e, const int32_t* ids, const int32_t* mask, int32_t B, int32_t S,
+                                 const rlx_encoder_weights_t* w, float* out, void* ws, size_t ws_bytes, void* stream) {
+    rlx_status_t s = check_forward_args(e, ids, mask, B, S, w, out, ws, ws_bytes, false);
+    if (s != RLX_OK) return s;
+    return forward_device(e, ids, mask, B, S, w, out, static_cast<unsigned char*>(ws), static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_encoder_forward_host(rlx_encoder_t* e, const int32_t* ids_h, const int32_t* mask_h, int32_t B,
+                                      int32_t S, const rlx_encoder_weights_t* w, float* out_h, void* ws,
+                                      size_t ws_bytes, void* stream) {
+    rlx_status_t s = check_forward_args(e, ids_h, mask_h, B, S, w, out_h, ws, ws_bytes, true);
+    if (s != RLX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    int32_t* ids_d = reinterpret_cast<int32_t*>(base + a.ids);
+    int32_t* mask_d = reinterpret_cast<int32_t*>(base + a.mask);
+    float* out_d = reinterpret_cast<float*>(base + a.out);
+    const size_t tok_bytes = (size_t)B * S * sizeof(int32_t);
+    RLX_CUDA_TRY(cudaMemcpyAsync(ids_d, ids_h, tok_bytes, cudaMemcpyHostToDevice, st));
+    RLX_CUDA_TRY(cudaMemcpyAsync(mask_d, mask_h, tok_bytes, cudaMemcpyHostToDevice, st));
+    s = forward_device(e, ids_d, mask_d, B, S, w, out_d, base, st);
+    if (s != RLX_OK) return s;
+    RLX_CUDA_TRY(cudaMemcpyAsync(out_h, out_d, (size_t)B * e->cfg.hidden * sizeof(float), cudaMemcpyDeviceToHost, st));
+    RLX_CUDA_TRY(cudaStreamSynchronize(st));
+    return RLX_OK;
+}
+
+rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t* e, void* ws, void* stream) {
+    if (!e || !ws) return RLX_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    RLX_CUDA_TRY(cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st));
+    RLX_CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(word), st));
+    RLX_CUDA_TRY(cudaStreamSynchronize(st));
+    if (word & RLX_DEVSTAT_TIMEOUT) return RLX_ERR_DEVICE_TIMEOUT;
+    if (word & RLX_DEVSTAT_TOKEN_RANGE) return RLX_ERR_TOKEN_RANGE;
+    return RLX_OK;
+}
+
+const char* rlx_status_string(rlx_status_t s) {
+    switch (s) {
+        case RLX_OK: return "ok";
+        case RLX_ERR_INVALID_ARG: return "invalid argument";
+        case RLX_ERR_UNSUPPORTED: return "unsupported shape";
+        case RLX_ERR_WORKSPACE: return "workspace too small";
+        case RLX_ERR_CUDA: return "CUDA call failed";
+        case RLX_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case RLX_ERR_TOKEN_RANGE: return "token id out of range (clamped)";
+    }
+    return "unknown status";
+}
+
+// ------------------------------------------------------------------- kernel-level entry points
+rlx_status_t rlx_embed_layernorm(const int32_t* ids, const void* word, const void* pos, const void* type,
+                                 const float* gamma, const float* beta, int32_t T, int32_t S, int32_t H, int32_t V,
+                                 float eps, void* out, int32_t* status, void* stream) {
+    if (!ids || !word || !pos || !type || !gamma || !beta || !out || T <= 0 || S <= 0 || V <= 0) return RLX_ERR_INVALID_ARG;
+    if (H <= 0 || H % 128 != 0 || H > 1024) return RLX_ERR_UNSUPPORTED;
+    if (!aligned16(word) || !aligned16(pos) || !aligned16(type) || !aligned16(gamma) || !aligned16(beta) || !aligned16(out))
+        return RLX_ERR_INVALID_ARG;
+    return launch_embed_ln(ids, (const bf16*)word, (const bf16*)pos, (const bf16*)type, gamma, beta, T, S, H, V, eps,
+                           (bf16*)out, status, static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_layernorm(const void* x, const float* gamma, const float* beta, int32_t rows, int32_t H, float eps,
+                           void* out, void* stream) {
+    if (!x || !gamma || !beta || !out || rows <= 0) return RLX_ERR_INVALID_ARG;
+    if (H <= 0 || H % 128 != 0 || H > 1024) return RLX_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(gamma) || !aligned16(beta) || !aligned16(out)) return RLX_ERR_INVALID_ARG;
+    return launch_layernorm((const bf16*)x, gamma, beta, rows, H, eps, (bf16*)out, static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_gemm_bf16(const void* A, const void* W, const float* bias, const void* residual, rlx_epilogue_t epi,
+                           int32_t M, int32_t N, int32_t K, void* out, rlx_gemm_impl_t impl, int32_t* status,
+                           void* stream) {
+    if (!A || !W || !bias || !out || M <= 0 || N <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
+    if ((int)epi < 0 || (int)epi > 2 || (epi == RLX_EPI_BIAS_RESIDUAL && !residual)) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(W) || !aligned16(bias) || !aligned16(out) || (residual && !aligned16(residual)))
+        return RLX_ERR_INVALID_ARG;
+    if (N % 64 != 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
+    if (impl != RLX_GEMM_TCGEN05 && impl != RLX_GEMM_SIMT) return RLX_ERR_INVALID_ARG;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return launch_gemm((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, (int)epi, M, N, K, (bf16*)out,
+                       impl == RLX_GEMM_SIMT, status, static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_attention_bf16(const void* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,
+                                void* ctx, void* stream) {
+    if (!qkv || !mask || !ctx || B <= 0 || S <= 0 || h <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(qkv) || !aligned16(ctx)) return RLX_ERR_INVALID_ARG;
+    if ((d != 32 && d != 64) || S > 512 || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return launch_attention_bf16((const bf16*)qkv, mask, B, S, h, d, (bf16*)ctx, static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,
+                               float* ctx, void* stream) {
+    if (!qkv || !mask || !ctx || B <= 0 || S <= 0 || h <= 0) return RLX_ERR_INVALID_ARG;
+    if ((d != 32 && d != 64) || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 grid((S + rlx::kAttF32Warps - 1) / rlx::kAttF32Warps, h, B);
+    const float scale = 1.0f / sqrtf((float)d);
+    if (d == 32)
+        rlx::attention_f32_kernel<32><<<grid, rlx::kAttF32Warps * 32, 0, st>>>(qkv, mask, ctx, S, h * d, scale);
+    else
+        rlx::attention_f32_kernel<64><<<grid, rlx::kAttF32Warps * 32, 0, st>>>(qkv, mask, ctx, S, h * d, scale);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t rlx_pool_l2norm(const void* x, const int32_t* mask, int32_t B, int32_t S, int32_t H, float* out,
+                             void* stream) {
+    if (!x || !mask || !out || B <= 0 || S <= 0) return RLX_ERR_INVALID_ARG;
+    if (H <= 0 || H % 128 != 0 || H > 1024) return RLX_ERR_UNSUPPORTED;
+    if (!aligned16(x)) return RLX_ERR_INVALID_ARG;
+    return launch_pool((const bf16*)x, mask, B, S, H, out, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every
+symbol the header declares, validates arguments before any launch, and sizes the workspace."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2609_37916_b200 import binding
+from paper_2609_37916_b200.build import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build()
+    return binding._load()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "rlx_encoder.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(rlx_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS), declared ^ set(binding.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings(lib):
+    seen = {lib.rlx_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+    assert lib.rlx_status_string(99).decode() == "unknown status"
+
+
+def _cfg(**kw):
+    base = dict(num_layers=6, hidden=384, num_heads=12, ffn=1536, vocab=30522, max_pos=512, type_vocab=2,
+                ln_eps=1e-12, max_batch=32, max_seq=128, device=0, flags=0)
+    base.update(kw)
+    return base
+
+
+def test_create_validates_shapes(lib):
+    enc = binding.Encoder(**_cfg())
+    assert enc.kernels_per_forward() == 2 + 7 * 6
+    enc.close()
+    for bad, status in [
+        (dict(hidden=400, num_heads=10), 2),    # H % 128
+        (dict(hidden=384, num_heads=8), 2),     # head_dim 48
+        (dict(hidden=2048, num_heads=32), 2),   # H > 1024
+        (dict(ffn=1000), 2),                    # F % 64
+        (dict(max_seq=1024, max_pos=512), 2),   # seq > max_pos
+        (dict(num_layers=0), 1),
+        (dict(max_batch=-1), 1),
+    ]:
+        with pytest.raises(binding.RlxError) as ei:
+            binding.Encoder(**_cfg(**bad))
+        assert ei.value.status == status, bad
+
+
+def test_create_rejects_wrong_struct_size_and_null(lib):
+    cfg = binding._Config(4, 6, 384, 12, 1536, 30522, 512, 2, 1e-12, 32, 128, 0, 0)
+    h = C.c_void_p()
+    assert lib.rlx_encoder_create(C.byref(cfg), C.byref(h)) == 1
+    assert lib.rlx_encoder_create(None, C.byref(h)) == 1
+    lib.rlx_encoder_destroy(None)  # no-op
+
+
+def test_workspace_bytes_layout(lib):
+    enc = binding.Encoder(**_cfg(max_batch=256, max_seq=256))
+    T, H, F = 256 * 256, 384, 1536
+    need = enc.workspace_bytes(256, 256)
+    acts = T * (H + 3 * H + H + H + H + F) * 2
+    assert acts <= need <= acts + 3 * T * 4 + (1 << 20)
+    assert need % 256 == 0
+    assert enc.workspace_bytes(257, 256) == 0 and enc.workspace_bytes(1, 0) == 0
+    assert enc.workspace_bytes(1, 16) < enc.workspace_bytes(2, 16)
+    enc.close()
+
+
+def test_forward_rejects_bad_arguments_before_touching_the_device(lib):
+    enc = binding.Encoder(**_cfg())
+    w = binding._Weights()
+    w.struct_size = C.sizeof(binding._Weights)
+    fake = C.c_void_p(0x1000)
+    # null pointers
+    assert lib.rlx_encoder_forward(enc._h, None, fake, 1, 16, C.byref(w), fake, fake, C.c_size_t(1 << 30), None) == 1
+    # sizes outside the configured bounds
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 64, 16, C.byref(w), fake, fake, C.c_size_t(1 << 30), None) == 1
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 1, 129, C.byref(w), fake, fake, C.c_size_t(1 << 30), None) == 1
+    # weights struct without layers
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 1, 16, C.byref(w), fake, fake, C.c_size_t(1 << 30), None) == 1
+    # misaligned workspace / ids
+    layers = (binding._Layer * 6)()
+    for l in layers:
+        for n in binding.LAYER_FIELDS:
+            setattr(l, n, 0x2000)
+    w.layers = layers
+    for n in ("word_emb", "pos_emb", "type_emb", "emb_ln_g", "emb_ln_b"):
+        setattr(w, n, 0x2000)
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 1, 16, C.byref(w), fake, C.c_void_p(0x1010),
+                                   C.c_size_t(1 << 30), None) == 1
+    assert lib.rlx_encoder_forward(enc._h, C.c_void_p(0x1004), fake, 1, 16, C.byref(w), fake, fake,
+                                   C.c_size_t(1 << 30), None) == 1
+    # workspace too small
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 1, 16, C.byref(w), fake, fake, C.c_size_t(1024), None) == 3
+    # a null weight pointer inside a layer
+    layers[3].w2 = 0
+    assert lib.rlx_encoder_forward(enc._h, fake, fake, 1, 16, C.byref(w), fake, fake, C.c_size_t(1 << 30), None) == 1
+    enc.close()
+
+
+def test_kernel_entry_points_validate_on_the_host(lib):
+    fake = C.c_void_p(0x1000)
+    assert lib.rlx_layernorm(fake, fake, fake, 4, 100, C.c_float(1e-12), fake, None) == 2   # H % 128
+    assert lib.rlx_layernorm(None, fake, fake, 4, 128, C.c_float(1e-12), fake, None) == 1
+    assert lib.rlx_gemm_bf16(fake, fake, fake, None, 0, 8, 100, 64, fake, 0, None, None) == 2  # N % 64
+    assert lib.rlx_gemm_bf16(fake, fake, fake, None, 0, 8, 128, 60, fake, 0, None, None) == 2  # K % 8
+    assert lib.rlx_gemm_bf16(fake, fake, fake, None, 2, 8, 128, 64, fake, 0, None, None) == 1  # residual missing
+    assert lib.rlx_attention_bf16(fake, fake, 1, 16, 12, 48, fake, None) == 2                   # head_dim
+    assert lib.rlx_attention_bf16(fake, fake, 1, 1024, 12, 32, fake, None) == 2                 # seq > 512
+    assert lib.rlx_attention_f32(fake, fake, 0, 16, 12, 32, fake, None) == 1
+    assert lib.rlx_pool_l2norm(fake, fake, 1, 16, 100, fake, None) == 2
+    assert lib.rlx_embed_layernorm(fake, fake, fake, fake, fake, fake, 16, 16, 2048, 100, C.c_float(0), fake,
+                                   None, None) == 2

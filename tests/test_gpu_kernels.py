@@ -1,0 +1,234 @@
+"""Each CUDA kernel, through the C ABI, against the fp64 oracle on the same seeded inputs.
+Sizes span several tiles plus ragged tails; tolerances are derived from bf16 storage
+(unit round-off u = 2^-9) with fp32 arithmetic inside the kernels."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import oracle  # noqa: E402
+from synth.inputs import CONFIGS, make_inputs, round_to_bf16  # noqa: E402
+from gpu_common import BF16_U, bf16_dev, f32_dev, i32_dev, rand_bf16, to_np64  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rlx():
+    import paper_2609_37916_b200 as pkg
+    from paper_2609_37916_b200.build import build
+    build()
+    return pkg
+
+
+def assert_close_bf16_out(got, ref, extra_abs=0.0):
+    """Output stored in bf16: |err| <= 2u|ref| + small absolute slack for fp32 accumulation."""
+    tol = 2 * BF16_U * np.abs(ref) + 1e-5 + extra_abs
+    bad = np.abs(got - ref) > tol
+    assert not bad.any(), (int(bad.sum()), float(np.abs(got - ref).max()))
+
+
+# ------------------------------------------------------------------ LayerNorm / embedding / pool
+@pytest.mark.parametrize("H", [128, 384, 768, 1024])
+@pytest.mark.parametrize("rows", [1, 7, 1000])
+def test_layernorm(rlx, H, rows):
+    rng = np.random.default_rng(H + rows)
+    x = rand_bf16(rng, (rows, H), 2.0) + round_to_bf16(np.float32(0.5))
+    x = round_to_bf16(x)
+    g = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    b = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    got = to_np64(rlx.layernorm(bf16_dev(x), f32_dev(g), f32_dev(b), 1e-12))
+    ref = oracle.layernorm(x.astype(np.float64), g, b, 1e-12)
+    assert_close_bf16_out(got, ref)
+
+
+def test_layernorm_constant_row_gives_beta(rlx):
+    H = 384
+    x = np.full((3, H), 1.5, np.float32)
+    b = round_to_bf16(np.linspace(-1, 1, H).astype(np.float32))
+    got = to_np64(rlx.layernorm(bf16_dev(x), f32_dev(np.ones(H)), f32_dev(b), 1e-12))
+    assert np.array_equal(got, np.broadcast_to(b.astype(np.float64), (3, H)))
+
+
+@pytest.mark.parametrize("name", ["c0", "c1"])
+def test_embed_layernorm_matches_oracle_stage(rlx, name):
+    inp = make_inputs(CONFIGS[name], ln_affine_random=True)
+    c = inp.cfg
+    # hit both ends of the vocabulary
+    inp.ids[0, 0], inp.ids[0, 1] = 0, c.vocab - 1
+    _, d = oracle.encoder_forward(c, inp.ids, inp.mask, inp.params, [],
+                                  compute_all_rows=True, dumps=True)
+    p = inp.params
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = rlx.embed_layernorm(i32_dev(inp.ids), bf16_dev(p["word_emb"]), bf16_dev(p["pos_emb"]),
+                              bf16_dev(p["type_emb"]), f32_dev(p["emb_ln_g"]), f32_dev(p["emb_ln_b"]),
+                              c.seq, c.vocab, c.ln_eps, status=status)
+    assert_close_bf16_out(to_np64(got).reshape(c.batch, c.seq, c.hidden), d["x_emb"])
+    assert int(status.item()) == 0
+
+
+def test_embed_out_of_range_id_is_clamped_and_flagged(rlx):
+    inp = make_inputs(CONFIGS["c0"])
+    c, p = inp.cfg, inp.params
+    ids = inp.ids.copy()
+    ids[0, 3] = c.vocab + 5
+    ids[0, 4] = -2
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (bf16_dev(p["word_emb"]), bf16_dev(p["pos_emb"]), bf16_dev(p["type_emb"]), f32_dev(p["emb_ln_g"]),
+            f32_dev(p["emb_ln_b"]), c.seq, c.vocab, c.ln_eps)
+    got = rlx.embed_layernorm(i32_dev(ids), *args, status=status)
+    assert int(status.item()) == 1
+    clamped = inp.ids.copy()
+    clamped[0, 3], clamped[0, 4] = c.vocab - 1, 0
+    want = rlx.embed_layernorm(i32_dev(clamped), *args)
+    assert torch.equal(got, want)
+
+
+@pytest.mark.parametrize("B,S,H", [(1, 16, 384), (5, 37, 384), (3, 512, 768), (2, 9, 1024), (4, 33, 128)])
+def test_pool_l2norm(rlx, B, S, H):
+    rng = np.random.default_rng(B * S + H)
+    x = rand_bf16(rng, (B, S, H))
+    mask = (rng.random((B, S)) < 0.6).astype(np.int32)
+    mask[0, :] = 0
+    mask[0, S // 2] = 1          # single valid token
+    if B > 1:
+        mask[1, :] = 0           # empty sequence -> zeros
+    got = to_np64(rlx.pool_l2norm(bf16_dev(x), i32_dev(mask)))
+    ref = oracle.pool_l2(x.astype(np.float64), mask)
+    assert np.abs(got - ref).max() < 2e-6
+    if B > 1:
+        assert np.array_equal(got[1], np.zeros(H))
+
+
+# ------------------------------------------------------------------ GEMM
+GEMM_SHAPES = [(128, 64, 64), (16, 1152, 384), (300, 384, 384), (257, 1536, 384), (1000, 384, 1536),
+               (129, 768, 768), (4096, 192, 72), (2048, 2304, 768)]
+
+
+@pytest.mark.parametrize("impl", [0, 1], ids=["tcgen05", "simt"])
+def test_gemm_small_integers_is_bit_exact(rlx, impl):
+    """Operands are small integers (exact in bf16, sums exact in fp32): any layout, descriptor or
+    indexing mistake shows up as a wrong integer, with no tolerance to hide behind."""
+    rng = np.random.default_rng(11)
+    for (M, N, K) in [(128, 64, 64), (128, 128, 128), (200, 192, 384), (384, 256, 136), (130, 384, 1536)]:
+        a = rng.integers(-3, 4, size=(M, K)).astype(np.float32)
+        w = rng.integers(-3, 4, size=(N, K)).astype(np.float32)
+        bias = rng.integers(-8, 9, size=N).astype(np.float32)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        got = to_np64(rlx.gemm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(bias), impl=impl, status=status))
+        ref = a.astype(np.float64) @ w.astype(np.float64).T + bias
+        assert int(status.item()) == 0
+        assert np.abs(ref).max() < 256  # integers below 2^8 are exact in bf16
+        assert np.array_equal(got, ref), (M, N, K, np.abs(got - ref).max())
+
+
+@pytest.mark.parametrize("impl", [0, 1], ids=["tcgen05", "simt"])
+@pytest.mark.parametrize("epi", [0, 1, 2], ids=["bias", "gelu", "residual"])
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+def test_gemm_matches_oracle_linear(rlx, shape, epi, impl):
+    M, N, K = shape
+    if impl == 1 and M * N * K > 2e9:
+        pytest.skip("bring-up GEMM: large case covered by the tensor-core path")
+    rng = np.random.default_rng(M + N + K + epi)
+    a = rand_bf16(rng, (M, K))
+    w = rand_bf16(rng, (N, K), 0.05)
+    bias = (0.1 * rng.standard_normal(N)).astype(np.float32)
+    res = rand_bf16(rng, (M, N)) if epi == 2 else None
+    got = to_np64(rlx.gemm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(bias),
+                                residual=bf16_dev(res) if res is not None else None, epilogue=epi, impl=impl))
+    ref = oracle.linear(a.astype(np.float64), w, bias)
+    if epi == 1:
+        ref = oracle.gelu(ref)
+    if epi == 2:
+        ref = ref + res.astype(np.float64)
+    # fp32 accumulation of K products of magnitude ~|a||w|: error ~ K * 2^-24 * sum|a_k w_k|
+    assert_close_bf16_out(got, ref, extra_abs=K * 2.0 ** -24 * 0.2)
+
+
+# ------------------------------------------------------------------ attention
+def _qkv_case(seed, B, S, h, d, gain=1.0, holes=0.0):
+    rng = np.random.default_rng(seed)
+    H = h * d
+    qkv = rand_bf16(rng, (B, S, 3 * H))
+    qkv[..., :H] = round_to_bf16(qkv[..., :H] * np.float32(gain))
+    lengths = rng.integers(1, S + 1, size=B)
+    lengths[0] = S
+    if B > 1:
+        lengths[1] = 1
+    mask = (np.arange(S)[None, :] < lengths[:, None]).astype(np.int32)
+    if holes > 0:
+        mask = (mask * (rng.random((B, S)) >= holes)).astype(np.int32)
+        mask[:, 0] = 1
+    return qkv, mask
+
+
+ATT_CASES = [(1, 16, 12, 32), (3, 128, 12, 32), (2, 129, 4, 32), (2, 1, 2, 32), (3, 200, 3, 64), (2, 512, 2, 64),
+             (4, 63, 12, 32), (2, 65, 2, 64)]
+
+
+@pytest.mark.parametrize("case", ATT_CASES)
+@pytest.mark.parametrize("variant", ["plain", "peaky", "holes"])
+def test_attention_f32_mode_within_1e4_relative(rlx, case, variant):
+    B, S, h, d = case
+    qkv, mask = _qkv_case(sum(case), B, S, h, d, gain=6.0 if variant == "peaky" else 1.0,
+                          holes=0.3 if variant == "holes" else 0.0)
+    got = to_np64(rlx.attention_f32(f32_dev(qkv), i32_dev(mask), h))
+    ref = oracle.attention(qkv.astype(np.float64), mask, h, compute_all_rows=True)
+    valid = mask != 0
+    ref_v, got_v = ref[valid], got[valid]
+    # per (sequence, head) scale-relative error and an element-wise bound
+    assert np.abs(got_v - ref_v).max() <= 1e-4 * np.abs(ref_v).max()
+    assert np.all(np.abs(got_v - ref_v) <= 1e-4 * np.abs(ref_v) + 1e-6)
+    for b in range(B):
+        for j in range(h):
+            r = ref[b][valid[b]][:, j * d:(j + 1) * d]
+            g = got[b][valid[b]][:, j * d:(j + 1) * d]
+            assert np.abs(g - r).max() <= 1e-4 * np.abs(r).max()
+
+
+@pytest.mark.parametrize("case", ATT_CASES)
+@pytest.mark.parametrize("variant", ["plain", "peaky", "holes"])
+def test_attention_bf16_mode(rlx, case, variant):
+    B, S, h, d = case
+    qkv, mask = _qkv_case(sum(case) + 1, B, S, h, d, gain=6.0 if variant == "peaky" else 1.0,
+                          holes=0.3 if variant == "holes" else 0.0)
+    got = to_np64(rlx.attention_bf16(bf16_dev(qkv), i32_dev(mask), h))
+    ref = oracle.attention(qkv.astype(np.float64), mask, h, compute_all_rows=True)
+    valid = mask != 0
+    # probabilities are rounded to bf16 before the PV product and the result is stored in bf16:
+    # |err| <= u * (max|v| + |out|) with margin 2
+    vmax = np.abs(qkv[..., 2 * h * d:]).max()
+    assert np.abs(got[valid] - ref[valid]).max() <= 2 * BF16_U * (vmax + np.abs(ref[valid]).max())
+    assert np.all(np.isfinite(got))
+
+
+def test_attention_adversarial_logits(rlx):
+    """One dominant key (+30), all-equal logits, and logits so negative that exp underflows."""
+    h, d, S = 1, 32, 64
+    H = h * d
+    for mode in ("dominant", "equal", "underflow"):
+        qkv = np.zeros((1, S, 3 * H), np.float32)
+        rng = np.random.default_rng(5)
+        qkv[..., 2 * H:] = rand_bf16(rng, (1, S, H))
+        if mode == "dominant":
+            qkv[0, :, :H] = 1.0
+            qkv[0, 7, H:2 * H] = round_to_bf16(np.float32(30.0 * np.sqrt(d) / d))
+        elif mode == "underflow":
+            qkv[0, :, :H] = 1.0
+            qkv[0, :, H:2 * H] = -40.0
+            qkv[0, 3, H:2 * H] = 0.0
+        mask = np.ones((1, S), np.int32)
+        ref = oracle.attention(qkv.astype(np.float64), mask, h)
+        got32 = to_np64(rlx.attention_f32(f32_dev(qkv), i32_dev(mask), h))
+        got16 = to_np64(rlx.attention_bf16(bf16_dev(qkv), i32_dev(mask), h))
+        assert np.abs(got32 - ref).max() <= 1e-4 * np.abs(ref).max(), mode
+        assert np.abs(got16 - ref).max() <= 4 * BF16_U * np.abs(qkv[..., 2 * H:]).max(), mode
+
+
+def test_attention_all_masked_sequence_gives_zeros(rlx):
+    qkv, mask = _qkv_case(3, 2, 70, 2, 32)
+    mask[1, :] = 0
+    got = rlx.attention_bf16(bf16_dev(qkv), i32_dev(mask), 2)
+    assert torch.count_nonzero(got[1]) == 0
+    got32 = rlx.attention_f32(f32_dev(qkv), i32_dev(mask), 2)
+    assert torch.count_nonzero(got32[1]) == 0
