@@ -25,6 +25,7 @@ using bf16 = __nv_bfloat16;
         cudaError_t _e = (expr);                \
         if (_e != cudaSuccess) {                \
             g_last_cuda_error = _e;             \
+            (void)cudaGetLastError();           \
             return RLX_ERR_CUDA;                \
         }                                       \
     } while (0)
@@ -249,6 +250,8 @@ struct rlx_encoder {
     rlx_encoder_weights_t weights;
     bool have_weights = false;
     std::vector<GraphEntry> graphs;
+    cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
+                                            // legacy default stream, which cannot be captured)
 };
 
 namespace {
@@ -339,9 +342,10 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
         }
     // capture once for this (batch, seq, pointer set)
     cudaGraph_t graph = nullptr;
-    RLX_CUDA_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, st);
-    cudaError_t ce = cudaStreamEndCapture(st, &graph);
+    if (!e->capture_stream) RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
+    RLX_CUDA_TRY(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal));
+    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream);
+    cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
     if (s != RLX_OK) {
         if (graph) cudaGraphDestroy(graph);
         return s;
@@ -388,6 +392,7 @@ rlx_status_t rlx_encoder_create(const rlx_encoder_config_t* c, rlx_encoder_t** o
 void rlx_encoder_destroy(rlx_encoder_t* e) {
     if (!e) return;
     drop_graphs(e);
+    if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
     delete e;
 }
 

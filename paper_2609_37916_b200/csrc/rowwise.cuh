@@ -17,14 +17,14 @@ __device__ __forceinline__ void ln_normalise_store(float (&v)[NV * 4], const flo
     float s = 0.f;
 #pragma unroll
     for (int i = 0; i < NV * 4; ++i) s += v[i];
-    const float mean = warp_sum(s) * (1.0f / H);
+    const float mean = warp_sum(s) / (float)H;  // true division: a constant row has exactly zero deviation
     float q = 0.f;
 #pragma unroll
     for (int i = 0; i < NV * 4; ++i) {
         v[i] -= mean;
         q += v[i] * v[i];
     }
-    const float var = warp_sum(q) * (1.0f / H);
+    const float var = warp_sum(q) / (float)H;
     const float rstd = 1.0f / sqrtf(var + eps);
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
