@@ -59,6 +59,7 @@ typedef enum {
 /* rlx_encoder_config_t.flags */
 #define RLX_FLAG_NO_GRAPH 0x1u  /* launch kernels one by one instead of replaying a CUDA graph */
 #define RLX_FLAG_GEMM_SIMT 0x2u /* use the plain CUDA-core GEMM (bring-up / cross-check only)  */
+#define RLX_FLAG_KERNEL_EVENTS 0x4u /* record a CUDA event between kernels (see rlx_encoder_kernel_times) */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */
@@ -174,6 +175,17 @@ rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t *encoder, void *worksp
 
 /* Number of kernels one forward of (batch, seq) launches (for launch accounting). */
 int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t *encoder);
+
+/*
+ * Per-kernel device times of the most recent forward of an encoder created with
+ * RLX_FLAG_KERNEL_EVENTS (the paper's runtime exposes per-operator reports, Section 4; this is
+ * the timing analogue).  Waits for that forward to finish, then writes `count` =
+ * rlx_encoder_kernels_per_forward() durations in milliseconds to ms_host (host memory), in
+ * launch order: embed+LN, then per layer [QKV GEMM, attention, out-proj GEMM, LN, FFN-up GEMM,
+ * FFN-down GEMM, LN], then pool.  In graph mode the events are nodes of the captured graph, so
+ * the figures contain no host launch gaps.  RLX_ERR_UNSUPPORTED if the flag was not set.
+ */
+rlx_status_t rlx_encoder_kernel_times(rlx_encoder_t *encoder, float *ms_host, int32_t count);
 
 /* Static string for a status code. */
 const char *rlx_status_string(rlx_status_t status);

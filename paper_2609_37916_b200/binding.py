@@ -21,12 +21,13 @@ STATUS_NAMES = {0: "RLX_OK", 1: "RLX_ERR_INVALID_ARG", 2: "RLX_ERR_UNSUPPORTED",
                 4: "RLX_ERR_CUDA", 5: "RLX_ERR_DEVICE_TIMEOUT", 6: "RLX_ERR_TOKEN_RANGE"}
 FLAG_NO_GRAPH = 0x1
 FLAG_GEMM_SIMT = 0x2
+FLAG_KERNEL_EVENTS = 0x4
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 
 EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
-    "rlx_encoder_forward_host", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward",
+    "rlx_encoder_forward_host", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
     "rlx_attention_f32", "rlx_pool_l2norm",
 )
@@ -190,6 +191,13 @@ class Encoder:
                                                 _ptr(out), _ptr(workspace), C.c_size_t(workspace.numel()),
                                                 _stream(stream)), "rlx_encoder_forward_host")
         return out
+
+    def kernel_times(self) -> List[float]:
+        """Milliseconds per kernel of the last forward (encoder created with FLAG_KERNEL_EVENTS)."""
+        n = self.kernels_per_forward()
+        buf = (C.c_float * n)()
+        _check(_load().rlx_encoder_kernel_times(self._h, buf, n), "rlx_encoder_kernel_times")
+        return list(buf)
 
     def last_device_status(self, workspace: torch.Tensor, stream=None) -> int:
         return int(_load().rlx_encoder_last_device_status(self._h, _ptr(workspace), _stream(stream)))

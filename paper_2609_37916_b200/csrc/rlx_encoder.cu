@@ -250,6 +250,7 @@ struct rlx_encoder {
     rlx_encoder_weights_t weights;
     bool have_weights = false;
     std::vector<GraphEntry> graphs;
+    std::vector<cudaEvent_t> events;        // RLX_FLAG_KERNEL_EVENTS: one before the first kernel, one after each
     cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
                                             // legacy default stream, which cannot be captured)
 };
@@ -271,7 +272,8 @@ void drop_graphs(rlx_encoder* e) {
 
 // The kernel sequence of one forward, enqueued on `st` (eagerly or under stream capture).
 rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
-                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
+                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st,
+                             bool capturing) {
     const rlx_encoder_config_t& c = e->cfg;
     const int H = c.hidden, F = c.ffn, T = B * S, h = c.num_heads, d = e->head_dim;
     const bool simt = (c.flags & RLX_FLAG_GEMM_SIMT) != 0;
@@ -284,7 +286,19 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     bf16* x1 = reinterpret_cast<bf16*>(ws + a.x1);
     bf16* g = reinterpret_cast<bf16*>(ws + a.g);
     rlx_status_t s;
-#define RLX_TRY(call) do { s = (call); if (s != RLX_OK) return s; } while (0)
+    size_t ev = 0;
+    // With RLX_FLAG_KERNEL_EVENTS an event is recorded between consecutive kernels; under stream
+    // capture the records become event-record nodes of the graph, so replays time each kernel on
+    // the device without any host launch gap.
+    auto mark = [&]() -> rlx_status_t {
+        if (e->events.empty()) return RLX_OK;
+        RLX_CUDA_TRY(cudaEventRecordWithFlags(e->events[ev++], st,
+                                              capturing ? cudaEventRecordExternal : cudaEventRecordDefault));
+        return RLX_OK;
+    };
+#define RLX_TRY(call) do { s = (call); if (s != RLX_OK) return s; s = mark(); if (s != RLX_OK) return s; } while (0)
+    s = mark();
+    if (s != RLX_OK) return s;
     RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
                             w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st));
     for (int l = 0; l < c.num_layers; ++l) {
@@ -326,7 +340,11 @@ rlx_status_t check_forward_args(const rlx_encoder* e, const void* ids, const voi
 rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
     RLX_CUDA_TRY(init_kernels_for_current_device());
-    if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st);
+    if ((e->cfg.flags & RLX_FLAG_KERNEL_EVENTS) && e->events.empty()) {
+        e->events.resize(3 + 7 * (size_t)e->cfg.num_layers);
+        for (auto& evt : e->events) RLX_CUDA_TRY(cudaEventCreate(&evt));
+    }
+    if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);
 
     if (!same_weights(e, w)) {
         drop_graphs(e);
@@ -344,7 +362,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
     cudaGraph_t graph = nullptr;
     if (!e->capture_stream) RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
     RLX_CUDA_TRY(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal));
-    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream);
+    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream, true);
     cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
     if (s != RLX_OK) {
         if (graph) cudaGraphDestroy(graph);
@@ -393,6 +411,7 @@ void rlx_encoder_destroy(rlx_encoder_t* e) {
     if (!e) return;
     drop_graphs(e);
     if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
+    for (auto& evt : e->events) cudaEventDestroy(evt);
     delete e;
 }
 
@@ -440,6 +459,14 @@ rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t* e, void* ws, void* st
     RLX_CUDA_TRY(cudaStreamSynchronize(st));
     if (word & RLX_DEVSTAT_TIMEOUT) return RLX_ERR_DEVICE_TIMEOUT;
     if (word & RLX_DEVSTAT_TOKEN_RANGE) return RLX_ERR_TOKEN_RANGE;
+    return RLX_OK;
+}
+
+rlx_status_t rlx_encoder_kernel_times(rlx_encoder_t* e, float* ms_host, int32_t count) {
+    if (!e || !ms_host || count != rlx_encoder_kernels_per_forward(e)) return RLX_ERR_INVALID_ARG;
+    if (e->events.size() != (size_t)count + 1) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(cudaEventSynchronize(e->events.back()));
+    for (int i = 0; i < count; ++i) RLX_CUDA_TRY(cudaEventElapsedTime(&ms_host[i], e->events[i], e->events[i + 1]));
     return RLX_OK;
 }
 
