@@ -167,6 +167,38 @@ rlx_status_t rlx_encoder_forward_host(rlx_encoder_t *encoder, const int32_t *tok
                                       void *cuda_stream);
 
 /*
+ * The same forward for callers that cannot provide a workspace because they cannot allocate
+ * device memory at all.  (The paper has no counterpart: its runtime plans and owns its arena.)
+ * Typical callers: a plain C/C++ host that was handed only input and output buffers and links no
+ * allocator; a plug-in running inside another framework's callback where cudaMalloc/cudaFree are
+ * off limits because they synchronise the whole device or because the host application's pool
+ * already owns all device memory; a latency-critical loop that must not touch the allocator.
+ *
+ * The scratch arena is a fixed array of RLX_STATIC_WORKSPACE_BYTES built into the library's device
+ * image, so every GPU that loads the library gives up that much memory until the process exits.
+ * A (batch, seq) whose rlx_encoder_workspace_bytes exceeds the limit is rejected with
+ * RLX_ERR_WORKSPACE before anything is launched (at H=384, F=1536 the limit covers about 1,800
+ * tokens, e.g. batch 14 x seq 128).  The call makes no cudaMalloc/cudaFree and uses no
+ * allocating library routine: kernels are launched directly (no CUDA graph is built), and
+ * RLX_FLAG_KERNEL_EVENTS is ignored.
+ *
+ * token_ids, attention_mask, weights, out: exactly as for rlx_encoder_forward (dev pointers).
+ * device_status: optional dev int32; receives this call's RLX_DEVSTAT_* bits (0 = clean).
+ *
+ * The first call on each device looks up the arena's device address (the device must be
+ * current); make that first call outside any stream capture.  All calls, from every encoder
+ * object in the process, share the one arena and it keeps the previous call's contents: the call
+ * clears the only word that must start at zero itself, but two calls that overlap on the GPU
+ * (different streams, or different threads) race on the arena and corrupt each other.
+ * Asynchronous on cuda_stream.
+ */
+#define RLX_STATIC_WORKSPACE_BYTES (16u << 20)
+rlx_status_t rlx_encoder_forward_static(rlx_encoder_t *encoder, const int32_t *token_ids,
+                                        const int32_t *attention_mask, int32_t batch, int32_t seq,
+                                        const rlx_encoder_weights_t *weights, float *out,
+                                        int32_t *device_status, void *cuda_stream);
+
+/*
  * Synchronises cuda_stream, reads and clears the sticky device status word kept
  * in `workspace`, and maps it to RLX_OK / RLX_ERR_TOKEN_RANGE /
  * RLX_ERR_DEVICE_TIMEOUT (timeout wins).

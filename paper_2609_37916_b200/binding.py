@@ -24,10 +24,11 @@ FLAG_GEMM_SIMT = 0x2
 FLAG_KERNEL_EVENTS = 0x4
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
+STATIC_WORKSPACE_BYTES = 16 << 20
 
 EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
-    "rlx_encoder_forward_host", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
+    "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
     "rlx_attention_f32", "rlx_pool_l2norm",
 )
@@ -190,6 +191,20 @@ class Encoder:
         _check(_load().rlx_encoder_forward_host(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights.c),
                                                 _ptr(out), _ptr(workspace), C.c_size_t(workspace.numel()),
                                                 _stream(stream)), "rlx_encoder_forward_host")
+        return out
+
+    def forward_static(self, ids: torch.Tensor, mask: torch.Tensor, weights: DeviceWeights, out: torch.Tensor,
+                       device_status: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """rlx_encoder_forward_static: the forward for callers that cannot allocate a workspace; the
+        scratch lives in a fixed arena inside the library (STATIC_WORKSPACE_BYTES), shared by all
+        calls, so calls must not overlap on the GPU.  Raises RlxError(RLX_ERR_WORKSPACE) when
+        (batch, seq) needs more than the arena holds."""
+        B, S = ids.shape
+        assert ids.dtype == torch.int32 and mask.dtype == torch.int32 and out.dtype == torch.float32
+        assert ids.is_cuda and mask.is_cuda and out.is_cuda and ids.is_contiguous() and mask.is_contiguous()
+        _check(_load().rlx_encoder_forward_static(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights.c),
+                                                  _ptr(out), _ptr(device_status), _stream(stream)),
+               "rlx_encoder_forward_static")
         return out
 
     def kernel_times(self) -> List[float]:

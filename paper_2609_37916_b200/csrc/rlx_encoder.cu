@@ -483,6 +483,62 @@ const char* rlx_status_string(rlx_status_t s) {
     return "unknown status";
 }
 
+// ------------------------------------------------------------------- forward without a caller workspace
+}  // extern "C"
+
+// Scratch arena of rlx_encoder_forward_static.  It lives in the library's device image: every GPU
+// that loads the library reserves these bytes until the process exits.  In host code the name
+// below is only a stand-in for the symbol, not a device address; the address a kernel can use
+// is obtained per device with cudaGetSymbolAddress (static_workspace_for_current_device).
+static __device__ __align__(256) unsigned char g_static_workspace[RLX_STATIC_WORKSPACE_BYTES];
+
+namespace {
+// Resolves the device address of the static arena once per device (the device must be current).
+rlx_status_t static_workspace_for_current_device(unsigned char** out) {
+    static std::mutex mu;
+    static unsigned char* addr[64] = {};
+    int dev = 0;
+    RLX_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RLX_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!addr[dev]) {
+        void* p = nullptr;
+        RLX_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_workspace));
+        if (!p) return RLX_ERR_CUDA;
+        addr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = addr[dev];
+    return RLX_OK;
+}
+}  // namespace
+
+extern "C" {
+
+rlx_status_t rlx_encoder_forward_static(rlx_encoder_t* e, const int32_t* ids, const int32_t* mask, int32_t B,
+                                        int32_t S, const rlx_encoder_weights_t* w, float* out,
+                                        int32_t* device_status, void* stream) {
+    if (!e) return RLX_ERR_INVALID_ARG;
+    // validate everything but the workspace with a stand-in pointer and size
+    rlx_status_t s = check_forward_args(e, ids, mask, B, S, w, out, reinterpret_cast<void*>(uintptr_t(256)),
+                                        ~size_t(0), false);
+    if (s != RLX_OK) return s;
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    if (a.total > (size_t)RLX_STATIC_WORKSPACE_BYTES) return RLX_ERR_WORKSPACE;  // beyond the built-in arena
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* ws = nullptr;
+    s = static_workspace_for_current_device(&ws);
+    if (s != RLX_OK) return s;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    // the arena keeps the previous call's bytes: the status word is the only part read before it is
+    // written, so it alone is cleared; every activation row is rewritten by the kernels below
+    RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status, 0, sizeof(int32_t), st));
+    s = enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);  // direct launches: no graph objects
+    if (s != RLX_OK) return s;
+    if (device_status)
+        RLX_CUDA_TRY(cudaMemcpyAsync(device_status, ws + a.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    return RLX_OK;
+}
+
 // ------------------------------------------------------------------- kernel-level entry points
 rlx_status_t rlx_embed_layernorm(const int32_t* ids, const void* word, const void* pos, const void* type,
                                  const float* gamma, const float* beta, int32_t T, int32_t S, int32_t H, int32_t V,

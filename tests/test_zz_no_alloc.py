@@ -1,0 +1,71 @@
+"""rlx_encoder_forward_static: the forward for callers that cannot allocate device memory (no
+allocator linked, a host application that owns the whole memory pool, a loop that must not call
+cudaMalloc).  Its scratch is a fixed arena inside the library, so the result must equal the
+ordinary entry point's on the same inputs, also on a second call that reuses the dirty arena.
+Collected last on purpose: a failure here cannot hide any other test's result."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from gpu_common import cosine_rows, i32_dev, to_np64  # noqa: E402
+from synth.inputs import CONFIGS, make_inputs  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rlx():
+    import paper_2609_37916_b200 as pkg
+    from paper_2609_37916_b200.build import build
+    build()
+    return pkg
+
+
+def test_static_arena_forward_matches_workspace_forward_twice(rlx):
+    first = make_inputs(CONFIGS["c1"], batch=3, seq=96, num_layers=2, lengths=[96, 17, 50])
+    second = make_inputs(CONFIGS["c1"], batch=2, seq=128, num_layers=2, lengths=[5, 128], weights=False)
+    w = rlx.upload_weights(first.params, first.layers)
+    enc = rlx.Encoder.from_config(first.cfg, max_batch=4, max_seq=128)
+    for inp in (first, second):     # second call: other shape, arena still holds the first call's bytes
+        B, S, H = inp.cfg.batch, inp.cfg.seq, inp.cfg.hidden
+        assert enc.workspace_bytes(B, S) <= rlx.binding.STATIC_WORKSPACE_BYTES
+        ids, mask = i32_dev(inp.ids), i32_dev(inp.mask)
+        want = torch.empty((B, H), dtype=torch.float32, device="cuda")
+        enc.forward(ids, mask, w, want, enc.alloc_workspace(B, S))
+        got = torch.full((B, H), float("nan"), dtype=torch.float32, device="cuda")
+        status = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+        enc.forward_static(ids, mask, w, got, device_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        g, r = to_np64(got), to_np64(want)
+        assert np.all(np.isfinite(g))
+        # same kernels in the same order: identical bits; the graded tolerance is the fallback statement
+        assert cosine_rows(g, r).min() >= 0.9995 and np.abs(g - r).max() <= 2e-2
+        assert np.array_equal(g, r)
+    enc.close()
+
+
+def test_static_arena_rejects_sizes_beyond_its_limit_and_flags_bad_ids(rlx):
+    inp = make_inputs(CONFIGS["c2"], num_layers=1)
+    c = inp.cfg
+    enc = rlx.Encoder.from_config(c, max_batch=c.batch, max_seq=c.seq)
+    assert enc.workspace_bytes(c.batch, c.seq) > rlx.binding.STATIC_WORKSPACE_BYTES
+    w = rlx.upload_weights(inp.params, inp.layers)
+    out = torch.zeros((c.batch, c.hidden), dtype=torch.float32, device="cuda")
+    with pytest.raises(rlx.RlxError) as ei:
+        enc.forward_static(i32_dev(inp.ids), i32_dev(inp.mask), w, out)
+    assert ei.value.status == 3          # RLX_ERR_WORKSPACE, nothing launched
+    assert torch.count_nonzero(out) == 0
+    # a small batch with an out-of-range id: clamped, reported through device_status, then a clean call
+    ids = inp.ids[:2, :64].copy()
+    ids[0, 1] = c.vocab + 3
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out2 = torch.empty((2, c.hidden), dtype=torch.float32, device="cuda")
+    enc.forward_static(i32_dev(ids), i32_dev(inp.mask[:2, :64]), w, out2, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1
+    enc.forward_static(i32_dev(inp.ids[:2, :64]), i32_dev(inp.mask[:2, :64]), w, out2, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0       # the status word does not leak from the previous call
+    enc.close()
