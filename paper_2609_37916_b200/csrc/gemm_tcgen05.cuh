@@ -1,15 +1,18 @@
 // bf16 "Linear" GEMM for sm_100a: out[M,N] = epilogue(A[M,K] * W[N,K]^T + bias).
 //
-// Structure (one persistent CTA per SM, 192 threads):
+// Structure (one persistent CTA per SM, 320 threads):
 //   warp 0      TMA producer: streams 128x64 A tiles and BLOCK_N x 64 W tiles (128-byte swizzle)
 //               through a STAGES-deep shared-memory ring guarded by full/empty mbarriers
 //   warp 1      allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N=BLOCK_N,
 //               K=16 per instruction) into one of two fp32 accumulator buffers in TMEM and
 //               commits stage releases / accumulator-ready signals to mbarriers
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (one TMEM lane quadrant per warp, one output
-//               row per thread), add bias, apply GELU or add the residual in fp32, round to bf16
-//               and store; the second accumulator buffer lets tile i's epilogue overlap tile
-//               i+1's main loop
+//   warps 2..9  epilogue: each warp owns one TMEM lane quadrant (32 rows) and one half of the tile's
+//               columns; per 32-column chunk it tcgen05.ld's the accumulator (the next chunk's load
+//               is in flight while this one is processed), adds bias, applies GELU or adds the
+//               residual in fp32, rounds to bf16, writes the chunk to a swizzled shared-memory
+//               staging buffer and hands it to a TMA store (rows past M are clipped by the copy).
+//               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop;
+//               a warp releases its accumulator as soon as its last tcgen05.ld has landed.
 // Every mbarrier wait is bounded by a wall-clock budget; on expiry the CTA raises an abort flag,
 // records RLX_DEVSTAT_TIMEOUT, drains, frees its tensor memory and returns.
 #pragma once
@@ -23,8 +26,10 @@ namespace tc {
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int kThreads = 192;
-constexpr int kEpiWarps = 4;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8;
+constexpr int kStageBufBytes = 32 * 32 * 2;          // one 32-row x 32-column bf16 chunk
+constexpr int kStagingBytes = kEpiWarps * 2 * kStageBufBytes;  // two buffers per epilogue warp
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
 
 template <int BLOCK_N>
@@ -32,11 +37,12 @@ struct Cfg {
     static constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;
     static constexpr int B_BYTES = BLOCK_N * BLOCK_K * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (220 * 1024 / STAGE_BYTES) > 8 ? 8 : (220 * 1024 / STAGE_BYTES);
+    static constexpr int RING_BUDGET = 222 * 1024 - kStagingBytes;
+    static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
     static constexpr int TMEM_COLS = (2 * BLOCK_N <= 32) ? 32 : (2 * BLOCK_N <= 64) ? 64 : (2 * BLOCK_N <= 128) ? 128
                                      : (2 * BLOCK_N <= 256) ? 256 : 512;
     static constexpr int BAR_BYTES = 256;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // +1024: manual alignment
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + kStagingBytes + BAR_BYTES + 1024;  // +1024: manual alignment
     static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128");
     static_assert(B_BYTES % 1024 == 0, "stage tiles must stay 1024-byte aligned");
     static_assert(STAGES >= 2, "ring too shallow");
@@ -87,6 +93,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// TMA store of one staged chunk (shared -> global), tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tmap, int x, int y, uint32_t smem_src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
@@ -148,25 +167,27 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 struct Params {
     const float* bias;               // [N]
     const __nv_bfloat16* residual;   // [M,N] or null
-    __nv_bfloat16* out;              // [M,N]
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
 };
 
 template <int BLOCK_N, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_out, const Params p) {
     using C = Cfg<BLOCK_N>;
     extern __shared__ unsigned char smem_raw[];
     // manual 1024-byte alignment (required by the 128-byte swizzle atoms)
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - raw);
-    const uint32_t bars = base + C::STAGES * C::STAGE_BYTES;
+    const uint32_t staging = base + C::STAGES * C::STAGE_BYTES;
+    const uint32_t bars = staging + kStagingBytes;
     // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem slot, abort flag
     const uint32_t full_bar = bars, empty_bar = bars + 8 * C::STAGES;
     const uint32_t tfull_bar = bars + 16 * C::STAGES, tempty_bar = tfull_bar + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + 16 * C::STAGES + 32);
+    uint32_t* tmem_slot =
+        reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + kStagingBytes + 16 * C::STAGES + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -188,6 +209,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         fence_barrier_init();
         prefetch_tmap(&tmap_a);
         prefetch_tmap(&tmap_b);
+        prefetch_tmap(&tmap_out);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -248,8 +270,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+        constexpr int HALF_N = BLOCK_N / 2;
+        constexpr int NC = HALF_N / 32;       // 32-column chunks per warp and tile
+        const int ew = warp - 2;
+        const int quad = warp & 3;            // TMEM lane quadrant this warp may read
+        const int half = ew >> 2;             // which half of the tile's columns
+        const uint32_t stg = staging + ew * 2 * kStageBufBytes;
+        const uint32_t row_off = lane * 64;             // 64-byte rows in the staging chunk
+        const uint32_t swz = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte chunk index ^ (row/2 % 4)
         int it = 0;
+        uint32_t nstore = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
             const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
@@ -257,57 +287,73 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             const uint32_t aphase = (it >> 1) & 1;
             if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int m = m_blk * BLOCK_M + quad * 32 + lane;
+            const int m_row0 = m_blk * BLOCK_M + quad * 32;
+            const int m = m_row0 + lane;
             const bool row_ok = m < p.M;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N;
-            __nv_bfloat16* orow = p.out + (size_t)m * p.N + n_blk * BLOCK_N;
-            const __nv_bfloat16* rrow = p.residual + (size_t)m * p.N + n_blk * BLOCK_N;
-            const float* brow = p.bias + n_blk * BLOCK_N;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BLOCK_N; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32(taddr + c0, r);
+            const int n0 = n_blk * BLOCK_N + half * HALF_N;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N + half * HALF_N;
+            const __nv_bfloat16* rrow = p.residual + (size_t)m * p.N + n0;
+            const float* brow = p.bias + n0;
+            uint32_t r[2][32];
+            tmem_ld_32x32(taddr, r[0]);
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
                 tmem_ld_wait();
+                if (c + 1 < NC) {
+                    tmem_ld_32x32(taddr + (c + 1) * 32, r[(c + 1) & 1]);
+                } else {
+                    // every accumulator value this warp needs is in registers: release the buffer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar + 8 * as);
+                }
+                const uint32_t(&acc)[32] = r[c & 1];
                 float v[32];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c0) + i);
-                    v[4 * i + 0] = __uint_as_float(r[4 * i + 0]) + b4.x;
-                    v[4 * i + 1] = __uint_as_float(r[4 * i + 1]) + b4.y;
-                    v[4 * i + 2] = __uint_as_float(r[4 * i + 2]) + b4.z;
-                    v[4 * i + 3] = __uint_as_float(r[4 * i + 3]) + b4.w;
+                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c * 32) + i);
+                    v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4.x;
+                    v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b4.y;
+                    v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b4.z;
+                    v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b4.w;
                 }
                 if (EPI == 1) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
                 }
-                if (row_ok) {
-                    if (EPI == 2) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint4 q = __ldg(reinterpret_cast<const uint4*>(rrow + c0) + i);
-                            v[8 * i + 0] += bf16lo(q.x); v[8 * i + 1] += bf16hi(q.x);
-                            v[8 * i + 2] += bf16lo(q.y); v[8 * i + 3] += bf16hi(q.y);
-                            v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
-                            v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
-                        }
-                    }
+                if (EPI == 2 && row_ok) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        uint4 q;
-                        q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
-                        q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
-                        q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
-                        q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-                        *(reinterpret_cast<uint4*>(orow + c0) + i) = q;
+                        const uint4 q = __ldg(reinterpret_cast<const uint4*>(rrow + c * 32) + i);
+                        v[8 * i + 0] += bf16lo(q.x); v[8 * i + 1] += bf16hi(q.x);
+                        v[8 * i + 2] += bf16lo(q.y); v[8 * i + 3] += bf16hi(q.y);
+                        v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
+                        v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
                     }
                 }
+                // the staging buffer used two chunks ago must have been read out by its TMA store
+                const uint32_t buf = stg + (nstore & 1) * kStageBufBytes;
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 q;
+                    q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
+                    q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+                    q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+                    q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+                    st_shared_v4(buf + row_off + (((uint32_t)i ^ swz) << 4), q);
+                }
+                fence_proxy_async();   // make the generic-proxy writes visible to the TMA engine
+                __syncwarp();
+                if (lane == 0) {
+                    if (m_row0 < p.M) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
+                    bulk_commit();
+                }
+                ++nstore;
             }
-            // release this accumulator buffer to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar + 8 * as);
         }
+        if (lane == 0) bulk_wait<0>();   // all of this warp's stores have completed
     }
 
     // ---------------------------------------------------------------- teardown

@@ -53,16 +53,19 @@ encode_tiled_fn get_encode_fn() {
     return fn;
 }
 
-// bf16 row-major [rows, cols] matrix, box = box_rows x 64 columns, 128-byte swizzle, zero OOB fill.
-bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// bf16 row-major [rows, cols] matrix, box = box_rows x box_cols; operand tiles use 64 columns with the
+// 128-byte swizzle, output chunks 32 columns with the 64-byte swizzle; zero OOB fill on loads,
+// out-of-range rows dropped on stores.
+bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows,
+               uint32_t box_cols = rlx::tc::BLOCK_K, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     encode_tiled_fn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * sizeof(bf16)};
-    cuuint32_t box[2] = {(cuuint32_t)rlx::tc::BLOCK_K, box_rows};
+    cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -164,15 +167,15 @@ int pick_block_n(int M, int N) {
 }
 
 template <int BN>
-rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const rlx::tc::Params& p, int epi,
-                               cudaStream_t st) {
+rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                               const rlx::tc::Params& p, int epi, cudaStream_t st) {
     const int tiles = ((p.M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M) * (p.N / BN);
     const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
     const int smem = rlx::tc::Cfg<BN>::SMEM_BYTES;
     switch (epi) {
-        case 0: rlx::tc::gemm_tcgen05_kernel<BN, 0><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
-        case 1: rlx::tc::gemm_tcgen05_kernel<BN, 1><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
-        case 2: rlx::tc::gemm_tcgen05_kernel<BN, 2><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, p); break;
+        case 0: rlx::tc::gemm_tcgen05_kernel<BN, 0><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
+        case 1: rlx::tc::gemm_tcgen05_kernel<BN, 1><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
+        case 2: rlx::tc::gemm_tcgen05_kernel<BN, 2><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
@@ -194,15 +197,16 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     }
     const int bn = pick_block_n(M, N);
     if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
-    CUtensorMap ta, tb;
+    CUtensorMap ta, tb, to;
     if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)bn)) return RLX_ERR_CUDA;
-    rlx::tc::Params p{bias, residual, out, M, N, K, status};
+    if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
+    rlx::tc::Params p{bias, residual, M, N, K, status};
     switch (bn) {
-        case 64: return launch_gemm_tc_bn<64>(ta, tb, p, epi, st);
-        case 128: return launch_gemm_tc_bn<128>(ta, tb, p, epi, st);
-        case 192: return launch_gemm_tc_bn<192>(ta, tb, p, epi, st);
-        case 256: return launch_gemm_tc_bn<256>(ta, tb, p, epi, st);
+        case 64: return launch_gemm_tc_bn<64>(ta, tb, to, p, epi, st);
+        case 128: return launch_gemm_tc_bn<128>(ta, tb, to, p, epi, st);
+        case 192: return launch_gemm_tc_bn<192>(ta, tb, to, p, epi, st);
+        case 256: return launch_gemm_tc_bn<256>(ta, tb, to, p, epi, st);
     }
     return RLX_ERR_UNSUPPORTED;
 }
