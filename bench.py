@@ -167,17 +167,23 @@ def workload_config(name: str, extra=None):
 
 # ---------------------------------------------------------------------------- roofline bookkeeping
 def kernel_classes(num_layers: int):
-    names = ["embed_ln"]
+    names = ["pack", "embed_ln"]
     for _ in range(num_layers):
         names += list(KERNEL_CLASSES)
     names.append("pool_l2")
     return names
 
 
-def algorithmic_work(cls: str, c, n_valid_tokens: int):
-    """(bound, work per launch, unit): algorithmic flops for the contractions (dense, all B*S rows:
-    the kernels compute padded rows too), algorithmic bytes for the streaming kernels."""
-    T, H, F, S, B = c.batch * c.seq, c.hidden, c.ffn, c.seq, c.batch
+def algorithmic_work(cls: str, c, lengths):
+    """(bound, work per launch, unit).  Valid tokens are packed, so only they are computed and only
+    they are counted: T = sum of valid lengths rows for the GEMMs and row kernels, sum of len^2
+    query-key pairs for attention.  Skipped (padded) work is never counted."""
+    H, F, S, B = c.hidden, c.ffn, c.seq, c.batch
+    T = int(np.sum(lengths))
+    n_valid_tokens = T
+    pairs = float(np.sum(np.asarray(lengths, dtype=np.float64) ** 2))
+    if cls == "pack":
+        return "hbm", B * S * 4.0 + T * 4.0 + B * 8.0, "byte"   # read the mask, write positions and offsets
     if cls == "gemm_qkv":
         return "tensor", 2.0 * T * 3 * H * H, "flop"
     if cls == "gemm_out":
@@ -185,13 +191,13 @@ def algorithmic_work(cls: str, c, n_valid_tokens: int):
     if cls in ("gemm_ffn1", "gemm_ffn2"):
         return "tensor", 2.0 * T * F * H, "flop"
     if cls == "attention":
-        return "tensor", 4.0 * B * S * S * H, "flop"          # QK^T and PV, dense S x S per head
+        return "tensor", 4.0 * pairs * H, "flop"              # QK^T and PV over len x len per head
     if cls in ("ln1", "ln2"):
         return "hbm", 2.0 * T * H * 2, "byte"                 # read + write one bf16 row per token
     if cls == "embed_ln":
         return "hbm", T * (2.0 * H * 2 + 4), "byte"           # word-row gather + output row + id
     if cls == "pool_l2":
-        return "hbm", n_valid_tokens * H * 2.0 + T * 4 + B * H * 4, "byte"
+        return "hbm", n_valid_tokens * H * 2.0 + B * 8 + B * H * 4, "byte"
     raise KeyError(cls)
 
 
@@ -319,7 +325,7 @@ def run_ours(args):
         for cls, vals in per_class.items():
             launches_per_step = names.count(cls)
             avg_ms = sum(vals) / len(vals)
-            bound, work, unit = algorithmic_work(cls, cfg, n_valid)
+            bound, work, unit = algorithmic_work(cls, cfg, mine.lengths)
             if bound == "tensor":
                 ach = work / (avg_ms * 1e-3) / 1e12
                 peak = peaks["bf16_tflops"]

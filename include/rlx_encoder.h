@@ -60,6 +60,7 @@ typedef enum {
 #define RLX_FLAG_NO_GRAPH 0x1u  /* launch kernels one by one instead of replaying a CUDA graph */
 #define RLX_FLAG_GEMM_SIMT 0x2u /* use the plain CUDA-core GEMM (bring-up / cross-check only)  */
 #define RLX_FLAG_KERNEL_EVENTS 0x4u /* record a CUDA event between kernels (see rlx_encoder_kernel_times) */
+#define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */
@@ -141,7 +142,8 @@ size_t rlx_encoder_workspace_bytes(const rlx_encoder_t *encoder, int32_t batch, 
  * weights         host struct of dev pointers (see above); read during the call only
  * out             dev f32 [batch, H]; a sequence with no valid position yields zeros
  * workspace       dev, 256-byte aligned, >= rlx_encoder_workspace_bytes(batch, seq);
- *                 scratch: contents are overwritten by every call
+ *                 scratch: contents are overwritten by every call.  Its first 256 bytes hold the
+ *                 sticky device status word: zero them once before the first call
  *
  * Asynchronous on cuda_stream.  Unless RLX_FLAG_NO_GRAPH is set the kernel
  * sequence is captured once per distinct (batch, seq, pointer set) into a CUDA
@@ -213,8 +215,8 @@ int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t *encoder);
  * RLX_FLAG_KERNEL_EVENTS (the paper's runtime exposes per-operator reports, Section 4; this is
  * the timing analogue).  Waits for that forward to finish, then writes `count` =
  * rlx_encoder_kernels_per_forward() durations in milliseconds to ms_host (host memory), in
- * launch order: embed+LN, then per layer [QKV GEMM, attention, out-proj GEMM, LN, FFN-up GEMM,
- * FFN-down GEMM, LN], then pool.  In graph mode the events are nodes of the captured graph, so
+ * launch order: [sequence packing,] embed+LN, then per layer [QKV GEMM, attention, out-proj GEMM,
+ * LN, FFN-up GEMM, FFN-down GEMM, LN], then pool.  In graph mode the events are nodes of the captured graph, so
  * the figures contain no host launch gaps.  RLX_ERR_UNSUPPORTED if the flag was not set.
  */
 rlx_status_t rlx_encoder_kernel_times(rlx_encoder_t *encoder, float *ms_host, int32_t count);
@@ -228,6 +230,19 @@ const char *rlx_status_string(rlx_status_t status);
  * checked against the oracle in isolation.  All pointers dev; `status` is an
  * optional dev int32 that receives RLX_DEVSTAT_* bits (may be NULL).
  * ------------------------------------------------------------------------- */
+
+/*
+ * Sequence packing (the forward's first kernel unless RLX_FLAG_NO_PACK): compacts the valid
+ * positions of every sequence so that all later kernels touch sum(valid) rows instead of
+ * batch*seq.  Exact for any 0/1 mask (Section 3.1's custom mask kind): positions keep their
+ * original index, attention and pooling only ever involve valid tokens.  Integer outputs, all dev:
+ *   seq_len[b]             number of valid positions of sequence b
+ *   seq_start[0..batch]    exclusive prefix sum of seq_len (seq_start[batch] = packed row count)
+ *   pos_of_rank[b*seq + r] original position of the r-th valid token of sequence b (r < seq_len[b])
+ *   ticket                 one uint32 that must be zero before the first call; the kernel leaves it zero
+ */
+rlx_status_t rlx_pack_sequences(const int32_t *attention_mask, int32_t batch, int32_t seq, int32_t *seq_len,
+                                int32_t *seq_start, int32_t *pos_of_rank, uint32_t *ticket, void *cuda_stream);
 
 /* x[t] = LN(word[ids[t]] + pos[t % seq] + type[0]) -> bf16 [tokens, H]. */
 rlx_status_t rlx_embed_layernorm(const int32_t *token_ids, const void *word_emb, const void *pos_emb,

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     embed_layernorm,
     gemm_bf16,
     layernorm,
+    pack_sequences,
     lib_path,
     pool_l2norm,
     upload_weights,

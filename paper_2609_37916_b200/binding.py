@@ -22,6 +22,7 @@ STATUS_NAMES = {0: "RLX_OK", 1: "RLX_ERR_INVALID_ARG", 2: "RLX_ERR_UNSUPPORTED",
 FLAG_NO_GRAPH = 0x1
 FLAG_GEMM_SIMT = 0x2
 FLAG_KERNEL_EVENTS = 0x4
+FLAG_NO_PACK = 0x8
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20
@@ -29,7 +30,7 @@ STATIC_WORKSPACE_BYTES = 16 << 20
 EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
-    "rlx_status_string", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
+    "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
     "rlx_attention_f32", "rlx_pool_l2norm",
 )
 
@@ -226,6 +227,18 @@ def embed_layernorm(ids, word, pos, type_, gamma, beta, seq: int, vocab: int, ep
                                        H, vocab, C.c_float(eps), _ptr(out), _ptr(status), _stream(stream)),
            "rlx_embed_layernorm")
     return out
+
+
+def pack_sequences(mask: torch.Tensor, stream=None):
+    """rlx_pack_sequences -> (seq_len [B], seq_start [B+1], pos_of_rank [B,S]) int32 device tensors."""
+    B, S = mask.shape
+    seq_len = torch.empty(B, dtype=torch.int32, device=mask.device)
+    seq_start = torch.empty(B + 1, dtype=torch.int32, device=mask.device)
+    pos_of_rank = torch.full((B, S), -1, dtype=torch.int32, device=mask.device)
+    ticket = torch.zeros(1, dtype=torch.int32, device=mask.device)
+    _check(_load().rlx_pack_sequences(_ptr(mask), B, S, _ptr(seq_len), _ptr(seq_start), _ptr(pos_of_rank),
+                                      _ptr(ticket), _stream(stream)), "rlx_pack_sequences")
+    return seq_len, seq_start, pos_of_rank, ticket
 
 
 def layernorm(x, gamma, beta, eps: float, stream=None):

@@ -1,11 +1,12 @@
 // Key-padding-masked scaled-dot-product attention with online softmax, reading q/k/v as strided
 // views of the packed [T, 3H] projection (no split / transpose copies).
 //
-//  attention_bf16_kernel: bf16 in/out.  One CTA = 64 query rows of one (sequence, head); 4 warps of
-//    16 rows each.  K/V stream through shared memory in 64-key blocks (cp.async double buffer),
-//    QK^T and PV run on the warp-level tensor-core path (mma.sync m16n8k16, fp32 accumulate), the
-//    softmax state (running max / sum) lives in registers and is reduced with quad shuffles.
-//    Key blocks beyond the last valid key are never loaded; masked keys get a -inf bias.
+//  attention_bf16_kernel: bf16 in/out.  One CTA = 128 query rows of one (sequence, head); 8 warps of
+//    16 rows each.  K/V stream through shared memory in 64-key blocks (cp.async, 4-stage ring, three
+//    blocks in flight), QK^T and PV run on the warp-level tensor-core path (mma.sync m16n8k16, fp32
+//    accumulate), the softmax state (running max / sum) lives in registers and is reduced with quad
+//    shuffles; the 1/sqrt(d)*log2(e) scale is folded into the exp2 argument.  Key blocks beyond the
+//    last valid key are never loaded; masking runs only in blocks that contain an invalid key.
 //  attention_f32_kernel: fp32 in/out CUDA-core kernel, one warp per query row, K/V staged in shared
 //    memory 32 keys at a time, warp-shuffle reductions.  Reference-precision mode for testing.
 #pragma once
@@ -41,24 +42,31 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-constexpr int kAttBlockM = 64;   // query rows per CTA
-constexpr int kAttBlockN = 64;   // keys per shared-memory block
-constexpr int kAttThreads = 128;
+constexpr int kAttBlockM = 128;  // query rows per CTA (8 warps x 16 rows)
+constexpr int kAttBlockN = 64;   // keys per shared-memory stage
+constexpr int kAttStages = 4;    // K/V ring depth (three blocks in flight ahead of the one being used)
+constexpr int kAttThreads = 256;
+constexpr int kAttMaxSeq = 512;
 
 template <int D>
 struct AttSmem {
     static constexpr int kStride = D + 8;  // +16 bytes per row: conflict-free ldmatrix
-    __nv_bfloat16 q[kAttBlockM * kStride];
-    __nv_bfloat16 k[2][kAttBlockN * kStride];
-    __nv_bfloat16 v[2][kAttBlockN * kStride];
-    float bias[512 + 64];  // 0 for a valid key, -inf for a masked one (seq <= 512 supported here)
+    __nv_bfloat16 q[kAttBlockM * kStride];  // Q tile; reused as the output staging tile at the end
+    __nv_bfloat16 k[kAttStages][kAttBlockN * kStride];
+    __nv_bfloat16 v[kAttStages][kAttBlockN * kStride];
+    float bias[kAttMaxSeq];                 // padded mode: 0 for a valid key, -inf for a masked one
+    int blk_full[kAttMaxSeq / kAttBlockN];  // padded mode: 1 when all 64 keys of the block are valid
     int kv_end;
     int q_any;
 };
 
+// Two addressing modes share the kernel:
+//   padded: seq_start == nullptr.  Sequence b occupies rows b*S .. b*S+S; `mask` flags valid keys.
+//   packed: rows of sequence b are seq_start[b] .. seq_start[b]+seq_len[b], all valid (mask unused).
 template <int D>
-__global__ void __launch_bounds__(kAttThreads)
+__global__ void __launch_bounds__(kAttThreads, D == 32 ? 3 : 2)
 attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ mask,
+                      const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
                       __nv_bfloat16* __restrict__ ctx, int S, int H, float scale_log2e) {
     using SM = AttSmem<D>;
     constexpr int STR = SM::kStride;
@@ -70,70 +78,85 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q0 = blockIdx.x * kAttBlockM, head = blockIdx.y, b = blockIdx.z;
-    const size_t row0 = (size_t)b * S;
+    const bool packed = seq_start != nullptr;
+    const size_t row0 = packed ? (size_t)__ldg(seq_start + b) : (size_t)b * S;
+    const int len = packed ? __ldg(seq_len + b) : S;   // rows of this sequence present in memory
+    if (q0 >= len) return;                              // whole CTA outside the sequence (uniform)
     const int ld = 3 * H;
     const __nv_bfloat16* qbase = qkv + row0 * ld + head * D;
     const __nv_bfloat16* kbase = qbase + H;
     const __nv_bfloat16* vbase = qbase + 2 * H;
 
-    if (tid == 0) { sm.kv_end = 0; sm.q_any = 0; }
-    __syncthreads();
-    {
+    int kv_end = len;
+    if (!packed) {
+        if (tid == 0) { sm.kv_end = 0; sm.q_any = 0; }
+        if (tid < kAttMaxSeq / kAttBlockN) sm.blk_full[tid] = 1;
+        __syncthreads();
         int last = 0, any = 0;
-        const int spad = (S + 63) & ~63;
+        const int spad = (S + kAttBlockN - 1) / kAttBlockN * kAttBlockN;
         for (int k = tid; k < spad; k += kAttThreads) {
             const bool valid = (k < S) && (__ldg(mask + row0 + k) != 0);
             sm.bias[k] = valid ? 0.f : -INFINITY;
             if (valid) {
                 last = k + 1;
                 any |= (k >= q0 && k < q0 + kAttBlockM);
+            } else {
+                sm.blk_full[k / kAttBlockN] = 0;   // benign race: every writer stores 0
             }
         }
         if (last) atomicMax(&sm.kv_end, last);
         if (any) atomicOr(&sm.q_any, 1);
-    }
-    __syncthreads();
-    const int kv_end = sm.kv_end;
-    if (kv_end == 0 || sm.q_any == 0) {
-        // nothing observable in this block: write zeros so later stages only ever see finite values
-        for (int i = tid; i < kAttBlockM * CH; i += kAttThreads) {
-            const int r = i / CH, c = i % CH;
-            if (q0 + r < S)
-                *reinterpret_cast<uint4*>(ctx + (row0 + q0 + r) * H + head * D + c * 8) = make_uint4(0, 0, 0, 0);
+        __syncthreads();
+        kv_end = sm.kv_end;
+        if (kv_end == 0 || sm.q_any == 0) {
+            // nothing observable in this block: write zeros so later stages only ever see finite values
+            for (int i = tid; i < kAttBlockM * CH; i += kAttThreads) {
+                const int r = i / CH, c = i % CH;
+                if (q0 + r < S)
+                    *reinterpret_cast<uint4*>(ctx + (row0 + q0 + r) * H + head * D + c * 8) = make_uint4(0, 0, 0, 0);
+            }
+            return;
         }
-        return;
     }
     const int nblk = (kv_end + kAttBlockN - 1) / kAttBlockN;
 
-    auto load_rows = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row) {
-        for (int i = tid; i < 64 * CH; i += kAttThreads) {
+    auto load_rows = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row, int nrows) {
+        for (int i = tid; i < nrows * CH; i += kAttThreads) {
             const int r = i / CH, c = i % CH;
-            const bool ok = first_row + r < S;
+            const bool ok = first_row + r < len;
             const __nv_bfloat16* src = base + (size_t)(ok ? first_row + r : 0) * ld + c * 8;
             cp_async16(smem_u32(dst + r * STR + c * 8), src, ok);
         }
     };
-    load_rows(qbase, sm.q, q0);
-    load_rows(kbase, sm.k[0], 0);
-    load_rows(vbase, sm.v[0], 0);
-    cp_async_commit();
+    load_rows(qbase, sm.q, q0, kAttBlockM);
+#pragma unroll
+    for (int j = 0; j < kAttStages - 1; ++j) {
+        if (j < nblk) {
+            load_rows(kbase, sm.k[j], j * kAttBlockN, kAttBlockN);
+            load_rows(vbase, sm.v[j], j * kAttBlockN, kAttBlockN);
+        }
+        cp_async_commit();
+    }
 
     uint32_t qf[KT][4];
     float o[ND][4];
 #pragma unroll
     for (int i = 0; i < ND; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // running max (scaled) and sum
     const int g = lane >> 2, t4 = lane & 3;
+    const bool warp_active = q0 + warp * 16 < len;   // warps whose 16 rows lie past the sequence only sync
 
     for (int j = 0; j < nblk; ++j) {
-        const int buf = j & 1;
-        if (j + 1 < nblk) {
-            load_rows(kbase, sm.k[buf ^ 1], (j + 1) * kAttBlockN);
-            load_rows(vbase, sm.v[buf ^ 1], (j + 1) * kAttBlockN);
+        const int buf = j % kAttStages;
+        cp_async_wait<kAttStages - 2>();   // block j (and Q) have landed
+        __syncthreads();                   // ... for every thread; and block j-1's stage is free
+        if (j + kAttStages - 1 < nblk) {
+            const int nb = (j + kAttStages - 1) % kAttStages;
+            load_rows(kbase, sm.k[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
+            load_rows(vbase, sm.v[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
         }
         cp_async_commit();
-        cp_async_wait<1>();
-        __syncthreads();
+        if (!warp_active) continue;
         if (j == 0) {
 #pragma unroll
             for (int kt = 0; kt < KT; ++kt) {
@@ -158,16 +181,23 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 mma_bf16_16816(s[nt], qf[2 * kp + 1][0], qf[2 * kp + 1][1], qf[2 * kp + 1][2], qf[2 * kp + 1][3], b2, b3);
             }
         }
-        // ---- scale, mask bias, running max ----
-        const float* bias = sm.bias + j * kAttBlockN;
+        // ---- masking only where the block has an invalid key ----
+        const int k0 = j * kAttBlockN;
+        const bool need_mask = packed ? (k0 + kAttBlockN > len) : (sm.blk_full[j] == 0);
+        if (need_mask) {
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                const int kk = k0 + nt * 8 + 2 * t4;
+                const bool v0 = packed ? (kk < len) : (sm.bias[kk] == 0.f);
+                const bool v1 = packed ? (kk + 1 < len) : (sm.bias[kk + 1] == 0.f);
+                if (!v0) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
+                if (!v1) { s[nt][1] = -INFINITY; s[nt][3] = -INFINITY; }
+            }
+        }
+        // ---- running max on raw scores (the positive scale commutes with max) ----
         float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
-            const float b0 = bias[nt * 8 + 2 * t4], b1 = bias[nt * 8 + 2 * t4 + 1];
-            s[nt][0] = s[nt][0] * scale_log2e + b0;
-            s[nt][1] = s[nt][1] * scale_log2e + b1;
-            s[nt][2] = s[nt][2] * scale_log2e + b0;
-            s[nt][3] = s[nt][3] * scale_log2e + b1;
             mx[0] = fmaxf(mx[0], fmaxf(s[nt][0], s[nt][1]));
             mx[1] = fmaxf(mx[1], fmaxf(s[nt][2], s[nt][3]));
         }
@@ -176,7 +206,7 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         for (int r = 0; r < 2; ++r) {
             mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
             mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-            const float m_new = fmaxf(m_run[r], mx[r]);
+            const float m_new = fmaxf(m_run[r], mx[r] * scale_log2e);
             msub[r] = (m_new == -INFINITY) ? 0.f : m_new;   // all keys so far masked: avoid inf - inf
             alpha[r] = fast_exp2(m_run[r] - msub[r]);        // m_run = -inf -> 0
             m_run[r] = m_new;
@@ -187,14 +217,14 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             o[nd][0] *= alpha[0]; o[nd][1] *= alpha[0];
             o[nd][2] *= alpha[1]; o[nd][3] *= alpha[1];
         }
-        // ---- P = exp2(S - m), row sums, pack to bf16 A fragments ----
+        // ---- P = exp2(S*c - m), row sums, pack to bf16 A fragments ----
         uint32_t pf[4][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
-            const float p0 = fast_exp2(s[nt][0] - msub[0]);
-            const float p1 = fast_exp2(s[nt][1] - msub[0]);
-            const float p2 = fast_exp2(s[nt][2] - msub[1]);
-            const float p3 = fast_exp2(s[nt][3] - msub[1]);
+            const float p0 = fast_exp2(fmaf(s[nt][0], scale_log2e, -msub[0]));
+            const float p1 = fast_exp2(fmaf(s[nt][1], scale_log2e, -msub[0]));
+            const float p2 = fast_exp2(fmaf(s[nt][2], scale_log2e, -msub[1]));
+            const float p3 = fast_exp2(fmaf(s[nt][3], scale_log2e, -msub[1]));
             l_run[0] += p0 + p1;
             l_run[1] += p2 + p3;
             pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
@@ -214,25 +244,30 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 mma_bf16_16816(o[2 * np + 1], pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], b2, b3);
             }
         }
-        __syncthreads();  // everyone is done with this buffer before the next prefetch overwrites it
     }
     cp_async_wait<0>();
+    if (!warp_active) return;
 
-    // ---- normalise and store ----
+    // ---- normalise, stage this warp's 16 x D tile in its own rows of the Q buffer, store 16 B / lane ----
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
         l_run[r] = l_run[r] > 0.f ? 1.0f / l_run[r] : 0.f;
     }
-    const int qr0 = q0 + warp * 16 + g, qr1 = qr0 + 8;
+    __nv_bfloat16* stage = sm.q + warp * 16 * STR;   // only this warp ever touched these rows
 #pragma unroll
     for (int nd = 0; nd < ND; ++nd) {
-        const int col = head * D + nd * 8 + 2 * t4;
-        if (qr0 < S)
-            *reinterpret_cast<uint32_t*>(ctx + (row0 + qr0) * H + col) = pack_bf16(o[nd][0] * l_run[0], o[nd][1] * l_run[0]);
-        if (qr1 < S)
-            *reinterpret_cast<uint32_t*>(ctx + (row0 + qr1) * H + col) = pack_bf16(o[nd][2] * l_run[1], o[nd][3] * l_run[1]);
+        *reinterpret_cast<uint32_t*>(stage + g * STR + nd * 8 + 2 * t4) = pack_bf16(o[nd][0] * l_run[0], o[nd][1] * l_run[0]);
+        *reinterpret_cast<uint32_t*>(stage + (g + 8) * STR + nd * 8 + 2 * t4) = pack_bf16(o[nd][2] * l_run[1], o[nd][3] * l_run[1]);
+    }
+    __syncwarp();
+    for (int i = lane; i < 16 * CH; i += 32) {
+        const int r = i / CH, c = i % CH;
+        const int qr = q0 + warp * 16 + r;
+        if (qr < len)
+            *reinterpret_cast<uint4*>(ctx + (row0 + qr) * H + head * D + c * 8) =
+                *reinterpret_cast<const uint4*>(stage + r * STR + c * 8);
     }
 }
 

@@ -169,6 +169,7 @@ struct Params {
     const __nv_bfloat16* residual;   // [M,N] or null
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
+    const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
 };
 
 template <int BLOCK_N, int EPI>
@@ -191,8 +192,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int M = p.M;
+    if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));   // packed activations: only sum(len) rows exist
     const int n_tiles = p.N / BLOCK_N;
-    const int m_tiles = (p.M + BLOCK_M - 1) / BLOCK_M;
+    const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
     const int num_tiles = n_tiles * m_tiles;
     const int num_kb = (p.K + BLOCK_K - 1) / BLOCK_K;
 
@@ -289,7 +292,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             tc_fence_after();
             const int m_row0 = m_blk * BLOCK_M + quad * 32;
             const int m = m_row0 + lane;
-            const bool row_ok = m < p.M;
+            const bool row_ok = m < M;
             const int n0 = n_blk * BLOCK_N + half * HALF_N;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N + half * HALF_N;
             const __nv_bfloat16* rrow = p.residual + (size_t)m * p.N + n0;
@@ -347,7 +350,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 fence_proxy_async();   // make the generic-proxy writes visible to the TMA engine
                 __syncwarp();
                 if (lane == 0) {
-                    if (m_row0 < p.M) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
+                    if (m_row0 < M) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
                     bulk_commit();
                 }
                 ++nstore;

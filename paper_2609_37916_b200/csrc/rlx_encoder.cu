@@ -105,12 +105,27 @@ cudaError_t init_kernels_for_current_device() {
 }
 
 // ------------------------------------------------------------------ launchers
+struct Packing {   // device arrays written by pack_sequences_kernel; all null in padded mode
+    const int32_t* seq_len = nullptr;
+    const int32_t* seq_start = nullptr;    // [B+1]; seq_start[B] = number of packed rows
+    const int32_t* pos_of_rank = nullptr;
+    int B = 0;
+    const int32_t* total() const { return seq_start ? seq_start + B : nullptr; }
+};
+
+rlx_status_t launch_pack(const int32_t* mask, int B, int S, int32_t* seq_len, int32_t* seq_start,
+                         int32_t* pos_of_rank, unsigned int* ticket, cudaStream_t st) {
+    rlx::pack_sequences_kernel<<<B, rlx::kPackThreads, 0, st>>>(mask, B, S, seq_len, seq_start, pos_of_rank, ticket);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
 rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* pos, const bf16* type,
                              const float* g, const float* b, int T, int S, int H, int V, float eps, bf16* out,
-                             int32_t* status, cudaStream_t st) {
+                             int32_t* status, cudaStream_t st, const Packing& pk = Packing()) {
     const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: rlx::embed_ln_kernel<NV><<<grid, thr, 0, st>>>(ids, word, pos, type, g, b, out, T, S, V, eps, status); break;
+#define RLX_CASE(NV) case NV: rlx::embed_ln_kernel<NV><<<grid, thr, 0, st>>>(ids, word, pos, type, g, b, out, T, S, V, eps, status, pk.seq_start, pk.pos_of_rank, pk.B); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE
         default: return RLX_ERR_UNSUPPORTED;
@@ -120,10 +135,10 @@ rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* p
 }
 
 rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int T, int H, float eps, bf16* out,
-                              cudaStream_t st) {
+                              cudaStream_t st, const int32_t* rows_ptr = nullptr) {
     const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: rlx::layernorm_kernel<NV><<<grid, thr, 0, st>>>(x, g, b, out, T, eps); break;
+#define RLX_CASE(NV) case NV: rlx::layernorm_kernel<NV><<<grid, thr, 0, st>>>(x, g, b, out, T, eps, rows_ptr); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE
         default: return RLX_ERR_UNSUPPORTED;
@@ -132,23 +147,24 @@ rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int
     return RLX_OK;
 }
 
-rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H, float* out, cudaStream_t st) {
+rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H, float* out, cudaStream_t st,
+                         const Packing& pk = Packing()) {
     const int vecs = H / 8, G = rlx::kPoolThreads / vecs;
     const size_t smem = (size_t)G * H * sizeof(float);
-    rlx::pool_l2norm_kernel<<<B, rlx::kPoolThreads, smem, st>>>(x, mask, out, S, H);
+    rlx::pool_l2norm_kernel<<<B, rlx::kPoolThreads, smem, st>>>(x, mask, out, S, H, pk.seq_start, pk.seq_len);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
 
-rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, int B, int S, int h, int d, bf16* ctx,
-                                   cudaStream_t st) {
+rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const int32_t* seq_start,
+                                   const int32_t* seq_len, int B, int S, int h, int d, bf16* ctx, cudaStream_t st) {
     const int H = h * d;
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
     dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
     if (d == 32)
-        rlx::attention_bf16_kernel<32><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st>>>(qkv, mask, ctx, S, H, scale_log2e);
+        rlx::attention_bf16_kernel<32><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st>>>(qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e);
     else if (d == 64)
-        rlx::attention_bf16_kernel<64><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st>>>(qkv, mask, ctx, S, H, scale_log2e);
+        rlx::attention_bf16_kernel<64><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st>>>(qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e);
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
@@ -183,7 +199,8 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
 }
 
 rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const bf16* residual, int epi, int M, int N,
-                         int K, bf16* out, bool simt, int32_t* status, cudaStream_t st) {
+                         int K, bf16* out, bool simt, int32_t* status, cudaStream_t st,
+                         const int32_t* m_ptr = nullptr) {
     if (simt) {
         dim3 grid((N + rlx::kSimtTile - 1) / rlx::kSimtTile, (M + rlx::kSimtTile - 1) / rlx::kSimtTile);
         switch (epi) {
@@ -201,7 +218,7 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)bn)) return RLX_ERR_CUDA;
     if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
-    rlx::tc::Params p{bias, residual, M, N, K, status};
+    rlx::tc::Params p{bias, residual, M, N, K, status, m_ptr};
     switch (bn) {
         case 64: return launch_gemm_tc_bn<64>(ta, tb, to, p, epi, st);
         case 128: return launch_gemm_tc_bn<128>(ta, tb, to, p, epi, st);
@@ -213,8 +230,9 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
 
 // ------------------------------------------------------------------ workspace arena
 struct Arena {
-    size_t status, ids, mask, out, x, qkv, ctx, y, x1, g, total;
+    size_t status, ids, mask, out, seq_len, seq_start, pos_of_rank, x, qkv, ctx, y, x1, g, total;
 };
+constexpr size_t kTicketOffset = 64;   // packing ticket counter inside the 256-byte status block
 
 Arena plan_arena(int B, int S, int H, int F) {
     const size_t T = (size_t)B * S;
@@ -229,6 +247,9 @@ Arena plan_arena(int B, int S, int H, int F) {
     a.ids = take(T * 4);
     a.mask = take(T * 4);
     a.out = take((size_t)B * H * 4);
+    a.seq_len = take((size_t)B * 4);
+    a.seq_start = take((size_t)(B + 1) * 4);
+    a.pos_of_rank = take(T * 4);
     a.x = take(T * H * 2);
     a.qkv = take(T * 3 * H * 2);
     a.ctx = take(T * H * 2);
@@ -281,6 +302,9 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     const rlx_encoder_config_t& c = e->cfg;
     const int H = c.hidden, F = c.ffn, T = B * S, h = c.num_heads, d = e->head_dim;
     const bool simt = (c.flags & RLX_FLAG_GEMM_SIMT) != 0;
+    // valid tokens are packed unless the caller asked for the padded layout (the bring-up GEMM has
+    // no dynamic row count, so it implies the padded layout too)
+    const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !simt;
     const Arena a = plan_arena(B, S, H, F);
     int32_t* status = reinterpret_cast<int32_t*>(ws + a.status);
     bf16* x = reinterpret_cast<bf16*>(ws + a.x);
@@ -303,19 +327,31 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
 #define RLX_TRY(call) do { s = (call); if (s != RLX_OK) return s; s = mark(); if (s != RLX_OK) return s; } while (0)
     s = mark();
     if (s != RLX_OK) return s;
+    Packing pk;
+    if (pack) {
+        int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
+        int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
+        int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
+        // the ticket must be zero when the packing kernel starts, whatever the workspace held before
+        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, sizeof(unsigned int), st));
+        RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
+                            reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
+        pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
+    }
+    const int32_t* rows = pk.total();
     RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
-                            w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st));
+                            w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
     for (int l = 0; l < c.num_layers; ++l) {
         const rlx_layer_weights_t& lw = w->layers[l];
-        RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, simt, status, st));
-        RLX_TRY(launch_attention_bf16(qkv, mask, B, S, h, d, ctx, st));
-        RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st));
-        RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st));
-        RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st));
-        RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st));
-        RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st));
+        RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, simt, status, st, rows));
+        RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
+        RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
+        RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
+        RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
+        RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st, rows));
+        RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
     }
-    RLX_TRY(launch_pool(x, mask, B, S, H, out, st));
+    RLX_TRY(launch_pool(x, mask, B, S, H, out, st, pk));
 #undef RLX_TRY
     return RLX_OK;
 }
@@ -345,7 +381,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
     RLX_CUDA_TRY(init_kernels_for_current_device());
     if ((e->cfg.flags & RLX_FLAG_KERNEL_EVENTS) && e->events.empty()) {
-        e->events.resize(3 + 7 * (size_t)e->cfg.num_layers);
+        e->events.resize((size_t)rlx_encoder_kernels_per_forward(e) + 1);
         for (auto& evt : e->events) RLX_CUDA_TRY(cudaEventCreate(&evt));
     }
     if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);
@@ -424,7 +460,11 @@ size_t rlx_encoder_workspace_bytes(const rlx_encoder_t* e, int32_t batch, int32_
     return plan_arena(batch, seq, e->cfg.hidden, e->cfg.ffn).total;
 }
 
-int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e) { return e ? 2 + 7 * e->cfg.num_layers : 0; }
+int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e) {
+    if (!e) return 0;
+    const bool pack = !(e->cfg.flags & RLX_FLAG_NO_PACK) && !(e->cfg.flags & RLX_FLAG_GEMM_SIMT);
+    return 2 + 7 * e->cfg.num_layers + (pack ? 1 : 0);
+}
 
 rlx_status_t rlx_encoder_forward(rlx_encoder_t* e, const int32_t* ids, const int32_t* mask, int32_t B, int32_t S,
                                  const rlx_encoder_weights_t* w, float* out, void* ws, size_t ws_bytes, void* stream) {
@@ -555,6 +595,12 @@ rlx_status_t rlx_embed_layernorm(const int32_t* ids, const void* word, const voi
                            (bf16*)out, status, static_cast<cudaStream_t>(stream));
 }
 
+rlx_status_t rlx_pack_sequences(const int32_t* mask, int32_t B, int32_t S, int32_t* seq_len, int32_t* seq_start,
+                                int32_t* pos_of_rank, uint32_t* ticket, void* stream) {
+    if (!mask || !seq_len || !seq_start || !pos_of_rank || !ticket || B <= 0 || S <= 0) return RLX_ERR_INVALID_ARG;
+    return launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank, ticket, static_cast<cudaStream_t>(stream));
+}
+
 rlx_status_t rlx_layernorm(const void* x, const float* gamma, const float* beta, int32_t rows, int32_t H, float eps,
                            void* out, void* stream) {
     if (!x || !gamma || !beta || !out || rows <= 0) return RLX_ERR_INVALID_ARG;
@@ -583,7 +629,8 @@ rlx_status_t rlx_attention_bf16(const void* qkv, const int32_t* mask, int32_t B,
     if (!aligned16(qkv) || !aligned16(ctx)) return RLX_ERR_INVALID_ARG;
     if ((d != 32 && d != 64) || S > 512 || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
-    return launch_attention_bf16((const bf16*)qkv, mask, B, S, h, d, (bf16*)ctx, static_cast<cudaStream_t>(stream));
+    return launch_attention_bf16((const bf16*)qkv, mask, nullptr, nullptr, B, S, h, d, (bf16*)ctx,
+                                 static_cast<cudaStream_t>(stream));
 }
 
 rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,

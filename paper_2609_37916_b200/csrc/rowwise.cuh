@@ -38,23 +38,108 @@ __device__ __forceinline__ void ln_normalise_store(float (&v)[NV * 4], const flo
     }
 }
 
-// x[t] = LN(word[ids[t]] + pos[t % S] + type[0]).  Ids outside [0, V) are clamped and flagged.
+// Sequence packing.  Valid tokens (mask != 0) are compacted so that sequence b owns the packed rows
+// seq_start[b] .. seq_start[b] + seq_len[b]; every later kernel then works on sum(len) rows instead
+// of B*S.  Exact for any 0/1 mask: positions are taken from the original index s, attention only
+// ever involves a sequence's valid tokens, pooling averages exactly those rows.
+//   seq_len[b]            number of valid positions of sequence b
+//   seq_start[0..B]       exclusive prefix sum of seq_len (seq_start[B] = total packed rows)
+//   pos_of_rank[b*S + r]  original position s of the r-th valid token of sequence b
+// One CTA per sequence; the last CTA to finish (ticket counter, reset for the next launch) scans
+// seq_len.  Integer work only.
+constexpr int kPackThreads = 128;
+
+__global__ void __launch_bounds__(kPackThreads)
+pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* __restrict__ seq_len,
+                      int32_t* __restrict__ seq_start, int32_t* __restrict__ pos_of_rank,
+                      unsigned int* __restrict__ ticket) {
+    __shared__ int warp_cnt[kPackThreads / 32];
+    __shared__ int is_last;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int running = 0;
+    for (int base = 0; base < S; base += kPackThreads) {
+        const int s = base + tid;
+        const bool valid = s < S && __ldg(mask + (size_t)b * S + s) != 0;
+        const unsigned bal = __ballot_sync(0xffffffffu, valid);
+        if (lane == 0) warp_cnt[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, chunk = 0;
+#pragma unroll
+        for (int w = 0; w < kPackThreads / 32; ++w) {
+            if (w < warp) before += warp_cnt[w];
+            chunk += warp_cnt[w];
+        }
+        if (valid) pos_of_rank[(size_t)b * S + running + before + __popc(bal & ((1u << lane) - 1u))] = s;
+        running += chunk;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        seq_len[b] = running;
+        __threadfence();
+        is_last = (atomicAdd(ticket, 1u) == (unsigned)(B - 1));
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // exclusive scan of seq_len by the last CTA: each warp-sized chunk with shuffles, carried serially
+    if (warp == 0) {
+        int carry = 0;
+        for (int base = 0; base < B; base += 32) {
+            const int i = base + lane;
+            const int v = i < B ? *((volatile int32_t*)seq_len + i) : 0;
+            int incl = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int n = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            if (i < B) seq_start[i] = carry + incl - v;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            seq_start[B] = carry;
+            *ticket = 0;   // ready for the next launch
+        }
+    }
+}
+
+// Largest b with seq_start[b] <= p (seq_start is non-decreasing, seq_start[B] = total > p).
+__device__ __forceinline__ int find_sequence(const int32_t* __restrict__ seq_start, int B, int p) {
+    int lo = 0, hi = B;   // invariant: seq_start[lo] <= p < seq_start[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(seq_start + mid) <= p) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// x[row] = LN(word[id] + pos[s] + type[0]).  Ids outside [0, V) are clamped and flagged.
+// Padded mode (seq_start == nullptr): row = token t = b*S + s for all T tokens.
+// Packed mode: row p < seq_start[B] belongs to sequence b = find_sequence(p) at position
+// s = pos_of_rank[b*S + (p - seq_start[b])].
 template <int NV>
 __global__ void __launch_bounds__(kRowWarps * 32)
 embed_ln_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict__ word,
                 const __nv_bfloat16* __restrict__ pos, const __nv_bfloat16* __restrict__ type,
                 const float* __restrict__ gamma, const float* __restrict__ beta,
-                __nv_bfloat16* __restrict__ out, int T, int S, int V, float eps, int32_t* status) {
+                __nv_bfloat16* __restrict__ out, int T, int S, int V, float eps, int32_t* status,
+                const int32_t* __restrict__ seq_start, const int32_t* __restrict__ pos_of_rank, int B) {
     constexpr int H = NV * 128;
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kRowWarps + (threadIdx.x >> 5);
     if (t >= T) return;
-    int id = __ldg(ids + t);
+    int tok = t, s = t % S;
+    if (seq_start != nullptr) {
+        if (t >= __ldg(seq_start + B)) return;
+        const int b = find_sequence(seq_start, B, t);
+        s = __ldg(pos_of_rank + (size_t)b * S + (t - __ldg(seq_start + b)));
+        tok = b * S + s;
+    }
+    int id = __ldg(ids + tok);
     if (id < 0 || id >= V) {
         if (lane == 0 && status) atomicOr(status, RLX_DEVSTAT_TOKEN_RANGE_BIT);
         id = id < 0 ? 0 : V - 1;
     }
-    const int s = t % S;
     const __nv_bfloat16* wrow = word + (size_t)id * H;
     const __nv_bfloat16* prow = pos + (size_t)s * H;
     float v[NV * 4];
@@ -76,11 +161,12 @@ embed_ln_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict
 template <int NV>
 __global__ void __launch_bounds__(kRowWarps * 32)
 layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ gamma,
-                 const float* __restrict__ beta, __nv_bfloat16* __restrict__ out, int T, float eps) {
+                 const float* __restrict__ beta, __nv_bfloat16* __restrict__ out, int T, float eps,
+                 const int32_t* __restrict__ rows_ptr) {
     constexpr int H = NV * 128;
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kRowWarps + (threadIdx.x >> 5);
-    if (t >= T) return;
+    if (t >= T || (rows_ptr != nullptr && t >= __ldg(rows_ptr))) return;   // rows_ptr: packed row count
     const __nv_bfloat16* row = x + (size_t)t * H;
     float v[NV * 4];
 #pragma unroll
@@ -102,19 +188,23 @@ constexpr int kPoolThreads = 384;
 
 __global__ void __launch_bounds__(kPoolThreads)
 pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restrict__ mask,
-                   float* __restrict__ out, int S, int H) {
+                   float* __restrict__ out, int S, int H, const int32_t* __restrict__ seq_start,
+                   const int32_t* __restrict__ seq_len) {
     extern __shared__ float pool_smem[];  // [G][H] partial sums, then [kPoolThreads/32] reductions
     const int b = blockIdx.x;
     const int vecs = H / 8;               // 16-byte vectors per row
     const int G = kPoolThreads / vecs;    // row groups (>= 1 since H <= 1024 -> vecs <= 128)
     const int g = threadIdx.x / vecs, c = threadIdx.x % vecs;
-    const __nv_bfloat16* xb = x + (size_t)b * S * H;
+    // packed mode (seq_start != nullptr): the sequence's rows are contiguous and all valid
+    const bool packed = seq_start != nullptr;
+    const __nv_bfloat16* xb = x + (packed ? (size_t)__ldg(seq_start + b) : (size_t)b * S) * H;
     const int32_t* mb = mask + (size_t)b * S;
+    const int nrows = packed ? __ldg(seq_len + b) : S;
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     int count = 0;
     if (g < G) {
-        for (int s = g; s < S; s += G) {
-            if (__ldg(mb + s) == 0) continue;
+        for (int s = g; s < nrows; s += G) {
+            if (!packed && __ldg(mb + s) == 0) continue;
             ++count;
             const uint4 a = __ldg(reinterpret_cast<const uint4*>(xb + (size_t)s * H + c * 8));
             acc[0] += bf16lo(a.x); acc[1] += bf16hi(a.x);

@@ -42,7 +42,7 @@ def _cfg(**kw):
 
 def test_create_validates_shapes(lib):
     enc = binding.Encoder(**_cfg())
-    assert enc.kernels_per_forward() == 2 + 7 * 6
+    assert enc.kernels_per_forward() == 3 + 7 * 6   # packing + embed + 7 per layer + pool
     enc.close()
     for bad, status in [
         (dict(hidden=400, num_heads=10), 2),    # H % 128

@@ -100,6 +100,29 @@ def test_pool_l2norm(rlx, B, S, H):
         assert np.array_equal(got[1], np.zeros(H))
 
 
+@pytest.mark.parametrize("B,S,holes", [(1, 16, 0.0), (7, 130, 0.0), (5, 512, 0.4), (300, 33, 0.3), (64, 128, 0.0)])
+def test_pack_sequences_is_bit_exact(rlx, B, S, holes):
+    rng = np.random.default_rng(B * S)
+    lengths = rng.integers(0, S + 1, size=B)
+    lengths[0] = S
+    if B > 2:
+        lengths[1], lengths[2] = 0, 1
+    mask = (np.arange(S)[None, :] < lengths[:, None]).astype(np.int32)
+    if holes:
+        mask = (mask * (rng.random((B, S)) >= holes)).astype(np.int32)
+    dmask = i32_dev(mask)
+    for _ in range(2):   # the ticket counter must be left ready for a second launch
+        seq_len, seq_start, pos, ticket = rlx.pack_sequences(dmask)
+        torch.cuda.synchronize()
+        assert int(ticket.item()) == 0
+        want_len = mask.astype(bool).sum(1)
+        assert np.array_equal(seq_len.cpu().numpy(), want_len)
+        assert np.array_equal(seq_start.cpu().numpy(), np.concatenate([[0], np.cumsum(want_len)]))
+        got = pos.cpu().numpy()
+        for b in range(B):
+            assert np.array_equal(got[b, :want_len[b]], np.nonzero(mask[b])[0])
+
+
 # ------------------------------------------------------------------ GEMM
 GEMM_SHAPES = [(128, 64, 64), (16, 1152, 384), (300, 384, 384), (257, 1536, 384), (1000, 384, 1536),
                (129, 768, 768), (4096, 192, 72), (2048, 2304, 768)]
