@@ -60,6 +60,7 @@ typedef enum {
 #define RLX_FLAG_NO_GRAPH 0x1u  /* launch kernels one by one instead of replaying a CUDA graph */
 #define RLX_FLAG_GEMM_SIMT 0x2u /* use the plain CUDA-core GEMM (bring-up / cross-check only)  */
 #define RLX_FLAG_KERNEL_EVENTS 0x4u /* record a CUDA event between kernels (see rlx_encoder_kernel_times) */
+#define RLX_FLAG_NO_PDL 0x10u   /* plain stream order between kernels (no programmatic dependent launch) */
 #define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
 
 typedef struct {

@@ -23,6 +23,7 @@ FLAG_NO_GRAPH = 0x1
 FLAG_GEMM_SIMT = 0x2
 FLAG_KERNEL_EVENTS = 0x4
 FLAG_NO_PACK = 0x8
+FLAG_NO_PDL = 0x10
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20

@@ -76,6 +76,8 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     extern __shared__ __align__(16) unsigned char att_smem_raw[];
     SM& sm = *reinterpret_cast<SM*>(att_smem_raw);
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q0 = blockIdx.x * kAttBlockM, head = blockIdx.y, b = blockIdx.z;
     const bool packed = seq_start != nullptr;

@@ -192,12 +192,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int M = p.M;
-    if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));   // packed activations: only sum(len) rows exist
-    const int n_tiles = p.N / BLOCK_N;
-    const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
-    const int num_tiles = n_tiles * m_tiles;
-    const int num_kb = (p.K + BLOCK_K - 1) / BLOCK_K;
+    pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::STAGES; ++i) {
@@ -222,6 +217,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+
+    // everything above is independent of the previous kernel; its outputs are read only from here on
+    pdl_wait();
+    int M = p.M;
+    if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));   // packed activations: only sum(len) rows exist
+    const int n_tiles = p.N / BLOCK_N;
+    const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
+    const int num_tiles = n_tiles * m_tiles;
+    const int num_kb = (p.K + BLOCK_K - 1) / BLOCK_K;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer

@@ -105,6 +105,26 @@ cudaError_t init_kernels_for_current_device() {
 }
 
 // ------------------------------------------------------------------ launchers
+// When set, kernels are launched with the programmatic-stream-serialization attribute so that each
+// kernel's prologue overlaps its predecessor's tail (the kernels call griddepcontrol.wait before
+// they read anything a predecessor wrote).  Set by enqueue_forward around its launches.
+thread_local bool g_pdl_launch = false;
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_pdl_launch ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 struct Packing {   // device arrays written by pack_sequences_kernel; all null in padded mode
     const int32_t* seq_len = nullptr;
     const int32_t* seq_start = nullptr;    // [B+1]; seq_start[B] = number of packed rows
@@ -125,7 +145,7 @@ rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* p
                              int32_t* status, cudaStream_t st, const Packing& pk = Packing()) {
     const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: rlx::embed_ln_kernel<NV><<<grid, thr, 0, st>>>(ids, word, pos, type, g, b, out, T, S, V, eps, status, pk.seq_start, pk.pos_of_rank, pk.B); break;
+#define RLX_CASE(NV) case NV: RLX_CUDA_TRY(launch_ex(rlx::embed_ln_kernel<NV>, grid, thr, 0, st, ids, word, pos, type, g, b, out, T, S, V, eps, status, pk.seq_start, pk.pos_of_rank, pk.B)); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE
         default: return RLX_ERR_UNSUPPORTED;
@@ -138,7 +158,7 @@ rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int
                               cudaStream_t st, const int32_t* rows_ptr = nullptr) {
     const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: rlx::layernorm_kernel<NV><<<grid, thr, 0, st>>>(x, g, b, out, T, eps, rows_ptr); break;
+#define RLX_CASE(NV) case NV: RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE
         default: return RLX_ERR_UNSUPPORTED;
@@ -151,7 +171,7 @@ rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H
                          const Packing& pk = Packing()) {
     const int vecs = H / 8, G = rlx::kPoolThreads / vecs;
     const size_t smem = (size_t)G * H * sizeof(float);
-    rlx::pool_l2norm_kernel<<<B, rlx::kPoolThreads, smem, st>>>(x, mask, out, S, H, pk.seq_start, pk.seq_len);
+    RLX_CUDA_TRY(launch_ex(rlx::pool_l2norm_kernel, B, rlx::kPoolThreads, smem, st, x, mask, out, S, H, pk.seq_start, pk.seq_len));
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -162,9 +182,9 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
     dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
     if (d == 32)
-        rlx::attention_bf16_kernel<32><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st>>>(qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e);
+        RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<32>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
     else if (d == 64)
-        rlx::attention_bf16_kernel<64><<<grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st>>>(qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e);
+        RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<64>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
@@ -189,9 +209,9 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
     const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
     const int smem = rlx::tc::Cfg<BN>::SMEM_BYTES;
     switch (epi) {
-        case 0: rlx::tc::gemm_tcgen05_kernel<BN, 0><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
-        case 1: rlx::tc::gemm_tcgen05_kernel<BN, 1><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
-        case 2: rlx::tc::gemm_tcgen05_kernel<BN, 2><<<grid, rlx::tc::kThreads, smem, st>>>(ta, tb, to, p); break;
+        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
@@ -327,6 +347,11 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
 #define RLX_TRY(call) do { s = (call); if (s != RLX_OK) return s; s = mark(); if (s != RLX_OK) return s; } while (0)
     s = mark();
     if (s != RLX_OK) return s;
+    // programmatic dependent launch between consecutive kernels; not combined with per-kernel events
+    struct PdlScope {
+        explicit PdlScope(bool on) { g_pdl_launch = on; }
+        ~PdlScope() { g_pdl_launch = false; }
+    } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && e->events.empty());
     Packing pk;
     if (pack) {
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);

@@ -55,6 +55,7 @@ pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* _
                       unsigned int* __restrict__ ticket) {
     __shared__ int warp_cnt[kPackThreads / 32];
     __shared__ int is_last;
+    pdl_launch_dependents();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int running = 0;
     for (int base = 0; base < S; base += kPackThreads) {
@@ -125,6 +126,8 @@ embed_ln_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict
                 __nv_bfloat16* __restrict__ out, int T, int S, int V, float eps, int32_t* status,
                 const int32_t* __restrict__ seq_start, const int32_t* __restrict__ pos_of_rank, int B) {
     constexpr int H = NV * 128;
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kRowWarps + (threadIdx.x >> 5);
     if (t >= T) return;
@@ -164,6 +167,8 @@ layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ 
                  const float* __restrict__ beta, __nv_bfloat16* __restrict__ out, int T, float eps,
                  const int32_t* __restrict__ rows_ptr) {
     constexpr int H = NV * 128;
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * kRowWarps + (threadIdx.x >> 5);
     if (t >= T || (rows_ptr != nullptr && t >= __ldg(rows_ptr))) return;   // rows_ptr: packed row count
@@ -191,6 +196,8 @@ pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restric
                    float* __restrict__ out, int S, int H, const int32_t* __restrict__ seq_start,
                    const int32_t* __restrict__ seq_len) {
     extern __shared__ float pool_smem[];  // [G][H] partial sums, then [kPoolThreads/32] reductions
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x;
     const int vecs = H / 8;               // 16-byte vectors per row
     const int G = kPoolThreads / vecs;    // row groups (>= 1 since H <= 1024 -> vecs <= 128)
