@@ -262,8 +262,11 @@ typedef enum {
 } rlx_epilogue_t;
 
 typedef enum {
-    RLX_GEMM_TCGEN05 = 0, /* TMA-fed tcgen05 MMA with TMEM accumulators (the product path) */
-    RLX_GEMM_SIMT = 1     /* plain CUDA-core tiles (bring-up / cross-check)                */
+    RLX_GEMM_TCGEN05 = 0,        /* TMA-fed tcgen05 MMA with TMEM accumulators; tile shape and CTA
+                                    grouping chosen from the problem size (the product path)      */
+    RLX_GEMM_SIMT = 1,           /* plain CUDA-core tiles (bring-up / cross-check)                 */
+    RLX_GEMM_TCGEN05_PAIR = 2,   /* force the CTA-pair variant (cta_group::2, 256-row tiles); N % 128 == 0 */
+    RLX_GEMM_TCGEN05_SINGLE = 3  /* force the one-CTA-per-tile variant                             */
 } rlx_gemm_impl_t;
 
 /*

@@ -13,6 +13,12 @@
 //               staging buffer and hands it to a TMA store (rows past M are clipped by the copy).
 //               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop;
 //               a warp releases its accumulator as soon as its last tcgen05.ld has landed.
+// Two instantiations per tile shape: CG = 1 (one CTA per 128 x BLOCK_N tile) and CG = 2, where a
+// cluster of two CTAs on neighbouring SMs computes a 256 x BLOCK_N tile with tcgen05.mma.cta_group::2:
+// each CTA loads its own 128 rows of A and only HALF of the W tile, the leader CTA issues the MMAs
+// for both, and each CTA finds its 128 accumulator rows in its own TMEM.  This halves the W bytes
+// every SM has to pull from L2 (the operand feed, not the tensor pipe, is what limits these GEMMs)
+// without any multicast load.  Completion is signalled to both CTAs with a multicast tcgen05.commit.
 // Every mbarrier wait is bounded by a wall-clock budget; on expiry the CTA raises an abort flag,
 // records RLX_DEVSTAT_TIMEOUT, drains, frees its tensor memory and returns.
 #pragma once
@@ -32,10 +38,11 @@ constexpr int kStageBufBytes = 32 * 32 * 2;          // one 32-row x 32-column b
 constexpr int kStagingBytes = kEpiWarps * 2 * kStageBufBytes;  // two buffers per epilogue warp
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
 
-template <int BLOCK_N>
+template <int BLOCK_N, int CG = 1>
 struct Cfg {
     static constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;
-    static constexpr int B_BYTES = BLOCK_N * BLOCK_K * 2;
+    static constexpr int B_ROWS = BLOCK_N / CG;                  // W rows this CTA loads per k-block
+    static constexpr int B_BYTES = B_ROWS * BLOCK_K * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int RING_BUDGET = 222 * 1024 - kStagingBytes;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
@@ -43,7 +50,8 @@ struct Cfg {
                                      : (2 * BLOCK_N <= 256) ? 256 : 512;
     static constexpr int BAR_BYTES = 256;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + kStagingBytes + BAR_BYTES + 1024;  // +1024: manual alignment
-    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128");
+    static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128 / M=256");
+    static_assert(CG == 1 || CG == 2, "cta_group");
     static_assert(B_BYTES % 1024 == 0, "stage tiles must stay 1024-byte aligned");
     static_assert(STAGES >= 2, "ring too shallow");
 };
@@ -85,6 +93,25 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return true;
 }
+// ---- cluster helpers (CG = 2) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `smem_addr` (a shared::cta address) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
@@ -107,31 +134,66 @@ __device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_g
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+// CG = 2 form: the mbarrier may live in the peer CTA (cluster address); the data lands in this CTA
+__device__ __forceinline__ void tma_load_2d_cg2(uint32_t smem_dst, const CUtensorMap* tmap, int x, int y, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar_cluster) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
+template <int CG>
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+    if constexpr (CG == 1)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+    else
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
 }
+template <int CG>
 __device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (CG == 1)
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    else
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
+template <int CG>
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    if constexpr (CG == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    if constexpr (CG == 1)
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+            "}\n" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    else
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "setp.ne.b32 p, %4, 0;\n"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+            "}\n" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed
+// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed.  CG = 2: the
+// arrive is multicast to the barrier at the same offset in both CTAs of the pair.
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if constexpr (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
 }
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (thread = lane = row)
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -170,13 +232,15 @@ struct Params {
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
     const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
+    int debug;                       // experiments only: bit 0 = epilogue releases the accumulator without reading it
 };
 
-template <int BLOCK_N, int EPI>
+template <int BLOCK_N, int EPI, int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_out, const Params p) {
-    using C = Cfg<BLOCK_N>;
+    using C = Cfg<BLOCK_N, CG>;
+    constexpr int TILE_M = BLOCK_M * CG;   // rows of one output tile (per CTA pair when CG = 2)
     extern __shared__ unsigned char smem_raw[];
     // manual 1024-byte alignment (required by the 128-byte swizzle atoms)
     const uint32_t raw = smem_u32(smem_raw);
@@ -192,6 +256,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = (CG == 2) ? cluster_ctarank() : 0u;   // rank 0 leads the pair
     pdl_launch_dependents();
 
     if (threadIdx.x == 0) {
@@ -201,7 +266,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(tfull_bar + 8 * i, 1);
-            mbar_init(tempty_bar + 8 * i, kEpiWarps);
+            mbar_init(tempty_bar + 8 * i, kEpiWarps * CG);   // the leader's barrier collects both CTAs' warps
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -210,11 +275,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         prefetch_tmap(&tmap_out);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc<CG>(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish<CG>();
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();   // the peer's barriers are initialised before any remote use
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -223,9 +289,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     int M = p.M;
     if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));   // packed activations: only sum(len) rows exist
     const int n_tiles = p.N / BLOCK_N;
-    const int m_tiles = (M + BLOCK_M - 1) / BLOCK_M;
+    const int m_tiles = (M + TILE_M - 1) / TILE_M;
     const int num_tiles = n_tiles * m_tiles;
     const int num_kb = (p.K + BLOCK_K - 1) / BLOCK_K;
+    const int tile0 = blockIdx.x / CG, tile_step = gridDim.x / CG;   // both CTAs of a pair walk the same tiles
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -233,27 +300,35 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int tile = tile0; tile < num_tiles && ok; tile += tile_step) {
                 const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-                    mbar_expect_tx(full_bar + 8 * stage, C::STAGE_BYTES);
-                    tma_load_2d(sa, &tmap_a, kb * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
-                    tma_load_2d(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                    if constexpr (CG == 1) {
+                        mbar_expect_tx(full_bar + 8 * stage, C::STAGE_BYTES);
+                        tma_load_2d(sa, &tmap_a, kb * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
+                        tma_load_2d(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                    } else {
+                        // both CTAs' copies complete on the LEADER's full barrier, which expects all bytes
+                        const uint32_t lead_full = map_to_cta(full_bar + 8 * stage, 0);
+                        if (cta_rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * C::STAGE_BYTES);
+                        tma_load_2d_cg2(sa, &tmap_a, kb * BLOCK_K, m_blk * TILE_M + (int)cta_rank * BLOCK_M, lead_full);
+                        tma_load_2d_cg2(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS, lead_full);
+                    }
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = make_idesc(TILE_M, BLOCK_N);
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+            for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (it >> 1) & 1;
                 if (!mbar_wait(tempty_bar + 8 * as, aphase ^ 1, abort_flag)) { ok = false; break; }
@@ -267,12 +342,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 #pragma unroll
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
-                        umma_bf16(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_bf16<CG>(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(empty_bar + 8 * stage);  // stage reusable once these MMAs have read it
+                    umma_commit<CG>(empty_bar + 8 * stage);  // stage reusable once these MMAs have read it
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit(tfull_bar + 8 * as);  // accumulator complete
+                if (ok) umma_commit<CG>(tfull_bar + 8 * as);  // accumulator complete
             }
         }
     } else {
@@ -288,19 +363,40 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         int it = 0;
         uint32_t nstore = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+        for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
             const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
             const int as = it & 1;
             const uint32_t aphase = (it >> 1) & 1;
-            if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const int m_row0 = m_blk * BLOCK_M + quad * 32;
+            const int m_row0 = m_blk * TILE_M + (int)cta_rank * BLOCK_M + quad * 32;
             const int m = m_row0 + lane;
             const bool row_ok = m < M;
             const int n0 = n_blk * BLOCK_N + half * HALF_N;
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N + half * HALF_N;
-            const __nv_bfloat16* rrow = p.residual + (size_t)m * p.N + n0;
             const float* brow = p.bias + n0;
+            // residual rows of this tile are fetched before waiting for the accumulator, so their
+            // latency hides behind the main loop
+            uint4 res[EPI == 2 ? NC : 1][4];
+            if (EPI == 2) {
+                const int m_pre = m_blk * TILE_M + (int)cta_rank * BLOCK_M + quad * 32 + lane;
+                if (m_pre < M) {
+                    const __nv_bfloat16* rpre = p.residual + (size_t)m_pre * p.N + n_blk * BLOCK_N + half * HALF_N;
+#pragma unroll
+                    for (int c = 0; c < NC; ++c)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) res[c][i] = __ldg(reinterpret_cast<const uint4*>(rpre + c * 32) + i);
+                }
+            }
+            if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            if (p.debug & 1) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 1 || cta_rank == 0) mbar_arrive(tempty_bar + 8 * as);
+                    else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * as, 0));
+                }
+                continue;
+            }
             uint32_t r[2][32];
             tmem_ld_32x32(taddr, r[0]);
 #pragma unroll
@@ -312,7 +408,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     // every accumulator value this warp needs is in registers: release the buffer
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar + 8 * as);
+                    if (lane == 0) {
+                        if (CG == 1 || cta_rank == 0) mbar_arrive(tempty_bar + 8 * as);
+                        else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * as, 0));
+                    }
                 }
                 const uint32_t(&acc)[32] = r[c & 1];
                 float v[32];
@@ -326,12 +425,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 }
                 if (EPI == 1) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = gelu_erf(v[i]);
+                    for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
                 }
                 if (EPI == 2 && row_ok) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        const uint4 q = __ldg(reinterpret_cast<const uint4*>(rrow + c * 32) + i);
+                        const uint4 q = res[c][i];
                         v[8 * i + 0] += bf16lo(q.x); v[8 * i + 1] += bf16hi(q.x);
                         v[8 * i + 2] += bf16lo(q.y); v[8 * i + 3] += bf16hi(q.y);
                         v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
@@ -351,10 +450,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
                     st_shared_v4(buf + row_off + (((uint32_t)i ^ swz) << 4), q);
                 }
-                fence_proxy_async();   // make the generic-proxy writes visible to the TMA engine
+                if (!(p.debug & 4)) fence_proxy_async();   // make the generic-proxy writes visible to the TMA engine
                 __syncwarp();
                 if (lane == 0) {
-                    if (m_row0 < M) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
+                    if (m_row0 < M && !(p.debug & 2)) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
                     bulk_commit();
                 }
                 ++nstore;
@@ -372,10 +471,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();   // neither CTA leaves while the pair still uses its memory
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem_base, C::TMEM_COLS);
+        tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
     }
 }
 

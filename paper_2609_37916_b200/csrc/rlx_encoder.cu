@@ -71,18 +71,21 @@ bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
 }
 
 // ------------------------------------------------------------------ one-time kernel attributes
-template <int BN, int EPI>
+template <int BN, int EPI, int CG>
 cudaError_t set_gemm_attr() {
-    return cudaFuncSetAttribute(rlx::tc::gemm_tcgen05_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                rlx::tc::Cfg<BN>::SMEM_BYTES);
+    return cudaFuncSetAttribute(rlx::tc::gemm_tcgen05_kernel<BN, EPI, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                rlx::tc::Cfg<BN, CG>::SMEM_BYTES);
 }
-template <int BN>
+template <int BN, int CG = 1>
 cudaError_t set_gemm_attr_all() {
     cudaError_t e;
-    if ((e = set_gemm_attr<BN, 0>()) != cudaSuccess) return e;
-    if ((e = set_gemm_attr<BN, 1>()) != cudaSuccess) return e;
-    return set_gemm_attr<BN, 2>();
+    if ((e = set_gemm_attr<BN, 0, CG>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr<BN, 1, CG>()) != cudaSuccess) return e;
+    return set_gemm_attr<BN, 2, CG>();
 }
+
+// Number of CTA pairs that can be resident at once (pairs must sit in one GPC), per device.
+int g_max_pairs[64] = {};
 
 cudaError_t init_kernels_for_current_device() {
     static std::mutex mu;
@@ -96,6 +99,25 @@ cudaError_t init_kernels_for_current_device() {
     if ((e = set_gemm_attr_all<128>()) != cudaSuccess) return e;
     if ((e = set_gemm_attr_all<192>()) != cudaSuccess) return e;
     if ((e = set_gemm_attr_all<256>()) != cudaSuccess) return e;
+    if ((e = (set_gemm_attr_all<128, 2>())) != cudaSuccess) return e;
+    if ((e = (set_gemm_attr_all<192, 2>())) != cudaSuccess) return e;
+    if ((e = (set_gemm_attr_all<256, 2>())) != cudaSuccess) return e;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * rlx::kNumSMs);
+        cfg.blockDim = dim3(rlx::tc::kThreads);
+        cfg.dynamicSmemBytes = rlx::tc::Cfg<256, 2>::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tc::gemm_tcgen05_kernel<256, 0, 2>, &cfg)) != cudaSuccess) return e;
+        if (dev < 64) g_max_pairs[dev] = n;
+    }
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)sizeof(rlx::AttSmem<32>))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -110,6 +132,8 @@ cudaError_t init_kernels_for_current_device() {
 // they read anything a predecessor wrote).  Set by enqueue_forward around its launches.
 thread_local bool g_pdl_launch = false;
 
+thread_local int g_cluster_x = 1;   // set by the CTA-pair GEMM launcher around its launch
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
@@ -117,11 +141,22 @@ cudaError_t launch_ex(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    if (g_pdl_launch) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (g_cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)g_cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = g_pdl_launch ? 1 : 0;
+    cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
@@ -156,9 +191,12 @@ rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* p
 
 rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int T, int H, float eps, bf16* out,
                               cudaStream_t st, const int32_t* rows_ptr = nullptr) {
-    const int grid = (T + rlx::kRowWarps - 1) / rlx::kRowWarps, thr = rlx::kRowWarps * 32;
+    const bool big = T >= 4 * rlx::kNumSMs * rlx::kRowWarps * 4;   // enough rows for 4 rows per warp on every SM
+    const int rows_per_cta = rlx::kRowWarps * (big ? 4 : 1);
+    const int grid = (T + rows_per_cta - 1) / rows_per_cta, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); break;
+#define RLX_CASE(NV) case NV: if (big) RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV, 4>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); \
+                     else RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV, 1>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE
         default: return RLX_ERR_UNSUPPORTED;
@@ -191,27 +229,57 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     return RLX_OK;
 }
 
-int pick_block_n(int M, int N) {
+struct TileChoice { int bn; int cg; };
+
+// Tile shape for an [M, N] output.  CTA pairs (cg = 2, 256-row tiles, each CTA loading half of the
+// W tile) are used when there are enough tiles to keep every pair busy for a few rounds; smaller
+// problems keep one CTA per 128-row tile and shrink BLOCK_N until every SM has work.
+TileChoice pick_tile(int M, int N, int K, int want_cg = 0) {
+    static const int env_cg = getenv("RLX_GEMM_CG") ? atoi(getenv("RLX_GEMM_CG")) : 0;   // tuning knobs
+    const int force_cg = want_cg ? want_cg : env_cg;
+    static const int force_bn = getenv("RLX_GEMM_BN") ? atoi(getenv("RLX_GEMM_BN")) : 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int pairs = (dev >= 0 && dev < 64) ? g_max_pairs[dev] : 0;
+    // pairs pay off once a tile's main loop is long enough to amortise the cross-CTA handshakes
+    if (force_cg != 1 && pairs > 0 && (force_cg == 2 || K >= 768)) {
+        const int m_tiles2 = (M + 255) / 256;
+        const int cand2[3] = {256, 192, 128};
+        for (int i = 0; i < 3; ++i) {
+            if (force_bn && cand2[i] != force_bn) continue;
+            if (N % cand2[i] == 0 && (force_cg == 2 || m_tiles2 * (N / cand2[i]) >= 3 * pairs)) return {cand2[i], 2};
+        }
+    }
     const int m_tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
     const int cand[4] = {256, 192, 128, 64};
+    if (force_bn && N % force_bn == 0 && (force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256))
+        return {force_bn, 1};
     // largest tile that still gives every SM work; otherwise the smallest that divides N
     for (int i = 0; i < 4; ++i)
-        if (N % cand[i] == 0 && m_tiles * (N / cand[i]) >= rlx::kNumSMs) return cand[i];
+        if (N % cand[i] == 0 && m_tiles * (N / cand[i]) >= rlx::kNumSMs) return {cand[i], 1};
     for (int i = 3; i >= 0; --i)
-        if (N % cand[i] == 0) return cand[i];
-    return 0;
+        if (N % cand[i] == 0) return {cand[i], 1};
+    return {0, 1};
 }
 
-template <int BN>
+template <int BN, int CG>
 rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
                                const rlx::tc::Params& p, int epi, cudaStream_t st) {
-    const int tiles = ((p.M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M) * (p.N / BN);
-    const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
-    const int smem = rlx::tc::Cfg<BN>::SMEM_BYTES;
+    const int tile_m = rlx::tc::BLOCK_M * CG;
+    const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN);
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int slots = CG == 1 ? rlx::kNumSMs : ((dev >= 0 && dev < 64) ? g_max_pairs[dev] : 1);
+    const int grid = CG * (tiles < slots ? tiles : slots);
+    const int smem = rlx::tc::Cfg<BN, CG>::SMEM_BYTES;
+    struct ClusterScope {
+        explicit ClusterScope(int x) { g_cluster_x = x; }
+        ~ClusterScope() { g_cluster_x = 1; }
+    } scope(CG);
     switch (epi) {
-        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
-        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
-        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
@@ -220,7 +288,7 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
 
 rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const bf16* residual, int epi, int M, int N,
                          int K, bf16* out, bool simt, int32_t* status, cudaStream_t st,
-                         const int32_t* m_ptr = nullptr) {
+                         const int32_t* m_ptr = nullptr, int want_cg = 0) {
     if (simt) {
         dim3 grid((N + rlx::kSimtTile - 1) / rlx::kSimtTile, (M + rlx::kSimtTile - 1) / rlx::kSimtTile);
         switch (epi) {
@@ -232,18 +300,28 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
         RLX_CUDA_TRY(cudaGetLastError());
         return RLX_OK;
     }
-    const int bn = pick_block_n(M, N);
+    const TileChoice tc = pick_tile(M, N, K, want_cg);
+    const int bn = tc.bn;
     if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
     CUtensorMap ta, tb, to;
     if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
-    if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)bn)) return RLX_ERR_CUDA;
+    if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / tc.cg))) return RLX_ERR_CUDA;
     if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
-    rlx::tc::Params p{bias, residual, M, N, K, status, m_ptr};
+    static const int dbg = getenv("RLX_GEMM_DEBUG") ? atoi(getenv("RLX_GEMM_DEBUG")) : 0;
+    rlx::tc::Params p{bias, residual, M, N, K, status, m_ptr, dbg};
+    if (tc.cg == 2) {
+        switch (bn) {
+            case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, to, p, epi, st);
+            case 192: return launch_gemm_tc_bn<192, 2>(ta, tb, to, p, epi, st);
+            case 256: return launch_gemm_tc_bn<256, 2>(ta, tb, to, p, epi, st);
+        }
+        return RLX_ERR_UNSUPPORTED;
+    }
     switch (bn) {
-        case 64: return launch_gemm_tc_bn<64>(ta, tb, to, p, epi, st);
-        case 128: return launch_gemm_tc_bn<128>(ta, tb, to, p, epi, st);
-        case 192: return launch_gemm_tc_bn<192>(ta, tb, to, p, epi, st);
-        case 256: return launch_gemm_tc_bn<256>(ta, tb, to, p, epi, st);
+        case 64: return launch_gemm_tc_bn<64, 1>(ta, tb, to, p, epi, st);
+        case 128: return launch_gemm_tc_bn<128, 1>(ta, tb, to, p, epi, st);
+        case 192: return launch_gemm_tc_bn<192, 1>(ta, tb, to, p, epi, st);
+        case 256: return launch_gemm_tc_bn<256, 1>(ta, tb, to, p, epi, st);
     }
     return RLX_ERR_UNSUPPORTED;
 }
@@ -642,10 +720,14 @@ rlx_status_t rlx_gemm_bf16(const void* A, const void* W, const float* bias, cons
     if (!aligned16(A) || !aligned16(W) || !aligned16(bias) || !aligned16(out) || (residual && !aligned16(residual)))
         return RLX_ERR_INVALID_ARG;
     if (N % 64 != 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
-    if (impl != RLX_GEMM_TCGEN05 && impl != RLX_GEMM_SIMT) return RLX_ERR_INVALID_ARG;
+    if (impl != RLX_GEMM_TCGEN05 && impl != RLX_GEMM_SIMT && impl != RLX_GEMM_TCGEN05_PAIR &&
+        impl != RLX_GEMM_TCGEN05_SINGLE)
+        return RLX_ERR_INVALID_ARG;
+    if (impl == RLX_GEMM_TCGEN05_PAIR && N % 128 != 0 && N % 192 != 0) return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
+    const int want_cg = impl == RLX_GEMM_TCGEN05_PAIR ? 2 : impl == RLX_GEMM_TCGEN05_SINGLE ? 1 : 0;
     return launch_gemm((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, (int)epi, M, N, K, (bf16*)out,
-                       impl == RLX_GEMM_SIMT, status, static_cast<cudaStream_t>(stream));
+                       impl == RLX_GEMM_SIMT, status, static_cast<cudaStream_t>(stream), nullptr, want_cg);
 }
 
 rlx_status_t rlx_attention_bf16(const void* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,

@@ -161,7 +161,10 @@ embed_ln_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict
 }
 
 // out = LN(x) row by row (the residual sum was already formed by the producing GEMM's epilogue).
-template <int NV>
+// Each warp handles kLnRowsPerWarp rows with all of their loads issued before the first reduction,
+// so with 4 rows per warp a warp keeps 3 KB (H=384) in flight and the grid is 4x smaller; small
+// problems use 1 row per warp so that every SM still gets CTAs.
+template <int NV, int kLnRowsPerWarp>
 __global__ void __launch_bounds__(kRowWarps * 32)
 layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ gamma,
                  const float* __restrict__ beta, __nv_bfloat16* __restrict__ out, int T, float eps,
@@ -170,20 +173,31 @@ layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ 
     pdl_launch_dependents();
     pdl_wait();
     const int lane = threadIdx.x & 31;
-    const int t = blockIdx.x * kRowWarps + (threadIdx.x >> 5);
-    if (t >= T || (rows_ptr != nullptr && t >= __ldg(rows_ptr))) return;   // rows_ptr: packed row count
-    const __nv_bfloat16* row = x + (size_t)t * H;
-    float v[NV * 4];
+    const int t0 = (blockIdx.x * kRowWarps + (threadIdx.x >> 5)) * kLnRowsPerWarp;
+    int rows = T;
+    if (rows_ptr != nullptr) rows = min(rows, __ldg(rows_ptr));   // rows_ptr: packed row count
+    if (t0 >= rows) return;
+    uint2 raw[kLnRowsPerWarp][NV];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        const int col = (i * 32 + lane) * 4;
-        const uint2 a = __ldg(reinterpret_cast<const uint2*>(row + col));
-        v[i * 4 + 0] = bf16lo(a.x);
-        v[i * 4 + 1] = bf16hi(a.x);
-        v[i * 4 + 2] = bf16lo(a.y);
-        v[i * 4 + 3] = bf16hi(a.y);
+    for (int r = 0; r < kLnRowsPerWarp; ++r) {
+        const int t = min(t0 + r, rows - 1);   // clamp: tail rows are loaded twice, stored once
+        const __nv_bfloat16* row = x + (size_t)t * H;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) raw[r][i] = __ldg(reinterpret_cast<const uint2*>(row + (i * 32 + lane) * 4));
     }
-    ln_normalise_store<NV>(v, gamma, beta, eps, lane, out + (size_t)t * H);
+#pragma unroll
+    for (int r = 0; r < kLnRowsPerWarp; ++r) {
+        if (t0 + r >= rows) break;
+        float v[NV * 4];
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            v[i * 4 + 0] = bf16lo(raw[r][i].x);
+            v[i * 4 + 1] = bf16hi(raw[r][i].x);
+            v[i * 4 + 2] = bf16lo(raw[r][i].y);
+            v[i * 4 + 3] = bf16hi(raw[r][i].y);
+        }
+        ln_normalise_store<NV>(v, gamma, beta, eps, lane, out + (size_t)(t0 + r) * H);
+    }
 }
 
 // Masked mean-pool + L2 normalisation.  One CTA per sequence.  Thread (g, c) owns the 8-column
