@@ -61,6 +61,7 @@ typedef enum {
 #define RLX_FLAG_GEMM_SIMT 0x2u /* use the plain CUDA-core GEMM (bring-up / cross-check only)  */
 #define RLX_FLAG_KERNEL_EVENTS 0x4u /* record a CUDA event between kernels (see rlx_encoder_kernel_times) */
 #define RLX_FLAG_NO_PDL 0x10u   /* plain stream order between kernels (no programmatic dependent launch) */
+#define RLX_FLAG_ATTN_TCGEN05 0x20u /* packed attention on the tcgen05/TMEM kernel instead of the mma.sync one */
 #define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
 
 typedef struct {
@@ -295,6 +296,18 @@ rlx_status_t rlx_attention_bf16(const void *qkv_bf16, const int32_t *attention_m
 rlx_status_t rlx_attention_f32(const float *qkv_f32, const int32_t *attention_mask, int32_t batch,
                                int32_t seq, int32_t num_heads, int32_t head_dim, float *ctx_f32,
                                void *cuda_stream);
+
+/*
+ * The same attention on PACKED rows (what the forward runs after sequence packing): qkv holds
+ * `rows` rows of [q | k | v]; sequence b owns rows seq_start[b] .. seq_start[b] + seq_len[b], all
+ * valid, seq_len[b] <= max_len <= 512; ctx uses the same row numbering.  impl 0: tcgen05/TMEM
+ * kernel (TMA-fed, S and P in tensor memory, one thread per query row in the softmax);
+ * impl 1: warp-level mma.sync kernel.  Rows outside every sequence are not written.
+ */
+rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const int32_t *seq_start,
+                                       const int32_t *seq_len, int32_t batch, int32_t max_len,
+                                       int32_t num_heads, int32_t head_dim, void *ctx_bf16, int32_t impl,
+                                       int32_t *status, void *cuda_stream);
 
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
 rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,

@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     RlxError,
     attention_bf16,
     attention_f32,
+    attention_packed_bf16,
     embed_layernorm,
     gemm_bf16,
     layernorm,

@@ -24,6 +24,7 @@ FLAG_GEMM_SIMT = 0x2
 FLAG_KERNEL_EVENTS = 0x4
 FLAG_NO_PACK = 0x8
 FLAG_NO_PDL = 0x10
+FLAG_ATTN_TCGEN05 = 0x20
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20
@@ -32,7 +33,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_pool_l2norm",
 )
 
 
@@ -265,6 +266,17 @@ def attention_bf16(qkv, mask, num_heads: int, stream=None):
     ctx = torch.empty((B, S, H), dtype=torch.bfloat16, device=qkv.device)
     _check(_load().rlx_attention_bf16(_ptr(qkv), _ptr(mask), B, S, num_heads, H // num_heads, _ptr(ctx), _stream(stream)),
            "rlx_attention_bf16")
+    return ctx
+
+
+def attention_packed_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, impl: int = 0, status=None, stream=None):
+    """qkv: packed [rows, 3H] bf16; returns ctx [rows, H] (rows outside every sequence stay zero)."""
+    rows, H3 = qkv.shape
+    H = H3 // 3
+    ctx = torch.zeros((rows, H), dtype=torch.bfloat16, device=qkv.device)
+    _check(_load().rlx_attention_packed_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len,
+                                             num_heads, H // num_heads, _ptr(ctx), impl, _ptr(status), _stream(stream)),
+           "rlx_attention_packed_bf16")
     return ctx
 
 

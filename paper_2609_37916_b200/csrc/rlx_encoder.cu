@@ -12,6 +12,7 @@
 
 #include "../../include/rlx_encoder.h"
 #include "attention.cuh"
+#include "attention_tc.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
 #include "rowwise.cuh"
@@ -118,6 +119,10 @@ cudaError_t init_kernels_for_current_device() {
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tc::gemm_tcgen05_kernel<256, 0, 2>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs[dev] = n;
     }
+    if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tca::Smem<32>::BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tca::Smem<64>::BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)sizeof(rlx::AttSmem<32>))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -223,6 +228,29 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
         RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<32>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
     else if (d == 64)
         RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<64>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
+    else
+        return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+unsigned long long* g_attn_dbg = nullptr;   // experiments only
+// Packed-sequence attention on tcgen05 (the product path): qkv is the packed [rows, 3H] projection.
+rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_start, const int32_t* seq_len, int B,
+                                 int S, int h, int d, bf16* ctx, int32_t* status, cudaStream_t st) {
+    const int H = h * d;
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
+    CUtensorMap tq;
+    if (!make_tmap(&tq, qkv, (uint64_t)rows, (uint64_t)3 * H, rlx::tca::kBlockN, (uint32_t)d,
+                   d == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
+        return RLX_ERR_CUDA;
+    dim3 grid((S + rlx::tca::kBlockM - 1) / rlx::tca::kBlockM, h, B);
+    if (d == 32)
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, grid, rlx::tca::kThreads, rlx::tca::Smem<32>::BYTES, st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, status, g_attn_dbg));
+    else if (d == 64)
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, grid, rlx::tca::kThreads, rlx::tca::Smem<64>::BYTES, st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, status, g_attn_dbg));
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
@@ -447,7 +475,10 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     for (int l = 0; l < c.num_layers; ++l) {
         const rlx_layer_weights_t& lw = w->layers[l];
         RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, simt, status, st, rows));
-        RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
+        if (pack && (c.flags & RLX_FLAG_ATTN_TCGEN05))
+            RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx, status, st));
+        else
+            RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
         RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
         RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
         RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
@@ -739,6 +770,23 @@ rlx_status_t rlx_attention_bf16(const void* qkv, const int32_t* mask, int32_t B,
     return launch_attention_bf16((const bf16*)qkv, mask, nullptr, nullptr, B, S, h, d, (bf16*)ctx,
                                  static_cast<cudaStream_t>(stream));
 }
+
+rlx_status_t rlx_attention_packed_bf16(const void* qkv, int32_t rows, const int32_t* seq_start, const int32_t* seq_len,
+                                       int32_t B, int32_t max_len, int32_t h, int32_t d, void* ctx, int32_t impl,
+                                       int32_t* status, void* stream) {
+    if (!qkv || !seq_start || !seq_len || !ctx || B <= 0 || max_len <= 0 || h <= 0 || rows <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(qkv) || !aligned16(ctx)) return RLX_ERR_INVALID_ARG;
+    if ((d != 32 && d != 64) || max_len > 512 || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (impl == 0)
+        return launch_attention_tc((const bf16*)qkv, rows, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, status, st);
+    if (impl == 1)
+        return launch_attention_bf16((const bf16*)qkv, nullptr, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, st);
+    return RLX_ERR_INVALID_ARG;
+}
+
+void rlx_debug_set_attn_trace(void* p) { g_attn_dbg = static_cast<unsigned long long*>(p); }
 
 rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,
                                float* ctx, void* stream) {

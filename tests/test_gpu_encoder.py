@@ -62,12 +62,12 @@ def check(got, ref, lengths, tight=True):
 
 
 @pytest.mark.parametrize("name", ["c0", "c1", "c2"])
-@pytest.mark.parametrize("mode", ["graph", "eager", "padded", "simt_gemm", "host_io"])
+@pytest.mark.parametrize("mode", ["graph", "eager", "padded", "attn_tcgen05", "simt_gemm", "host_io"])
 def test_full_config_matches_oracle(rlx, name, mode):
     if mode == "simt_gemm" and name == "c2":
         pytest.skip("bring-up GEMM is covered on c0/c1")
     inp = make_inputs(CONFIGS[name])
-    flags = {"graph": 0, "eager": 1, "padded": 8, "simt_gemm": 1 | 2, "host_io": 0}[mode]
+    flags = {"graph": 0, "eager": 1, "padded": 8, "attn_tcgen05": 0x20, "simt_gemm": 1 | 2, "host_io": 0}[mode]
     got, status = run_gpu(rlx, inp, flags=flags, host_io=(mode == "host_io"))
     assert status == 0
     ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
@@ -81,12 +81,13 @@ def test_c0_matches_stored_golden(rlx):
     check(got, want.reshape(1, -1), inp.lengths)
 
 
+@pytest.mark.parametrize("flags", [0, 0x20], ids=["default", "attn_tcgen05"])
 @pytest.mark.parametrize("name,sample", [("c3", [0, 1, 100, 255]), ("c4", [0, 63])])
-def test_large_config_sampled_sequences_match_oracle(rlx, name, sample):
+def test_large_config_sampled_sequences_match_oracle(rlx, name, sample, flags):
     """Full-size run in the benchmark's launch configuration; the oracle recomputes a sample of the
     sequences one by one (sequences are independent, so a batch-1 oracle call is the same function)."""
     inp = make_inputs(CONFIGS[name])
-    got, status = run_gpu(rlx, inp)
+    got, status = run_gpu(rlx, inp, flags=flags)
     assert status == 0
     assert np.all(np.isfinite(got))
     assert np.allclose(np.linalg.norm(got, axis=1), 1.0, atol=1e-5)

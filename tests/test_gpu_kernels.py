@@ -234,6 +234,37 @@ def test_attention_bf16_mode(rlx, case, variant):
     assert np.all(np.isfinite(got))
 
 
+PACKED_CASES = [([11], 12, 32), ([128], 2, 32), ([5, 128, 64, 1, 129, 200], 3, 32), ([512, 17, 300], 2, 64),
+                ([256, 255, 257, 16, 15], 12, 32), ([130, 1, 511], 1, 64)]
+
+
+@pytest.mark.parametrize("impl", [0, 1], ids=["tcgen05", "mma_sync"])
+@pytest.mark.parametrize("lengths,h,d", PACKED_CASES)
+@pytest.mark.parametrize("gain", [1.0, 6.0], ids=["plain", "peaky"])
+def test_attention_packed_matches_oracle(rlx, lengths, h, d, gain, impl):
+    """Packed rows (what the forward runs): every sequence is a dense block of valid rows.  The oracle
+    sees each sequence as a batch-1 problem with an all-ones mask."""
+    rng = np.random.default_rng(sum(lengths) + h + d)
+    H = h * d
+    total = sum(lengths)
+    rows = total + 7                                  # a few rows past the last sequence
+    qkv = rand_bf16(rng, (rows, 3 * H))
+    qkv[:, :H] = round_to_bf16(qkv[:, :H] * np.float32(gain))
+    qkv[total:] = np.float32("nan")                   # junk after the last sequence must not leak in
+    start = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.attention_packed_bf16(bf16_dev(qkv), i32_dev(start[:-1]), i32_dev(np.array(lengths)),
+                                            max(lengths), h, impl=impl, status=status))
+    assert int(status.item()) == 0
+    vmax = np.abs(qkv[:total, 2 * H:]).max()
+    for b, n in enumerate(lengths):
+        seq = qkv[start[b]:start[b] + n].astype(np.float64)[None]
+        ref = oracle.attention(seq, np.ones((1, n), np.int32), h)[0]
+        err = np.abs(got[start[b]:start[b] + n] - ref).max()
+        assert np.isfinite(err) and err <= 2 * BF16_U * (vmax + np.abs(ref).max()), (b, n, err)
+    assert np.array_equal(got[total:], np.zeros((rows - total, H)))
+
+
 def test_attention_adversarial_logits(rlx):
     """One dominant key (+30), all-equal logits, and logits so negative that exp underflows."""
     h, d, S = 1, 32, 64
