@@ -166,10 +166,11 @@ def workload_config(name: str, extra=None):
 
 
 # ---------------------------------------------------------------------------- roofline bookkeeping
-def kernel_classes(num_layers: int):
+def kernel_classes(num_layers: int, fused_ln: bool):
+    per_layer = [k for k in KERNEL_CLASSES if not (fused_ln and k in ("ln1", "ln2"))]
     names = ["pack", "embed_ln"]
     for _ in range(num_layers):
-        names += list(KERNEL_CLASSES)
+        names += per_layer
     names.append("pool_l2")
     return names
 
@@ -295,11 +296,13 @@ def run_ours(args):
     barrier()
 
     # ---- timed region 3: per-kernel device times from event nodes inside the replayed graph ----
-    names = kernel_classes(cfg.num_layers)
+    n_kernels = enc.kernels_per_forward(B, S)
+    names = kernel_classes(cfg.num_layers, fused_ln=(n_kernels == 3 + 5 * cfg.num_layers))
+    assert len(names) == n_kernels
     per_class = {}
     for _ in range(args.steps):
         step_device(enc_t, ws_t)
-        times = enc_t.kernel_times()
+        times = enc_t.kernel_times(B, S)
         for n, t in zip(names, times):
             per_class.setdefault(n, []).append(t)
     barrier()
@@ -359,7 +362,7 @@ def run_ours(args):
             "e2e": {"value": seqs * args.steps / (e2e_total / 1e3), "unit": "sequences/s", "p50_ms": e2e_p50,
                     "h2d_bytes_per_step": 2 * B * S * 4, "d2h_bytes_per_step": B * H * 4,
                     "timing": "host wall clock around rlx_encoder_forward_host (copies + forward + sync)"},
-            "gpu_launches": args.steps * enc.kernels_per_forward(),
+            "gpu_launches": args.steps * n_kernels,
             "clocks": sampler.summary(),
             "roofline": roofline,
             "kernels": ktab,

@@ -14,6 +14,7 @@ from .binding import (  # noqa: F401
     attention_packed_bf16,
     embed_layernorm,
     gemm_bf16,
+    gemm_residual_layernorm_bf16,
     layernorm,
     pack_sequences,
     lib_path,

@@ -25,6 +25,7 @@ FLAG_KERNEL_EVENTS = 0x4
 FLAG_NO_PACK = 0x8
 FLAG_NO_PDL = 0x10
 FLAG_ATTN_TCGEN05 = 0x20
+FLAG_FUSED_LN = 0x40
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20
@@ -32,7 +33,7 @@ STATIC_WORKSPACE_BYTES = 16 << 20
 EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
-    "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_attention_bf16",
+    "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
     "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_pool_l2norm",
 )
 
@@ -167,8 +168,8 @@ class Encoder:
     def workspace_bytes(self, batch: int, seq: int) -> int:
         return int(_load().rlx_encoder_workspace_bytes(self._h, batch, seq))
 
-    def kernels_per_forward(self) -> int:
-        return int(_load().rlx_encoder_kernels_per_forward(self._h))
+    def kernels_per_forward(self, batch: int, seq: int) -> int:
+        return int(_load().rlx_encoder_kernels_per_forward(self._h, batch, seq))
 
     def alloc_workspace(self, batch: int, seq: int, device="cuda") -> torch.Tensor:
         n = self.workspace_bytes(batch, seq)
@@ -210,9 +211,9 @@ class Encoder:
                "rlx_encoder_forward_static")
         return out
 
-    def kernel_times(self) -> List[float]:
+    def kernel_times(self, batch: int, seq: int) -> List[float]:
         """Milliseconds per kernel of the last forward (encoder created with FLAG_KERNEL_EVENTS)."""
-        n = self.kernels_per_forward()
+        n = self.kernels_per_forward(batch, seq)
         buf = (C.c_float * n)()
         _check(_load().rlx_encoder_kernel_times(self._h, buf, n), "rlx_encoder_kernel_times")
         return list(buf)
@@ -257,6 +258,16 @@ def gemm_bf16(a, w, bias, residual=None, epilogue: int = EPI_BIAS, impl: int = G
     out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
     _check(_load().rlx_gemm_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(residual), epilogue, M, N, K, _ptr(out), impl,
                                  _ptr(status), _stream(stream)), "rlx_gemm_bf16")
+    return out
+
+
+def gemm_residual_layernorm_bf16(a, w, bias, residual, gamma, beta, eps: float, status=None, stream=None):
+    M, K = a.shape
+    N = w.shape[0]
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
+    _check(_load().rlx_gemm_residual_layernorm_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(residual), _ptr(gamma),
+                                                    _ptr(beta), C.c_float(eps), M, N, K, _ptr(out), _ptr(status),
+                                                    _stream(stream)), "rlx_gemm_residual_layernorm_bf16")
     return out
 
 

@@ -1,16 +1,18 @@
 // bf16 "Linear" GEMM for sm_100a: out[M,N] = epilogue(A[M,K] * W[N,K]^T + bias).
 //
-// Structure (one persistent CTA per SM, 320 threads):
+// Structure (one persistent CTA per SM, 320 to 576 threads):
 //   warp 0      TMA producer: streams 128x64 A tiles and BLOCK_N x 64 W tiles (128-byte swizzle)
 //               through a STAGES-deep shared-memory ring guarded by full/empty mbarriers
 //   warp 1      allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N=BLOCK_N,
 //               K=16 per instruction) into one of two fp32 accumulator buffers in TMEM and
 //               commits stage releases / accumulator-ready signals to mbarriers
-//   warps 2..9  epilogue: each warp owns one TMEM lane quadrant (32 rows) and one half of the tile's
-//               columns; per 32-column chunk it tcgen05.ld's the accumulator (the next chunk's load
+//   warps 2..   epilogue (8 to 16 warps): each warp owns one TMEM lane quadrant (32 rows) and one 64-column
+//               slab of the tile; per 32-column chunk it tcgen05.ld's the accumulator (the next chunk's load
 //               is in flight while this one is processed), adds bias, applies GELU or adds the
-//               residual in fp32, rounds to bf16, writes the chunk to a swizzled shared-memory
-//               staging buffer and hands it to a TMA store (rows past M are clipped by the copy).
+//               residual in fp32, rounds to bf16, transposes the chunk through a swizzled
+//               shared-memory buffer and stores it with 16-byte stores that cover whole 64-byte row
+//               segments (a TMA store per chunk was tried: waiting for it to drain its staging buffer
+//               stalled the warp for about a microsecond per chunk).
 //               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop;
 //               a warp releases its accumulator as soon as its last tcgen05.ld has landed.
 // Two instantiations per tile shape: CG = 1 (one CTA per 128 x BLOCK_N tile) and CG = 2, where a
@@ -32,10 +34,7 @@ namespace tc {
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;   // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int kThreads = 320;
-constexpr int kEpiWarps = 8;
 constexpr int kStageBufBytes = 32 * 32 * 2;          // one 32-row x 32-column bf16 chunk
-constexpr int kStagingBytes = kEpiWarps * 2 * kStageBufBytes;  // two buffers per epilogue warp
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
 
 template <int BLOCK_N, int CG = 1>
@@ -44,12 +43,19 @@ struct Cfg {
     static constexpr int B_ROWS = BLOCK_N / CG;                  // W rows this CTA loads per k-block
     static constexpr int B_BYTES = B_ROWS * BLOCK_K * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int RING_BUDGET = 222 * 1024 - kStagingBytes;
+    // epilogue: EPI_SPLIT warps share each 32-row TMEM quadrant, each taking a 64-column slab (32 for
+    // the narrowest tile); many short per-warp chains hide the TMEM / memory latencies of the epilogue
+    static constexpr int EPI_SPLIT = BLOCK_N >= 192 ? BLOCK_N / 64 : 2;
+    static constexpr int EPI_WARPS = 4 * EPI_SPLIT;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static constexpr int SLAB = BLOCK_N / EPI_SPLIT;
+    static constexpr int STAGING_BYTES = EPI_WARPS * kStageBufBytes;   // one transpose buffer per epilogue warp
+    static constexpr int RING_BUDGET = 222 * 1024 - STAGING_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
     static constexpr int TMEM_COLS = (2 * BLOCK_N <= 32) ? 32 : (2 * BLOCK_N <= 64) ? 64 : (2 * BLOCK_N <= 128) ? 128
                                      : (2 * BLOCK_N <= 256) ? 256 : 512;
     static constexpr int BAR_BYTES = 256;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + kStagingBytes + BAR_BYTES + 1024;  // +1024: manual alignment
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;  // +1024: manual alignment
     static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128 / M=256");
     static_assert(CG == 1 || CG == 2, "cta_group");
     static_assert(B_BYTES % 1024 == 0, "stage tiles must stay 1024-byte aligned");
@@ -131,6 +137,11 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -229,6 +240,7 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 struct Params {
     const float* bias;               // [N]
     const __nv_bfloat16* residual;   // [M,N] or null
+    __nv_bfloat16* out;              // [M,N]
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
     const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
@@ -236,9 +248,8 @@ struct Params {
 };
 
 template <int BLOCK_N, int EPI, int CG>
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                    const __grid_constant__ CUtensorMap tmap_out, const Params p) {
+__global__ void __launch_bounds__((Cfg<BLOCK_N, CG>::THREADS), 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
     using C = Cfg<BLOCK_N, CG>;
     constexpr int TILE_M = BLOCK_M * CG;   // rows of one output tile (per CTA pair when CG = 2)
     extern __shared__ unsigned char smem_raw[];
@@ -247,12 +258,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - raw);
     const uint32_t staging = base + C::STAGES * C::STAGE_BYTES;
-    const uint32_t bars = staging + kStagingBytes;
+    const uint32_t bars = staging + C::STAGING_BYTES;
     // barrier block: full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem slot, abort flag
     const uint32_t full_bar = bars, empty_bar = bars + 8 * C::STAGES;
     const uint32_t tfull_bar = bars + 16 * C::STAGES, tempty_bar = tfull_bar + 16;
     uint32_t* tmem_slot =
-        reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + kStagingBytes + 16 * C::STAGES + 32);
+        reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + C::STAGING_BYTES + 16 * C::STAGES + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -266,13 +277,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(tfull_bar + 8 * i, 1);
-            mbar_init(tempty_bar + 8 * i, kEpiWarps * CG);   // the leader's barrier collects both CTAs' warps
+            mbar_init(tempty_bar + 8 * i, C::EPI_WARPS * CG);   // the leader's barrier collects both CTAs' warps
         }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_a);
         prefetch_tmap(&tmap_b);
-        prefetch_tmap(&tmap_out);
     }
     if (warp == 1) {
         tmem_alloc<CG>(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -352,16 +362,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        constexpr int HALF_N = BLOCK_N / 2;
+        constexpr int HALF_N = C::SLAB;       // columns of the tile this warp handles
         constexpr int NC = HALF_N / 32;       // 32-column chunks per warp and tile
         const int ew = warp - 2;
         const int quad = warp & 3;            // TMEM lane quadrant this warp may read
-        const int half = ew >> 2;             // which half of the tile's columns
-        const uint32_t stg = staging + ew * 2 * kStageBufBytes;
+        const int half = ew >> 2;             // which column slab of the tile
+        const uint32_t stg = staging + ew * kStageBufBytes;
         const uint32_t row_off = lane * 64;             // 64-byte rows in the staging chunk
         const uint32_t swz = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte chunk index ^ (row/2 % 4)
         int it = 0;
-        uint32_t nstore = 0;
         bool ok = true;
         for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
             const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
@@ -437,10 +446,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                         v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
                     }
                 }
-                // the staging buffer used two chunks ago must have been read out by its TMA store
-                const uint32_t buf = stg + (nstore & 1) * kStageBufBytes;
-                if (lane == 0) bulk_wait_read<1>();
-                __syncwarp();
+                // transpose through this warp's staging buffer so that every store instruction writes
+                // whole 64-byte row segments (8 rows x 64 B per instruction, full sectors)
+                __syncwarp();   // the previous chunk has been read out of the buffer
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     uint4 q;
@@ -448,18 +456,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
                     q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
                     q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-                    st_shared_v4(buf + row_off + (((uint32_t)i ^ swz) << 4), q);
+                    st_shared_v4(stg + row_off + (((uint32_t)i ^ swz) << 4), q);
                 }
-                if (!(p.debug & 4)) fence_proxy_async();   // make the generic-proxy writes visible to the TMA engine
                 __syncwarp();
-                if (lane == 0) {
-                    if (m_row0 < M && !(p.debug & 2)) tma_store_2d(&tmap_out, n0 + c * 32, m_row0, buf);  // never start past the extent
-                    bulk_commit();
+                if (!(p.debug & 2)) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int rr = i * 8 + (lane >> 2), cc = lane & 3;
+                        const uint4 q = ld_shared_v4(stg + rr * 64 + (((uint32_t)cc ^ (uint32_t)((rr >> 1) & 3)) << 4));
+                        if (m_row0 + rr < M)
+                            *reinterpret_cast<uint4*>(p.out + (size_t)(m_row0 + rr) * p.N + n0 + c * 32 + cc * 8) = q;
+                    }
                 }
-                ++nstore;
             }
         }
-        if (lane == 0) bulk_wait<0>();   // all of this warp's stores have completed
     }
 
     // ---------------------------------------------------------------- teardown

@@ -15,6 +15,7 @@
 #include "attention_tc.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
+#include "gemm_ln_tcgen05.cuh"
 #include "rowwise.cuh"
 
 namespace {
@@ -100,13 +101,19 @@ cudaError_t init_kernels_for_current_device() {
     if ((e = set_gemm_attr_all<128>()) != cudaSuccess) return e;
     if ((e = set_gemm_attr_all<192>()) != cudaSuccess) return e;
     if ((e = set_gemm_attr_all<256>()) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcln::gemm_ln_tcgen05_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcln::Cfg<128>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcln::gemm_ln_tcgen05_kernel<192>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcln::Cfg<192>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcln::gemm_ln_tcgen05_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcln::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<128, 2>())) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<192, 2>())) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<256, 2>())) != cudaSuccess) return e;
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2 * rlx::kNumSMs);
-        cfg.blockDim = dim3(rlx::tc::kThreads);
+        cfg.blockDim = dim3(rlx::tc::Cfg<256, 2>::THREADS);
         cfg.dynamicSmemBytes = rlx::tc::Cfg<256, 2>::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -132,6 +139,7 @@ cudaError_t init_kernels_for_current_device() {
 }
 
 // ------------------------------------------------------------------ launchers
+unsigned long long* g_attn_dbg = nullptr;   // experiments only: device buffer for in-kernel phase timestamps
 // When set, kernels are launched with the programmatic-stream-serialization attribute so that each
 // kernel's prologue overlaps its predecessor's tail (the kernels call griddepcontrol.wait before
 // they read anything a predecessor wrote).  Set by enqueue_forward around its launches.
@@ -234,7 +242,6 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     return RLX_OK;
 }
 
-unsigned long long* g_attn_dbg = nullptr;   // experiments only
 // Packed-sequence attention on tcgen05 (the product path): qkv is the packed [rows, 3H] projection.
 rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_start, const int32_t* seq_len, int B,
                                  int S, int h, int d, bf16* ctx, int32_t* status, cudaStream_t st) {
@@ -291,8 +298,8 @@ TileChoice pick_tile(int M, int N, int K, int want_cg = 0) {
 }
 
 template <int BN, int CG>
-rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
-                               const rlx::tc::Params& p, int epi, cudaStream_t st) {
+rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const rlx::tc::Params& p, int epi,
+                               cudaStream_t st) {
     const int tile_m = rlx::tc::BLOCK_M * CG;
     const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN);
     int dev = 0;
@@ -305,9 +312,9 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
         ~ClusterScope() { g_cluster_x = 1; }
     } scope(CG);
     switch (epi) {
-        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
-        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
-        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::kThreads, smem, st, ta, tb, to, p)); break;
+        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
@@ -331,27 +338,47 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     const TileChoice tc = pick_tile(M, N, K, want_cg);
     const int bn = tc.bn;
     if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
-    CUtensorMap ta, tb, to;
+    CUtensorMap ta, tb;
     if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / tc.cg))) return RLX_ERR_CUDA;
-    if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
     static const int dbg = getenv("RLX_GEMM_DEBUG") ? atoi(getenv("RLX_GEMM_DEBUG")) : 0;
-    rlx::tc::Params p{bias, residual, M, N, K, status, m_ptr, dbg};
+    rlx::tc::Params p{bias, residual, out, M, N, K, status, m_ptr, dbg};
     if (tc.cg == 2) {
         switch (bn) {
-            case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, to, p, epi, st);
-            case 192: return launch_gemm_tc_bn<192, 2>(ta, tb, to, p, epi, st);
-            case 256: return launch_gemm_tc_bn<256, 2>(ta, tb, to, p, epi, st);
+            case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, p, epi, st);
+            case 192: return launch_gemm_tc_bn<192, 2>(ta, tb, p, epi, st);
+            case 256: return launch_gemm_tc_bn<256, 2>(ta, tb, p, epi, st);
         }
         return RLX_ERR_UNSUPPORTED;
     }
     switch (bn) {
-        case 64: return launch_gemm_tc_bn<64, 1>(ta, tb, to, p, epi, st);
-        case 128: return launch_gemm_tc_bn<128, 1>(ta, tb, to, p, epi, st);
-        case 192: return launch_gemm_tc_bn<192, 1>(ta, tb, to, p, epi, st);
-        case 256: return launch_gemm_tc_bn<256, 1>(ta, tb, to, p, epi, st);
+        case 64: return launch_gemm_tc_bn<64, 1>(ta, tb, p, epi, st);
+        case 128: return launch_gemm_tc_bn<128, 1>(ta, tb, p, epi, st);
+        case 192: return launch_gemm_tc_bn<192, 1>(ta, tb, p, epi, st);
+        case 256: return launch_gemm_tc_bn<256, 1>(ta, tb, p, epi, st);
     }
     return RLX_ERR_UNSUPPORTED;
+}
+
+// out = LN(A W^T + bias + residual): whole rows per CTA (N = 256, 384 or 512).
+rlx_status_t launch_gemm_ln(const bf16* A, const bf16* W, const float* bias, const bf16* residual, const float* gamma,
+                            const float* beta, float eps, int M, int N, int K, bf16* out, int32_t* status,
+                            cudaStream_t st, const int32_t* m_ptr = nullptr) {
+    if ((N != 256 && N != 384 && N != 512) || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
+    const int nh = N / 2;
+    CUtensorMap ta, tb;
+    if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
+    if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)nh)) return RLX_ERR_CUDA;
+    rlx::tcln::Params p{bias, residual, gamma, beta, out, eps, M, K, status, m_ptr, g_attn_dbg};
+    const int tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
+    const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
+    switch (nh) {
+        case 128: RLX_CUDA_TRY(launch_ex(rlx::tcln::gemm_ln_tcgen05_kernel<128>, grid, rlx::tcln::kThreads, rlx::tcln::Cfg<128>::SMEM_BYTES, st, ta, tb, p)); break;
+        case 192: RLX_CUDA_TRY(launch_ex(rlx::tcln::gemm_ln_tcgen05_kernel<192>, grid, rlx::tcln::kThreads, rlx::tcln::Cfg<192>::SMEM_BYTES, st, ta, tb, p)); break;
+        case 256: RLX_CUDA_TRY(launch_ex(rlx::tcln::gemm_ln_tcgen05_kernel<256>, grid, rlx::tcln::kThreads, rlx::tcln::Cfg<256>::SMEM_BYTES, st, ta, tb, p)); break;
+    }
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
 }
 
 // ------------------------------------------------------------------ workspace arena
@@ -386,6 +413,21 @@ Arena plan_arena(int B, int S, int H, int F) {
     return a;
 }
 
+// With RLX_FLAG_FUSED_LN the out-projection and FFN-down GEMMs absorb the residual LayerNorm when a
+// whole row fits in tensor memory and there are enough 128-row tiles to give every SM one (whole-row
+// tiles cannot be split across SMs, so small batches keep the separate GEMM + LayerNorm kernels).
+// Opt-in: measured on the 256x256 batch it is on par with the separate kernels, not ahead of them.
+bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
+    if ((c.flags & RLX_FLAG_GEMM_SIMT) || !(c.flags & RLX_FLAG_FUSED_LN)) return false;
+    if (c.hidden != 256 && c.hidden != 384 && c.hidden != 512) return false;
+    return (long long)B * S >= 128ll * rlx::kNumSMs;
+}
+
+int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
+    const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
+    return 2 + (uses_fused_ln(c, B, S) ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
+}
+
 struct GraphEntry {
     int B, S;
     const void *ids, *mask, *out, *ws;
@@ -401,6 +443,7 @@ struct rlx_encoder {
     rlx_encoder_weights_t weights;
     bool have_weights = false;
     std::vector<GraphEntry> graphs;
+    int last_kernels = 0;                   // kernels of the most recent forward (for kernel_times)
     std::vector<cudaEvent_t> events;        // RLX_FLAG_KERNEL_EVENTS: one before the first kernel, one after each
     cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
                                             // legacy default stream, which cannot be captured)
@@ -470,6 +513,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
     }
     const int32_t* rows = pk.total();
+    const bool fuse_ln = uses_fused_ln(c, B, S);
     RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
                             w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
     for (int l = 0; l < c.num_layers; ++l) {
@@ -479,11 +523,20 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
             RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx, status, st));
         else
             RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
-        RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
-        RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
+        if (fuse_ln) {
+            RLX_TRY(launch_gemm_ln(ctx, (const bf16*)lw.wo, lw.bo, x, lw.ln1_g, lw.ln1_b, c.ln_eps, T, H, H, x1, status, st, rows));
+        } else {
+            RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
+            RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
+        }
         RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
-        RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st, rows));
-        RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
+        if (fuse_ln) {
+            // x1 is both the residual and (after this kernel) dead; the result goes to x
+            RLX_TRY(launch_gemm_ln(g, (const bf16*)lw.w2, lw.b2, x1, lw.ln2_g, lw.ln2_b, c.ln_eps, T, H, F, x, status, st, rows));
+        } else {
+            RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st, rows));
+            RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
+        }
     }
     RLX_TRY(launch_pool(x, mask, B, S, H, out, st, pk));
 #undef RLX_TRY
@@ -515,9 +568,11 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
     RLX_CUDA_TRY(init_kernels_for_current_device());
     if ((e->cfg.flags & RLX_FLAG_KERNEL_EVENTS) && e->events.empty()) {
-        e->events.resize((size_t)rlx_encoder_kernels_per_forward(e) + 1);
+        e->events.resize(4 + 7 * (size_t)e->cfg.num_layers);   // upper bound: one per kernel + 1
+        e->last_kernels = 0;
         for (auto& evt : e->events) RLX_CUDA_TRY(cudaEventCreate(&evt));
     }
+    e->last_kernels = kernels_in_forward(e->cfg, B, S);
     if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);
 
     if (!same_weights(e, w)) {
@@ -594,10 +649,9 @@ size_t rlx_encoder_workspace_bytes(const rlx_encoder_t* e, int32_t batch, int32_
     return plan_arena(batch, seq, e->cfg.hidden, e->cfg.ffn).total;
 }
 
-int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e) {
-    if (!e) return 0;
-    const bool pack = !(e->cfg.flags & RLX_FLAG_NO_PACK) && !(e->cfg.flags & RLX_FLAG_GEMM_SIMT);
-    return 2 + 7 * e->cfg.num_layers + (pack ? 1 : 0);
+int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e, int32_t batch, int32_t seq) {
+    if (!e || batch <= 0 || seq <= 0) return 0;
+    return kernels_in_forward(e->cfg, batch, seq);
 }
 
 rlx_status_t rlx_encoder_forward(rlx_encoder_t* e, const int32_t* ids, const int32_t* mask, int32_t B, int32_t S,
@@ -641,9 +695,10 @@ rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t* e, void* ws, void* st
 }
 
 rlx_status_t rlx_encoder_kernel_times(rlx_encoder_t* e, float* ms_host, int32_t count) {
-    if (!e || !ms_host || count != rlx_encoder_kernels_per_forward(e)) return RLX_ERR_INVALID_ARG;
-    if (e->events.size() != (size_t)count + 1) return RLX_ERR_UNSUPPORTED;
-    RLX_CUDA_TRY(cudaEventSynchronize(e->events.back()));
+    if (!e || !ms_host) return RLX_ERR_INVALID_ARG;
+    if (e->events.empty() || e->last_kernels <= 0) return RLX_ERR_UNSUPPORTED;
+    if (count != e->last_kernels) return RLX_ERR_INVALID_ARG;
+    RLX_CUDA_TRY(cudaEventSynchronize(e->events[count]));
     for (int i = 0; i < count; ++i) RLX_CUDA_TRY(cudaEventElapsedTime(&ms_host[i], e->events[i], e->events[i + 1]));
     return RLX_OK;
 }
@@ -759,6 +814,18 @@ rlx_status_t rlx_gemm_bf16(const void* A, const void* W, const float* bias, cons
     const int want_cg = impl == RLX_GEMM_TCGEN05_PAIR ? 2 : impl == RLX_GEMM_TCGEN05_SINGLE ? 1 : 0;
     return launch_gemm((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, (int)epi, M, N, K, (bf16*)out,
                        impl == RLX_GEMM_SIMT, status, static_cast<cudaStream_t>(stream), nullptr, want_cg);
+}
+
+rlx_status_t rlx_gemm_residual_layernorm_bf16(const void* A, const void* W, const float* bias, const void* residual,
+                                              const float* gamma, const float* beta, float eps, int32_t M, int32_t N,
+                                              int32_t K, void* out, int32_t* status, void* stream) {
+    if (!A || !W || !bias || !residual || !gamma || !beta || !out || M <= 0 || N <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(W) || !aligned16(bias) || !aligned16(residual) || !aligned16(gamma) ||
+        !aligned16(beta) || !aligned16(out))
+        return RLX_ERR_INVALID_ARG;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return launch_gemm_ln((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, gamma, beta, eps, M, N, K,
+                          (bf16*)out, status, static_cast<cudaStream_t>(stream));
 }
 
 rlx_status_t rlx_attention_bf16(const void* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,

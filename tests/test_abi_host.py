@@ -42,7 +42,7 @@ def _cfg(**kw):
 
 def test_create_validates_shapes(lib):
     enc = binding.Encoder(**_cfg())
-    assert enc.kernels_per_forward() == 3 + 7 * 6   # packing + embed + 7 per layer + pool
+    assert enc.kernels_per_forward(32, 128) == 3 + 7 * 6   # packing + embed + 7 per layer + pool
     enc.close()
     for bad, status in [
         (dict(hidden=400, num_heads=10), 2),    # H % 128
@@ -56,6 +56,20 @@ def test_create_validates_shapes(lib):
         with pytest.raises(binding.RlxError) as ei:
             binding.Encoder(**_cfg(**bad))
         assert ei.value.status == status, bad
+
+
+def test_kernel_count_drops_when_layernorm_is_fused(lib):
+    enc = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_FUSED_LN))
+    assert enc.kernels_per_forward(256, 256) == 3 + 5 * 6     # enough 128-row tiles for every SM: LN fused
+    assert enc.kernels_per_forward(32, 128) == 3 + 7 * 6
+    enc.close()
+    plain = binding.Encoder(**_cfg(max_batch=256, max_seq=256))
+    assert plain.kernels_per_forward(256, 256) == 3 + 7 * 6
+    plain.close()
+    big = binding.Encoder(**_cfg(hidden=768, num_heads=12, ffn=3072, max_batch=64, max_seq=512,
+                                 flags=binding.FLAG_FUSED_LN))
+    assert big.kernels_per_forward(64, 512) == 3 + 7 * 6      # a 768-wide row does not fit in tensor memory
+    big.close()
 
 
 def test_create_rejects_wrong_struct_size_and_null(lib):

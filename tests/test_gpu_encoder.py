@@ -81,7 +81,7 @@ def test_c0_matches_stored_golden(rlx):
     check(got, want.reshape(1, -1), inp.lengths)
 
 
-@pytest.mark.parametrize("flags", [0, 0x20], ids=["default", "attn_tcgen05"])
+@pytest.mark.parametrize("flags", [0, 0x20, 0x40], ids=["default", "attn_tcgen05", "fused_ln"])
 @pytest.mark.parametrize("name,sample", [("c3", [0, 1, 100, 255]), ("c4", [0, 63])])
 def test_large_config_sampled_sequences_match_oracle(rlx, name, sample, flags):
     """Full-size run in the benchmark's launch configuration; the oracle recomputes a sample of the

@@ -173,6 +173,38 @@ def test_gemm_matches_oracle_linear(rlx, shape, epi, impl):
     assert_close_bf16_out(got, ref, extra_abs=K * 2.0 ** -24 * 0.2)
 
 
+@pytest.mark.parametrize("shape", [(128, 384, 384), (300, 384, 1536), (1000, 256, 320), (129, 512, 512),
+                                   (20000, 384, 384), (19000, 384, 1536)])
+def test_gemm_residual_layernorm_fused(rlx, shape):
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    a = rand_bf16(rng, (M, K))
+    w = rand_bf16(rng, (N, K), 0.05)
+    bias = (0.1 * rng.standard_normal(N)).astype(np.float32)
+    res = rand_bf16(rng, (M, N))
+    g = (1 + 0.1 * rng.standard_normal(N)).astype(np.float32)
+    b = (0.1 * rng.standard_normal(N)).astype(np.float32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.gemm_residual_layernorm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(bias), bf16_dev(res), f32_dev(g),
+                                                   f32_dev(b), 1e-12, status=status))
+    assert int(status.item()) == 0
+    ref = oracle.layernorm(oracle.linear(a.astype(np.float64), w, bias) + res.astype(np.float64), g, b, 1e-12)
+    # the pre-LayerNorm sum stays in fp32 here (no bf16 round trip), so the plain bf16-output bound holds
+    assert_close_bf16_out(got, ref, extra_abs=K * 2.0 ** -24 * 0.5)
+
+
+def test_gemm_residual_layernorm_constant_rows_give_beta(rlx):
+    """Zero weights, zero bias and a constant residual row: LayerNorm of a constant row is exactly beta."""
+    M, N, K = 200, 384, 384
+    a = np.ones((M, K), np.float32)
+    w = np.zeros((N, K), np.float32)
+    res = np.full((M, N), 1.5, np.float32)
+    beta = round_to_bf16(np.linspace(-1, 1, N).astype(np.float32))
+    got = to_np64(rlx.gemm_residual_layernorm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(np.zeros(N)), bf16_dev(res),
+                                                   f32_dev(np.ones(N)), f32_dev(beta), 1e-12))
+    assert np.array_equal(got, np.broadcast_to(beta.astype(np.float64), (M, N)))
+
+
 # ------------------------------------------------------------------ attention
 def _qkv_case(seed, B, S, h, d, gain=1.0, holes=0.0):
     rng = np.random.default_rng(seed)
