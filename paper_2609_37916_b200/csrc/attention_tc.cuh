@@ -1,7 +1,7 @@
 // Packed-sequence attention on the 5th-generation tensor cores (tcgen05 + TMEM), head_dim 32 or 64,
 // up to 512 keys per sequence.  One CTA = 128 query rows of one (sequence, head):
 //
-//   warp 0 (1 lane)   TMA: Q tile and all K / V blocks of the sequence (128 keys each) straight out
+//   warp 0 (1 lane)   TMA: Q tile and all K / V blocks of the sequence (64 keys each) straight out
 //                     of the packed [rows, 3H] projection, one mbarrier per block
 //   warp 1 (1 lane)   MMA issue:  S = Q K^T  (M=128, N=keys, K=d; both operands K-major)
 //                                 O += P V    (M=128, N=d, K=keys; P read from TMEM, V MN-major)
@@ -12,7 +12,10 @@
 //                     then O / sum -> bf16 -> global.
 // Two passes over S (the QK^T product is simply issued twice when there is more than one key block)
 // mean the final row max is known before any exponential is taken: no running rescale of O.
-// TMEM columns per CTA: S [0,128), P [128,192), O [192,192+d)  (256 allocated, two CTAs fit per SM).
+// Keys come in blocks of 64; P overwrites S in place (chunk c of P lands in columns that chunk <= c
+// of S occupied), so a CTA needs only 128 TMEM columns (S/P [0,64), O [64,64+d)) and four CTAs share
+// an SM: each CTA is a chain of short dependent steps, and it is the number of chains in flight
+// that fills the machine.
 // All mbarrier waits are bounded; on expiry the CTA sets the status bit and leaves.
 #pragma once
 #include <cuda.h>
@@ -26,17 +29,19 @@ using namespace rlx::tc;
 
 constexpr int kThreads = 192;
 constexpr int kBlockM = 128;   // query rows per CTA
-constexpr int kBlockN = 128;   // keys per block
-constexpr int kMaxBlocks = 4;  // 512 keys
-constexpr int kTmemCols = 256;
-constexpr int kColS = 0, kColP = 128, kColO = 192;
+constexpr int kBlockN = 64;    // keys per block
+constexpr int kMaxBlocks = 8;  // 512 keys
+constexpr int kTmemCols = 128; // four CTAs per SM: the kernel is a chain of short dependent steps, so
+                               // throughput comes from many CTAs in flight, not from a long one
+constexpr int kColS = 0, kColP = 0, kColO = 64;   // P (bf16) overwrites S in place, chunk by chunk
 
 template <int D>
 struct Smem {
     static constexpr int ROW_BYTES = D * 2;                  // 64 (64-byte swizzle) or 128 (128-byte swizzle)
-    static constexpr int TILE_BYTES = kBlockN * ROW_BYTES;   // one 128-row tile of Q, K or V
-    static constexpr int BAR_OFFSET = (1 + 2 * kMaxBlocks) * TILE_BYTES;
-    static constexpr int BYTES = BAR_OFFSET + 256 + 1024;    // + barriers + alignment slack
+    static constexpr int TILE_BYTES = kBlockN * ROW_BYTES;   // one 64-row tile of K or V (Q is two of them)
+    // Q (128 rows), then nblk K tiles, then nblk V tiles, then the barrier block
+    __host__ __device__ static constexpr int bar_offset(int nblk) { return (2 + 2 * nblk) * TILE_BYTES; }
+    __host__ __device__ static constexpr int bytes(int nblk) { return bar_offset(nblk) + 256 + 1024; }
 };
 
 // K-major operand tile with rows of ROW_BYTES (= the swizzle span): 8-row groups are 8*ROW_BYTES apart.
@@ -86,7 +91,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t* __restrict__ seq_start,
                     const int32_t* __restrict__ seq_len, __nv_bfloat16* __restrict__ ctx, int H,
-                    float scale_log2e, int32_t* status, unsigned long long* dbg) {
+                    float scale_log2e, int max_blocks, int32_t* status, unsigned long long* dbg) {
     using SM = Smem<D>;
     pdl_launch_dependents();
     pdl_wait();
@@ -100,12 +105,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - raw);
-    const uint32_t sq = base, sk = base + SM::TILE_BYTES, sv = sk + kMaxBlocks * SM::TILE_BYTES;
-    const uint32_t bars = base + SM::BAR_OFFSET;
+    const uint32_t sq = base, sk = base + 2 * SM::TILE_BYTES, sv = sk + max_blocks * SM::TILE_BYTES;
+    const uint32_t bars = base + SM::bar_offset(max_blocks);
     // barriers: q_full, k_full[4], v_full[4], s_full, s_free, p_full, pv_done
     const uint32_t q_full = bars, k_full = bars + 8, v_full = bars + 8 + 8 * kMaxBlocks;
     const uint32_t s_full = bars + 8 + 16 * kMaxBlocks, s_free = s_full + 8, p_full = s_full + 16, pv_done = s_full + 24;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + SM::BAR_OFFSET + 8 + 16 * kMaxBlocks + 32);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + SM::bar_offset(max_blocks) + 8 + 16 * kMaxBlocks + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,8 +142,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
     if (warp == 0) {
         // ------------------------------------------------------------ TMA: Q, then K_j and V_j
         if (lane == 0) {
-            mbar_expect_tx(q_full, SM::TILE_BYTES);
+            mbar_expect_tx(q_full, 2 * SM::TILE_BYTES);
             tma_load_2d(sq, &tmap_qkv, head * D, row0 + q0, q_full);
+            tma_load_2d(sq + SM::TILE_BYTES, &tmap_qkv, head * D, row0 + q0 + kBlockN, q_full);
             for (int j = 0; j < nkb; ++j) {
                 mbar_expect_tx(k_full + 8 * j, SM::TILE_BYTES);
                 tma_load_2d(sk + j * SM::TILE_BYTES, &tmap_qkv, H + head * D, row0 + j * kBlockN, k_full + 8 * j);
@@ -173,11 +179,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
                 tc_fence_after();
                 issue_s(j);
             }
-            // pass 2: S_j again (unless the single block is still in TMEM), then O += P_j V_j
+            // pass 2: S_j again (unless the single block is still in TMEM), then O += P_j V_j.  P_j lives in
+            // S_j's columns, so S_{j+1} may only be issued once P_j V_j has finished reading them.
+            uint32_t n_pvdone = 0;
             for (int j = 0; j < nkb && ok; ++j) {
                 if (nkb > 1) {
-                    if (!(ok = mbar_wait(s_free, n_sfree & 1, abort_flag))) break;
-                    ++n_sfree;
+                    if (j == 0) {
+                        if (!(ok = mbar_wait(s_free, n_sfree & 1, abort_flag))) break;   // last pass-1 read
+                        ++n_sfree;
+                    } else {
+                        if (!(ok = mbar_wait(pv_done, n_pvdone & 1, abort_flag))) break;
+                        ++n_pvdone;
+                    }
                     tc_fence_after();
                     issue_s(j);
                 }
@@ -241,7 +254,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
                 ++n_sfull;
                 tc_fence_after();
             }
-            if (j > 0) {   // P buffer is free once the previous P V product has read it
+            if (j > 0) {   // keeps this thread's view of the pv_done phases in step (S_j was issued after it)
                 if (!(ok = mbar_wait(pv_done, n_pvdone & 1, abort_flag))) break;
                 ++n_pvdone;
                 tc_fence_after();
@@ -277,10 +290,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
             tc_fence_before();
             __syncwarp();
             stamp();   // P written
-            if (lane == 0) {
-                mbar_arrive(p_full);
-                if (nkb > 1) mbar_arrive(s_free);
-            }
+            if (lane == 0) mbar_arrive(p_full);
         }
         // ---- O / sum -> bf16 -> global ----
         if (ok && (ok = mbar_wait(pv_done, n_pvdone & 1, abort_flag))) {

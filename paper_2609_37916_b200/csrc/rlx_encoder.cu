@@ -127,9 +127,9 @@ cudaError_t init_kernels_for_current_device() {
         if (dev < 64) g_max_pairs[dev] = n;
     }
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tca::Smem<32>::BYTES)) != cudaSuccess) return e;
+                                  rlx::tca::Smem<32>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tca::Smem<64>::BYTES)) != cudaSuccess) return e;
+                                  rlx::tca::Smem<64>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   (int)sizeof(rlx::AttSmem<32>))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -252,12 +252,13 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
                    d == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
         return RLX_ERR_CUDA;
     dim3 grid((S + rlx::tca::kBlockM - 1) / rlx::tca::kBlockM, h, B);
+    const int nblk = (S + rlx::tca::kBlockN - 1) / rlx::tca::kBlockN;   // K/V tiles held in shared memory
     if (d == 32)
-        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, grid, rlx::tca::kThreads, rlx::tca::Smem<32>::BYTES, st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, status, g_attn_dbg));
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, grid, rlx::tca::kThreads, rlx::tca::Smem<32>::bytes(nblk), st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status, g_attn_dbg));
     else if (d == 64)
-        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, grid, rlx::tca::kThreads, rlx::tca::Smem<64>::BYTES, st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, status, g_attn_dbg));
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, grid, rlx::tca::kThreads, rlx::tca::Smem<64>::bytes(nblk), st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status, g_attn_dbg));
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
