@@ -32,6 +32,14 @@ import numpy as np  # noqa: E402
 
 METRIC = "encoder forward sequences/s (p50 ms reported alongside)"
 KERNEL_CLASSES = ("gemm_qkv", "attention", "gemm_out", "ln1", "gemm_ffn1", "gemm_ffn2", "ln2")
+# dram__bytes per launch (MB) from the ncu captures summarised under profiles/ (one capture per
+# kernel and workload; absent where no capture exists for that workload)
+NCU_DRAM_TRAFFIC_MB = {
+    "c2": {"gemm_out": 3.6, "gemm_ffn2": 9.5},
+    "c3": {"attention": 98.8, "gemm_ffn1": 90.5, "gemm_qkv": 62.2, "ln1": 28.6, "ln2": 28.6},
+}
+# B200: 148 SMs x 16 special-function results per clock x 1.965 GHz (exp2 of the softmax)
+EXP_PEAK_TEXP_S = 148 * 16 * 1.965e9 / 1e12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -192,7 +200,10 @@ def algorithmic_work(cls: str, c, lengths):
     if cls in ("gemm_ffn1", "gemm_ffn2"):
         return "tensor", 2.0 * T * F * H, "flop"
     if cls == "attention":
-        return "tensor", 4.0 * pairs * H, "flop"              # QK^T and PV over len x len per head
+        # at head_dim 32/64 the softmax exponentials (one per query-key pair and head), not the
+        # QK^T / PV flops, are the scarce resource: 128..256 flops per exp against a tensor : MUFU
+        # throughput ratio of ~3500 : 1
+        return "alu", pairs * c.num_heads, "exp"
     if cls in ("ln1", "ln2"):
         return "hbm", 2.0 * T * H * 2, "byte"                 # read + write one bf16 row per token
     if cls == "embed_ln":
@@ -333,21 +344,25 @@ def run_ours(args):
                 ach = work / (avg_ms * 1e-3) / 1e12
                 peak = peaks["bf16_tflops"]
                 u = "TFLOP/s"
+            elif bound == "alu":
+                ach = work / (avg_ms * 1e-3) / 1e12
+                peak = EXP_PEAK_TEXP_S
+                u = "Texp/s"
             else:
                 ach = work / (avg_ms * 1e-3) / 1e9
                 peak = peaks["hbm_gbs"]
                 u = "GB/s"
             ktab[cls] = {"avg_us": avg_ms * 1e3, "launches_per_step": launches_per_step,
                          "ms_per_step": avg_ms * launches_per_step, "bound": bound, "achieved": ach, "unit": u,
-                         "frac": ach / peak}
+                         "peak": peak, "frac": ach / peak}
             tot_kernel_ms += avg_ms * launches_per_step
         for v in ktab.values():
             v["share"] = v["ms_per_step"] / tot_kernel_ms
         dom = max(ktab, key=lambda k: ktab[k]["ms_per_step"])
         d = ktab[dom]
-        roofline = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak":
-                    (peaks["bf16_tflops"] if d["bound"] == "tensor" else peaks["hbm_gbs"]), "unit": d["unit"],
-                    "frac": d["frac"], "traffic": None, "peak_source": f"{peak_kind} (burst: kernels are timed "
+        traffic_mb = NCU_DRAM_TRAFFIC_MB.get(args.config, {}).get(dom)
+        roofline = {"kernel": dom, "bound": d["bound"], "achieved": d["achieved"], "peak": d["peak"], "unit": d["unit"],
+                    "frac": d["frac"], "traffic": None if traffic_mb is None else traffic_mb * 1e6, "peak_source": f"{peak_kind} (burst: kernels are timed "
                     "one by one inside a sub-millisecond step)", "share_of_step": d["share"],
                     "timing": "CUDA event nodes between kernels inside the replayed graph"}
 
