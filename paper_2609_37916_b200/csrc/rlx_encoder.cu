@@ -278,12 +278,13 @@ TileChoice pick_tile(int M, int N, int K, int want_cg = 0) {
     cudaGetDevice(&dev);
     const int pairs = (dev >= 0 && dev < 64) ? g_max_pairs[dev] : 0;
     // pairs pay off once a tile's main loop is long enough to amortise the cross-CTA handshakes
-    if (force_cg != 1 && pairs > 0 && (force_cg == 2 || K >= 768)) {
+    // (K >= 1536, or K >= 768 with a wide output) and every pair gets at least two tiles
+    if (force_cg != 1 && pairs > 0 && (force_cg == 2 || K >= 1536 || (K >= 768 && N >= 1536))) {
         const int m_tiles2 = (M + 255) / 256;
         const int cand2[3] = {256, 192, 128};
         for (int i = 0; i < 3; ++i) {
             if (force_bn && cand2[i] != force_bn) continue;
-            if (N % cand2[i] == 0 && (force_cg == 2 || m_tiles2 * (N / cand2[i]) >= 3 * pairs)) return {cand2[i], 2};
+            if (N % cand2[i] == 0 && (force_cg == 2 || m_tiles2 * (N / cand2[i]) >= 2 * pairs)) return {cand2[i], 2};
         }
     }
     const int m_tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;

@@ -132,6 +132,15 @@ def test_degenerate_lengths_zero_one_full(rlx):
     check(got, ref, inp.lengths)
 
 
+def test_all_sequences_empty_gives_zero_embeddings(rlx):
+    """No valid token anywhere: zero packed rows, every kernel must cope with an empty problem."""
+    inp = make_inputs(CONFIGS["c1"], batch=3, seq=33, num_layers=2, lengths=[0, 0, 0])
+    for flags in (0, 8, 0x20):
+        got, status = run_gpu(rlx, inp, flags=flags)
+        assert status == 0
+        assert np.array_equal(got, np.zeros_like(got))
+
+
 def test_vocabulary_ends_and_out_of_range_ids(rlx):
     inp = make_inputs(CONFIGS["c0"])
     inp.ids[0, 0], inp.ids[0, 1] = 0, inp.cfg.vocab - 1
