@@ -204,11 +204,14 @@ rlx_status_t launch_embed_ln(const int32_t* ids, const bf16* word, const bf16* p
 
 rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int T, int H, float eps, bf16* out,
                               cudaStream_t st, const int32_t* rows_ptr = nullptr) {
-    const bool big = T >= 4 * rlx::kNumSMs * rlx::kRowWarps * 4;   // enough rows for 4 rows per warp on every SM
-    const int rows_per_cta = rlx::kRowWarps * (big ? 4 : 1);
+    // rows per warp: as many as still leave ~4 CTAs for every SM (static row bound T), so that large
+    // problems run as about one full wave of fat CTAs and small ones still cover all SMs
+    const int want_ctas = 4 * rlx::kNumSMs;
+    const int rpw = (T >= want_ctas * rlx::kRowWarps * 4) ? 4 : 1;   // 8 rows per warp measured slower
+    const int rows_per_cta = rlx::kRowWarps * rpw;
     const int grid = (T + rows_per_cta - 1) / rows_per_cta, thr = rlx::kRowWarps * 32;
     switch (H / 128) {
-#define RLX_CASE(NV) case NV: if (big) RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV, 4>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); \
+#define RLX_CASE(NV) case NV: if (rpw == 4) RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV, 4>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); \
                      else RLX_CUDA_TRY(launch_ex(rlx::layernorm_kernel<NV, 1>, grid, thr, 0, st, x, g, b, out, T, eps, rows_ptr)); break;
         RLX_CASE(1) RLX_CASE(2) RLX_CASE(3) RLX_CASE(4) RLX_CASE(5) RLX_CASE(6) RLX_CASE(7) RLX_CASE(8)
 #undef RLX_CASE

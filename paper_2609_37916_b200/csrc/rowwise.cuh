@@ -224,14 +224,33 @@ pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restric
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     int count = 0;
     if (g < G) {
-        for (int s = g; s < nrows; s += G) {
-            if (!packed && __ldg(mb + s) == 0) continue;
-            ++count;
-            const uint4 a = __ldg(reinterpret_cast<const uint4*>(xb + (size_t)s * H + c * 8));
+        auto add_row = [&](const uint4& a) {
             acc[0] += bf16lo(a.x); acc[1] += bf16hi(a.x);
             acc[2] += bf16lo(a.y); acc[3] += bf16hi(a.y);
             acc[4] += bf16lo(a.z); acc[5] += bf16hi(a.z);
             acc[6] += bf16lo(a.w); acc[7] += bf16hi(a.w);
+        };
+        if (packed) {
+            // all rows valid: four independent 16-byte loads in flight per thread
+            int s = g;
+            for (; s + 3 * G < nrows; s += 4 * G) {
+                uint4 a[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) a[u] = __ldg(reinterpret_cast<const uint4*>(xb + (size_t)(s + u * G) * H + c * 8));
+#pragma unroll
+                for (int u = 0; u < 4; ++u) add_row(a[u]);
+                count += 4;
+            }
+            for (; s < nrows; s += G) {
+                add_row(__ldg(reinterpret_cast<const uint4*>(xb + (size_t)s * H + c * 8)));
+                ++count;
+            }
+        } else {
+            for (int s = g; s < nrows; s += G) {
+                if (__ldg(mb + s) == 0) continue;
+                ++count;
+                add_row(__ldg(reinterpret_cast<const uint4*>(xb + (size_t)s * H + c * 8)));
+            }
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) pool_smem[g * H + c * 8 + i] = acc[i];
