@@ -123,6 +123,34 @@ def test_odd_shapes(rlx, B, S):
     check(got, ref, inp.lengths)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small_problems_match_oracle(rlx, seed):
+    """Randomised sweep over batch, sequence length, valid lengths (incl. 0 and full), holes, LayerNorm
+    affine parameters and layer count, each compared with the oracle and between the execution modes."""
+    rng = np.random.default_rng(1000 + seed)
+    B = int(rng.integers(1, 9))
+    S = int(rng.choice([1, 2, 15, 16, 17, 31, 33, 63, 64, 65, 100, 128, 130, 200, 255, 256]))
+    L = int(rng.integers(1, 4))
+    lengths = rng.integers(0, S + 1, size=B)
+    lengths[rng.integers(0, B)] = S
+    inp = make_inputs(CONFIGS["c1"], batch=B, seq=S, num_layers=L, lengths=lengths,
+                      ln_affine_random=bool(seed % 2), mask_holes=0.25 if seed % 3 == 0 else 0.0,
+                      qk_gain=3.0 if seed % 4 == 0 else 1.0)
+    ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
+    w = rlx.upload_weights(inp.params, inp.layers)
+    base, status = run_gpu(rlx, inp, weights=w)
+    assert status == 0
+    check(base, ref, inp.lengths, tight=(seed % 4 != 0))
+    assert np.array_equal(base[inp.lengths == 0], np.zeros_like(base[inp.lengths == 0]))
+    for flags in (0x10, 1, 0x20, 0x40, 8):   # no PDL, eager, tcgen05 attention, fused LN, padded layout
+        other, status = run_gpu(rlx, inp, weights=w, flags=flags)
+        assert status == 0
+        if flags in (0x10, 1):
+            assert np.array_equal(base, other), hex(flags)     # same kernels, other launch mechanics
+        else:
+            check(other, ref, inp.lengths, tight=(seed % 4 != 0))
+
+
 def test_degenerate_lengths_zero_one_full(rlx):
     inp = make_inputs(CONFIGS["c1"], batch=3, seq=40, num_layers=2, lengths=[0, 1, 40])
     got, status = run_gpu(rlx, inp)
