@@ -62,7 +62,8 @@ typedef enum {
 #define RLX_FLAG_KERNEL_EVENTS 0x4u /* record a CUDA event between kernels (see rlx_encoder_kernel_times) */
 #define RLX_FLAG_NO_PDL 0x10u   /* plain stream order between kernels (no programmatic dependent launch) */
 #define RLX_FLAG_ATTN_TCGEN05 0x20u /* packed attention on the tcgen05/TMEM kernel instead of the mma.sync one */
-#define RLX_FLAG_FUSED_LN 0x40u /* fold the residual LayerNorms into the out-proj / FFN-down GEMMs (see rlx_gemm_residual_layernorm_bf16) */
+#define RLX_FLAG_FUSED_LN 0x40u /* fold the residual LayerNorms into the out-proj / FFN-down GEMMs, whole rows per CTA */
+#define RLX_FLAG_CLUSTER_LN 0x80u /* fold the residual LayerNorms into the GEMMs with cluster-wide row statistics */
 #define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
 
 typedef struct {
@@ -219,8 +220,9 @@ int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t *encoder, int32_t ba
  * the timing analogue).  Waits for that forward to finish, then writes `count` =
  * rlx_encoder_kernels_per_forward(batch, seq) durations in milliseconds to ms_host (host memory),
  * in launch order: [sequence packing,] embed+LN, then per layer [QKV GEMM, attention, out-proj
- * GEMM, LN, FFN-up GEMM, FFN-down GEMM, LN], then pool; with RLX_FLAG_FUSED_LN (and hidden
- * 256/384/512, batch*seq >= 128*148) the two LN entries per layer are absent.  In graph mode the events are nodes of the captured graph, so
+ * GEMM, LN, FFN-up GEMM, FFN-down GEMM, LN], then pool; with RLX_FLAG_CLUSTER_LN, or with
+ * RLX_FLAG_FUSED_LN (hidden 256/384/512 and batch*seq >= 128*148), the two LN entries per layer
+ * are absent.  In graph mode the events are nodes of the captured graph, so
  * the figures contain no host launch gaps.  RLX_ERR_UNSUPPORTED if the flag was not set.
  */
 rlx_status_t rlx_encoder_kernel_times(rlx_encoder_t *encoder, float *ms_host, int32_t count);
@@ -283,15 +285,18 @@ rlx_status_t rlx_gemm_bf16(const void *A, const void *W, const float *bias, cons
                            rlx_gemm_impl_t impl, int32_t *status, void *cuda_stream);
 
 /*
- * out = LN(A W^T + bias + residual; gamma, beta) in ONE kernel: each CTA owns 128 whole rows in
- * tensor memory, so the residual sum and the row statistics never reach HBM (the fused
- * "Linear + add + norm" region of Section 3.2).  N must be 256, 384 or 512; K % 8 == 0.
- * A bf16 [M,K], W bf16 [N,K], residual bf16 [M,N], bias/gamma/beta f32 [N], out bf16 [M,N].
+ * out = LN(A W^T + bias + residual; gamma, beta) in ONE kernel, so the residual sum and the row
+ * statistics never reach HBM (the fused "Linear + add + norm" region of Section 3.2).
+ * A bf16 [M,K], W bf16 [N,K], residual bf16 [M,N], bias/gamma/beta f32 [N], out bf16 [M,N]; K % 8 == 0.
+ *   impl 0: thread-block clusters along N: each CTA owns a 64/128/192-column slab of 128 rows and the
+ *           partial row sums are exchanged through distributed shared memory (N % 64 == 0 and at
+ *           most 8 slabs, i.e. any supported hidden size);
+ *   impl 1: one CTA owns 128 whole rows in tensor memory (N must be 256, 384 or 512).
  */
 rlx_status_t rlx_gemm_residual_layernorm_bf16(const void *A, const void *W, const float *bias,
                                               const void *residual, const float *gamma, const float *beta,
                                               float eps, int32_t M, int32_t N, int32_t K, void *out,
-                                              int32_t *status, void *cuda_stream);
+                                              int32_t impl, int32_t *status, void *cuda_stream);
 
 /*
  * Key-padding-masked scaled-dot-product attention over the packed projection

@@ -26,6 +26,7 @@ FLAG_NO_PACK = 0x8
 FLAG_NO_PDL = 0x10
 FLAG_ATTN_TCGEN05 = 0x20
 FLAG_FUSED_LN = 0x40
+FLAG_CLUSTER_LN = 0x80
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20
@@ -261,12 +262,12 @@ def gemm_bf16(a, w, bias, residual=None, epilogue: int = EPI_BIAS, impl: int = G
     return out
 
 
-def gemm_residual_layernorm_bf16(a, w, bias, residual, gamma, beta, eps: float, status=None, stream=None):
+def gemm_residual_layernorm_bf16(a, w, bias, residual, gamma, beta, eps: float, impl: int = 0, status=None, stream=None):
     M, K = a.shape
     N = w.shape[0]
     out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device)
     _check(_load().rlx_gemm_residual_layernorm_bf16(_ptr(a), _ptr(w), _ptr(bias), _ptr(residual), _ptr(gamma),
-                                                    _ptr(beta), C.c_float(eps), M, N, K, _ptr(out), _ptr(status),
+                                                    _ptr(beta), C.c_float(eps), M, N, K, _ptr(out), impl, _ptr(status),
                                                     _stream(stream)), "rlx_gemm_residual_layernorm_bf16")
     return out
 

@@ -16,6 +16,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_ln_tcgen05.cuh"
+#include "gemm_cln_tcgen05.cuh"
 #include "rowwise.cuh"
 
 namespace {
@@ -107,6 +108,12 @@ cudaError_t init_kernels_for_current_device() {
                                   rlx::tcln::Cfg<192>::SMEM_BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tcln::gemm_ln_tcgen05_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcln::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tccl::gemm_cln_tcgen05_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tccl::Cfg<64>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tccl::gemm_cln_tcgen05_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tccl::Cfg<128>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tccl::gemm_cln_tcgen05_kernel<192>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tccl::Cfg<192>::SMEM_BYTES)) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<128, 2>())) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<192, 2>())) != cudaSuccess) return e;
     if ((e = (set_gemm_attr_all<256, 2>())) != cudaSuccess) return e;
@@ -386,6 +393,75 @@ rlx_status_t launch_gemm_ln(const bf16* A, const bf16* W, const float* bias, con
     return RLX_OK;
 }
 
+// out = LN(A W^T + bias + residual) with cluster-wide row statistics: N / BLOCK_N CTAs per cluster.
+template <int BN>
+rlx_status_t launch_gemm_cln_bn(const bf16* A, const bf16* W, const rlx::tccl::Params& p, cudaStream_t st) {
+    const int nranks = p.N / BN;
+    CUtensorMap ta, tb;
+    if (!make_tmap(&ta, A, (uint64_t)p.M, (uint64_t)p.K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
+    if (!make_tmap(&tb, W, (uint64_t)p.N, (uint64_t)p.K, (uint32_t)BN)) return RLX_ERR_CUDA;
+    const int m_tiles = (p.M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
+    // clusters that can be resident at once for this cluster size (cached per device and size)
+    static int max_clusters[64][rlx::tccl::kMaxCluster + 1] = {};
+    int dev = 0;
+    RLX_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return RLX_ERR_UNSUPPORTED;
+    if (max_clusters[dev][nranks] == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(nranks * rlx::kNumSMs);
+        cfg.blockDim = dim3(rlx::tccl::Cfg<BN>::THREADS);
+        cfg.dynamicSmemBytes = rlx::tccl::Cfg<BN>::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)nranks;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        RLX_CUDA_TRY(cudaOccupancyMaxActiveClusters(&n, rlx::tccl::gemm_cln_tcgen05_kernel<BN>, &cfg));
+        if (n <= 0) return RLX_ERR_UNSUPPORTED;
+        max_clusters[dev][nranks] = n;
+    }
+    const int clusters = m_tiles < max_clusters[dev][nranks] ? m_tiles : max_clusters[dev][nranks];
+    struct ClusterScope {
+        explicit ClusterScope(int x) { g_cluster_x = x; }
+        ~ClusterScope() { g_cluster_x = 1; }
+    } scope(nranks);
+    RLX_CUDA_TRY(launch_ex(rlx::tccl::gemm_cln_tcgen05_kernel<BN>, nranks * clusters, rlx::tccl::Cfg<BN>::THREADS,
+                           rlx::tccl::Cfg<BN>::SMEM_BYTES, st, ta, tb, p));
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+// Slab width for the clustered LayerNorm GEMM: the widest slab (fewest operand re-reads) that still
+// gives every SM a CTA, among those with N / BLOCK_N <= 8 CTAs per cluster; 0 if none fits.
+int pick_cln_block_n(int M, int N) {
+    const int m_tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
+    const int cand[3] = {192, 128, 64};
+    int fallback = 0;
+    for (int i = 0; i < 3; ++i) {
+        if (N % cand[i] != 0 || N / cand[i] > rlx::tccl::kMaxCluster) continue;
+        if (m_tiles * (N / cand[i]) >= rlx::kNumSMs) return cand[i];
+        fallback = cand[i];   // keeps the narrowest admissible slab
+    }
+    return fallback;
+}
+
+rlx_status_t launch_gemm_cln(const bf16* A, const bf16* W, const float* bias, const bf16* residual, const float* gamma,
+                             const float* beta, float eps, int M, int N, int K, bf16* out, int32_t* status,
+                             cudaStream_t st, const int32_t* m_ptr = nullptr) {
+    const int bn = pick_cln_block_n(M, N);
+    if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
+    rlx::tccl::Params p{bias, residual, gamma, beta, out, eps, M, N, K, status, m_ptr};
+    switch (bn) {
+        case 64: return launch_gemm_cln_bn<64>(A, W, p, st);
+        case 128: return launch_gemm_cln_bn<128>(A, W, p, st);
+        case 192: return launch_gemm_cln_bn<192>(A, W, p, st);
+    }
+    return RLX_ERR_UNSUPPORTED;
+}
+
 // ------------------------------------------------------------------ workspace arena
 struct Arena {
     size_t status, ids, mask, out, seq_len, seq_start, pos_of_rank, x, qkv, ctx, y, x1, g, total;
@@ -428,9 +504,17 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
     return (long long)B * S >= 128ll * rlx::kNumSMs;
 }
 
+// RLX_FLAG_CLUSTER_LN: LayerNorm folded into the out-proj / FFN-down GEMMs with cluster-wide row
+// statistics.  Opt-in: the two exchanges per tile cost about what the separate LayerNorm kernel costs.
+bool uses_cluster_ln(const rlx_encoder_config_t& c) {
+    if ((c.flags & RLX_FLAG_GEMM_SIMT) || !(c.flags & RLX_FLAG_CLUSTER_LN)) return false;
+    return pick_cln_block_n(128, c.hidden) != 0;
+}
+
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
-    return 2 + (uses_fused_ln(c, B, S) ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
+    const bool fused = uses_fused_ln(c, B, S) || uses_cluster_ln(c);
+    return 2 + (fused ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
 }
 
 struct GraphEntry {
@@ -519,6 +603,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     }
     const int32_t* rows = pk.total();
     const bool fuse_ln = uses_fused_ln(c, B, S);
+    const bool fuse_cln = !fuse_ln && uses_cluster_ln(c);
     RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
                             w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
     for (int l = 0; l < c.num_layers; ++l) {
@@ -530,6 +615,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
             RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
         if (fuse_ln) {
             RLX_TRY(launch_gemm_ln(ctx, (const bf16*)lw.wo, lw.bo, x, lw.ln1_g, lw.ln1_b, c.ln_eps, T, H, H, x1, status, st, rows));
+        } else if (fuse_cln) {
+            RLX_TRY(launch_gemm_cln(ctx, (const bf16*)lw.wo, lw.bo, x, lw.ln1_g, lw.ln1_b, c.ln_eps, T, H, H, x1, status, st, rows));
         } else {
             RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
             RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
@@ -538,6 +625,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         if (fuse_ln) {
             // x1 is both the residual and (after this kernel) dead; the result goes to x
             RLX_TRY(launch_gemm_ln(g, (const bf16*)lw.w2, lw.b2, x1, lw.ln2_g, lw.ln2_b, c.ln_eps, T, H, F, x, status, st, rows));
+        } else if (fuse_cln) {
+            RLX_TRY(launch_gemm_cln(g, (const bf16*)lw.w2, lw.b2, x1, lw.ln2_g, lw.ln2_b, c.ln_eps, T, H, F, x, status, st, rows));
         } else {
             RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, x1, RLX_EPI_BIAS_RESIDUAL, T, H, F, y, simt, status, st, rows));
             RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
@@ -823,12 +912,16 @@ rlx_status_t rlx_gemm_bf16(const void* A, const void* W, const float* bias, cons
 
 rlx_status_t rlx_gemm_residual_layernorm_bf16(const void* A, const void* W, const float* bias, const void* residual,
                                               const float* gamma, const float* beta, float eps, int32_t M, int32_t N,
-                                              int32_t K, void* out, int32_t* status, void* stream) {
+                                              int32_t K, void* out, int32_t impl, int32_t* status, void* stream) {
     if (!A || !W || !bias || !residual || !gamma || !beta || !out || M <= 0 || N <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
     if (!aligned16(A) || !aligned16(W) || !aligned16(bias) || !aligned16(residual) || !aligned16(gamma) ||
         !aligned16(beta) || !aligned16(out))
         return RLX_ERR_INVALID_ARG;
     RLX_CUDA_TRY(init_kernels_for_current_device());
+    if (impl == 0)
+        return launch_gemm_cln((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, gamma, beta, eps, M, N, K,
+                               (bf16*)out, status, static_cast<cudaStream_t>(stream));
+    if (impl != 1) return RLX_ERR_INVALID_ARG;
     return launch_gemm_ln((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, gamma, beta, eps, M, N, K,
                           (bf16*)out, status, static_cast<cudaStream_t>(stream));
 }

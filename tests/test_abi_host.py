@@ -58,17 +58,21 @@ def test_create_validates_shapes(lib):
         assert ei.value.status == status, bad
 
 
-def test_kernel_count_drops_when_layernorm_is_fused(lib):
-    enc = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_FUSED_LN))
-    assert enc.kernels_per_forward(256, 256) == 3 + 5 * 6     # enough 128-row tiles for every SM: LN fused
-    assert enc.kernels_per_forward(32, 128) == 3 + 7 * 6
+def test_kernel_count_follows_the_layernorm_fusion_flags(lib):
+    enc = binding.Encoder(**_cfg(max_batch=256, max_seq=256))
+    assert enc.kernels_per_forward(256, 256) == 3 + 7 * 6     # default: LayerNorm is its own kernel
     enc.close()
-    plain = binding.Encoder(**_cfg(max_batch=256, max_seq=256))
-    assert plain.kernels_per_forward(256, 256) == 3 + 7 * 6
-    plain.close()
+    cl = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_CLUSTER_LN))
+    assert cl.kernels_per_forward(256, 256) == 3 + 5 * 6      # folded into the GEMMs (cluster statistics)
+    assert cl.kernels_per_forward(1, 16) == 3 + 5 * 6
+    cl.close()
+    whole = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_FUSED_LN))
+    assert whole.kernels_per_forward(256, 256) == 3 + 5 * 6   # whole-row variant: enough 128-row tiles for every SM
+    assert whole.kernels_per_forward(32, 128) == 3 + 7 * 6
+    whole.close()
     big = binding.Encoder(**_cfg(hidden=768, num_heads=12, ffn=3072, max_batch=64, max_seq=512,
-                                 flags=binding.FLAG_FUSED_LN))
-    assert big.kernels_per_forward(64, 512) == 3 + 7 * 6      # a 768-wide row does not fit in tensor memory
+                                 flags=binding.FLAG_CLUSTER_LN))
+    assert big.kernels_per_forward(64, 512) == 3 + 5 * 6      # 768 = 4 slabs of 192 columns per cluster
     big.close()
 
 

@@ -173,10 +173,14 @@ def test_gemm_matches_oracle_linear(rlx, shape, epi, impl):
     assert_close_bf16_out(got, ref, extra_abs=K * 2.0 ** -24 * 0.2)
 
 
+@pytest.mark.parametrize("impl", [0, 1], ids=["cluster", "whole_row"])
 @pytest.mark.parametrize("shape", [(128, 384, 384), (300, 384, 1536), (1000, 256, 320), (129, 512, 512),
-                                   (20000, 384, 384), (19000, 384, 1536)])
-def test_gemm_residual_layernorm_fused(rlx, shape):
+                                   (20000, 384, 384), (19000, 384, 1536), (2200, 768, 768), (5000, 768, 3072),
+                                   (700, 1024, 256), (333, 128, 128), (16, 384, 384)])
+def test_gemm_residual_layernorm_fused(rlx, shape, impl):
     M, N, K = shape
+    if impl == 1 and N not in (256, 384, 512):
+        pytest.skip("whole-row variant: the row must fit in tensor memory")
     rng = np.random.default_rng(M + N + K)
     a = rand_bf16(rng, (M, K))
     w = rand_bf16(rng, (N, K), 0.05)
@@ -186,14 +190,15 @@ def test_gemm_residual_layernorm_fused(rlx, shape):
     b = (0.1 * rng.standard_normal(N)).astype(np.float32)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     got = to_np64(rlx.gemm_residual_layernorm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(bias), bf16_dev(res), f32_dev(g),
-                                                   f32_dev(b), 1e-12, status=status))
+                                                   f32_dev(b), 1e-12, impl=impl, status=status))
     assert int(status.item()) == 0
     ref = oracle.layernorm(oracle.linear(a.astype(np.float64), w, bias) + res.astype(np.float64), g, b, 1e-12)
     # the pre-LayerNorm sum stays in fp32 here (no bf16 round trip), so the plain bf16-output bound holds
     assert_close_bf16_out(got, ref, extra_abs=K * 2.0 ** -24 * 0.5)
 
 
-def test_gemm_residual_layernorm_constant_rows_give_beta(rlx):
+@pytest.mark.parametrize("impl", [0, 1], ids=["cluster", "whole_row"])
+def test_gemm_residual_layernorm_constant_rows_give_beta(rlx, impl):
     """Zero weights, zero bias and a constant residual row: LayerNorm of a constant row is exactly beta."""
     M, N, K = 200, 384, 384
     a = np.ones((M, K), np.float32)
@@ -201,7 +206,7 @@ def test_gemm_residual_layernorm_constant_rows_give_beta(rlx):
     res = np.full((M, N), 1.5, np.float32)
     beta = round_to_bf16(np.linspace(-1, 1, N).astype(np.float32))
     got = to_np64(rlx.gemm_residual_layernorm_bf16(bf16_dev(a), bf16_dev(w), f32_dev(np.zeros(N)), bf16_dev(res),
-                                                   f32_dev(np.ones(N)), f32_dev(beta), 1e-12))
+                                                   f32_dev(np.ones(N)), f32_dev(beta), 1e-12, impl=impl))
     assert np.array_equal(got, np.broadcast_to(beta.astype(np.float64), (M, N)))
 
 
