@@ -64,6 +64,7 @@ typedef enum {
 #define RLX_FLAG_ATTN_TCGEN05 0x20u /* packed attention on the tcgen05/TMEM kernel instead of the mma.sync one */
 #define RLX_FLAG_FUSED_LN 0x40u /* fold the residual LayerNorms into the out-proj / FFN-down GEMMs, whole rows per CTA */
 #define RLX_FLAG_CLUSTER_LN 0x80u /* fold the residual LayerNorms into the GEMMs with cluster-wide row statistics */
+#define RLX_FLAG_NO_PREFETCH 0x100u /* no L2 prefetch of the Linear weights on a side branch of the captured graph */
 #define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
 
 typedef struct {

@@ -534,6 +534,8 @@ struct rlx_encoder {
     std::vector<GraphEntry> graphs;
     int last_kernels = 0;                   // kernels of the most recent forward (for kernel_times)
     std::vector<cudaEvent_t> events;        // RLX_FLAG_KERNEL_EVENTS: one before the first kernel, one after each
+    cudaStream_t side_stream = nullptr;     // side branch of the captured graph (weight prefetch)
+    cudaEvent_t fork_event = nullptr, join_event = nullptr;
     cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
                                             // legacy default stream, which cannot be captured)
 };
@@ -590,6 +592,32 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         explicit PdlScope(bool on) { g_pdl_launch = on; }
         ~PdlScope() { g_pdl_launch = false; }
     } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && e->events.empty());
+    // side branch (captured graphs only): prefetch the Linear weights into L2 when they all fit
+    bool forked = false;
+    if (capturing && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH)) {
+        const size_t per_layer = ((size_t)3 * H * H + (size_t)H * H + (size_t)2 * H * F) * sizeof(bf16);
+        if (per_layer * c.num_layers <= ((size_t)48 << 20) && 4 * c.num_layers <= rlx::kMaxPrefetch) {
+            rlx::PrefetchList pf = {};
+            for (int l = 0; l < c.num_layers; ++l) {
+                const rlx_layer_weights_t& lw = w->layers[l];
+                const void* ptrs[4] = {lw.wqkv, lw.wo, lw.w1, lw.w2};
+                const size_t bytes[4] = {(size_t)3 * H * H * 2, (size_t)H * H * 2, (size_t)F * H * 2, (size_t)H * F * 2};
+                for (int i = 0; i < 4; ++i) {
+                    pf.ptr[pf.n] = ptrs[i];
+                    pf.bytes[pf.n] = (uint32_t)bytes[i];
+                    pf.first_piece[pf.n] = pf.total_pieces;
+                    pf.total_pieces += (uint32_t)((bytes[i] + rlx::kPrefetchPiece - 1) / rlx::kPrefetchPiece);
+                    ++pf.n;
+                }
+            }
+            RLX_CUDA_TRY(cudaEventRecord(e->fork_event, st));
+            RLX_CUDA_TRY(cudaStreamWaitEvent(e->side_stream, e->fork_event, 0));
+            rlx::prefetch_l2_kernel<<<rlx::kNumSMs, 32, 0, e->side_stream>>>(pf);
+            RLX_CUDA_TRY(cudaGetLastError());
+            RLX_CUDA_TRY(cudaEventRecord(e->join_event, e->side_stream));
+            forked = true;
+        }
+    }
     Packing pk;
     if (pack) {
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
@@ -634,6 +662,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     }
     RLX_TRY(launch_pool(x, mask, B, S, H, out, st, pk));
 #undef RLX_TRY
+    if (forked) RLX_CUDA_TRY(cudaStreamWaitEvent(st, e->join_event, 0));   // join the side branch
     return RLX_OK;
 }
 
@@ -684,6 +713,11 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
     // capture once for this (batch, seq, pointer set)
     cudaGraph_t graph = nullptr;
     if (!e->capture_stream) RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
+    if (!e->side_stream) {
+        RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->side_stream, cudaStreamNonBlocking));
+        RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->fork_event, cudaEventDisableTiming));
+        RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->join_event, cudaEventDisableTiming));
+    }
     RLX_CUDA_TRY(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal));
     rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream, true);
     cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
@@ -734,6 +768,9 @@ void rlx_encoder_destroy(rlx_encoder_t* e) {
     if (!e) return;
     drop_graphs(e);
     if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
+    if (e->side_stream) cudaStreamDestroy(e->side_stream);
+    if (e->fork_event) cudaEventDestroy(e->fork_event);
+    if (e->join_event) cudaEventDestroy(e->join_event);
     for (auto& evt : e->events) cudaEventDestroy(evt);
     delete e;
 }

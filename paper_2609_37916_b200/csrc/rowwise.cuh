@@ -104,6 +104,32 @@ pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* _
     }
 }
 
+// Weight matrices to pull into L2 while the first kernels of a forward run: a small batch starts from
+// a cold L2 and would otherwise pay an HBM round trip at the head of every GEMM.  Runs as a side
+// branch of the captured graph (nothing on the main chain waits for it).  Pieces are issued in list
+// order (layer by layer) as asynchronous bulk prefetches.
+constexpr int kMaxPrefetch = 96;
+constexpr uint32_t kPrefetchPiece = 32 * 1024;
+struct PrefetchList {
+    const void* ptr[kMaxPrefetch];
+    uint32_t bytes[kMaxPrefetch];        // multiples of 16
+    uint32_t first_piece[kMaxPrefetch];  // running count of pieces before this matrix
+    int n;
+    uint32_t total_pieces;
+};
+
+__global__ void __launch_bounds__(32)
+prefetch_l2_kernel(const PrefetchList pf) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t piece = blockIdx.x * blockDim.x + threadIdx.x; piece < pf.total_pieces; piece += stride) {
+        int m = 0;
+        while (m + 1 < pf.n && pf.first_piece[m + 1] <= piece) ++m;
+        const uint32_t off = (piece - pf.first_piece[m]) * kPrefetchPiece;
+        const uint32_t sz = min(kPrefetchPiece, pf.bytes[m] - off);
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(static_cast<const char*>(pf.ptr[m]) + off), "r"(sz) : "memory");
+    }
+}
+
 // Largest b with seq_start[b] <= p (seq_start is non-decreasing, seq_start[B] = total > p).
 __device__ __forceinline__ int find_sequence(const int32_t* __restrict__ seq_start, int B, int p) {
     int lo = 0, hi = B;   // invariant: seq_start[lo] <= p < seq_start[hi]

@@ -142,10 +142,10 @@ def test_random_small_problems_match_oracle(rlx, seed):
     assert status == 0
     check(base, ref, inp.lengths, tight=(seed % 4 != 0))
     assert np.array_equal(base[inp.lengths == 0], np.zeros_like(base[inp.lengths == 0]))
-    for flags in (0x10, 1, 0x20, 0x80, 8):   # no PDL, eager, tcgen05 attention, cluster LayerNorm, padded layout
+    for flags in (0x10, 0x100, 1, 0x20, 0x80, 8):   # no PDL, no prefetch, eager, tcgen05 attn, cluster LN, padded
         other, status = run_gpu(rlx, inp, weights=w, flags=flags)
         assert status == 0
-        if flags in (0x10, 1):
+        if flags in (0x10, 0x100, 1):
             assert np.array_equal(base, other), hex(flags)     # same kernels, other launch mechanics
         else:
             check(other, ref, inp.lengths, tight=(seed % 4 != 0))
