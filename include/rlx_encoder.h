@@ -150,6 +150,7 @@ size_t rlx_encoder_workspace_bytes(const rlx_encoder_t *encoder, int32_t batch, 
  *                 scratch: contents are overwritten by every call.  Its first 256 bytes hold the
  *                 sticky device status word: zero them once before the first call
  *
+ * config->device must be the current CUDA device (RLX_ERR_INVALID_ARG otherwise).
  * Asynchronous on cuda_stream.  Unless RLX_FLAG_NO_GRAPH is set the kernel
  * sequence is captured once per distinct (batch, seq, pointer set) into a CUDA
  * graph and replayed afterwards.  Activations are computed in bf16 storage

@@ -689,6 +689,9 @@ rlx_status_t check_forward_args(const rlx_encoder* e, const void* ids, const voi
 
 rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
                             const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st) {
+    int dev = -1;
+    RLX_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != e->cfg.device) return RLX_ERR_INVALID_ARG;   // the object is bound to one device; make it current
     RLX_CUDA_TRY(init_kernels_for_current_device());
     if ((e->cfg.flags & RLX_FLAG_KERNEL_EVENTS) && e->events.empty()) {
         e->events.resize(4 + 7 * (size_t)e->cfg.num_layers);   // upper bound: one per kernel + 1
@@ -889,6 +892,9 @@ rlx_status_t rlx_encoder_forward_static(rlx_encoder_t* e, const int32_t* ids, co
     const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
     if (a.total > (size_t)RLX_STATIC_WORKSPACE_BYTES) return RLX_ERR_WORKSPACE;  // beyond the built-in arena
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = -1;
+    RLX_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != e->cfg.device) return RLX_ERR_INVALID_ARG;
     unsigned char* ws = nullptr;
     s = static_workspace_for_current_device(&ws);
     if (s != RLX_OK) return s;

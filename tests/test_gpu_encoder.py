@@ -204,6 +204,18 @@ def test_padding_invariance_and_determinism_are_bitwise(rlx):
     assert np.array_equal(a[perm], d)                  # batch-permutation equivariance
 
 
+def test_forward_refuses_an_encoder_bound_to_another_device(rlx):
+    inp = make_inputs(CONFIGS["c0"])
+    c = inp.cfg
+    enc = rlx.Encoder.from_config(c, max_batch=1, max_seq=c.seq, device=torch.cuda.device_count())  # not current
+    w = rlx.upload_weights(inp.params, inp.layers)
+    out = torch.zeros((1, c.hidden), dtype=torch.float32, device="cuda")
+    with pytest.raises(rlx.RlxError) as ei:
+        enc.forward(i32_dev(inp.ids), i32_dev(inp.mask), w, out, enc.alloc_workspace(1, c.seq))
+    assert ei.value.status == 1 and torch.count_nonzero(out) == 0
+    enc.close()
+
+
 def test_graph_cache_reuse_and_new_inputs(rlx):
     """Same encoder object, several calls: the captured graph must be replayed for the same
     pointer set and rebuilt when the buffers or the weights change."""
