@@ -42,6 +42,32 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Blackwell packed fp32 arithmetic: one issue slot per register PAIR.  The MMA accumulator quads are
+// even-aligned, so (c0,c1) and (c2,c3) pack without a move.
+__device__ __forceinline__ uint64_t att_pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void att_unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t att_fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t att_mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 constexpr int kAttBlockM = 128;  // query rows per CTA (8 warps x 16 rows)
 constexpr int kAttBlockN = 64;   // keys per shared-memory stage
 constexpr int kAttStages = 4;    // K/V ring depth (three blocks in flight ahead of the one being used)
@@ -144,7 +170,12 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     float o[ND][4];
 #pragma unroll
     for (int i = 0; i < ND; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};   // running max (scaled) and sum
+    float m_run[2] = {-INFINITY, -INFINITY};   // running max (scaled)
+    // Running row sums come out of the tensor cores: P times a column of ones accumulates, in every
+    // column of this extra n-tile, the sum of the bf16-rounded probabilities -- the same values the
+    // P V product uses, so numerator and denominator of the softmax agree.
+    float l_acc[4] = {0.f, 0.f, 0.f, 0.f};
+    constexpr uint32_t kOnesBf16x2 = 0x3F803F80u;
     const int g = lane >> 2, t4 = lane & 3;
     const bool warp_active = q0 + warp * 16 < len;   // warps whose 16 rows lie past the sequence only sync
 
@@ -197,11 +228,11 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             }
         }
         // ---- running max on raw scores (the positive scale commutes with max) ----
-        float mx[2] = {-INFINITY, -INFINITY};
+        float mx[2] = {fmaxf(s[0][0], s[0][1]), fmaxf(s[0][2], s[0][3])};
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            mx[0] = fmaxf(mx[0], fmaxf(s[nt][0], s[nt][1]));
-            mx[1] = fmaxf(mx[1], fmaxf(s[nt][2], s[nt][3]));
+        for (int nt = 1; nt < 8; ++nt) {
+            mx[0] = fmax3(mx[0], s[nt][0], s[nt][1]);
+            mx[1] = fmax3(mx[1], s[nt][2], s[nt][3]);
         }
         float alpha[2], msub[2];
 #pragma unroll
@@ -212,29 +243,31 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             msub[r] = (m_new == -INFINITY) ? 0.f : m_new;   // all keys so far masked: avoid inf - inf
             alpha[r] = fast_exp2(m_run[r] - msub[r]);        // m_run = -inf -> 0
             m_run[r] = m_new;
-            l_run[r] *= alpha[r];
         }
+        const uint64_t a0 = att_pack2(alpha[0], alpha[0]), a1 = att_pack2(alpha[1], alpha[1]);
 #pragma unroll
         for (int nd = 0; nd < ND; ++nd) {
-            o[nd][0] *= alpha[0]; o[nd][1] *= alpha[0];
-            o[nd][2] *= alpha[1]; o[nd][3] *= alpha[1];
+            att_unpack2(att_mul2(att_pack2(o[nd][0], o[nd][1]), a0), o[nd][0], o[nd][1]);
+            att_unpack2(att_mul2(att_pack2(o[nd][2], o[nd][3]), a1), o[nd][2], o[nd][3]);
         }
-        // ---- P = exp2(S*c - m), row sums, pack to bf16 A fragments ----
+        l_acc[0] *= alpha[0];
+        l_acc[2] *= alpha[1];
+        // ---- P = exp2(S*c - m), packed to bf16 A fragments ----
         uint32_t pf[4][4];
+        const uint64_t c2 = att_pack2(scale_log2e, scale_log2e);
+        const uint64_t nm0 = att_pack2(-msub[0], -msub[0]), nm1 = att_pack2(-msub[1], -msub[1]);
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
-            const float p0 = fast_exp2(fmaf(s[nt][0], scale_log2e, -msub[0]));
-            const float p1 = fast_exp2(fmaf(s[nt][1], scale_log2e, -msub[0]));
-            const float p2 = fast_exp2(fmaf(s[nt][2], scale_log2e, -msub[1]));
-            const float p3 = fast_exp2(fmaf(s[nt][3], scale_log2e, -msub[1]));
-            l_run[0] += p0 + p1;
-            l_run[1] += p2 + p3;
-            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p0, p1);
-            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p2, p3);
+            float x0, x1, x2, x3;
+            att_unpack2(att_fma2(att_pack2(s[nt][0], s[nt][1]), c2, nm0), x0, x1);
+            att_unpack2(att_fma2(att_pack2(s[nt][2], s[nt][3]), c2, nm1), x2, x3);
+            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(fast_exp2(x0), fast_exp2(x1));
+            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(fast_exp2(x2), fast_exp2(x3));
         }
         // ---- O += P V ----
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
+            mma_bf16_16816(l_acc, pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], kOnesBf16x2, kOnesBf16x2);
 #pragma unroll
             for (int np = 0; np < ND / 2; ++np) {  // two n-tiles per ldmatrix.x4.trans
                 uint32_t b0, b1, b2, b3;
@@ -251,12 +284,9 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     if (!warp_active) return;
 
     // ---- normalise, stage this warp's 16 x D tile in its own rows of the Q buffer, store 16 B / lane ----
+    float l_run[2] = {l_acc[0], l_acc[2]};   // every column of the ones n-tile holds the full row sum
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-        l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-        l_run[r] = l_run[r] > 0.f ? 1.0f / l_run[r] : 0.f;
-    }
+    for (int r = 0; r < 2; ++r) l_run[r] = l_run[r] > 0.f ? 1.0f / l_run[r] : 0.f;
     __nv_bfloat16* stage = sm.q + warp * 16 * STR;   // only this warp ever touched these rows
 #pragma unroll
     for (int nd = 0; nd < ND; ++nd) {
