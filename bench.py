@@ -408,6 +408,165 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------- attention under other mask kinds
+def attention_kind_workload(seed: int = 7, batch: int = 16, lo: int = 1024, hi: int = 4096):
+    rng = np.random.default_rng(seed)
+    return rng.integers(lo, hi + 1, size=batch).astype(np.int32)
+
+
+def visible_pairs(lengths, kind: str, window: int) -> int:
+    tot = 0
+    for n in (int(x) for x in lengths):
+        if kind == "none":
+            tot += n * n
+        elif kind == "causal":
+            tot += n * (n + 1) // 2
+        else:
+            i = np.arange(n, dtype=np.int64)
+            tot += int(np.minimum(i + 1, window).sum())
+    return tot
+
+
+def run_attention_kind(args):
+    """`--op attention_kind`: one step = one launch of rlx_attention_kind_bf16 over a packed batch of
+    decoder-shaped sequences (16 heads x 64, lengths 1024..4096, seeded), device-timed with an L2 flush
+    between steps; the oracle is timed on the first sequence."""
+    import torch
+    import paper_2609_37916_b200 as rlx
+
+    h, d = 16, 64
+    H = h * d
+    lengths = attention_kind_workload()
+    total, max_len = int(lengths.sum()), int(lengths.max())
+    start = np.concatenate([[0], np.cumsum(lengths)])[:-1].astype(np.int32)
+    kind_id = {"none": rlx.binding.MASK_NONE, "causal": rlx.binding.MASK_CAUSAL, "sliding": rlx.binding.MASK_SLIDING_WINDOW}[args.mask]
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    qkv = torch.randn(total, 3 * H, device="cuda", generator=g).to(torch.bfloat16)
+    ss, sl = torch.from_numpy(start).cuda(), torch.from_numpy(lengths).cuda()
+    rope = rlx.rope_tables(max_len, d) if args.rope else None
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    ctx = torch.zeros(total, H, dtype=torch.bfloat16, device="cuda")
+    sampler = ClockSampler(0)
+    sampler.start()
+
+    def step():
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = rlx.binding.attention_kind_bf16(qkv, ss, sl, max_len, h, kind_id, args.window, rope, out=ctx)
+        e1.record()
+        return e0, e1, out
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler.active.set()
+    evs = [step() for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    sampler.active.clear()
+    sampler.stop()
+    ms = [a.elapsed_time(b) for a, b, _ in evs]
+    p50 = statistics.median(ms)
+    pairs = visible_pairs(lengths, args.mask, args.window)
+    flops, exps, bytes_ = 4.0 * pairs * d * h, float(pairs) * h, 4.0 * total * H * 2
+    peaks, peak_kind = load_peaks()
+    # oracle on the first sequence
+    from oracle import attention_kinds as ak
+    n0 = int(lengths[0])
+    seq = qkv[:n0].float().cpu().numpy().astype(np.float64)
+    t0 = time.perf_counter()
+    ref = ak.attention_one(seq, h, kind_id, args.window, 10000.0 if args.rope else None)
+    t_or = time.perf_counter() - t0
+    got = evs[-1][2][:n0].float().cpu().numpy().astype(np.float64)
+    line = {
+        "metric": "attention (mask kind / rotary) tokens/s (p50 ms reported alongside)", "op": "attention_kind",
+        "value": total * args.steps / (sum(ms) / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "p50_ms": p50, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), 16 heads x 64, "
+                               f"mask {args.mask}" + (f"({args.window})" if args.mask == "sliding" else "") +
+                               (", rotary q,k" if args.rope else ""), "l2": "256 MiB flush write between steps"},
+        "gpu_launches": args.steps, "clocks": sampler.summary(),
+        "roofline": {"kernel": "attention_bf16_kernel<64>", "bound": "alu", "achieved": exps / (p50 * 1e-3) / 1e12,
+                     "peak": EXP_PEAK_TEXP_S, "unit": "Texp/s", "frac": exps / (p50 * 1e-3) / 1e12 / EXP_PEAK_TEXP_S,
+                     "traffic": None, "tensor_tflops": flops / (p50 * 1e-3) / 1e12,
+                     "tensor_frac_of_" + peak_kind: flops / (p50 * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "hbm_gbs": bytes_ / (p50 * 1e-3) / 1e9,
+                     "work": "visible (query, key) pairs only"},
+        "cpu_baseline": {"value": n0 / t_or, "unit": "tokens/s", "cores": usable_cores(), "kind": "oracle",
+                         "sample": f"first sequence ({n0} tokens), 1 run, {t_or:.2f} s"},
+        "parity_on_sample": {"max_abs_err": float(np.abs(got - ref).max()), "max_abs_ref": float(np.abs(ref).max())},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_qk_rope(args):
+    """`--op qk_rope`: one step = one launch of rlx_qk_rope_bf16 (in-place rotation of the q and k column
+    blocks) over the packed batch of `--op attention_kind`; HBM-bound: 2/3 of qkv read and written."""
+    import torch
+    import paper_2609_37916_b200 as rlx
+
+    h, d = 16, 64
+    H = h * d
+    lengths = attention_kind_workload()
+    total, max_len = int(lengths.sum()), int(lengths.max())
+    start = np.concatenate([[0], np.cumsum(lengths)])[:-1].astype(np.int32)
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    qkv0 = torch.randn(total, 3 * H, device="cuda", generator=g).to(torch.bfloat16)
+    qkv = qkv0.clone()
+    ss, sl = torch.from_numpy(start).cuda(), torch.from_numpy(lengths).cuda()
+    rope = rlx.rope_tables(max_len, d)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(0)
+    sampler.start()
+
+    def step():
+        qkv.copy_(qkv0)          # keep magnitudes fixed: the rotation is applied to fresh data every step
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        rlx.binding.qk_rope_bf16(qkv, ss, sl, max_len, h, rope)
+        e1.record()
+        return e0, e1
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler.active.set()
+    evs = [step() for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    sampler.active.clear()
+    sampler.stop()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    p50 = statistics.median(ms)
+    bytes_ = 2.0 * total * 2 * H * 2          # q and k blocks, read and written, bf16
+    peaks, peak_kind = load_peaks()
+    from oracle import attention_kinds as ak
+    n0 = int(lengths[0])
+    t0 = time.perf_counter()
+    ref = ak.rope_qk_packed(qkv0[:n0].float().cpu().numpy().astype(np.float64), [0], [n0], h, 10000.0)
+    t_or = time.perf_counter() - t0
+    got = qkv[:n0].float().cpu().numpy().astype(np.float64)
+    ach = bytes_ / (p50 * 1e-3) / 1e9
+    line = {
+        "metric": "fused QK-RoPE tokens/s (p50 ms reported alongside)", "op": "qk_rope",
+        "value": total * args.steps / (sum(ms) / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "p50_ms": p50, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), 16 heads x 64",
+                   "l2": "256 MiB flush write between steps"},
+        "gpu_launches": args.steps, "clocks": sampler.summary(),
+        "roofline": {"kernel": "qk_rope_kernel<64>", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peak_kind},
+        "cpu_baseline": {"value": n0 / t_or, "unit": "tokens/s", "cores": usable_cores(), "kind": "oracle",
+                         "sample": f"first sequence ({n0} tokens), 1 run, {t_or:.3f} s"},
+        "parity_on_sample": {"max_abs_err": float(np.abs(got - ref).max()), "max_abs_ref": float(np.abs(ref).max())},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -415,7 +574,16 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="c2", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope"])
+    ap.add_argument("--mask", default="causal", choices=["none", "causal", "sliding"])
+    ap.add_argument("--window", type=int, default=512)
+    ap.add_argument("--rope", type=int, default=1)
     args = ap.parse_args()
+    if args.op != "encoder":
+        if args.impl != "ours" or args.gpus != 1:
+            raise SystemExit(f"--op {args.op} runs on one GPU with --impl ours")
+        (run_attention_kind if args.op == "attention_kind" else run_qk_rope)(args)
+        return
     if args.impl == "reference":
         run_reference_arm(args)
     else:

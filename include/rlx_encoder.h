@@ -329,6 +329,52 @@ rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const
                                        int32_t num_heads, int32_t head_dim, void *ctx_bf16, int32_t impl,
                                        int32_t *status, void *cuda_stream);
 
+/*
+ * Attention under the other mask kinds of Section 3.1, with the rotary embedding of the fused
+ * QK-RoPE region (Section 3.2) applied to q and k as they are loaded.  The paper names the kinds and
+ * the region without defining them; this entry point reads them as the decoder families of its
+ * model zoo do:
+ *   RLX_MASK_NONE            every key of the sequence is visible;
+ *   RLX_MASK_CAUSAL          key k is visible to query i  iff  k <= i;
+ *   RLX_MASK_SLIDING_WINDOW  key k is visible to query i  iff  i - window < k <= i  (window >= 1);
+ *   rotary embedding         column j < head_dim/2 of every q and k head is paired with column
+ *                            j + head_dim/2 and the pair is rotated by the angle of the row's position
+ *                            in its sequence: lo' = lo*cos - hi*sin, hi' = hi*cos + lo*sin, in fp32,
+ *                            rounded to bf16 before the tensor-core product.  v is not touched.
+ * Arguments: qkv / seq_start / seq_len / ctx as in rlx_attention_packed_bf16 (packed rows, device
+ * memory, 16-byte aligned; seq_len[b] <= max_len <= RLX_ATTENTION_KIND_MAX_LEN).  rope_cos and
+ * rope_sin are device fp32 tables [max_len, head_dim/2] (row = position, 16-byte aligned) holding
+ * cos / sin of position * theta^(-2j/head_dim), or both NULL for no rotation.  `window` is read for
+ * RLX_MASK_SLIDING_WINDOW only.  head_dim in {32, 64}.  Key blocks that no row of a 128-row query
+ * tile can see are neither loaded nor multiplied.  Asynchronous on cuda_stream; the caller owns
+ * every buffer; nothing is allocated.  Errors: RLX_ERR_INVALID_ARG for null / misaligned pointers,
+ * a lone rope table, an unknown kind or window < 1; RLX_ERR_UNSUPPORTED for other head sizes or
+ * lengths beyond the maximum.
+ */
+#define RLX_MASK_NONE 0
+#define RLX_MASK_CAUSAL 1
+#define RLX_MASK_SLIDING_WINDOW 2
+#define RLX_ATTENTION_KIND_MAX_LEN 32768
+rlx_status_t rlx_attention_kind_bf16(const void *qkv_bf16, int32_t rows, const int32_t *seq_start,
+                                     const int32_t *seq_len, int32_t batch, int32_t max_len,
+                                     int32_t num_heads, int32_t head_dim, int32_t mask_kind,
+                                     int32_t window, const float *rope_cos, const float *rope_sin,
+                                     void *ctx_bf16, void *cuda_stream);
+
+/*
+ * The fused QK-RoPE region of Section 3.2 on its own: rotates the q and the k column blocks of the
+ * packed projection IN PLACE (one pass over both; v is not touched), with the pairing, positions and
+ * tables of rlx_attention_kind_bf16 -- after this call, rlx_attention_kind_bf16 with NULL tables gives
+ * bit for bit what it gives on the unrotated buffer with the tables.  One pass over 2/3 of qkv at HBM
+ * speed, where the in-attention form rotates every key block once per 128-row query tile: prefer this
+ * call for sequences of more than a few hundred rows, the in-attention form when qkv must stay
+ * read-only.  qkv: device bf16 [rows, 3*num_heads*head_dim], 16-byte aligned, modified; other
+ * arguments and error behaviour as in rlx_attention_kind_bf16 (both tables required).
+ */
+rlx_status_t rlx_qk_rope_bf16(void *qkv_bf16, int32_t rows, const int32_t *seq_start, const int32_t *seq_len,
+                              int32_t batch, int32_t max_len, int32_t num_heads, int32_t head_dim,
+                              const float *rope_cos, const float *rope_sin, void *cuda_stream);
+
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
 rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,
                              int32_t seq, int32_t hidden, float *out, void *cuda_stream);

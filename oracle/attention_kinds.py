@@ -90,3 +90,17 @@ def attention_packed(qkv: np.ndarray, seq_start, seq_len, num_heads: int, kind: 
         if n > 0:
             out[s0:s0 + n] = attention_one(qkv[s0:s0 + n], num_heads, kind, window, rope_theta)
     return out
+
+
+def rope_qk_packed(qkv: np.ndarray, seq_start, seq_len, num_heads: int, theta: float = 10000.0) -> np.ndarray:
+    """The QK-RoPE region on packed rows: q and k column blocks rotated by each row's position within its
+    sequence, v and rows outside every sequence returned unchanged."""
+    out = np.array(qkv, dtype=np.float64, copy=True)
+    H = out.shape[1] // 3
+    d = H // num_heads
+    for s0, n in zip(np.asarray(seq_start), np.asarray(seq_len)):
+        s0, n = int(s0), int(n)
+        for part in (0, 1):
+            blk = out[s0:s0 + n, part * H:(part + 1) * H].reshape(n, num_heads, d)
+            out[s0:s0 + n, part * H:(part + 1) * H] = rope(blk, theta).reshape(n, H)
+    return out

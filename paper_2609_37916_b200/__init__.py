@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     RlxError,
     attention_bf16,
     attention_f32,
+    attention_kind_bf16,
     attention_packed_bf16,
     embed_layernorm,
     gemm_bf16,
@@ -19,5 +20,7 @@ from .binding import (  # noqa: F401
     pack_sequences,
     lib_path,
     pool_l2norm,
+    qk_rope_bf16,
+    rope_tables,
     upload_weights,
 )

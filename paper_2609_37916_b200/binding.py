@@ -36,7 +36,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_pool_l2norm",
 )
 
 
@@ -291,6 +291,43 @@ def attention_packed_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int,
                                              num_heads, H // num_heads, _ptr(ctx), impl, _ptr(status), _stream(stream)),
            "rlx_attention_packed_bf16")
     return ctx
+
+
+MASK_NONE, MASK_CAUSAL, MASK_SLIDING_WINDOW = 0, 1, 2
+ATTENTION_KIND_MAX_LEN = 32768
+
+
+def rope_tables(max_len: int, head_dim: int, theta: float = 10000.0, device="cuda"):
+    """cos / sin of position * theta^(-2j/head_dim) as fp32 device tables [max_len, head_dim/2] (the
+    constant inputs rlx_attention_kind_bf16 takes; angles are formed in fp64 on the host)."""
+    j = torch.arange(head_dim // 2, dtype=torch.float64)
+    ang = torch.arange(max_len, dtype=torch.float64)[:, None] * torch.pow(torch.tensor(theta, dtype=torch.float64),
+                                                                         -2.0 * j / head_dim)[None, :]
+    return ang.cos().float().contiguous().to(device), ang.sin().float().contiguous().to(device)
+
+
+def attention_kind_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, mask_kind: int, window: int = 0,
+                        rope=None, out=None, stream=None):
+    """qkv: packed [rows, 3H] bf16; rope: None or the (cos, sin) pair of rope_tables; returns ctx [rows, H]
+    (a fresh zero-filled tensor, or `out` with rows outside every sequence left as they were)."""
+    rows, H3 = qkv.shape
+    H = H3 // 3
+    ctx = torch.zeros((rows, H), dtype=torch.bfloat16, device=qkv.device) if out is None else out
+    cos, sin = rope if rope is not None else (None, None)
+    _check(_load().rlx_attention_kind_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len,
+                                           num_heads, H // num_heads, mask_kind, window, _ptr(cos), _ptr(sin),
+                                           _ptr(ctx), _stream(stream)),
+           "rlx_attention_kind_bf16")
+    return ctx
+
+
+def qk_rope_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, rope, stream=None):
+    """Rotates the q and k column blocks of packed qkv [rows, 3H] bf16 IN PLACE; returns qkv."""
+    rows, H3 = qkv.shape
+    cos, sin = rope
+    _check(_load().rlx_qk_rope_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len, num_heads,
+                                    H3 // 3 // num_heads, _ptr(cos), _ptr(sin), _stream(stream)), "rlx_qk_rope_bf16")
+    return qkv
 
 
 def attention_f32(qkv, mask, num_heads: int, stream=None):

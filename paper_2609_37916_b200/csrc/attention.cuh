@@ -86,14 +86,30 @@ struct AttSmem {
     int q_any;
 };
 
+// Positional visibility and rotary embedding (packed mode only; template switches, so the encoder's
+// instantiation carries none of it):
+//   MK = 1: key k is visible to query i iff  i - window < k <= i  (causal when window >= the sequence
+//           length).  Key blocks wholly outside a CTA's rows are never loaded, blocks wholly outside a
+//           warp's 16 rows are skipped by that warp, and the element test runs only in blocks that a
+//           boundary crosses.
+//   ROPE:   q and k rows are rotated in shared memory after they land ("rotate-half" pairing of column
+//           j with j + D/2 by the angle whose cosine / sine the caller tabulates per position), in fp32,
+//           and rounded back to bf16 for the tensor-core products.  Each thread rotates what it copied
+//           itself, one key block ahead of the block being multiplied, so no barrier is added.
+struct AttKind {
+    int window;
+    const float* rope_cos;   // [max_len, D/2]
+    const float* rope_sin;
+};
+
 // Two addressing modes share the kernel:
 //   padded: seq_start == nullptr.  Sequence b occupies rows b*S .. b*S+S; `mask` flags valid keys.
 //   packed: rows of sequence b are seq_start[b] .. seq_start[b]+seq_len[b], all valid (mask unused).
-template <int D>
+template <int D, int MK = 0, bool ROPE = false>
 __global__ void __launch_bounds__(kAttThreads, D == 32 ? 3 : 2)
 attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ mask,
                       const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
-                      __nv_bfloat16* __restrict__ ctx, int S, int H, float scale_log2e) {
+                      __nv_bfloat16* __restrict__ ctx, int S, int H, float scale_log2e, AttKind kind) {
     using SM = AttSmem<D>;
     constexpr int STR = SM::kStride;
     constexpr int KT = D / 16;       // k-tiles of the QK^T product
@@ -146,7 +162,12 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             return;
         }
     }
-    const int nblk = (kv_end + kAttBlockN - 1) / kAttBlockN;
+    int jb0 = 0, nblk = (kv_end + kAttBlockN - 1) / kAttBlockN;   // key blocks jb0 .. nblk-1
+    if (MK) {
+        const int q_hi = min(q0 + kAttBlockM, len);                // one past this CTA's last real row
+        jb0 = max(0, q0 - kind.window + 1) / kAttBlockN;
+        nblk = (q_hi + kAttBlockN - 1) / kAttBlockN;
+    }
 
     auto load_rows = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row, int nrows) {
         for (int i = tid; i < nrows * CH; i += kAttThreads) {
@@ -156,15 +177,50 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             cp_async16(smem_u32(dst + r * STR + c * 8), src, ok);
         }
     };
-    load_rows(qbase, sm.q, q0, kAttBlockM);
+    // Rotary mode: a thread copies BOTH halves of the column pairs it will rotate (chunk c and chunk
+    // c + CH/2 of a row), so that once its own copies have completed it can rotate them in place with no
+    // CTA barrier in between; the barrier that publishes the tile to the other warps comes afterwards.
+    auto load_rows_paired = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row, int nrows) {
+        constexpr int CPR = D / 16;
+        for (int i = tid; i < nrows * CPR; i += kAttThreads) {
+            const int r = i / CPR, c = i % CPR;
+            const bool ok = first_row + r < len;
+            const __nv_bfloat16* src = base + (size_t)(ok ? first_row + r : 0) * ld + c * 8;
+            cp_async16(smem_u32(dst + r * STR + c * 8), src, ok);
+            cp_async16(smem_u32(dst + r * STR + D / 2 + c * 8), src + D / 2, ok);
+        }
+    };
+    auto load_qk = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row, int nrows) {
+        if (ROPE) load_rows_paired(base, dst, first_row, nrows);
+        else load_rows(base, dst, first_row, nrows);
+    };
+    load_qk(qbase, sm.q, q0, kAttBlockM);
 #pragma unroll
     for (int j = 0; j < kAttStages - 1; ++j) {
-        if (j < nblk) {
-            load_rows(kbase, sm.k[j], j * kAttBlockN, kAttBlockN);
-            load_rows(vbase, sm.v[j], j * kAttBlockN, kAttBlockN);
+        if (jb0 + j < nblk) {
+            load_qk(kbase, sm.k[j], (jb0 + j) * kAttBlockN, kAttBlockN);
+            load_rows(vbase, sm.v[j], (jb0 + j) * kAttBlockN, kAttBlockN);
         }
         cp_async_commit();
     }
+    // rotate, in place, the column pairs of a q or k tile that THIS thread copied (same task mapping as
+    // load_rows_paired); row r holds position first_pos + r
+    auto rope_rows = [&](__nv_bfloat16* tile, int first_pos, int nrows) {
+        constexpr int CPR = D / 16;   // tasks per row: 8 (lo, hi) column pairs each
+        for (int i = tid; i < nrows * CPR; i += kAttThreads) {
+            const int r = i / CPR, c = i % CPR;
+            const int pos = first_pos + r;
+            if (pos >= len) continue;   // zero-filled row
+            uint4* plo = reinterpret_cast<uint4*>(tile + r * STR + c * 8);
+            uint4* phi = reinterpret_cast<uint4*>(tile + r * STR + D / 2 + c * 8);
+            uint4 lo = *plo, hi = *phi;
+            const float4* pc = reinterpret_cast<const float4*>(kind.rope_cos + (size_t)pos * (D / 2) + c * 8);
+            const float4* ps = reinterpret_cast<const float4*>(kind.rope_sin + (size_t)pos * (D / 2) + c * 8);
+            rope_rotate8(lo, hi, __ldg(pc), __ldg(pc + 1), __ldg(ps), __ldg(ps + 1));
+            *plo = lo;
+            *phi = hi;
+        }
+    };
 
     uint32_t qf[KT][4];
     float o[ND][4];
@@ -179,18 +235,29 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     const int g = lane >> 2, t4 = lane & 3;
     const bool warp_active = q0 + warp * 16 < len;   // warps whose 16 rows lie past the sequence only sync
 
-    for (int j = 0; j < nblk; ++j) {
-        const int buf = j % kAttStages;
+    const int r0 = q0 + warp * 16;   // first query row of this warp (index within the sequence)
+    for (int j = jb0; j < nblk; ++j) {
+        const int buf = (j - jb0) % kAttStages;
         cp_async_wait<kAttStages - 2>();   // block j (and Q) have landed
+        if (ROPE && j == jb0) {            // own copies of Q and the first key block: rotate before publishing
+            rope_rows(sm.q, q0, kAttBlockM);
+            rope_rows(sm.k[buf], j * kAttBlockN, kAttBlockN);
+        }
         __syncthreads();                   // ... for every thread; and block j-1's stage is free
         if (j + kAttStages - 1 < nblk) {
-            const int nb = (j + kAttStages - 1) % kAttStages;
-            load_rows(kbase, sm.k[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
+            const int nb = (j - jb0 + kAttStages - 1) % kAttStages;
+            load_qk(kbase, sm.k[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
             load_rows(vbase, sm.v[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
         }
         cp_async_commit();
+        if (ROPE && j + 1 < nblk) {
+            // block j+1 is rotated one step ahead by the threads that copied it; nobody reads it before
+            // the barrier at the top of the next iteration
+            cp_async_wait<kAttStages - 2>();
+            rope_rows(sm.k[(j + 1 - jb0) % kAttStages], (j + 1) * kAttBlockN, kAttBlockN);
+        }
         if (!warp_active) continue;
-        if (j == 0) {
+        if (j == jb0) {
 #pragma unroll
             for (int kt = 0; kt < KT; ++kt) {
                 const int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
@@ -198,6 +265,8 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 ldmatrix_x4(smem_u32(sm.q + r * STR + c), qf[kt][0], qf[kt][1], qf[kt][2], qf[kt][3]);
             }
         }
+        const int k0 = j * kAttBlockN;
+        if (MK && (k0 > r0 + 15 || k0 + kAttBlockN - 1 <= r0 - kind.window)) continue;   // nothing visible
         // ---- S = Q K^T for 64 keys: 8 n-tiles x 4 accumulators ----
         float s[8][4];
 #pragma unroll
@@ -215,16 +284,30 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             }
         }
         // ---- masking only where the block has an invalid key ----
-        const int k0 = j * kAttBlockN;
-        const bool need_mask = packed ? (k0 + kAttBlockN > len) : (sm.blk_full[j] == 0);
-        if (need_mask) {
+        if (MK) {
+            // the block needs the element test unless every key is visible to all 16 rows
+            if (k0 + kAttBlockN > len || k0 + kAttBlockN - 1 > r0 || k0 <= r0 + 15 - kind.window) {
+                const int ia = r0 + g, ib = ia + 8;   // rows of accumulators {0,1} and {2,3}
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                const int kk = k0 + nt * 8 + 2 * t4;
-                const bool v0 = packed ? (kk < len) : (sm.bias[kk] == 0.f);
-                const bool v1 = packed ? (kk + 1 < len) : (sm.bias[kk + 1] == 0.f);
-                if (!v0) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
-                if (!v1) { s[nt][1] = -INFINITY; s[nt][3] = -INFINITY; }
+                for (int nt = 0; nt < 8; ++nt) {
+                    const int kk = k0 + nt * 8 + 2 * t4;
+                    if (!(kk < len && kk <= ia && kk > ia - kind.window)) s[nt][0] = -INFINITY;
+                    if (!(kk + 1 < len && kk + 1 <= ia && kk + 1 > ia - kind.window)) s[nt][1] = -INFINITY;
+                    if (!(kk < len && kk <= ib && kk > ib - kind.window)) s[nt][2] = -INFINITY;
+                    if (!(kk + 1 < len && kk + 1 <= ib && kk + 1 > ib - kind.window)) s[nt][3] = -INFINITY;
+                }
+            }
+        } else {
+            const bool need_mask = packed ? (k0 + kAttBlockN > len) : (sm.blk_full[j] == 0);
+            if (need_mask) {
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    const int kk = k0 + nt * 8 + 2 * t4;
+                    const bool v0 = packed ? (kk < len) : (sm.bias[kk] == 0.f);
+                    const bool v1 = packed ? (kk + 1 < len) : (sm.bias[kk + 1] == 0.f);
+                    if (!v0) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
+                    if (!v1) { s[nt][1] = -INFINITY; s[nt][3] = -INFINITY; }
+                }
             }
         }
         // ---- running max on raw scores (the positive scale commutes with max) ----

@@ -137,10 +137,16 @@ cudaError_t init_kernels_for_current_device() {
                                   rlx::tca::Smem<32>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tca::Smem<64>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)sizeof(rlx::AttSmem<32>))) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  (int)sizeof(rlx::AttSmem<64>))) != cudaSuccess) return e;
+#define RLX_ATT_SMEM_ATTR(D, MK, ROPE)                                                                       \
+    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<D, MK, ROPE>,                                  \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(rlx::AttSmem<D>))) != \
+        cudaSuccess)                                                                                        \
+        return e;
+    RLX_ATT_SMEM_ATTR(32, 0, false) RLX_ATT_SMEM_ATTR(64, 0, false)
+    RLX_ATT_SMEM_ATTR(32, 0, true) RLX_ATT_SMEM_ATTR(64, 0, true)
+    RLX_ATT_SMEM_ATTR(32, 1, false) RLX_ATT_SMEM_ATTR(64, 1, false)
+    RLX_ATT_SMEM_ATTR(32, 1, true) RLX_ATT_SMEM_ATTR(64, 1, true)
+#undef RLX_ATT_SMEM_ATTR
     if (dev < 64) done[dev] = true;
     return cudaSuccess;
 }
@@ -237,17 +243,33 @@ rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H
     return RLX_OK;
 }
 
+// positional = false: every key of the sequence is visible (the encoder's attention); true: the window
+// rule of the kernel's MK = 1 mode (packed rows only).  rope_cos == nullptr: no rotary embedding.
 rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const int32_t* seq_start,
-                                   const int32_t* seq_len, int B, int S, int h, int d, bf16* ctx, cudaStream_t st) {
+                                   const int32_t* seq_len, int B, int S, int h, int d, bf16* ctx, cudaStream_t st,
+                                   bool positional = false, int window = 0, const float* rope_cos = nullptr,
+                                   const float* rope_sin = nullptr) {
     const int H = h * d;
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
     dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
-    if (d == 32)
-        RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<32>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<32>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
-    else if (d == 64)
-        RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<64>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<64>), st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e));
-    else
-        return RLX_ERR_UNSUPPORTED;
+    const rlx::AttKind kind{window, rope_cos, rope_sin};
+    const bool rope = rope_cos != nullptr;
+    if (d != 32 && d != 64) return RLX_ERR_UNSUPPORTED;
+#define RLX_ATT_LAUNCH(D, MK, ROPE)                                                                              \
+    RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<D, MK, ROPE>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<D>), \
+                           st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e, kind))
+    if (d == 32) {
+        if (!positional && !rope) RLX_ATT_LAUNCH(32, 0, false);
+        else if (!positional) RLX_ATT_LAUNCH(32, 0, true);
+        else if (!rope) RLX_ATT_LAUNCH(32, 1, false);
+        else RLX_ATT_LAUNCH(32, 1, true);
+    } else {
+        if (!positional && !rope) RLX_ATT_LAUNCH(64, 0, false);
+        else if (!positional) RLX_ATT_LAUNCH(64, 0, true);
+        else if (!rope) RLX_ATT_LAUNCH(64, 1, false);
+        else RLX_ATT_LAUNCH(64, 1, true);
+    }
+#undef RLX_ATT_LAUNCH
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -992,6 +1014,41 @@ rlx_status_t rlx_attention_packed_bf16(const void* qkv, int32_t rows, const int3
     if (impl == 1)
         return launch_attention_bf16((const bf16*)qkv, nullptr, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, st);
     return RLX_ERR_INVALID_ARG;
+}
+
+rlx_status_t rlx_attention_kind_bf16(const void* qkv, int32_t rows, const int32_t* seq_start, const int32_t* seq_len,
+                                     int32_t B, int32_t max_len, int32_t h, int32_t d, int32_t mask_kind,
+                                     int32_t window, const float* rope_cos, const float* rope_sin, void* ctx,
+                                     void* stream) {
+    if (!qkv || !seq_start || !seq_len || !ctx || B <= 0 || max_len <= 0 || h <= 0 || rows <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(qkv) || !aligned16(ctx) || !aligned16(rope_cos) || !aligned16(rope_sin)) return RLX_ERR_INVALID_ARG;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr)) return RLX_ERR_INVALID_ARG;
+    if (mask_kind != RLX_MASK_NONE && mask_kind != RLX_MASK_CAUSAL && mask_kind != RLX_MASK_SLIDING_WINDOW)
+        return RLX_ERR_INVALID_ARG;
+    if (mask_kind == RLX_MASK_SLIDING_WINDOW && window < 1) return RLX_ERR_INVALID_ARG;
+    if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    const bool positional = mask_kind != RLX_MASK_NONE;
+    const int w = mask_kind == RLX_MASK_SLIDING_WINDOW ? window : (1 << 30);   // causal: the window never cuts
+    return launch_attention_bf16((const bf16*)qkv, nullptr, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx,
+                                 static_cast<cudaStream_t>(stream), positional, w, rope_cos, rope_sin);
+}
+
+rlx_status_t rlx_qk_rope_bf16(void* qkv, int32_t rows, const int32_t* seq_start, const int32_t* seq_len, int32_t B,
+                              int32_t max_len, int32_t h, int32_t d, const float* rope_cos, const float* rope_sin,
+                              void* stream) {
+    if (!qkv || !seq_start || !seq_len || !rope_cos || !rope_sin || B <= 0 || max_len <= 0 || h <= 0 || rows <= 0)
+        return RLX_ERR_INVALID_ARG;
+    if (!aligned16(qkv) || !aligned16(rope_cos) || !aligned16(rope_sin)) return RLX_ERR_INVALID_ARG;
+    if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    dim3 grid((max_len + rlx::kRopeRows - 1) / rlx::kRopeRows, B);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (d == 32)
+        rlx::qk_rope_kernel<32><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h, rope_cos, rope_sin);
+    else
+        rlx::qk_rope_kernel<64><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h, rope_cos, rope_sin);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
 }
 
 void rlx_debug_set_attn_trace(void* p) { g_attn_dbg = static_cast<unsigned long long*>(p); }

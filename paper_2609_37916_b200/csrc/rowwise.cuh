@@ -140,6 +140,40 @@ __device__ __forceinline__ int find_sequence(const int32_t* __restrict__ seq_sta
     return lo;
 }
 
+// Fused QK-RoPE: rotates, in place, the q and k column blocks of packed [rows, 3H] projections (v is
+// left alone).  grid = (row tiles of kRopeRows, sequences); one task = eight (j, j + D/2) column pairs
+// of one head of q or k of one row: 2 x 16 bytes in, 2 x 16 bytes out, consecutive lanes on consecutive
+// 16-byte chunks.  A row's position is its index within its sequence.
+constexpr int kRopeRows = 16;
+constexpr int kRopeThreads = 256;
+template <int D>
+__global__ void __launch_bounds__(kRopeThreads)
+qk_rope_kernel(__nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ seq_start,
+               const int32_t* __restrict__ seq_len, int heads, const float* __restrict__ rope_cos,
+               const float* __restrict__ rope_sin) {
+    constexpr int CPR = D / 16;                 // tasks per head
+    const int b = blockIdx.y;
+    const int len = __ldg(seq_len + b);
+    const int p0 = blockIdx.x * kRopeRows;
+    if (p0 >= len) return;
+    const int H = heads * D;
+    const size_t row0 = (size_t)__ldg(seq_start + b);
+    const int per_row = 2 * heads * CPR;        // q heads then k heads: columns 0 .. 2H are contiguous
+    const int nrows = min(kRopeRows, len - p0);
+    for (int i = threadIdx.x; i < nrows * per_row; i += kRopeThreads) {
+        const int r = i / per_row, t = i % per_row;
+        const int hd = t / CPR, c = t % CPR;    // hd in [0, 2*heads): head of q (first H columns) or k
+        const int pos = p0 + r;
+        __nv_bfloat16* base = qkv + (row0 + pos) * (size_t)(3 * H) + hd * D + c * 8;
+        uint4 lo = *reinterpret_cast<const uint4*>(base), hi = *reinterpret_cast<const uint4*>(base + D / 2);
+        const float4* pc = reinterpret_cast<const float4*>(rope_cos + (size_t)pos * (D / 2) + c * 8);
+        const float4* ps = reinterpret_cast<const float4*>(rope_sin + (size_t)pos * (D / 2) + c * 8);
+        rope_rotate8(lo, hi, __ldg(pc), __ldg(pc + 1), __ldg(ps), __ldg(ps + 1));
+        *reinterpret_cast<uint4*>(base) = lo;
+        *reinterpret_cast<uint4*>(base + D / 2) = hi;
+    }
+}
+
 // x[row] = LN(word[id] + pos[s] + type[0]).  Ids outside [0, V) are clamped and flagged.
 // Padded mode (seq_start == nullptr): row = token t = b*S + s for all T tokens.
 // Packed mode: row p < seq_start[B] belongs to sequence b = find_sequence(p) at position

@@ -247,3 +247,20 @@ def test_rope_leaves_values_alone_and_changes_attention():
     qkv = _rand_qkv(rng, L, h, d, 2.0)
     assert not np.allclose(ak.attention_one(qkv, h, ak.KIND_CAUSAL, 0, 10000.0),
                            ak.attention_one(qkv, h, ak.KIND_CAUSAL, 0, None))
+
+
+def test_rope_qk_packed_composes_with_attention():
+    """Rotating q,k first and then attending without rotation is the rotary attention; v, and rows that
+    belong to no sequence, pass through untouched."""
+    rng = np.random.default_rng(10)
+    h, d = 2, 8
+    H = h * d
+    lens = [6, 1, 9]
+    start = np.concatenate([[0], np.cumsum(lens)])[:-1]
+    qkv = _rand_qkv(rng, sum(lens) + 3, h, d)
+    rot = ak.rope_qk_packed(qkv, start, lens, h, 10000.0)
+    assert np.array_equal(rot[:, 2 * H:], qkv[:, 2 * H:]) and np.array_equal(rot[sum(lens):], qkv[sum(lens):])
+    assert np.array_equal(rot[start], qkv[start])                  # position 0 of every sequence: identity
+    a = ak.attention_packed(rot, start, lens, h, ak.KIND_CAUSAL, 0, None)
+    b = ak.attention_packed(qkv, start, lens, h, ak.KIND_CAUSAL, 0, 10000.0)
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-15)
