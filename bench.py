@@ -567,6 +567,92 @@ def run_qk_rope(args):
     print(json.dumps(line), flush=True)
 
 
+def run_scaled_matmul(args):
+    """`--op scaled_matmul`: one step = rlx_scaled_matmul_bf16 (block-scaled minifloat weights dequantised
+    to bf16, then the tcgen05 GEMM with bias) at the BERT-base FFN-up shape over 32,768 tokens; the
+    dequantisation pass is also timed alone on a matrix larger than L2."""
+    import torch
+    import paper_2609_37916_b200 as rlx
+    from synth.inputs import make_block_scaled_weights, pack_nibbles
+
+    fmts = {"fp8_e4m3": (rlx.binding.FMT_FP8_E4M3, 8, 0x7E, False, "E4M3"), "fp4_e2m1": (rlx.binding.FMT_FP4_E2M1, 4, 7, True, "E2M1")}
+    word, bits, maxmag, packed, oname = fmts[args.fmt]
+    M, N, K = 32768, 3072, 768
+    torch.cuda.set_device(0)
+    g = torch.Generator(device="cuda").manual_seed(3)
+    a = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+    bias = torch.randn(N, device="cuda", generator=g)
+    codes, scales = make_block_scaled_weights(3, N, K, bits, maxmag, 122, 128)
+    dev_codes = torch.from_numpy(pack_nibbles(codes) if packed else codes).cuda()
+    dev_scales = torch.from_numpy(scales).cuda()
+    w_scratch = torch.empty(N, K, dtype=torch.bfloat16, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    # the big matrix for the dequantisation pass alone
+    N2, K2 = 16384, 8192
+    codes2, scales2 = make_block_scaled_weights(4, N2, K2, bits, maxmag, 122, 128)
+    dev_codes2 = torch.from_numpy(pack_nibbles(codes2) if packed else codes2).cuda()
+    dev_scales2 = torch.from_numpy(scales2).cuda()
+    w2 = torch.empty(N2, K2, dtype=torch.bfloat16, device="cuda")
+    sampler = ClockSampler(0)
+    sampler.start()
+
+    def timed(fn):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        out = fn()
+        e1.record()
+        return e0, e1, out
+
+    y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    mm = lambda: rlx.scaled_matmul_bf16(a, dev_codes, dev_scales, word, bias, w_scratch=w_scratch, out=y)
+    dq = lambda: rlx.dequant_block_scaled_bf16(dev_codes2, dev_scales2, N2, K2, word, out=w2)
+    for _ in range(max(args.warmup, 3)):
+        timed(mm)
+        timed(dq)
+    torch.cuda.synchronize()
+    sampler.active.set()
+    ev_mm = [timed(mm) for _ in range(args.steps)]
+    ev_dq = [timed(dq) for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    sampler.active.clear()
+    sampler.stop()
+    ms = [x.elapsed_time(y) for x, y, _ in ev_mm]
+    ms_dq = [x.elapsed_time(y) for x, y, _ in ev_dq]
+    p50, p50_dq = statistics.median(ms), statistics.median(ms_dq)
+    peaks, peak_kind = load_peaks()
+    flops = 2.0 * M * N * K
+    dq_bytes = N2 * K2 * (0.5 if packed else 1.0) + N2 * K2 / 32 + 2.0 * N2 * K2
+    # oracle: fp64 matmul on the dequantised grid for the first rows
+    from oracle import scaled_matmul as osm
+    m0 = 256
+    t0 = time.perf_counter()
+    ref = osm.scaled_matmul(a[:m0].float().cpu().numpy().astype(np.float64), codes, scales, getattr(osm, oname),
+                            bias.cpu().numpy().astype(np.float64))
+    t_or = time.perf_counter() - t0
+    got = ev_mm[-1][2][:m0].float().cpu().numpy().astype(np.float64)
+    ach = flops / (p50 * 1e-3) / 1e12
+    line = {
+        "metric": "ScaledMatMul tokens/s (p50 ms reported alongside)", "op": "scaled_matmul",
+        "value": M * args.steps / (sum(ms) / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "p50_ms": p50, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"M={M} tokens, N={N}, K={K} (BERT-base FFN-up), weights {args.fmt} with E8M0 scales per 32, "
+                               "dequantise + GEMM(+bias) per step", "l2": "256 MiB flush write between steps"},
+        "gpu_launches": 2 * args.steps, "clocks": sampler.summary(),
+        "roofline": {"kernel": "gemm_tcgen05_kernel", "bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"], "traffic": None, "peak_source": peak_kind,
+                     "note": "interval = dequantisation pass + GEMM"},
+        "dequant": {"workload": f"{N2} x {K2} weights", "p50_ms": p50_dq, "bound": "hbm",
+                    "achieved": dq_bytes / (p50_dq * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": dq_bytes / (p50_dq * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "cpu_baseline": {"value": m0 / t_or, "unit": "tokens/s", "cores": usable_cores(), "kind": "oracle",
+                         "sample": f"first {m0} rows, 1 run, {t_or:.2f} s"},
+        "parity_on_sample": {"max_abs_err": float(np.abs(got - ref).max()), "max_abs_ref": float(np.abs(ref).max())},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -574,7 +660,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="c2", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope"])
+    ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope", "scaled_matmul"])
+    ap.add_argument("--fmt", default="fp8_e4m3", choices=["fp8_e4m3", "fp4_e2m1"])
     ap.add_argument("--mask", default="causal", choices=["none", "causal", "sliding"])
     ap.add_argument("--window", type=int, default=512)
     ap.add_argument("--rope", type=int, default=1)
@@ -582,7 +669,7 @@ def main():
     if args.op != "encoder":
         if args.impl != "ours" or args.gpus != 1:
             raise SystemExit(f"--op {args.op} runs on one GPU with --impl ours")
-        (run_attention_kind if args.op == "attention_kind" else run_qk_rope)(args)
+        {"attention_kind": run_attention_kind, "qk_rope": run_qk_rope, "scaled_matmul": run_scaled_matmul}[args.op](args)
         return
     if args.impl == "reference":
         run_reference_arm(args)

@@ -375,6 +375,41 @@ rlx_status_t rlx_qk_rope_bf16(void *qkv_bf16, int32_t rows, const int32_t *seq_s
                               int32_t batch, int32_t max_len, int32_t num_heads, int32_t head_dim,
                               const float *rope_cos, const float *rope_sin, void *cuda_stream);
 
+/*
+ * ScaledMatMul (Section 3.2 "block-scaled tensor-core minifloats -- the FP8/FP6/FP4 grids and arbitrary
+ * fNeXmY formats"; Section 5): weight-only quantisation, the paper fixing neither layout nor block
+ * size.  Reading used here (the open microscaling convention):
+ *   code    sign | X exponent bits | Y mantissa bits, bias 2^(X-1)-1, gradual underflow; one code per
+ *           byte (low bits), or two 4-bit codes per byte with RLX_MINIFLOAT_PACKED4 (low nibble = the
+ *           smaller k).  special = 0: every code finite; 1: all-ones magnitude is NaN (FP8 E4M3);
+ *           2: top exponent is infinity / NaN (FP8 E5M2).
+ *   scale   one E8M0 byte per 32 consecutive k of a row: 2^(byte - 127), 255 = NaN.
+ *   weight  W[n,k] = value(code[n,k]) * scale[n, k/32].
+ * rlx_dequant_block_scaled_bf16 writes W as bf16 [N,K]: exact whenever the product lies in bf16's
+ * range (these grids carry at most 7 significant bits), correctly rounded otherwise (down to 2^-149
+ * in magnitude).  rlx_scaled_matmul_bf16 = that pass into `w_scratch_bf16` ([N,K] bf16, caller's)
+ * followed by rlx_gemm_bf16 on it (tcgen05 path, fp32 accumulation, fused epilogue), i.e. the F32
+ * reference on the dequantised grid with bf16 activations.  The weights of an encoder are static, so
+ * the intended use is to dequantise once and keep W resident (a B200 has the HBM for it); a GEMM
+ * that re-decodes codes per tile would add work to the tensor-core loop and save no traffic here.
+ * codes: device, 16-byte aligned, [N,K] bytes or [N,K/2]; scales: device [N,K/32]; K % 32 == 0
+ * (RLX_ERR_UNSUPPORTED otherwise); a malformed format word or a code wider than its container gives
+ * RLX_ERR_INVALID_ARG.  Asynchronous on cuda_stream; nothing is allocated.
+ */
+#define RLX_MINIFLOAT(ebits, mbits, special) (((ebits) << 8) | ((mbits) << 4) | (special))
+#define RLX_MINIFLOAT_PACKED4 0x1000
+#define RLX_FMT_FP8_E4M3 RLX_MINIFLOAT(4, 3, 1)
+#define RLX_FMT_FP8_E5M2 RLX_MINIFLOAT(5, 2, 2)
+#define RLX_FMT_FP6_E3M2 RLX_MINIFLOAT(3, 2, 0)
+#define RLX_FMT_FP6_E2M3 RLX_MINIFLOAT(2, 3, 0)
+#define RLX_FMT_FP4_E2M1 (RLX_MINIFLOAT(2, 1, 0) | RLX_MINIFLOAT_PACKED4)
+rlx_status_t rlx_dequant_block_scaled_bf16(const void *codes, const void *scales_e8m0, int32_t N, int32_t K,
+                                           int32_t format, void *w_bf16, void *cuda_stream);
+rlx_status_t rlx_scaled_matmul_bf16(const void *A, const void *codes, const void *scales_e8m0, int32_t format,
+                                    const float *bias, const void *residual, rlx_epilogue_t epilogue,
+                                    int32_t M, int32_t N, int32_t K, void *w_scratch_bf16, void *out,
+                                    int32_t *status, void *cuda_stream);
+
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
 rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,
                              int32_t seq, int32_t hidden, float *out, void *cuda_stream);

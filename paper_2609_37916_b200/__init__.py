@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     attention_f32,
     attention_kind_bf16,
     attention_packed_bf16,
+    dequant_block_scaled_bf16,
     embed_layernorm,
     gemm_bf16,
     gemm_residual_layernorm_bf16,
@@ -22,5 +23,6 @@ from .binding import (  # noqa: F401
     pool_l2norm,
     qk_rope_bf16,
     rope_tables,
+    scaled_matmul_bf16,
     upload_weights,
 )

@@ -36,7 +36,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_pool_l2norm",
 )
 
 
@@ -328,6 +328,37 @@ def qk_rope_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, rope, st
     _check(_load().rlx_qk_rope_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len, num_heads,
                                     H3 // 3 // num_heads, _ptr(cos), _ptr(sin), _stream(stream)), "rlx_qk_rope_bf16")
     return qkv
+
+
+def minifloat(ebits: int, mbits: int, special: int = 0, packed4: bool = False) -> int:
+    """Format word of rlx_dequant_block_scaled_bf16 (special: 0 none, 1 all-ones magnitude NaN, 2 IEEE)."""
+    return (ebits << 8) | (mbits << 4) | special | (0x1000 if packed4 else 0)
+
+
+FMT_FP8_E4M3, FMT_FP8_E5M2 = minifloat(4, 3, 1), minifloat(5, 2, 2)
+FMT_FP6_E3M2, FMT_FP6_E2M3 = minifloat(3, 2, 0), minifloat(2, 3, 0)
+FMT_FP4_E2M1 = minifloat(2, 1, 0, packed4=True)
+
+
+def dequant_block_scaled_bf16(codes, scales, N: int, K: int, fmt: int, out=None, stream=None):
+    """codes uint8 [N,K] (or [N,K/2] packed nibbles), scales uint8 [N,K/32] -> W bf16 [N,K]."""
+    w = torch.empty((N, K), dtype=torch.bfloat16, device=codes.device) if out is None else out
+    _check(_load().rlx_dequant_block_scaled_bf16(_ptr(codes), _ptr(scales), N, K, fmt, _ptr(w), _stream(stream)),
+           "rlx_dequant_block_scaled_bf16")
+    return w
+
+
+def scaled_matmul_bf16(a, codes, scales, fmt: int, bias, residual=None, epilogue: int = EPI_BIAS, w_scratch=None,
+                       out=None, status=None, stream=None):
+    """out bf16 [M,N] = epilogue(a [M,K] . dequant(codes, scales)^T + bias); N = rows of codes."""
+    M, K = a.shape
+    N = codes.shape[0]
+    w = torch.empty((N, K), dtype=torch.bfloat16, device=a.device) if w_scratch is None else w_scratch
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device) if out is None else out
+    _check(_load().rlx_scaled_matmul_bf16(_ptr(a), _ptr(codes), _ptr(scales), fmt, _ptr(bias), _ptr(residual), epilogue,
+                                          M, N, K, _ptr(w), _ptr(out), _ptr(status), _stream(stream)),
+           "rlx_scaled_matmul_bf16")
+    return out
 
 
 def attention_f32(qkv, mask, num_heads: int, stream=None):

@@ -13,6 +13,7 @@
 #include "../../include/rlx_encoder.h"
 #include "attention.cuh"
 #include "attention_tc.cuh"
+#include "dequant.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
 #include "gemm_ln_tcgen05.cuh"
@@ -1049,6 +1050,57 @@ rlx_status_t rlx_qk_rope_bf16(void* qkv, int32_t rows, const int32_t* seq_start,
         rlx::qk_rope_kernel<64><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h, rope_cos, rope_sin);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
+}
+
+namespace {
+// format word: (ebits << 8) | (mbits << 4) | special, plus RLX_MINIFLOAT_PACKED4
+rlx_status_t parse_minifloat(int32_t format, rlx::MiniFloatFormat* f, bool* packed4) {
+    if (format < 0 || (format & ~0x1fff)) return RLX_ERR_INVALID_ARG;
+    f->ebits = (format >> 8) & 0xf;
+    f->mbits = (format >> 4) & 0xf;
+    f->special = format & 0xf;
+    *packed4 = (format & RLX_MINIFLOAT_PACKED4) != 0;
+    if (f->ebits < 1 || f->special > 2) return RLX_ERR_INVALID_ARG;
+    if (1 + f->ebits + f->mbits > (*packed4 ? 4 : 8)) return RLX_ERR_INVALID_ARG;
+    return RLX_OK;
+}
+}  // namespace
+
+rlx_status_t rlx_dequant_block_scaled_bf16(const void* codes, const void* scales, int32_t N, int32_t K, int32_t format,
+                                           void* w_bf16, void* stream) {
+    if (!codes || !scales || !w_bf16 || N <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(w_bf16)) return RLX_ERR_INVALID_ARG;
+    rlx::MiniFloatFormat f;
+    bool packed4;
+    const rlx_status_t fs = parse_minifloat(format, &f, &packed4);
+    if (fs != RLX_OK) return fs;
+    if (K % 32 != 0) return RLX_ERR_UNSUPPORTED;
+    const long long tasks = (long long)N * (K / rlx::kDequantElemsPerThread);
+    const int blocks = (int)std::min<long long>((tasks + rlx::kDequantThreads - 1) / rlx::kDequantThreads,
+                                                (long long)rlx::kNumSMs * 16);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (packed4)
+        rlx::dequant_block_scaled_kernel<true><<<blocks, rlx::kDequantThreads, 0, st>>>(
+            (const uint8_t*)codes, (const uint8_t*)scales, (bf16*)w_bf16, N, K, f);
+    else
+        rlx::dequant_block_scaled_kernel<false><<<blocks, rlx::kDequantThreads, 0, st>>>(
+            (const uint8_t*)codes, (const uint8_t*)scales, (bf16*)w_bf16, N, K, f);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t rlx_scaled_matmul_bf16(const void* A, const void* codes, const void* scales, int32_t format,
+                                    const float* bias, const void* residual, rlx_epilogue_t epi, int32_t M, int32_t N,
+                                    int32_t K, void* w_scratch, void* out, int32_t* status, void* stream) {
+    if (!A || !bias || !out || M <= 0) return RLX_ERR_INVALID_ARG;
+    if ((int)epi < 0 || (int)epi > 2 || (epi == RLX_EPI_BIAS_RESIDUAL && !residual)) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(A) || !aligned16(bias) || !aligned16(out) || (residual && !aligned16(residual))) return RLX_ERR_INVALID_ARG;
+    if (N > 0 && N % 64 != 0) return RLX_ERR_UNSUPPORTED;
+    const rlx_status_t ds = rlx_dequant_block_scaled_bf16(codes, scales, N, K, format, w_scratch, stream);
+    if (ds != RLX_OK) return ds;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return launch_gemm((const bf16*)A, (const bf16*)w_scratch, bias, (const bf16*)residual, (int)epi, M, N, K, (bf16*)out,
+                       false, status, static_cast<cudaStream_t>(stream), nullptr, 0);
 }
 
 void rlx_debug_set_attn_trace(void* p) { g_attn_dbg = static_cast<unsigned long long*>(p); }

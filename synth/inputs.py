@@ -196,3 +196,22 @@ def make_inputs(
 def random_mask_case(seed: int, batch: int, seq: int, lo: int = 1) -> np.ndarray:
     """Prefix-mask lengths for ad-hoc test cases: uniform in [lo, seq]."""
     return np.random.default_rng(seed).integers(lo, seq + 1, size=batch)
+
+
+def make_block_scaled_weights(seed: int, n: int, k: int, code_bits: int, max_magnitude: int,
+                              scale_lo: int = 118, scale_hi: int = 136):
+    """Seeded block-scaled minifloat weights: codes uint8 [n, k] with a random sign bit (bit code_bits-1)
+    over a uniform magnitude code in [0, max_magnitude] (callers pass the largest magnitude code that is
+    a finite number in their format), and one scale byte per 32 consecutive k drawn uniformly from
+    [scale_lo, scale_hi].  Holds no decoding arithmetic."""
+    rng = np.random.default_rng(seed)
+    mag = rng.integers(0, max_magnitude + 1, size=(n, k))
+    sign = rng.integers(0, 2, size=(n, k)) << (code_bits - 1)
+    scales = rng.integers(scale_lo, scale_hi + 1, size=(n, k // 32))
+    return (mag | sign).astype(np.uint8), scales.astype(np.uint8)
+
+
+def pack_nibbles(codes: np.ndarray) -> np.ndarray:
+    """[n, k] 4-bit codes -> [n, k/2] bytes, the element with the smaller k in the low nibble."""
+    codes = np.asarray(codes, np.uint8)
+    return (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)

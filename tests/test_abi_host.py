@@ -172,3 +172,20 @@ def test_qk_rope_validates_on_the_host(lib):
     assert call(fake, 0, fake, fake, 1, 8, 2, 32, fake, fake, None) == 1
     assert call(fake, 8, fake, fake, 1, 8, 2, 48, fake, fake, None) == 2      # head size
     assert call(fake, 8, fake, fake, 1, 40000, 2, 32, fake, fake, None) == 2  # beyond the maximum length
+
+
+def test_scaled_matmul_validates_on_the_host(lib):
+    fake, odd = C.c_void_p(0x1000), C.c_void_p(0x1001)
+    fmt = lambda e, m, s=0, p=False: (e << 8) | (m << 4) | s | (0x1000 if p else 0)
+    dq = lib.rlx_dequant_block_scaled_bf16
+    assert dq(None, fake, 8, 32, fmt(4, 3, 1), fake, None) == 1
+    assert dq(odd, fake, 8, 32, fmt(4, 3, 1), fake, None) == 1                 # misaligned codes
+    assert dq(fake, fake, 8, 32, fmt(0, 3), fake, None) == 1                    # no exponent bits
+    assert dq(fake, fake, 8, 32, fmt(5, 3), fake, None) == 1                    # 9-bit code in a byte
+    assert dq(fake, fake, 8, 32, fmt(2, 2, 0, True), fake, None) == 1           # 5-bit code in a nibble
+    assert dq(fake, fake, 8, 32, fmt(4, 3, 3), fake, None) == 1                 # unknown special mode
+    assert dq(fake, fake, 8, 48, fmt(4, 3, 1), fake, None) == 2                 # K % 32
+    sm = lib.rlx_scaled_matmul_bf16
+    assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 2, 8, 64, 32, fake, fake, None, None) == 1   # residual missing
+    assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 0, 8, 100, 32, fake, fake, None, None) == 2  # N % 64
+    assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 0, 8, 64, 32, None, fake, None, None) == 1   # no scratch
