@@ -377,7 +377,7 @@ rlx_status_t rlx_qk_rope_bf16(void *qkv_bf16, int32_t rows, const int32_t *seq_s
 
 /*
  * ScaledMatMul (Section 3.2 "block-scaled tensor-core minifloats -- the FP8/FP6/FP4 grids and arbitrary
- * fNeXmY formats"; Section 5): weight-only quantisation, the paper fixing neither layout nor block
+ * fNeXmY formats"; Section 6): weight-only quantisation, the paper fixing neither layout nor block
  * size.  Reading used here (the open microscaling convention):
  *   code    sign | X exponent bits | Y mantissa bits, bias 2^(X-1)-1, gradual underflow; one code per
  *           byte (low bits), or two 4-bit codes per byte with RLX_MINIFLOAT_PACKED4 (low nibble = the

@@ -7,7 +7,7 @@ module; the product path never does, and it shares no code with the CUDA kernels
 What it follows.  Section 3.1 parameterises masked attention by MaskKind in {None, Causal,
 SlidingWindow(w), Custom}; Section 3.2 names a fused QK-RoPE region ahead of attention.  The paper
 defines none of them further, so the readings used here are the ones of the decoder families its model
-zoo (Section 9) names:
+zoo (Section 8.5) names:
 
   None              every key of the sequence is visible to every query.
   Causal            key k is visible to query i  iff  k <= i.

@@ -5,7 +5,7 @@ module; the product path never does, and it shares no code with the CUDA kernels
 
 What it follows.  Section 3.2 (numeric precision) lists weight-only quantisation down to "block-scaled
 tensor-core minifloats -- the FP8/FP6/FP4 grids and arbitrary fNeXmY formats, selectable per matmul";
-Section 5 names the operator (ScaledMatMul) and its bar: agreement with the F32 reference on the
+Section 6 names the operator (ScaledMatMul) and its bar: agreement with the F32 reference on the
 dequantised grid.  The paper gives no layout, block size or scale format; the readings used here are
 those of the open microscaling (MX) convention its llama.cpp scheme list also names:
 

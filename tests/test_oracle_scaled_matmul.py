@@ -1,5 +1,5 @@
 """Pins for the fp64 oracle of the block-scaled minifloat matmul (Section 3.2 numeric precision;
-Section 5 ScaledMatMul): published value grids, library decoders, closed forms, brute force.  No GPU."""
+Section 6 ScaledMatMul): published value grids, library decoders, closed forms, brute force.  No GPU."""
 import numpy as np
 import pytest
 import torch
