@@ -174,6 +174,22 @@ qk_rope_kernel(__nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ seq_
     }
 }
 
+// The same search done by a whole warp (p warp-uniform): every round samples 32 evenly spaced entries
+// of the remaining range and a ballot picks the sub-range, so 256 sequences take two dependent loads
+// instead of eight.
+__device__ __forceinline__ int find_sequence_warp(const int32_t* __restrict__ seq_start, int B, int p, int lane) {
+    int lo = 0, n = B;   // invariant: the answer lies in [lo, lo + n) and seq_start[lo] <= p
+    while (n > 1) {
+        const int step = (n + 31) >> 5;
+        const int idx = lo + lane * step;
+        const bool le = idx < lo + n && __ldg(seq_start + idx) <= p;   // true for a prefix of the lanes
+        const int k = 31 - __clz(__ballot_sync(0xffffffffu, le));       // lane 0 is always true
+        lo += k * step;
+        n = min(step, n - k * step);
+    }
+    return lo;
+}
+
 // x[row] = LN(word[id] + pos[s] + type[0]).  Ids outside [0, V) are clamped and flagged.
 // Padded mode (seq_start == nullptr): row = token t = b*S + s for all T tokens.
 // Packed mode: row p < seq_start[B] belongs to sequence b = find_sequence(p) at position
@@ -194,7 +210,7 @@ embed_ln_kernel(const int32_t* __restrict__ ids, const __nv_bfloat16* __restrict
     int tok = t, s = t % S;
     if (seq_start != nullptr) {
         if (t >= __ldg(seq_start + B)) return;
-        const int b = find_sequence(seq_start, B, t);
+        const int b = find_sequence_warp(seq_start, B, t, lane);
         s = __ldg(pos_of_rank + (size_t)b * S + (t - __ldg(seq_start + b)));
         tok = b * S + s;
     }
@@ -291,8 +307,16 @@ pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restric
             acc[6] += bf16lo(a.w); acc[7] += bf16hi(a.w);
         };
         if (packed) {
-            // all rows valid: four independent 16-byte loads in flight per thread
+            // all rows valid: eight, then four, independent 16-byte loads in flight per thread
             int s = g;
+            for (; s + 7 * G < nrows; s += 8 * G) {
+                uint4 a[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) a[u] = __ldg(reinterpret_cast<const uint4*>(xb + (size_t)(s + u * G) * H + c * 8));
+#pragma unroll
+                for (int u = 0; u < 8; ++u) add_row(a[u]);
+                count += 8;
+            }
             for (; s + 3 * G < nrows; s += 4 * G) {
                 uint4 a[4];
 #pragma unroll
@@ -315,12 +339,20 @@ pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restric
 #pragma unroll
         for (int i = 0; i < 8; ++i) pool_smem[g * H + c * 8 + i] = acc[i];
     }
-    __shared__ int s_count[kPoolThreads];
-    s_count[threadIdx.x] = (g < G && c == 0) ? count : 0;
+    // number of pooled rows: every group counted its own (integer sums: any order gives the same value)
+    __shared__ int s_count[kPoolThreads / 32];
+    {
+        int cnt = (g < G && c == 0) ? count : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if ((threadIdx.x & 31) == 0) s_count[threadIdx.x >> 5] = cnt;
+    }
     __syncthreads();
     // column sums: thread j < H owns column j
-    float n_valid = 0.f;
-    for (int i = 0; i < kPoolThreads; ++i) n_valid += (float)s_count[i];  // same value in every thread
+    int n_rows = 0;
+#pragma unroll
+    for (int i = 0; i < kPoolThreads / 32; ++i) n_rows += s_count[i];
+    const float n_valid = (float)n_rows;
     float colsum[3] = {0.f, 0.f, 0.f};  // H <= 1024 -> at most ceil(1024/384) = 3 columns per thread
     float sq = 0.f;
     const float inv_n = 1.0f / fmaxf(n_valid, 1e-9f);
