@@ -4,8 +4,11 @@
 //  attention_bf16_kernel: bf16 in/out.  One CTA = 128 query rows of one (sequence, head); 8 warps of
 //    16 rows each.  K/V stream through shared memory in 64-key blocks (cp.async, 4-stage ring, three
 //    blocks in flight), QK^T and PV run on the warp-level tensor-core path (mma.sync m16n8k16, fp32
-//    accumulate), the softmax state (running max / sum) lives in registers and is reduced with quad
-//    shuffles; the 1/sqrt(d)*log2(e) scale is folded into the exp2 argument.  Key blocks beyond the
+//    accumulate), the softmax state (running max) lives in registers and is reduced with quad
+//    shuffles, the row sums come from an extra ones column of the PV product; the 1/sqrt(d)*log2(e)
+//    scale is folded into the exp2 argument.  At head_dim 32 the online-softmax step is 32 keys (half a
+//    staged block): 64 registers per thread, four CTAs per SM instead of three (-6 % on the 256 x 256
+//    workload; at head_dim 64, and in the mask-kind / rotary modes, the 64-key step is kept).  Key blocks beyond the
 //    last valid key are never loaded; masking runs only in blocks that contain an invalid key.
 //  attention_f32_kernel: fp32 in/out CUDA-core kernel, one warp per query row, K/V staged in shared
 //    memory 32 keys at a time, warp-shuffle reductions.  Reference-precision mode for testing.
@@ -105,8 +108,9 @@ struct AttKind {
 // Two addressing modes share the kernel:
 //   padded: seq_start == nullptr.  Sequence b occupies rows b*S .. b*S+S; `mask` flags valid keys.
 //   packed: rows of sequence b are seq_start[b] .. seq_start[b]+seq_len[b], all valid (mask unused).
-template <int D, int MK = 0, bool ROPE = false>
-__global__ void __launch_bounds__(kAttThreads, D == 32 ? 3 : 2)
+template <int D, int MK = 0, bool ROPE = false, int KS = ((D == 32 && MK == 0 && !ROPE) ? 32 : 64),
+          int MINB = (D == 32 ? (KS == 32 ? 4 : 3) : 2)>
+__global__ void __launch_bounds__(kAttThreads, MINB)
 attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ mask,
                       const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
                       __nv_bfloat16* __restrict__ ctx, int S, int H, float scale_log2e, AttKind kind) {
@@ -267,16 +271,21 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         }
         const int k0 = j * kAttBlockN;
         if (MK && (k0 > r0 + 15 || k0 + kAttBlockN - 1 <= r0 - kind.window)) continue;   // nothing visible
-        // ---- S = Q K^T for 64 keys: 8 n-tiles x 4 accumulators ----
-        float s[8][4];
+        // The online-softmax step covers KS keys (64: the whole staged block; 32: half of it, which halves
+        // the score and probability registers and lets a fourth CTA fit on the SM at head_dim 32).
+        constexpr int NT = KS / 8;   // score n-tiles per step
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
+        for (int hf = 0; hf < kAttBlockN / KS; ++hf) {
+        // ---- S = Q K^T for KS keys: NT n-tiles x 4 accumulators ----
+        float s[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
             s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
             for (int kp = 0; kp < KT / 2; ++kp) {  // two k-tiles per ldmatrix.x4
                 uint32_t b0, b1, b2, b3;
                 const int mi = lane >> 3;
-                const int r = nt * 8 + (lane & 7);
+                const int r = (hf * NT + nt) * 8 + (lane & 7);
                 const int c = kp * 32 + (mi & 1) * 8 + (mi >> 1) * 16;
                 ldmatrix_x4(smem_u32(sm.k[buf] + r * STR + c), b0, b1, b2, b3);
                 mma_bf16_16816(s[nt], qf[2 * kp][0], qf[2 * kp][1], qf[2 * kp][2], qf[2 * kp][3], b0, b1);
@@ -289,8 +298,8 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             if (k0 + kAttBlockN > len || k0 + kAttBlockN - 1 > r0 || k0 <= r0 + 15 - kind.window) {
                 const int ia = r0 + g, ib = ia + 8;   // rows of accumulators {0,1} and {2,3}
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
-                    const int kk = k0 + nt * 8 + 2 * t4;
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int kk = k0 + (hf * NT + nt) * 8 + 2 * t4;
                     if (!(kk < len && kk <= ia && kk > ia - kind.window)) s[nt][0] = -INFINITY;
                     if (!(kk + 1 < len && kk + 1 <= ia && kk + 1 > ia - kind.window)) s[nt][1] = -INFINITY;
                     if (!(kk < len && kk <= ib && kk > ib - kind.window)) s[nt][2] = -INFINITY;
@@ -301,8 +310,8 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             const bool need_mask = packed ? (k0 + kAttBlockN > len) : (sm.blk_full[j] == 0);
             if (need_mask) {
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
-                    const int kk = k0 + nt * 8 + 2 * t4;
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int kk = k0 + (hf * NT + nt) * 8 + 2 * t4;
                     const bool v0 = packed ? (kk < len) : (sm.bias[kk] == 0.f);
                     const bool v1 = packed ? (kk + 1 < len) : (sm.bias[kk + 1] == 0.f);
                     if (!v0) { s[nt][0] = -INFINITY; s[nt][2] = -INFINITY; }
@@ -313,7 +322,7 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         // ---- running max on raw scores (the positive scale commutes with max) ----
         float mx[2] = {fmaxf(s[0][0], s[0][1]), fmaxf(s[0][2], s[0][3])};
 #pragma unroll
-        for (int nt = 1; nt < 8; ++nt) {
+        for (int nt = 1; nt < NT; ++nt) {
             mx[0] = fmax3(mx[0], s[nt][0], s[nt][1]);
             mx[1] = fmax3(mx[1], s[nt][2], s[nt][3]);
         }
@@ -336,11 +345,11 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         l_acc[0] *= alpha[0];
         l_acc[2] *= alpha[1];
         // ---- P = exp2(S*c - m), packed to bf16 A fragments ----
-        uint32_t pf[4][4];
+        uint32_t pf[NT / 2][4];
         const uint64_t c2 = att_pack2(scale_log2e, scale_log2e);
         const uint64_t nm0 = att_pack2(-msub[0], -msub[0]), nm1 = att_pack2(-msub[1], -msub[1]);
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
+        for (int nt = 0; nt < NT; ++nt) {
             float x0, x1, x2, x3;
             att_unpack2(att_fma2(att_pack2(s[nt][0], s[nt][1]), c2, nm0), x0, x1);
             att_unpack2(att_fma2(att_pack2(s[nt][2], s[nt][3]), c2, nm1), x2, x3);
@@ -349,19 +358,20 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         }
         // ---- O += P V ----
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < NT / 2; ++kk) {
             mma_bf16_16816(l_acc, pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], kOnesBf16x2, kOnesBf16x2);
 #pragma unroll
             for (int np = 0; np < ND / 2; ++np) {  // two n-tiles per ldmatrix.x4.trans
                 uint32_t b0, b1, b2, b3;
                 const int mi = lane >> 3;
-                const int r = kk * 16 + (mi & 1) * 8 + (lane & 7);
+                const int r = (hf * (NT / 2) + kk) * 16 + (mi & 1) * 8 + (lane & 7);
                 const int c = np * 16 + (mi >> 1) * 8;
                 ldmatrix_x4_trans(smem_u32(sm.v[buf] + r * STR + c), b0, b1, b2, b3);
                 mma_bf16_16816(o[2 * np], pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], b0, b1);
                 mma_bf16_16816(o[2 * np + 1], pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], b2, b3);
             }
         }
+        }   // hf
     }
     cp_async_wait<0>();
     if (!warp_active) return;
