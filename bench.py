@@ -36,7 +36,8 @@ KERNEL_CLASSES = ("gemm_qkv", "attention", "gemm_out", "ln1", "gemm_ffn1", "gemm
 # kernel and workload; absent where no capture exists for that workload)
 NCU_DRAM_TRAFFIC_MB = {
     "c2": {"gemm_out": 3.6, "gemm_ffn2": 9.5},
-    "c3": {"attention": 98.8, "gemm_ffn1": 90.5, "gemm_qkv": 62.2, "ln1": 28.6, "ln2": 28.6, "gemm_out": 62.2,
+    "c4": {"attention": 107.9},
+    "c3": {"attention": 98.7, "gemm_ffn1": 90.5, "gemm_qkv": 62.2, "ln1": 28.6, "ln2": 28.6, "gemm_out": 62.2,
            "gemm_ffn2": 158.2, "embed_ln": 17.1, "pool_l2": 28.6, "pack": 0.3},
 }
 # B200: 148 SMs x 16 special-function results per clock x 1.965 GHz (exp2 of the softmax)
