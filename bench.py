@@ -113,7 +113,7 @@ class ClockSampler(threading.Thread):
 
 
 # ---------------------------------------------------------------------------- oracle timing
-def time_oracle(cfg_name: str, budget_s: float, steps: int = 1, warmup: int = 0):
+def time_oracle(cfg_name: str, budget_s: float, steps: int = 1, warmup: int = 0, all_valid: bool = False):
     """Times the fp64 oracle (as it stands) on host cores on a bounded sample of the workload:
     the first n sequences of the seeded batch, n chosen from a one-sequence calibration run so
     that one step costs about `budget_s` seconds."""
@@ -121,7 +121,7 @@ def time_oracle(cfg_name: str, budget_s: float, steps: int = 1, warmup: int = 0)
     from synth.inputs import CONFIGS, EncoderConfig, make_inputs
 
     cfg = CONFIGS[cfg_name]
-    inp = make_inputs(cfg)
+    inp = make_inputs(cfg, lengths=np.full(cfg.batch, cfg.seq, dtype=np.int64) if all_valid else None)
     cores = usable_cores()
     oracle.set_threads(cores)
 
@@ -147,7 +147,7 @@ def run_reference_arm(args):
         return
     total_budget = 150.0
     per_step = total_budget / max(args.steps + args.warmup, 1)
-    r = time_oracle(args.config, per_step, steps=args.steps, warmup=args.warmup)
+    r = time_oracle(args.config, per_step, steps=args.steps, warmup=args.warmup, all_valid=args.all_valid)
     mean_t = sum(r["times"]) / len(r["times"])
     value = r["n"] / mean_t
     sample = f"first {r['n']} of {r['batch']} sequences of {args.config} per step"
@@ -172,6 +172,8 @@ def workload_config(name: str, extra=None):
          "parallelism": "replicated weights, batch sharded across ranks, no collective"}
     if extra:
         d.update(extra)
+        if "valid_lengths" in extra:
+            d["workload"] = d["workload"].replace(f"valid lengths uniform in [{c.len_lo},{c.len_hi}]", "every sequence full length")
     return d
 
 
@@ -239,11 +241,14 @@ def run_ours(args):
         dist.barrier()
 
     cfg = CONFIGS[args.config]
-    base = make_inputs(cfg)
+    # --all-valid: every sequence fills the whole padded length (mask all ones), for like-for-like context
+    # with benchmarks that feed unpadded inputs; the seeded draw order of everything else is unchanged
+    full = np.full(cfg.batch, cfg.seq, dtype=np.int64) if args.all_valid else None
+    base = make_inputs(cfg, lengths=full)
     if rank == 0:
         mine = base
     else:  # every rank gets its own batch (ids, lengths) and the same replicated weights
-        mine = make_inputs(EncoderConfig(**{**cfg.__dict__, "seed": cfg.seed + 1000 * rank}), weights=False)
+        mine = make_inputs(EncoderConfig(**{**cfg.__dict__, "seed": cfg.seed + 1000 * rank}), weights=False, lengths=full)
     weights = rlx.upload_weights(base.params, base.layers)
     B, S, H = cfg.batch, cfg.seq, cfg.hidden
 
@@ -376,14 +381,15 @@ def run_ours(args):
                     "event_overhead_us_per_launch": overhead_us,
                     "frac_net_of_event_overhead": d["frac"] * d["avg_us"] / net_us}
 
-        cb = time_oracle(args.config, budget_s=15.0, steps=1)
+        cb = time_oracle(args.config, budget_s=15.0, steps=1, all_valid=args.all_valid)
         cb_value = cb["n"] / cb["times"][0]
         seqs = B * world
         line = {
             "metric": METRIC, "value": seqs * args.steps / (total_ms / 1e3), "unit": "sequences/s",
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
             "p50_ms": p50_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": workload_config(args.config),
+            "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(args.config, {"valid_lengths": f"all {cfg.seq} (--all-valid)"} if args.all_valid else None),
             "e2e": {"value": seqs * args.steps / (e2e_total / 1e3), "unit": "sequences/s", "p50_ms": e2e_p50,
                     "h2d_bytes_per_step": 2 * B * S * 4, "d2h_bytes_per_step": B * H * 4,
                     "timing": "host wall clock around rlx_encoder_forward_host (copies + forward + sync)"},
@@ -662,6 +668,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="c2", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--all-valid", action="store_true", help="encoder op: every sequence has the full length")
     ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope", "scaled_matmul"])
     ap.add_argument("--fmt", default="fp8_e4m3", choices=["fp8_e4m3", "fp4_e2m1"])
     ap.add_argument("--mask", default="causal", choices=["none", "causal", "sliding"])
