@@ -59,48 +59,64 @@ def rope(x: np.ndarray, theta: float = 10000.0, positions: Optional[np.ndarray] 
     return np.concatenate([lo * c - hi * s, hi * c + lo * s], axis=-1)
 
 
+def split_qkv(qkv: np.ndarray, num_heads: int, num_kv_heads: Optional[int] = None):
+    """qkv [L, (hq + 2 hkv) d] -> q [L, hq, d], k [L, hkv, d], v [L, hkv, d]: q heads, then k heads, then v heads."""
+    hkv = num_heads if num_kv_heads is None else num_kv_heads
+    L, W = qkv.shape
+    d = W // (num_heads + 2 * hkv)
+    assert d * (num_heads + 2 * hkv) == W and num_heads % hkv == 0
+    q = qkv[:, :num_heads * d].reshape(L, num_heads, d)
+    k = qkv[:, num_heads * d:(num_heads + hkv) * d].reshape(L, hkv, d)
+    v = qkv[:, (num_heads + hkv) * d:].reshape(L, hkv, d)
+    return q, k, v
+
+
 def attention_one(qkv: np.ndarray, num_heads: int, kind: int, window: int = 0,
-                  rope_theta: Optional[float] = None) -> np.ndarray:
-    """One sequence: qkv [L, 3H] (q | k | v column blocks, head j = columns j*d..(j+1)*d) -> ctx [L, H]."""
+                  rope_theta: Optional[float] = None, num_kv_heads: Optional[int] = None) -> np.ndarray:
+    """One sequence: qkv [L, (hq + 2 hkv) d] (q | k | v column blocks, head j = columns j*d..(j+1)*d of its
+    block) -> ctx [L, hq d].  With fewer k/v heads than q heads (grouped-query attention, the layout of the
+    decoder families the paper's model zoo names), q head j reads k/v head j // (hq / hkv)."""
     qkv = np.asarray(qkv, np.float64)
-    L, H3 = qkv.shape
-    H = H3 // 3
-    d = H // num_heads
-    q, k, v = (qkv[:, i * H:(i + 1) * H].reshape(L, num_heads, d) for i in range(3))
+    L = qkv.shape[0]
+    q, k, v = split_qkv(qkv, num_heads, num_kv_heads)
+    d = q.shape[2]
+    group = num_heads // k.shape[1]
     if rope_theta is not None:
         q, k = rope(q, rope_theta), rope(k, rope_theta)
     vis = visible(L, kind, window)
     ctx = np.zeros((L, num_heads, d))
     for j in range(num_heads):
-        s = (q[:, j, :] @ k[:, j, :].T) / sqrt(d)
+        s = (q[:, j, :] @ k[:, j // group, :].T) / sqrt(d)
         s = np.where(vis, s, -np.inf)
         m = s.max(axis=1, keepdims=True)                         # every row sees at least itself
         e = np.where(vis, np.exp(s - m), 0.0)
-        ctx[:, j, :] = (e / e.sum(axis=1, keepdims=True)) @ v[:, j, :]
-    return ctx.reshape(L, H)
+        ctx[:, j, :] = (e / e.sum(axis=1, keepdims=True)) @ v[:, j // group, :]
+    return ctx.reshape(L, num_heads * d)
 
 
 def attention_packed(qkv: np.ndarray, seq_start, seq_len, num_heads: int, kind: int, window: int = 0,
-                     rope_theta: Optional[float] = None) -> np.ndarray:
+                     rope_theta: Optional[float] = None, num_kv_heads: Optional[int] = None) -> np.ndarray:
     """Packed rows: sequence b owns rows seq_start[b] .. seq_start[b]+seq_len[b]; other rows stay 0."""
     qkv = np.asarray(qkv, np.float64)
-    out = np.zeros((qkv.shape[0], qkv.shape[1] // 3))
+    hkv = num_heads if num_kv_heads is None else num_kv_heads
+    out = np.zeros((qkv.shape[0], qkv.shape[1] // (num_heads + 2 * hkv) * num_heads))
     for s0, n in zip(np.asarray(seq_start), np.asarray(seq_len)):
         s0, n = int(s0), int(n)
         if n > 0:
-            out[s0:s0 + n] = attention_one(qkv[s0:s0 + n], num_heads, kind, window, rope_theta)
+            out[s0:s0 + n] = attention_one(qkv[s0:s0 + n], num_heads, kind, window, rope_theta, num_kv_heads)
     return out
 
 
-def rope_qk_packed(qkv: np.ndarray, seq_start, seq_len, num_heads: int, theta: float = 10000.0) -> np.ndarray:
+def rope_qk_packed(qkv: np.ndarray, seq_start, seq_len, num_heads: int, theta: float = 10000.0,
+                   num_kv_heads: Optional[int] = None) -> np.ndarray:
     """The QK-RoPE region on packed rows: q and k column blocks rotated by each row's position within its
     sequence, v and rows outside every sequence returned unchanged."""
     out = np.array(qkv, dtype=np.float64, copy=True)
-    H = out.shape[1] // 3
-    d = H // num_heads
+    hkv = num_heads if num_kv_heads is None else num_kv_heads
+    d = out.shape[1] // (num_heads + 2 * hkv)
+    rot = (num_heads + hkv) * d                                   # q heads then k heads: one contiguous block
     for s0, n in zip(np.asarray(seq_start), np.asarray(seq_len)):
         s0, n = int(s0), int(n)
-        for part in (0, 1):
-            blk = out[s0:s0 + n, part * H:(part + 1) * H].reshape(n, num_heads, d)
-            out[s0:s0 + n, part * H:(part + 1) * H] = rope(blk, theta).reshape(n, H)
+        blk = out[s0:s0 + n, :rot].reshape(n, num_heads + hkv, d)
+        out[s0:s0 + n, :rot] = rope(blk, theta).reshape(n, rot)
     return out

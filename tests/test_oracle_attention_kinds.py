@@ -264,3 +264,33 @@ def test_rope_qk_packed_composes_with_attention():
     a = ak.attention_packed(rot, start, lens, h, ak.KIND_CAUSAL, 0, None)
     b = ak.attention_packed(qkv, start, lens, h, ak.KIND_CAUSAL, 0, 10000.0)
     np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-15)
+
+
+# ---------------------------------------------------------------- grouped-query layout
+def test_grouped_query_equals_repeated_kv_heads_and_library():
+    rng = np.random.default_rng(11)
+    L, hq, hkv, d = 21, 6, 2, 8
+    qkv = rng.standard_normal((L, (hq + 2 * hkv) * d)) * 1.5
+    got = ak.attention_one(qkv, hq, ak.KIND_CAUSAL, 0, 10000.0, num_kv_heads=hkv)
+    # the same thing with every k/v head written out once per q head of its group (plain multi-head layout)
+    q, k, v = ak.split_qkv(qkv, hq, hkv)
+    full = np.concatenate([q.reshape(L, -1), np.repeat(k, hq // hkv, axis=1).reshape(L, -1),
+                           np.repeat(v, hq // hkv, axis=1).reshape(L, -1)], axis=1)
+    np.testing.assert_allclose(got, ak.attention_one(full, hq, ak.KIND_CAUSAL, 0, 10000.0), rtol=1e-13, atol=1e-15)
+    # library routine with its own grouped-query switch (no rotation)
+    tq = torch.from_numpy(q).transpose(0, 1)[None]
+    tk = torch.from_numpy(k).transpose(0, 1)[None]
+    tv = torch.from_numpy(v).transpose(0, 1)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, enable_gqa=True)
+    ref = ref[0].transpose(0, 1).reshape(L, hq * d).numpy()
+    np.testing.assert_allclose(ak.attention_one(qkv, hq, ak.KIND_CAUSAL, 0, None, num_kv_heads=hkv), ref,
+                               rtol=1e-12, atol=1e-14)
+    # perturbing one k/v head reaches exactly the q heads of its group
+    pert = qkv.copy()
+    pert[:, (hq + 1) * d:(hq + 2) * d] += 0.25                      # k head 1
+    out2 = ak.attention_one(pert, hq, ak.KIND_CAUSAL, 0, 10000.0, num_kv_heads=hkv)
+    changed = [bool(np.any(got[:, j * d:(j + 1) * d] != out2[:, j * d:(j + 1) * d])) for j in range(hq)]
+    assert changed == [False, False, False, True, True, True]
+    # the packed rotation touches q and k heads only
+    rot = ak.rope_qk_packed(qkv, [0], [L], hq, 10000.0, num_kv_heads=hkv)
+    assert np.array_equal(rot[:, (hq + hkv) * d:], qkv[:, (hq + hkv) * d:]) and not np.allclose(rot[1:, :hq * d], qkv[1:, :hq * d])
