@@ -442,7 +442,8 @@ def run_attention_kind(args):
     import torch
     import paper_2609_37916_b200 as rlx
 
-    h, d = 16, 64
+    h, d = args.heads, 64
+    hkv = args.kv_heads or h
     H = h * d
     lengths = attention_kind_workload()
     total, max_len = int(lengths.sum()), int(lengths.max())
@@ -450,7 +451,7 @@ def run_attention_kind(args):
     kind_id = {"none": rlx.binding.MASK_NONE, "causal": rlx.binding.MASK_CAUSAL, "sliding": rlx.binding.MASK_SLIDING_WINDOW}[args.mask]
     torch.cuda.set_device(0)
     g = torch.Generator(device="cuda").manual_seed(7)
-    qkv = torch.randn(total, 3 * H, device="cuda", generator=g).to(torch.bfloat16)
+    qkv = torch.randn(total, (h + 2 * hkv) * d, device="cuda", generator=g).to(torch.bfloat16)
     ss, sl = torch.from_numpy(start).cuda(), torch.from_numpy(lengths).cuda()
     rope = rlx.rope_tables(max_len, d) if args.rope else None
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -462,7 +463,7 @@ def run_attention_kind(args):
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        out = rlx.binding.attention_kind_bf16(qkv, ss, sl, max_len, h, kind_id, args.window, rope, out=ctx)
+        out = rlx.binding.attention_kind_bf16(qkv, ss, sl, max_len, h, kind_id, args.window, rope, out=ctx, num_kv_heads=hkv)
         e1.record()
         return e0, e1, out
 
@@ -477,14 +478,14 @@ def run_attention_kind(args):
     ms = [a.elapsed_time(b) for a, b, _ in evs]
     p50 = statistics.median(ms)
     pairs = visible_pairs(lengths, args.mask, args.window)
-    flops, exps, bytes_ = 4.0 * pairs * d * h, float(pairs) * h, 4.0 * total * H * 2
+    flops, exps, bytes_ = 4.0 * pairs * d * h, float(pairs) * h, 2.0 * total * (2 * h + 2 * hkv) * d
     peaks, peak_kind = load_peaks()
     # oracle on the first sequence
     from oracle import attention_kinds as ak
     n0 = int(lengths[0])
     seq = qkv[:n0].float().cpu().numpy().astype(np.float64)
     t0 = time.perf_counter()
-    ref = ak.attention_one(seq, h, kind_id, args.window, 10000.0 if args.rope else None)
+    ref = ak.attention_one(seq, h, kind_id, args.window, 10000.0 if args.rope else None, num_kv_heads=hkv)
     t_or = time.perf_counter() - t0
     got = evs[-1][2][:n0].float().cpu().numpy().astype(np.float64)
     line = {
@@ -492,7 +493,7 @@ def run_attention_kind(args):
         "value": total * args.steps / (sum(ms) / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "p50_ms": p50, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), 16 heads x 64, "
+        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), {h} q heads / {hkv} kv heads x 64, "
                                f"mask {args.mask}" + (f"({args.window})" if args.mask == "sliding" else "") +
                                (", rotary q,k" if args.rope else ""), "l2": "256 MiB flush write between steps"},
         "gpu_launches": args.steps, "clocks": sampler.summary(),
@@ -674,6 +675,8 @@ def main():
     ap.add_argument("--mask", default="causal", choices=["none", "causal", "sliding"])
     ap.add_argument("--window", type=int, default=512)
     ap.add_argument("--rope", type=int, default=1)
+    ap.add_argument("--heads", type=int, default=16, help="attention_kind op: q heads (head_dim 64)")
+    ap.add_argument("--kv-heads", type=int, default=0, help="attention_kind op: k/v heads (0 = same as --heads)")
     args = ap.parse_args()
     if args.op != "encoder":
         if args.impl != "ours" or args.gpus != 1:

@@ -341,6 +341,10 @@ rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const
  *                            j + head_dim/2 and the pair is rotated by the angle of the row's position
  *                            in its sequence: lo' = lo*cos - hi*sin, hi' = hi*cos + lo*sin, in fp32,
  *                            rounded to bf16 before the tensor-core product.  v is not touched.
+ *   grouped-query layout     num_kv_heads < num_heads (a divisor of it): a row of qkv holds num_heads q
+ *                            heads, then num_kv_heads k heads, then num_kv_heads v heads, and q head j
+ *                            reads k / v head j / (num_heads / num_kv_heads); num_kv_heads ==
+ *                            num_heads is the plain [q | k | v] layout.  ctx is [rows, num_heads*head_dim].
  * Arguments: qkv / seq_start / seq_len / ctx as in rlx_attention_packed_bf16 (packed rows, device
  * memory, 16-byte aligned; seq_len[b] <= max_len <= RLX_ATTENTION_KIND_MAX_LEN).  rope_cos and
  * rope_sin are device fp32 tables [max_len, head_dim/2] (row = position, 16-byte aligned) holding
@@ -357,7 +361,7 @@ rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const
 #define RLX_ATTENTION_KIND_MAX_LEN 32768
 rlx_status_t rlx_attention_kind_bf16(const void *qkv_bf16, int32_t rows, const int32_t *seq_start,
                                      const int32_t *seq_len, int32_t batch, int32_t max_len,
-                                     int32_t num_heads, int32_t head_dim, int32_t mask_kind,
+                                     int32_t num_heads, int32_t num_kv_heads, int32_t head_dim, int32_t mask_kind,
                                      int32_t window, const float *rope_cos, const float *rope_sin,
                                      void *ctx_bf16, void *cuda_stream);
 
@@ -368,11 +372,11 @@ rlx_status_t rlx_attention_kind_bf16(const void *qkv_bf16, int32_t rows, const i
  * bit for bit what it gives on the unrotated buffer with the tables.  One pass over 2/3 of qkv at HBM
  * speed, where the in-attention form rotates every key block once per 128-row query tile: prefer this
  * call for sequences of more than a few hundred rows, the in-attention form when qkv must stay
- * read-only.  qkv: device bf16 [rows, 3*num_heads*head_dim], 16-byte aligned, modified; other
+ * read-only.  qkv: device bf16 [rows, (num_heads + 2*num_kv_heads)*head_dim], 16-byte aligned, modified; other
  * arguments and error behaviour as in rlx_attention_kind_bf16 (both tables required).
  */
 rlx_status_t rlx_qk_rope_bf16(void *qkv_bf16, int32_t rows, const int32_t *seq_start, const int32_t *seq_len,
-                              int32_t batch, int32_t max_len, int32_t num_heads, int32_t head_dim,
+                              int32_t batch, int32_t max_len, int32_t num_heads, int32_t num_kv_heads, int32_t head_dim,
                               const float *rope_cos, const float *rope_sin, void *cuda_stream);
 
 /*

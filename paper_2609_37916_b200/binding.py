@@ -307,26 +307,31 @@ def rope_tables(max_len: int, head_dim: int, theta: float = 10000.0, device="cud
 
 
 def attention_kind_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, mask_kind: int, window: int = 0,
-                        rope=None, out=None, stream=None):
-    """qkv: packed [rows, 3H] bf16; rope: None or the (cos, sin) pair of rope_tables; returns ctx [rows, H]
-    (a fresh zero-filled tensor, or `out` with rows outside every sequence left as they were)."""
-    rows, H3 = qkv.shape
-    H = H3 // 3
-    ctx = torch.zeros((rows, H), dtype=torch.bfloat16, device=qkv.device) if out is None else out
+                        rope=None, out=None, stream=None, num_kv_heads: Optional[int] = None):
+    """qkv: packed [rows, (hq + 2 hkv) d] bf16 (hkv = hq unless num_kv_heads is given); rope: None or the
+    (cos, sin) pair of rope_tables; returns ctx [rows, hq d] (a fresh zero-filled tensor, or `out` with rows
+    outside every sequence left as they were)."""
+    rows, W = qkv.shape
+    hkv = num_heads if num_kv_heads is None else num_kv_heads
+    d = W // (num_heads + 2 * hkv)
+    ctx = torch.zeros((rows, num_heads * d), dtype=torch.bfloat16, device=qkv.device) if out is None else out
     cos, sin = rope if rope is not None else (None, None)
     _check(_load().rlx_attention_kind_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len,
-                                           num_heads, H // num_heads, mask_kind, window, _ptr(cos), _ptr(sin),
+                                           num_heads, hkv, d, mask_kind, window, _ptr(cos), _ptr(sin),
                                            _ptr(ctx), _stream(stream)),
            "rlx_attention_kind_bf16")
     return ctx
 
 
-def qk_rope_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, rope, stream=None):
-    """Rotates the q and k column blocks of packed qkv [rows, 3H] bf16 IN PLACE; returns qkv."""
-    rows, H3 = qkv.shape
+def qk_rope_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, rope, stream=None,
+                 num_kv_heads: Optional[int] = None):
+    """Rotates the q and k column blocks of packed qkv [rows, (hq + 2 hkv) d] bf16 IN PLACE; returns qkv."""
+    rows, W = qkv.shape
+    hkv = num_heads if num_kv_heads is None else num_kv_heads
     cos, sin = rope
     _check(_load().rlx_qk_rope_bf16(_ptr(qkv), rows, _ptr(seq_start), _ptr(seq_len), seq_len.numel(), max_len, num_heads,
-                                    H3 // 3 // num_heads, _ptr(cos), _ptr(sin), _stream(stream)), "rlx_qk_rope_bf16")
+                                    hkv, W // (num_heads + 2 * hkv), _ptr(cos), _ptr(sin), _stream(stream)),
+           "rlx_qk_rope_bf16")
     return qkv
 
 

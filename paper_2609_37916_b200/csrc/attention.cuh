@@ -95,6 +95,7 @@ struct AttSmem {
 //           length).  Key blocks wholly outside a CTA's rows are never loaded, blocks wholly outside a
 //           warp's 16 rows are skipped by that warp, and the element test runs only in blocks that a
 //           boundary crosses.
+//   kv_group > 1: grouped-query layout, q head j reads k/v head j / kv_group (packed mode only).
 //   ROPE:   q and k rows are rotated in shared memory after they land ("rotate-half" pairing of column
 //           j with j + D/2 by the angle whose cosine / sine the caller tabulates per position), in fp32,
 //           and rounded back to bf16 for the tensor-core products.  Each thread rotates what it copied
@@ -103,6 +104,7 @@ struct AttKind {
     int window;
     const float* rope_cos;   // [max_len, D/2]
     const float* rope_sin;
+    int kv_group;            // q heads per k/v head (1: plain multi-head layout [q | k | v] of width 3H)
 };
 
 // Two addressing modes share the kernel:
@@ -130,10 +132,12 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     const size_t row0 = packed ? (size_t)__ldg(seq_start + b) : (size_t)b * S;
     const int len = packed ? __ldg(seq_len + b) : S;   // rows of this sequence present in memory
     if (q0 >= len) return;                              // whole CTA outside the sequence (uniform)
-    const int ld = 3 * H;
+    // row layout: H columns of q heads, then H / kv_group of k heads, then as many of v heads
+    const int Hkv = H / kind.kv_group;
+    const int ld = H + 2 * Hkv;
     const __nv_bfloat16* qbase = qkv + row0 * ld + head * D;
-    const __nv_bfloat16* kbase = qbase + H;
-    const __nv_bfloat16* vbase = qbase + 2 * H;
+    const __nv_bfloat16* kbase = qkv + row0 * ld + H + (head / kind.kv_group) * D;
+    const __nv_bfloat16* vbase = kbase + Hkv;
 
     int kv_end = len;
     if (!packed) {

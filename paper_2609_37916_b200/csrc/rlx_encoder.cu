@@ -249,11 +249,11 @@ rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H
 rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const int32_t* seq_start,
                                    const int32_t* seq_len, int B, int S, int h, int d, bf16* ctx, cudaStream_t st,
                                    bool positional = false, int window = 0, const float* rope_cos = nullptr,
-                                   const float* rope_sin = nullptr) {
+                                   const float* rope_sin = nullptr, int kv_group = 1) {
     const int H = h * d;
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
     dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
-    const rlx::AttKind kind{window, rope_cos, rope_sin};
+    const rlx::AttKind kind{window, rope_cos, rope_sin, kv_group};
     const bool rope = rope_cos != nullptr;
     if (d != 32 && d != 64) return RLX_ERR_UNSUPPORTED;
 #define RLX_ATT_LAUNCH(D, MK, ROPE)                                                                              \
@@ -1018,7 +1018,7 @@ rlx_status_t rlx_attention_packed_bf16(const void* qkv, int32_t rows, const int3
 }
 
 rlx_status_t rlx_attention_kind_bf16(const void* qkv, int32_t rows, const int32_t* seq_start, const int32_t* seq_len,
-                                     int32_t B, int32_t max_len, int32_t h, int32_t d, int32_t mask_kind,
+                                     int32_t B, int32_t max_len, int32_t h, int32_t hkv, int32_t d, int32_t mask_kind,
                                      int32_t window, const float* rope_cos, const float* rope_sin, void* ctx,
                                      void* stream) {
     if (!qkv || !seq_start || !seq_len || !ctx || B <= 0 || max_len <= 0 || h <= 0 || rows <= 0) return RLX_ERR_INVALID_ARG;
@@ -1027,27 +1027,31 @@ rlx_status_t rlx_attention_kind_bf16(const void* qkv, int32_t rows, const int32_
     if (mask_kind != RLX_MASK_NONE && mask_kind != RLX_MASK_CAUSAL && mask_kind != RLX_MASK_SLIDING_WINDOW)
         return RLX_ERR_INVALID_ARG;
     if (mask_kind == RLX_MASK_SLIDING_WINDOW && window < 1) return RLX_ERR_INVALID_ARG;
+    if (hkv <= 0 || h % hkv != 0) return RLX_ERR_INVALID_ARG;
     if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
     const bool positional = mask_kind != RLX_MASK_NONE;
     const int w = mask_kind == RLX_MASK_SLIDING_WINDOW ? window : (1 << 30);   // causal: the window never cuts
     return launch_attention_bf16((const bf16*)qkv, nullptr, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx,
-                                 static_cast<cudaStream_t>(stream), positional, w, rope_cos, rope_sin);
+                                 static_cast<cudaStream_t>(stream), positional, w, rope_cos, rope_sin, h / hkv);
 }
 
 rlx_status_t rlx_qk_rope_bf16(void* qkv, int32_t rows, const int32_t* seq_start, const int32_t* seq_len, int32_t B,
-                              int32_t max_len, int32_t h, int32_t d, const float* rope_cos, const float* rope_sin,
-                              void* stream) {
+                              int32_t max_len, int32_t h, int32_t hkv, int32_t d, const float* rope_cos,
+                              const float* rope_sin, void* stream) {
     if (!qkv || !seq_start || !seq_len || !rope_cos || !rope_sin || B <= 0 || max_len <= 0 || h <= 0 || rows <= 0)
         return RLX_ERR_INVALID_ARG;
+    if (hkv <= 0 || h % hkv != 0) return RLX_ERR_INVALID_ARG;
     if (!aligned16(qkv) || !aligned16(rope_cos) || !aligned16(rope_sin)) return RLX_ERR_INVALID_ARG;
     if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
     dim3 grid((max_len + rlx::kRopeRows - 1) / rlx::kRopeRows, B);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d == 32)
-        rlx::qk_rope_kernel<32><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h, rope_cos, rope_sin);
+        rlx::qk_rope_kernel<32><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
+                                                                    rope_cos, rope_sin);
     else
-        rlx::qk_rope_kernel<64><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h, rope_cos, rope_sin);
+        rlx::qk_rope_kernel<64><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
+                                                                    rope_cos, rope_sin);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }

@@ -140,8 +140,8 @@ __device__ __forceinline__ int find_sequence(const int32_t* __restrict__ seq_sta
     return lo;
 }
 
-// Fused QK-RoPE: rotates, in place, the q and k column blocks of packed [rows, 3H] projections (v is
-// left alone).  grid = (row tiles of kRopeRows, sequences); one task = eight (j, j + D/2) column pairs
+// Fused QK-RoPE: rotates, in place, the q and k column blocks of packed [rows, ld] projections (v is
+// left alone; ld = 3H, or (hq + 2 hkv) D in the grouped-query layout).  grid = (row tiles of kRopeRows, sequences); one task = eight (j, j + D/2) column pairs
 // of one head of q or k of one row: 2 x 16 bytes in, 2 x 16 bytes out, consecutive lanes on consecutive
 // 16-byte chunks.  A row's position is its index within its sequence.
 constexpr int kRopeRows = 16;
@@ -149,22 +149,21 @@ constexpr int kRopeThreads = 256;
 template <int D>
 __global__ void __launch_bounds__(kRopeThreads)
 qk_rope_kernel(__nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ seq_start,
-               const int32_t* __restrict__ seq_len, int heads, const float* __restrict__ rope_cos,
+               const int32_t* __restrict__ seq_len, int rot_heads, int ld, const float* __restrict__ rope_cos,
                const float* __restrict__ rope_sin) {
     constexpr int CPR = D / 16;                 // tasks per head
     const int b = blockIdx.y;
     const int len = __ldg(seq_len + b);
     const int p0 = blockIdx.x * kRopeRows;
     if (p0 >= len) return;
-    const int H = heads * D;
     const size_t row0 = (size_t)__ldg(seq_start + b);
-    const int per_row = 2 * heads * CPR;        // q heads then k heads: columns 0 .. 2H are contiguous
+    const int per_row = rot_heads * CPR;        // q heads then k heads: one contiguous block of rot_heads * D columns
     const int nrows = min(kRopeRows, len - p0);
     for (int i = threadIdx.x; i < nrows * per_row; i += kRopeThreads) {
         const int r = i / per_row, t = i % per_row;
-        const int hd = t / CPR, c = t % CPR;    // hd in [0, 2*heads): head of q (first H columns) or k
+        const int hd = t / CPR, c = t % CPR;    // hd in [0, rot_heads): a q head, then the k heads
         const int pos = p0 + r;
-        __nv_bfloat16* base = qkv + (row0 + pos) * (size_t)(3 * H) + hd * D + c * 8;
+        __nv_bfloat16* base = qkv + (row0 + pos) * (size_t)ld + hd * D + c * 8;
         uint4 lo = *reinterpret_cast<const uint4*>(base), hi = *reinterpret_cast<const uint4*>(base + D / 2);
         const float4* pc = reinterpret_cast<const float4*>(rope_cos + (size_t)pos * (D / 2) + c * 8);
         const float4* ps = reinterpret_cast<const float4*>(rope_sin + (size_t)pos * (D / 2) + c * 8);

@@ -146,12 +146,12 @@ def test_kernel_entry_points_validate_on_the_host(lib):
 def test_attention_kind_validates_on_the_host(lib):
     fake, odd = C.c_void_p(0x1000), C.c_void_p(0x1004)
     call = lib.rlx_attention_kind_bf16
-    ok_args = dict(rows=64, batch=1, max_len=64, h=2, d=32, kind=1, window=0, cos=None, sin=None)
+    ok_args = dict(rows=64, batch=1, max_len=64, h=2, hkv=2, d=32, kind=1, window=0, cos=None, sin=None)
 
     def run(qkv=fake, start=fake, length=fake, ctx=fake, **kw):
         a = dict(ok_args, **kw)
-        return call(qkv, a["rows"], start, length, a["batch"], a["max_len"], a["h"], a["d"], a["kind"], a["window"],
-                    a["cos"], a["sin"], ctx, None)
+        return call(qkv, a["rows"], start, length, a["batch"], a["max_len"], a["h"], a["hkv"], a["d"], a["kind"],
+                    a["window"], a["cos"], a["sin"], ctx, None)
 
     assert run(qkv=None) == 1 and run(start=None) == 1 and run(length=None) == 1 and run(ctx=None) == 1
     assert run(rows=0) == 1 and run(batch=0) == 1 and run(max_len=0) == 1
@@ -159,6 +159,7 @@ def test_attention_kind_validates_on_the_host(lib):
     assert run(kind=2, window=0) == 1                      # sliding window needs w >= 1
     assert run(cos=fake, sin=None) == 1 and run(cos=None, sin=fake) == 1   # a lone table
     assert run(cos=odd, sin=fake) == 1                     # misaligned table
+    assert run(h=6, hkv=4) == 1 and run(hkv=0) == 1       # k/v heads must divide the q heads
     assert run(d=48) == 2 and run(d=128) == 2              # head sizes other than 32 / 64
     assert run(max_len=32769) == 2                         # beyond RLX_ATTENTION_KIND_MAX_LEN
 
@@ -166,12 +167,13 @@ def test_attention_kind_validates_on_the_host(lib):
 def test_qk_rope_validates_on_the_host(lib):
     fake, odd = C.c_void_p(0x1000), C.c_void_p(0x1008)
     call = lib.rlx_qk_rope_bf16
-    assert call(None, 8, fake, fake, 1, 8, 2, 32, fake, fake, None) == 1
-    assert call(fake, 8, fake, fake, 1, 8, 2, 32, None, fake, None) == 1      # both tables are required
-    assert call(fake, 8, fake, fake, 1, 8, 2, 32, fake, odd, None) == 1       # misaligned table
-    assert call(fake, 0, fake, fake, 1, 8, 2, 32, fake, fake, None) == 1
-    assert call(fake, 8, fake, fake, 1, 8, 2, 48, fake, fake, None) == 2      # head size
-    assert call(fake, 8, fake, fake, 1, 40000, 2, 32, fake, fake, None) == 2  # beyond the maximum length
+    assert call(None, 8, fake, fake, 1, 8, 2, 2, 32, fake, fake, None) == 1
+    assert call(fake, 8, fake, fake, 1, 8, 2, 2, 32, None, fake, None) == 1      # both tables are required
+    assert call(fake, 8, fake, fake, 1, 8, 2, 2, 32, fake, odd, None) == 1       # misaligned table
+    assert call(fake, 0, fake, fake, 1, 8, 2, 2, 32, fake, fake, None) == 1
+    assert call(fake, 8, fake, fake, 1, 8, 3, 2, 32, fake, fake, None) == 1      # 2 k/v heads do not divide 3
+    assert call(fake, 8, fake, fake, 1, 8, 2, 2, 48, fake, fake, None) == 2      # head size
+    assert call(fake, 8, fake, fake, 1, 40000, 2, 2, 32, fake, fake, None) == 2  # beyond the maximum length
 
 
 def test_scaled_matmul_validates_on_the_host(lib):

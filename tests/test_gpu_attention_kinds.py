@@ -166,3 +166,38 @@ def test_separate_and_in_attention_rotation_agree_bitwise(rlx, d):
     rot = rlx.qk_rope_bf16(bf16_dev(qkv), start, slen, max(lengths), h, rope)
     split = rlx.attention_kind_bf16(rot, start, slen, max(lengths), h, CAUSAL, 0, None)
     assert torch.equal(fused, split)
+
+
+@pytest.mark.parametrize("d,hq,hkv", [(64, 8, 2), (32, 6, 3), (64, 4, 1)])
+@pytest.mark.parametrize("kind,window,theta", [(CAUSAL, 0, 10000.0), (SLIDING, 70, None), (NONE, 0, None)])
+def test_grouped_query_layout_matches_oracle(rlx, d, hq, hkv, kind, window, theta):
+    """Fewer k/v heads than q heads: rows are [hq q heads | hkv k heads | hkv v heads]."""
+    rng = np.random.default_rng(d + hq + hkv + kind)
+    lengths = [130, 1, 257, 64]
+    total = sum(lengths)
+    W = (hq + 2 * hkv) * d
+    qkv = rand_bf16(rng, (total, W))
+    qkv[:, :hq * d] = round_to_bf16(qkv[:, :hq * d] * np.float32(3.0))
+    start = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    rope = None if theta is None else rlx.rope_tables(max(lengths), d, theta)
+    got = to_np64(rlx.attention_kind_bf16(bf16_dev(qkv), i32_dev(start[:-1]), i32_dev(np.array(lengths)), max(lengths), hq,
+                                          kind, window, rope, num_kv_heads=hkv))
+    ref = ak.attention_packed(qkv.astype(np.float64), start[:-1], lengths, hq, kind, window, theta, num_kv_heads=hkv)
+    vmax = float(np.abs(qkv[:, (hq + hkv) * d:]).max())
+    tol = 2 * BF16_U * (vmax + np.abs(ref).max())
+    if theta is not None:
+        q = np.abs(qkv[:, :hq * d].astype(np.float64)).reshape(total, hq, d)
+        k = np.abs(qkv[:, hq * d:(hq + hkv) * d].astype(np.float64)).reshape(total, hkv, d)
+        ds = 2 * BF16_U * float(np.sqrt((q ** 2).sum(-1)).max() * np.sqrt((k ** 2).sum(-1)).max()) / np.sqrt(d)
+        tol += 2 * ds * vmax
+    err = np.abs(got - ref)
+    assert np.isfinite(err).all() and err.max() <= tol, (float(err.max()), tol)
+    if theta is not None:
+        # the separate in-place rotation, then attention without tables: the same bits
+        rot = rlx.qk_rope_bf16(bf16_dev(qkv), i32_dev(start[:-1]), i32_dev(np.array(lengths)), max(lengths), hq, rope,
+                               num_kv_heads=hkv)
+        want = ak.rope_qk_packed(qkv.astype(np.float64), start[:-1], lengths, hq, theta, num_kv_heads=hkv)
+        assert (np.abs(to_np64(rot) - want) <= 2 * BF16_U * np.abs(want) * 1.01 + 1e-6 * np.abs(qkv).max()).all()
+        split = rlx.attention_kind_bf16(rot, i32_dev(start[:-1]), i32_dev(np.array(lengths)), max(lengths), hq, kind,
+                                        window, None, num_kv_heads=hkv)
+        assert np.array_equal(to_np64(split), got)
