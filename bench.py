@@ -253,8 +253,8 @@ def run_ours(args):
     B, S, H = cfg.batch, cfg.seq, cfg.hidden
 
     stream = torch.cuda.Stream()
-    enc = rlx.Encoder.from_config(cfg, max_batch=B, max_seq=S, device=local)
-    enc_t = rlx.Encoder.from_config(cfg, max_batch=B, max_seq=S, device=local, flags=binding.FLAG_KERNEL_EVENTS)
+    enc = rlx.Encoder.from_config(cfg, max_batch=B, max_seq=S, device=local, flags=args.flags)
+    enc_t = rlx.Encoder.from_config(cfg, max_batch=B, max_seq=S, device=local, flags=args.flags | binding.FLAG_KERNEL_EVENTS)
     ws = enc.alloc_workspace(B, S)
     ws_t = enc_t.alloc_workspace(B, S)
     ids_d = torch.from_numpy(mine.ids).cuda()
@@ -669,6 +669,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="c2", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--flags", type=lambda v: int(v, 0), default=0, help="encoder op: rlx_encoder_config_t.flags (e.g. 0x200)")
     ap.add_argument("--all-valid", action="store_true", help="encoder op: every sequence has the full length")
     ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope", "scaled_matmul"])
     ap.add_argument("--fmt", default="fp8_e4m3", choices=["fp8_e4m3", "fp4_e2m1"])

@@ -66,6 +66,13 @@ typedef enum {
 #define RLX_FLAG_CLUSTER_LN 0x80u /* fold the residual LayerNorms into the GEMMs with cluster-wide row statistics */
 #define RLX_FLAG_NO_PREFETCH 0x100u /* no L2 prefetch of the Linear weights on a side branch of the captured graph */
 #define RLX_FLAG_NO_PACK 0x8u   /* keep the padded [batch*seq] row layout instead of packing valid tokens */
+#define RLX_FLAG_FOLD_LN 0x200u /* no LayerNorm kernels inside the layers: every GEMM that consumes a LayerNorm
+                                   output runs on the raw activation with gamma-scaled weights and rebuilds the
+                                   normalisation per row in its epilogue from partial row statistics written by
+                                   the producing GEMM; the residual adds and the pooling normalise on the fly.
+                                   5 kernels per layer instead of 7; needs a larger workspace (see
+                                   rlx_encoder_workspace_bytes).  Ignored with RLX_FLAG_GEMM_SIMT; takes
+                                   precedence over RLX_FLAG_FUSED_LN / RLX_FLAG_CLUSTER_LN */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */

@@ -28,6 +28,7 @@ FLAG_ATTN_TCGEN05 = 0x20
 FLAG_FUSED_LN = 0x40
 FLAG_CLUSTER_LN = 0x80
 FLAG_NO_PREFETCH = 0x100
+FLAG_FOLD_LN = 0x200
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT = 0, 1
 STATIC_WORKSPACE_BYTES = 16 << 20

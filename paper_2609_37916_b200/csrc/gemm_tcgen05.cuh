@@ -15,6 +15,15 @@
 //               stalled the warp for about a microsecond per chunk).
 //               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop;
 //               a warp releases its accumulator as soon as its last tcgen05.ld has landed.
+// Epilogue modes (template EPI): 0 bias; 1 bias + GELU; 2 bias + residual; and the LayerNorm-folding
+// modes that let a post-LN encoder drop its LayerNorm kernels:
+//   3 / 4  the A operand is a RAW pre-LayerNorm activation y and W was pre-multiplied by gamma:
+//          out = rstd_m * (acc - mu_m * c_n) + d_n  (then GELU for 4), with c_n = sum_k W'[n,k],
+//          d_n = sum_k beta_k W[n,k] + bias_n, and (mu_m, rstd_m) rebuilt per row from per-32-column
+//          partial (mean, M2) pairs written by the GEMM that produced y  ==  LN(y) W^T + bias;
+//   5      bias + residual (already normalised), and the partial statistics of the result are written;
+//   6      bias + LN(raw residual) rebuilt on the fly from the residual's partial statistics, gamma
+//          and beta, and the partial statistics of the result are written.
 // Two instantiations per tile shape: CG = 1 (one CTA per 128 x BLOCK_N tile) and CG = 2, where a
 // cluster of two CTAs on neighbouring SMs computes a 256 x BLOCK_N tile with tcgen05.mma.cta_group::2:
 // each CTA loads its own 128 rows of A and only HALF of the W tile, the leader CTA issues the MMAs
@@ -245,7 +254,30 @@ struct Params {
     int32_t* status;                 // device status word (may be null)
     const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
     int debug;                       // experiments only: bit 0 = epilogue releases the accumulator without reading it
+    // LayerNorm folding (EPI 3..6); unused fields stay null
+    const float* cvec;               // [N] EPI 3/4: column sums of the gamma-scaled weights
+    const float* dvec;               // [N] EPI 3/4: beta . W + bias
+    const float2* stats_in;          // [M, stats_in_p] partial (mean, M2) per 32 columns: of A's rows (3/4) or the residual's (6)
+    int stats_in_p;
+    const float* ln_gamma;           // [N] EPI 6
+    const float* ln_beta;            // [N] EPI 6
+    float2* stats_out;               // [M, N/32] EPI 5/6
+    float ln_eps;
 };
+
+// (mu, rstd) of one row from its per-32-column partials (equal counts: Chan's combination)
+__device__ __forceinline__ void row_stats_from_partials(const float2* __restrict__ sp, int P, float eps, float& mu, float& rstd) {
+    float sm = 0.f;
+    for (int i = 0; i < P; ++i) sm += __ldg(&sp[i]).x;
+    mu = sm / (float)P;
+    float m2 = 0.f;
+    for (int i = 0; i < P; ++i) {
+        const float2 q = __ldg(&sp[i]);
+        const float dlt = q.x - mu;
+        m2 += q.y + 32.f * dlt * dlt;
+    }
+    rstd = 1.0f / sqrtf(m2 / (32.f * (float)P) + eps);
+}
 
 template <int BLOCK_N, int EPI, int CG>
 __global__ void __launch_bounds__((Cfg<BLOCK_N, CG>::THREADS), 1)
@@ -384,15 +416,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             const float* brow = p.bias + n0;
             // residual rows of this tile are fetched before waiting for the accumulator, so their
             // latency hides behind the main loop
-            uint4 res[EPI == 2 ? NC : 1][4];
-            if (EPI == 2) {
+            constexpr bool kRes = EPI == 2 || EPI == 5 || EPI == 6;     // a residual tile is added
+            constexpr bool kFold = EPI == 3 || EPI == 4;                // LayerNorm folded into this GEMM's input
+            constexpr bool kStatsIn = kFold || EPI == 6;
+            constexpr bool kStatsOut = EPI == 5 || EPI == 6;
+            uint4 res[kRes ? NC : 1][4];
+            float ln_a = 1.f, ln_b = 0.f;   // x_norm = x * ln_a + ln_b  (ln_a = rstd, ln_b = -rstd * mu)
+            {
                 const int m_pre = m_blk * TILE_M + (int)cta_rank * BLOCK_M + quad * 32 + lane;
-                if (m_pre < M) {
+                if (kRes && m_pre < M) {
                     const __nv_bfloat16* rpre = p.residual + (size_t)m_pre * p.N + n_blk * BLOCK_N + half * HALF_N;
 #pragma unroll
                     for (int c = 0; c < NC; ++c)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) res[c][i] = __ldg(reinterpret_cast<const uint4*>(rpre + c * 32) + i);
+                }
+                if (kStatsIn && m_pre < M) {
+                    float mu, rstd;
+                    row_stats_from_partials(p.stats_in + (size_t)m_pre * p.stats_in_p, p.stats_in_p, p.ln_eps, mu, rstd);
+                    ln_a = rstd;
+                    ln_b = -rstd * mu;
                 }
             }
             if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
@@ -424,19 +467,33 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 }
                 const uint32_t(&acc)[32] = r[c & 1];
                 float v[32];
+                if constexpr (kFold) {
+                    const float* crow = p.cvec + n0 + c * 32;
+                    const float* drow = p.dvec + n0 + c * 32;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c * 32) + i);
-                    v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4.x;
-                    v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b4.y;
-                    v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b4.z;
-                    v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b4.w;
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(crow) + i);
+                        const float4 d4 = __ldg(reinterpret_cast<const float4*>(drow) + i);
+                        v[4 * i + 0] = fmaf(ln_a, __uint_as_float(acc[4 * i + 0]), fmaf(ln_b, c4.x, d4.x));
+                        v[4 * i + 1] = fmaf(ln_a, __uint_as_float(acc[4 * i + 1]), fmaf(ln_b, c4.y, d4.y));
+                        v[4 * i + 2] = fmaf(ln_a, __uint_as_float(acc[4 * i + 2]), fmaf(ln_b, c4.z, d4.z));
+                        v[4 * i + 3] = fmaf(ln_a, __uint_as_float(acc[4 * i + 3]), fmaf(ln_b, c4.w, d4.w));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c * 32) + i);
+                        v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4.x;
+                        v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b4.y;
+                        v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b4.z;
+                        v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b4.w;
+                    }
                 }
-                if (EPI == 1) {
+                if (EPI == 1 || EPI == 4) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
                 }
-                if (EPI == 2 && row_ok) {
+                if ((EPI == 2 || EPI == 5) && row_ok) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const uint4 q = res[c][i];
@@ -445,6 +502,41 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                         v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
                         v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
                     }
+                }
+                if (EPI == 6 && row_ok) {
+                    // residual = LN(raw residual row): (x * rstd - rstd * mu) * gamma_n + beta_n
+                    const float* grow = p.ln_gamma + n0 + c * 32;
+                    const float* berow = p.ln_beta + n0 + c * 32;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 q = res[c][i];
+                        const float4 g0 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i);
+                        const float4 g1 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i + 1);
+                        const float4 e0 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i);
+                        const float4 e1 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i + 1);
+                        v[8 * i + 0] += fmaf(fmaf(bf16lo(q.x), ln_a, ln_b), g0.x, e0.x);
+                        v[8 * i + 1] += fmaf(fmaf(bf16hi(q.x), ln_a, ln_b), g0.y, e0.y);
+                        v[8 * i + 2] += fmaf(fmaf(bf16lo(q.y), ln_a, ln_b), g0.z, e0.z);
+                        v[8 * i + 3] += fmaf(fmaf(bf16hi(q.y), ln_a, ln_b), g0.w, e0.w);
+                        v[8 * i + 4] += fmaf(fmaf(bf16lo(q.z), ln_a, ln_b), g1.x, e1.x);
+                        v[8 * i + 5] += fmaf(fmaf(bf16hi(q.z), ln_a, ln_b), g1.y, e1.y);
+                        v[8 * i + 6] += fmaf(fmaf(bf16lo(q.w), ln_a, ln_b), g1.z, e1.z);
+                        v[8 * i + 7] += fmaf(fmaf(bf16hi(q.w), ln_a, ln_b), g1.w, e1.w);
+                    }
+                }
+                if (kStatsOut && row_ok) {
+                    // partial statistics of this row's 32 results (two-pass inside the chunk)
+                    float sm = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) sm += v[i];
+                    const float mean = sm * (1.0f / 32.0f);
+                    float m2 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float dl = v[i] - mean;
+                        m2 = fmaf(dl, dl, m2);
+                    }
+                    p.stats_out[(size_t)m * (p.N / 32) + (n0 + c * 32) / 32] = make_float2(mean, m2);
                 }
                 // transpose through this warp's staging buffer so that every store instruction writes
                 // whole 64-byte row segments (8 rows x 64 B per instruction, full sectors)

@@ -85,7 +85,11 @@ cudaError_t set_gemm_attr_all() {
     cudaError_t e;
     if ((e = set_gemm_attr<BN, 0, CG>()) != cudaSuccess) return e;
     if ((e = set_gemm_attr<BN, 1, CG>()) != cudaSuccess) return e;
-    return set_gemm_attr<BN, 2, CG>();
+    if ((e = set_gemm_attr<BN, 2, CG>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr<BN, 3, CG>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr<BN, 4, CG>()) != cudaSuccess) return e;
+    if ((e = set_gemm_attr<BN, 5, CG>()) != cudaSuccess) return e;
+    return set_gemm_attr<BN, 6, CG>();
 }
 
 // Number of CTA pairs that can be resident at once (pairs must sit in one GPC), per device.
@@ -244,6 +248,17 @@ rlx_status_t launch_pool(const bf16* x, const int32_t* mask, int B, int S, int H
     return RLX_OK;
 }
 
+rlx_status_t launch_pool_ln(const bf16* z, const int32_t* mask, int B, int S, int H, float* out, cudaStream_t st,
+                            const Packing& pk, const float2* stats, const float* gamma, const float* beta, float eps) {
+    if (S > rlx::kPoolMaxRows) return RLX_ERR_UNSUPPORTED;
+    const int vecs = H / 8, G = rlx::kPoolThreads / vecs;
+    const size_t smem = (size_t)G * H * sizeof(float);
+    RLX_CUDA_TRY(launch_ex(rlx::pool_ln_l2norm_kernel, B, rlx::kPoolThreads, smem, st, z, mask, out, S, H, pk.seq_start,
+                           pk.seq_len, stats, H / 32, gamma, beta, eps));
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
 // positional = false: every key of the sequence is visible (the encoder's attention); true: the window
 // rule of the kernel's MK = 1 mode (packed rows only).  rope_cos == nullptr: no rotary embedding.
 rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const int32_t* seq_start,
@@ -350,16 +365,33 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
         case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
         case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
         case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 3: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 3, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 4: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 4, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 5: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 5, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 6: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 6, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
 
+// Extra operands of the LayerNorm-folding epilogues (EPI 3..6 of the tcgen05 GEMM).
+struct LnFold {
+    const float* cvec = nullptr;
+    const float* dvec = nullptr;
+    const float2* stats_in = nullptr;
+    int stats_in_p = 0;
+    const float* gamma = nullptr;
+    const float* beta = nullptr;
+    float2* stats_out = nullptr;
+    float eps = 0.f;
+};
+
 rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const bf16* residual, int epi, int M, int N,
                          int K, bf16* out, bool simt, int32_t* status, cudaStream_t st,
-                         const int32_t* m_ptr = nullptr, int want_cg = 0) {
+                         const int32_t* m_ptr = nullptr, int want_cg = 0, const LnFold* lf = nullptr) {
     if (simt) {
+        if (epi >= 3) return RLX_ERR_UNSUPPORTED;
         dim3 grid((N + rlx::kSimtTile - 1) / rlx::kSimtTile, (M + rlx::kSimtTile - 1) / rlx::kSimtTile);
         switch (epi) {
             case 0: rlx::gemm_simt_kernel<0><<<grid, 256, 0, st>>>(A, W, bias, residual, out, M, N, K); break;
@@ -378,6 +410,11 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / tc.cg))) return RLX_ERR_CUDA;
     static const int dbg = getenv("RLX_GEMM_DEBUG") ? atoi(getenv("RLX_GEMM_DEBUG")) : 0;
     rlx::tc::Params p{bias, residual, out, M, N, K, status, m_ptr, dbg};
+    if (epi >= 3) {
+        if (!lf || N % 32 != 0) return RLX_ERR_INVALID_ARG;
+        p.cvec = lf->cvec; p.dvec = lf->dvec; p.stats_in = lf->stats_in; p.stats_in_p = lf->stats_in_p;
+        p.ln_gamma = lf->gamma; p.ln_beta = lf->beta; p.stats_out = lf->stats_out; p.ln_eps = lf->eps;
+    }
     if (tc.cg == 2) {
         switch (bn) {
             case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, p, epi, st);
@@ -488,10 +525,13 @@ rlx_status_t launch_gemm_cln(const bf16* A, const bf16* W, const float* bias, co
 // ------------------------------------------------------------------ workspace arena
 struct Arena {
     size_t status, ids, mask, out, seq_len, seq_start, pos_of_rank, x, qkv, ctx, y, x1, g, total;
+    // RLX_FLAG_FOLD_LN: partial row statistics of y and z, and per layer the gamma-scaled weights with
+    // their c / d vectors (fold_layer bytes per layer: Wqkv' | W1' | cqkv | dqkv | c1 | d1)
+    size_t stats_y, stats_z, fold, fold_layer, f_wqkv, f_w1, f_cqkv, f_dqkv, f_c1, f_d1;
 };
 constexpr size_t kTicketOffset = 64;   // packing ticket counter inside the 256-byte status block
 
-Arena plan_arena(int B, int S, int H, int F) {
+Arena plan_arena(int B, int S, int H, int F, int L = 0, bool fold = false) {
     const size_t T = (size_t)B * S;
     Arena a{};
     size_t off = 0;
@@ -513,6 +553,20 @@ Arena plan_arena(int B, int S, int H, int F) {
     a.y = take(T * H * 2);
     a.x1 = take(T * H * 2);
     a.g = take(T * F * 2);
+    if (fold) {
+        a.stats_y = take(T * (size_t)(H / 32) * sizeof(float2));
+        a.stats_z = take(T * (size_t)(H / 32) * sizeof(float2));
+        size_t lo = 0;
+        auto sub = [&](size_t bytes) { size_t o = lo; lo += round_up(bytes, 256); return o; };
+        a.f_wqkv = sub((size_t)3 * H * H * 2);
+        a.f_w1 = sub((size_t)F * H * 2);
+        a.f_cqkv = sub((size_t)3 * H * 4);
+        a.f_dqkv = sub((size_t)3 * H * 4);
+        a.f_c1 = sub((size_t)F * 4);
+        a.f_d1 = sub((size_t)F * 4);
+        a.fold_layer = lo;
+        a.fold = take(lo * (size_t)L);
+    }
     a.total = off;
     return a;
 }
@@ -534,9 +588,15 @@ bool uses_cluster_ln(const rlx_encoder_config_t& c) {
     return pick_cln_block_n(128, c.hidden) != 0;
 }
 
+// RLX_FLAG_FOLD_LN: LayerNorm folded algebraically into the consuming GEMMs (hidden % 32 == 0, seq <= 512).
+bool uses_fold_ln(const rlx_encoder_config_t& c) {
+    return (c.flags & RLX_FLAG_FOLD_LN) && !(c.flags & RLX_FLAG_GEMM_SIMT) && c.hidden % 32 == 0 &&
+           c.max_seq <= rlx::kPoolMaxRows;
+}
+
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
-    const bool fused = uses_fused_ln(c, B, S) || uses_cluster_ln(c);
+    const bool fused = uses_fold_ln(c) || uses_fused_ln(c, B, S) || uses_cluster_ln(c);
     return 2 + (fused ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
 }
 
@@ -558,7 +618,7 @@ struct rlx_encoder {
     int last_kernels = 0;                   // kernels of the most recent forward (for kernel_times)
     std::vector<cudaEvent_t> events;        // RLX_FLAG_KERNEL_EVENTS: one before the first kernel, one after each
     cudaStream_t side_stream = nullptr;     // side branch of the captured graph (weight prefetch)
-    cudaEvent_t fork_event = nullptr, join_event = nullptr;
+    cudaEvent_t fork_event = nullptr, join_event = nullptr, fold_event = nullptr;
     cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
                                             // legacy default stream, which cannot be captured)
 };
@@ -588,7 +648,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     // valid tokens are packed unless the caller asked for the padded layout (the bring-up GEMM has
     // no dynamic row count, so it implies the padded layout too)
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !simt;
-    const Arena a = plan_arena(B, S, H, F);
+    const bool fold = uses_fold_ln(c);
+    const Arena a = plan_arena(B, S, H, F, c.num_layers, fold);
     int32_t* status = reinterpret_cast<int32_t*>(ws + a.status);
     bf16* x = reinterpret_cast<bf16*>(ws + a.x);
     bf16* qkv = reinterpret_cast<bf16*>(ws + a.qkv);
@@ -617,7 +678,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && e->events.empty());
     // side branch (captured graphs only): prefetch the Linear weights into L2 when they all fit
     bool forked = false;
-    if (capturing && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH)) {
+    if (capturing && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH) && !fold) {   // the fold pass reads the weights anyway
         const size_t per_layer = ((size_t)3 * H * H + (size_t)H * H + (size_t)2 * H * F) * sizeof(bf16);
         if (per_layer * c.num_layers <= ((size_t)48 << 20) && 4 * c.num_layers <= rlx::kMaxPrefetch) {
             rlx::PrefetchList pf = {};
@@ -653,8 +714,106 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
     }
     const int32_t* rows = pk.total();
-    const bool fuse_ln = uses_fused_ln(c, B, S);
-    const bool fuse_cln = !fuse_ln && uses_cluster_ln(c);
+    const bool fuse_ln = !fold && uses_fused_ln(c, B, S);
+    const bool fuse_cln = !fold && !fuse_ln && uses_cluster_ln(c);
+    if (fold) {
+        // ---- LayerNorm folded into the GEMMs: 5 kernels per layer, no LayerNorm kernel ----
+        // gamma-scaled weights and their c / d vectors, rebuilt inside every forward (weights may change
+        // behind the same pointers).  Under capture the fold runs on the side branch and is joined before
+        // the first GEMM that needs it; eager launches run it first on the main stream.
+        rlx::FoldList fl = {};
+        fl.K = H;
+        auto add_job = [&](const void* wm, const float* gm, const float* bt, const float* bias, size_t wf_off, size_t c_off,
+                           size_t d_off, int l, int nrows) {
+            unsigned char* base = ws + a.fold + (size_t)l * a.fold_layer;
+            fl.w[fl.n] = (const bf16*)wm; fl.gamma[fl.n] = gm; fl.beta[fl.n] = bt; fl.bias[fl.n] = bias;
+            fl.wf[fl.n] = (bf16*)(base + wf_off); fl.c[fl.n] = (float*)(base + c_off); fl.d[fl.n] = (float*)(base + d_off);
+            fl.first_row[fl.n + 1] = fl.first_row[fl.n] + nrows;
+            ++fl.n;
+        };
+        const bool fold_on_side = capturing && e->side_stream != nullptr;
+        cudaStream_t fold_st = fold_on_side ? e->side_stream : st;
+        if (fold_on_side && !forked) {
+            RLX_CUDA_TRY(cudaEventRecord(e->fork_event, st));
+            RLX_CUDA_TRY(cudaStreamWaitEvent(e->side_stream, e->fork_event, 0));
+            forked = true;
+        }
+        auto flush_jobs = [&]() -> rlx_status_t {
+            if (fl.n == 0) return RLX_OK;
+            const int total_rows = fl.first_row[fl.n];
+            rlx::ln_fold_weights_kernel<<<(total_rows + rlx::kFoldWarps - 1) / rlx::kFoldWarps, rlx::kFoldWarps * 32, 0, fold_st>>>(fl);
+            RLX_CUDA_TRY(cudaGetLastError());
+            fl.n = 0;
+            fl.first_row[0] = 0;
+            return RLX_OK;
+        };
+        for (int l = 0; l < c.num_layers; ++l) {
+            const rlx_layer_weights_t& lw = w->layers[l];
+            if (l > 0) {   // the QKV projection of layer l consumes LN2 of layer l-1
+                const rlx_layer_weights_t& pw = w->layers[l - 1];
+                add_job(lw.wqkv, pw.ln2_g, pw.ln2_b, lw.bqkv, a.f_wqkv, a.f_cqkv, a.f_dqkv, l, 3 * H);
+                if (fl.n == rlx::kFoldMaxJobs) { s = flush_jobs(); if (s != RLX_OK) return s; }
+            }
+            add_job(lw.w1, lw.ln1_g, lw.ln1_b, lw.b1, a.f_w1, a.f_c1, a.f_d1, l, F);
+            if (fl.n == rlx::kFoldMaxJobs) { s = flush_jobs(); if (s != RLX_OK) return s; }
+        }
+        s = flush_jobs();
+        if (s != RLX_OK) return s;
+        if (fold_on_side) RLX_CUDA_TRY(cudaEventRecord(e->fold_event, e->side_stream));
+        if (forked) RLX_CUDA_TRY(cudaEventRecord(e->join_event, e->side_stream));
+
+        float2* stats_y = reinterpret_cast<float2*>(ws + a.stats_y);
+        float2* stats_z = reinterpret_cast<float2*>(ws + a.stats_z);
+        bf16* z = x1;   // raw output of the FFN-down projection (pre-LayerNorm), reused across layers
+        const int P = H / 32;
+        RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
+                                w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
+        for (int l = 0; l < c.num_layers; ++l) {
+            const rlx_layer_weights_t& lw = w->layers[l];
+            unsigned char* fb = ws + a.fold + (size_t)l * a.fold_layer;
+            LnFold lf;
+            lf.eps = c.ln_eps;
+            if (l == 0) {
+                RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, false, status, st, rows));
+            } else {
+                lf.cvec = (const float*)(fb + a.f_cqkv); lf.dvec = (const float*)(fb + a.f_dqkv);
+                lf.stats_in = stats_z; lf.stats_in_p = P;
+                RLX_TRY(launch_gemm(z, (const bf16*)(fb + a.f_wqkv), lw.bqkv, nullptr, 3, T, 3 * H, H, qkv, false, status, st, rows, 0, &lf));
+            }
+            if (pack && (c.flags & RLX_FLAG_ATTN_TCGEN05))
+                RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx, status, st));
+            else
+                RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
+            // y = ctx Wo^T + bo + (l == 0 ? x : LN2_{l-1}(z)); partial statistics of y
+            lf = LnFold();
+            lf.eps = c.ln_eps;
+            lf.stats_out = stats_y;
+            if (l == 0) {
+                RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, 5, T, H, H, y, false, status, st, rows, 0, &lf));
+            } else {
+                const rlx_layer_weights_t& pw = w->layers[l - 1];
+                lf.stats_in = stats_z; lf.stats_in_p = P; lf.gamma = pw.ln2_g; lf.beta = pw.ln2_b;
+                RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, z, 6, T, H, H, y, false, status, st, rows, 0, &lf));
+            }
+            // g = gelu(LN1(y) W1^T + b1) on the raw y with the folded weights
+            if (l == 0 && fold_on_side) RLX_CUDA_TRY(cudaStreamWaitEvent(st, e->fold_event, 0));
+            lf = LnFold();
+            lf.eps = c.ln_eps;
+            lf.cvec = (const float*)(fb + a.f_c1); lf.dvec = (const float*)(fb + a.f_d1);
+            lf.stats_in = stats_y; lf.stats_in_p = P;
+            RLX_TRY(launch_gemm(y, (const bf16*)(fb + a.f_w1), lw.b1, nullptr, 4, T, F, H, g, false, status, st, rows, 0, &lf));
+            // z = g W2^T + b2 + LN1(y); partial statistics of z.  The previous z is dead by now (its last
+            // readers were this layer's QKV and out-projection GEMMs).
+            lf = LnFold();
+            lf.eps = c.ln_eps;
+            lf.stats_in = stats_y; lf.stats_in_p = P; lf.gamma = lw.ln1_g; lf.beta = lw.ln1_b; lf.stats_out = stats_z;
+            RLX_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, y, 6, T, H, F, z, false, status, st, rows, 0, &lf));
+        }
+        const rlx_layer_weights_t& last = w->layers[c.num_layers - 1];
+        RLX_TRY(launch_pool_ln(z, mask, B, S, H, out, st, pk, stats_z, last.ln2_g, last.ln2_b, c.ln_eps));
+        if (forked) RLX_CUDA_TRY(cudaStreamWaitEvent(st, e->join_event, 0));   // join the side branch
+        return RLX_OK;
+    }
     RLX_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
                             w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
     for (int l = 0; l < c.num_layers; ++l) {
@@ -705,7 +864,7 @@ rlx_status_t check_forward_args(const rlx_encoder* e, const void* ids, const voi
         for (size_t i = 0; i < sizeof(rlx_layer_weights_t) / sizeof(void*); ++i)
             if (!ptrs[i] || !aligned16(ptrs[i])) return RLX_ERR_INVALID_ARG;
     }
-    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn, e->cfg.num_layers, uses_fold_ln(e->cfg));
     if (ws_bytes < a.total) return RLX_ERR_WORKSPACE;
     return RLX_OK;
 }
@@ -743,6 +902,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
         RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->side_stream, cudaStreamNonBlocking));
         RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->fork_event, cudaEventDisableTiming));
         RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->join_event, cudaEventDisableTiming));
+        RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->fold_event, cudaEventDisableTiming));
     }
     RLX_CUDA_TRY(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal));
     rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream, true);
@@ -797,13 +957,14 @@ void rlx_encoder_destroy(rlx_encoder_t* e) {
     if (e->side_stream) cudaStreamDestroy(e->side_stream);
     if (e->fork_event) cudaEventDestroy(e->fork_event);
     if (e->join_event) cudaEventDestroy(e->join_event);
+    if (e->fold_event) cudaEventDestroy(e->fold_event);
     for (auto& evt : e->events) cudaEventDestroy(evt);
     delete e;
 }
 
 size_t rlx_encoder_workspace_bytes(const rlx_encoder_t* e, int32_t batch, int32_t seq) {
     if (!e || batch <= 0 || seq <= 0 || batch > e->cfg.max_batch || seq > e->cfg.max_seq) return 0;
-    return plan_arena(batch, seq, e->cfg.hidden, e->cfg.ffn).total;
+    return plan_arena(batch, seq, e->cfg.hidden, e->cfg.ffn, e->cfg.num_layers, uses_fold_ln(e->cfg)).total;
 }
 
 int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t* e, int32_t batch, int32_t seq) {
@@ -825,7 +986,7 @@ rlx_status_t rlx_encoder_forward_host(rlx_encoder_t* e, const int32_t* ids_h, co
     if (s != RLX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned char* base = static_cast<unsigned char*>(ws);
-    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn, e->cfg.num_layers, uses_fold_ln(e->cfg));
     int32_t* ids_d = reinterpret_cast<int32_t*>(base + a.ids);
     int32_t* mask_d = reinterpret_cast<int32_t*>(base + a.mask);
     float* out_d = reinterpret_cast<float*>(base + a.out);
@@ -912,7 +1073,7 @@ rlx_status_t rlx_encoder_forward_static(rlx_encoder_t* e, const int32_t* ids, co
     rlx_status_t s = check_forward_args(e, ids, mask, B, S, w, out, reinterpret_cast<void*>(uintptr_t(256)),
                                         ~size_t(0), false);
     if (s != RLX_OK) return s;
-    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn);
+    const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn, e->cfg.num_layers, uses_fold_ln(e->cfg));
     if (a.total > (size_t)RLX_STATIC_WORKSPACE_BYTES) return RLX_ERR_WORKSPACE;  // beyond the built-in arena
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int dev = -1;

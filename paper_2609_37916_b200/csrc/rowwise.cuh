@@ -381,4 +381,177 @@ pool_l2norm_kernel(const __nv_bfloat16* __restrict__ x, const int32_t* __restric
     }
 }
 
+// ----------------------------------------------------------------------------------------------
+// LayerNorm folding (post-LN encoders without LayerNorm kernels).
+//
+// LN(y) W^T + b = rstd * (y (gamma o W)^T - mu * c) + d  with  c_n = sum_k gamma_k W_nk,
+// d_n = sum_k beta_k W_nk + b_n: the GEMM that consumes a LayerNorm output can run on the RAW
+// activation y with gamma-scaled weights and fix the result up per row in its epilogue.  This kernel
+// prepares W' = bf16(gamma o W) (c is summed over the ROUNDED W', so the identity holds exactly for the
+// weights the tensor cores see), c and d for a list of matrices in one launch: one warp per output row.
+constexpr int kFoldMaxJobs = 24;
+constexpr int kFoldWarps = 8;
+struct FoldList {
+    const __nv_bfloat16* w[kFoldMaxJobs];
+    const float* gamma[kFoldMaxJobs];
+    const float* beta[kFoldMaxJobs];
+    const float* bias[kFoldMaxJobs];
+    __nv_bfloat16* wf[kFoldMaxJobs];
+    float* c[kFoldMaxJobs];
+    float* d[kFoldMaxJobs];
+    int first_row[kFoldMaxJobs + 1];   // prefix sums of the jobs' row counts
+    int n;
+    int K;                              // row length (the LayerNorm width), K % 256 == 0 not required: K % 8 == 0
+};
+
+__global__ void __launch_bounds__(kFoldWarps * 32)
+ln_fold_weights_kernel(const __grid_constant__ FoldList fl) {
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * kFoldWarps + (threadIdx.x >> 5);
+    if (row >= fl.first_row[fl.n]) return;
+    int j = 0;
+    while (row >= fl.first_row[j + 1]) ++j;
+    const int n = row - fl.first_row[j];
+    const int K = fl.K;
+    const __nv_bfloat16* wr = fl.w[j] + (size_t)n * K;
+    __nv_bfloat16* wo = fl.wf[j] + (size_t)n * K;
+    float cs = 0.f, ds = 0.f;
+    for (int k = lane * 8; k < K; k += 256) {
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(wr + k));
+        const float4 g0 = __ldg(reinterpret_cast<const float4*>(fl.gamma[j] + k)), g1 = __ldg(reinterpret_cast<const float4*>(fl.gamma[j] + k) + 1);
+        const float4 b0 = __ldg(reinterpret_cast<const float4*>(fl.beta[j] + k)), b1 = __ldg(reinterpret_cast<const float4*>(fl.beta[j] + k) + 1);
+        const float wv[8] = {bf16lo(q.x), bf16hi(q.x), bf16lo(q.y), bf16hi(q.y), bf16lo(q.z), bf16hi(q.z), bf16lo(q.w), bf16hi(q.w)};
+        const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        const float bv[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            o[i] = pack_bf16(wv[2 * i] * gv[2 * i], wv[2 * i + 1] * gv[2 * i + 1]);
+            cs += bf16lo(o[i]) + bf16hi(o[i]);
+            ds = fmaf(bv[2 * i], wv[2 * i], fmaf(bv[2 * i + 1], wv[2 * i + 1], ds));
+        }
+        *reinterpret_cast<uint4*>(wo + k) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    cs = warp_sum(cs);
+    ds = warp_sum(ds);
+    if (lane == 0) {
+        fl.c[j][n] = cs;
+        fl.d[j][n] = ds + __ldg(fl.bias[j] + n);
+    }
+}
+
+// Masked mean-pool + L2 normalisation of LN(z), z being the RAW last activation and its row statistics
+// arriving as per-32-column partials (the form the folding GEMM epilogues write).  One CTA per
+// sequence: first every row's (rstd, -rstd*mu) goes to shared memory, then thread (g, c) accumulates
+// z * rstd over its rows for its 8 columns; sum_r LN(z)_rc = gamma_c * (sum_r z_rc rstd_r + sum_r b_r)
+// + n * beta_c.  Fixed-order reductions (deterministic).
+constexpr int kPoolMaxRows = 512;
+__global__ void __launch_bounds__(kPoolThreads)
+pool_ln_l2norm_kernel(const __nv_bfloat16* __restrict__ z, const int32_t* __restrict__ mask, float* __restrict__ out, int S,
+                      int H, const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
+                      const float2* __restrict__ stats, int P, const float* __restrict__ gamma,
+                      const float* __restrict__ beta, float eps) {
+    extern __shared__ float pool_smem[];   // [G][H] partial sums
+    __shared__ float s_a[kPoolMaxRows], s_b[kPoolThreads / 32];
+    __shared__ float s_red[kPoolThreads / 32];
+    __shared__ int s_cnt[kPoolThreads / 32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int b = blockIdx.x;
+    const int vecs = H / 8, G = kPoolThreads / vecs;
+    const int g = threadIdx.x / vecs, c = threadIdx.x % vecs;
+    const bool packed = seq_start != nullptr;
+    const size_t row0 = packed ? (size_t)__ldg(seq_start + b) : (size_t)b * S;
+    const int nrows = packed ? __ldg(seq_len + b) : S;
+    const int32_t* mb = mask + (size_t)b * S;
+    // phase 0: row statistics -> (a, b) per row; a = 0 marks a row that is not pooled
+    float bsum = 0.f;
+    int cnt = 0;
+    for (int r = threadIdx.x; r < nrows; r += kPoolThreads) {
+        float a = 0.f, bb = 0.f;
+        if (packed || __ldg(mb + r) != 0) {
+            float mu, rstd;
+            // inline Chan combination of the row's partials
+            const float2* sp = stats + (row0 + r) * (size_t)P;
+            float sm = 0.f;
+            for (int i = 0; i < P; ++i) sm += __ldg(&sp[i]).x;
+            mu = sm / (float)P;
+            float m2 = 0.f;
+            for (int i = 0; i < P; ++i) {
+                const float2 q = __ldg(&sp[i]);
+                const float dl = q.x - mu;
+                m2 += q.y + 32.f * dl * dl;
+            }
+            rstd = 1.0f / sqrtf(m2 / (32.f * (float)P) + eps);
+            a = rstd;
+            bb = -rstd * mu;
+            ++cnt;
+        }
+        s_a[r] = a;
+        bsum += bb;
+    }
+    // sum of the b terms and the row count: warp butterflies, then the warps' values in index order
+    // (a fixed order, so every thread and every run gets the same bits)
+    {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            bsum += __shfl_xor_sync(0xffffffffu, bsum, o);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            s_cnt[threadIdx.x >> 5] = cnt;
+            s_b[threadIdx.x >> 5] = bsum;
+        }
+    }
+    __syncthreads();
+    bsum = 0.f;
+#pragma unroll
+    for (int i = 0; i < kPoolThreads / 32; ++i) bsum += s_b[i];
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (g < G) {
+        const __nv_bfloat16* zb = z + row0 * H + c * 8;
+        for (int r = g; r < nrows; r += G) {
+            const float a = s_a[r];
+            if (a == 0.f) continue;
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(zb + (size_t)r * H));
+            acc[0] = fmaf(bf16lo(q.x), a, acc[0]); acc[1] = fmaf(bf16hi(q.x), a, acc[1]);
+            acc[2] = fmaf(bf16lo(q.y), a, acc[2]); acc[3] = fmaf(bf16hi(q.y), a, acc[3]);
+            acc[4] = fmaf(bf16lo(q.z), a, acc[4]); acc[5] = fmaf(bf16hi(q.z), a, acc[5]);
+            acc[6] = fmaf(bf16lo(q.w), a, acc[6]); acc[7] = fmaf(bf16hi(q.w), a, acc[7]);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pool_smem[g * H + c * 8 + i] = acc[i];
+    }
+    __syncthreads();
+    int n_rows = 0;
+#pragma unroll
+    for (int i = 0; i < kPoolThreads / 32; ++i) n_rows += s_cnt[i];
+    const float n_valid = (float)n_rows;
+    const float inv_n = 1.0f / fmaxf(n_valid, 1e-9f);
+    float colsum[3] = {0.f, 0.f, 0.f};
+    float sq = 0.f;
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr) {
+        const int j = threadIdx.x + rr * kPoolThreads;
+        if (j < H) {
+            float t = 0.f;
+            for (int gg = 0; gg < G; ++gg) t += pool_smem[gg * H + j];
+            t = (__ldg(gamma + j) * (t + bsum) + n_valid * __ldg(beta + j)) * inv_n;
+            colsum[rr] = t;
+            sq += t * t;
+        }
+    }
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    float tot = 0.f;
+    for (int i = 0; i < kPoolThreads / 32; ++i) tot += s_red[i];
+    const float inv_norm = 1.0f / fmaxf(sqrtf(tot), 1e-12f);
+#pragma unroll
+    for (int rr = 0; rr < 3; ++rr) {
+        const int j = threadIdx.x + rr * kPoolThreads;
+        if (j < H) out[(size_t)b * H + j] = colsum[rr] * inv_norm;
+    }
+}
+
 }  // namespace rlx
