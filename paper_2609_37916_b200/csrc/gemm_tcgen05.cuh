@@ -266,17 +266,28 @@ struct Params {
 };
 
 // (mu, rstd) of one row from its per-32-column partials (equal counts: Chan's combination)
+// One pass over 16-byte loads (two partials each, all in flight together): sum of the means, of the M2
+// terms and of the squared means; the between-chunk part  32 * (sum mean_i^2 - P mu^2)  is a difference
+// of small numbers of one sign-definite kind (clamped at zero), accurate unless |mu| exceeds the row's
+// standard deviation by three orders of magnitude.
 __device__ __forceinline__ void row_stats_from_partials(const float2* __restrict__ sp, int P, float eps, float& mu, float& rstd) {
-    float sm = 0.f;
-    for (int i = 0; i < P; ++i) sm += __ldg(&sp[i]).x;
-    mu = sm / (float)P;
-    float m2 = 0.f;
-    for (int i = 0; i < P; ++i) {
-        const float2 q = __ldg(&sp[i]);
-        const float dlt = q.x - mu;
-        m2 += q.y + 32.f * dlt * dlt;
+    float sm = 0.f, sq = 0.f, m2 = 0.f;
+    const float4* sp4 = reinterpret_cast<const float4*>(sp);
+    for (int i = 0; i < P / 2; ++i) {
+        const float4 q = __ldg(sp4 + i);
+        sm += q.x + q.z;
+        sq = fmaf(q.x, q.x, fmaf(q.z, q.z, sq));
+        m2 += q.y + q.w;
     }
-    rstd = 1.0f / sqrtf(m2 / (32.f * (float)P) + eps);
+    if (P & 1) {
+        const float2 q = __ldg(sp + P - 1);
+        sm += q.x;
+        sq = fmaf(q.x, q.x, sq);
+        m2 += q.y;
+    }
+    mu = sm / (float)P;
+    const float between = fmaxf(sq - (float)P * mu * mu, 0.f);
+    rstd = 1.0f / sqrtf((m2 + 32.f * between) / (32.f * (float)P) + eps);
 }
 
 template <int BLOCK_N, int EPI, int CG>
