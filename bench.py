@@ -442,7 +442,7 @@ def run_attention_kind(args):
     import torch
     import paper_2609_37916_b200 as rlx
 
-    h, d = args.heads, 64
+    h, d = args.heads, args.head_dim
     hkv = args.kv_heads or h
     H = h * d
     lengths = attention_kind_workload()
@@ -493,11 +493,11 @@ def run_attention_kind(args):
         "value": total * args.steps / (sum(ms) / 1e3), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": sum(ms) / args.steps, "p50_ms": p50, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), {h} q heads / {hkv} kv heads x 64, "
+        "config": {"workload": f"packed batch of 16 sequences, lengths 1024..4096 (seed 7, {total} tokens), {h} q heads / {hkv} kv heads x {d}, "
                                f"mask {args.mask}" + (f"({args.window})" if args.mask == "sliding" else "") +
                                (", rotary q,k" if args.rope else ""), "l2": "256 MiB flush write between steps"},
         "gpu_launches": args.steps, "clocks": sampler.summary(),
-        "roofline": {"kernel": "attention_bf16_kernel<64>", "bound": "alu", "achieved": exps / (p50 * 1e-3) / 1e12,
+        "roofline": {"kernel": f"attention_bf16_kernel<{d}>", "bound": "alu", "achieved": exps / (p50 * 1e-3) / 1e12,
                      "peak": EXP_PEAK_TEXP_S, "unit": "Texp/s", "frac": exps / (p50 * 1e-3) / 1e12 / EXP_PEAK_TEXP_S,
                      "traffic": None, "tensor_tflops": flops / (p50 * 1e-3) / 1e12,
                      "tensor_frac_of_" + peak_kind: flops / (p50 * 1e-3) / 1e12 / peaks["bf16_tflops"],
@@ -677,6 +677,7 @@ def main():
     ap.add_argument("--window", type=int, default=512)
     ap.add_argument("--rope", type=int, default=1)
     ap.add_argument("--heads", type=int, default=16, help="attention_kind op: q heads (head_dim 64)")
+    ap.add_argument("--head-dim", type=int, default=64, choices=[32, 64, 128], help="attention_kind op: head size")
     ap.add_argument("--kv-heads", type=int, default=0, help="attention_kind op: k/v heads (0 = same as --heads)")
     args = ap.parse_args()
     if args.op != "encoder":

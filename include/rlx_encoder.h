@@ -356,7 +356,8 @@ rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const
  * memory, 16-byte aligned; seq_len[b] <= max_len <= RLX_ATTENTION_KIND_MAX_LEN).  rope_cos and
  * rope_sin are device fp32 tables [max_len, head_dim/2] (row = position, 16-byte aligned) holding
  * cos / sin of position * theta^(-2j/head_dim), or both NULL for no rotation.  `window` is read for
- * RLX_MASK_SLIDING_WINDOW only.  head_dim in {32, 64}.  Key blocks that no row of a 128-row query
+ * RLX_MASK_SLIDING_WINDOW only.  head_dim in {32, 64, 128} (128: one CTA per SM, the accumulator tile
+ * fills the register file).  Key blocks that no row of a 128-row query
  * tile can see are neither loaded nor multiplied.  Asynchronous on cuda_stream; the caller owns
  * every buffer; nothing is allocated.  Errors: RLX_ERR_INVALID_ARG for null / misaligned pointers,
  * a lone rope table, an unknown kind or window < 1; RLX_ERR_UNSUPPORTED for other head sizes or

@@ -8,7 +8,9 @@
 //    shuffles, the row sums come from an extra ones column of the PV product; the 1/sqrt(d)*log2(e)
 //    scale is folded into the exp2 argument.  At head_dim 32 the online-softmax step is 32 keys (half a
 //    staged block): 64 registers per thread, four CTAs per SM instead of three (-6 % on the 256 x 256
-//    workload; at head_dim 64, and in the mask-kind / rotary modes, the 64-key step is kept).  Key blocks beyond the
+//    workload; at head_dim 64, and in the mask-kind / rotary modes, the 64-key step is kept).  head_dim 128
+//    (mask-kind entry point only) runs one CTA per SM with the 32-key step: 64 output accumulators and
+//    32 Q-fragment registers per thread leave no room for more.  Key blocks beyond the
 //    last valid key are never loaded; masking runs only in blocks that contain an invalid key.
 //  attention_f32_kernel: fp32 in/out CUDA-core kernel, one warp per query row, K/V staged in shared
 //    memory 32 keys at a time, warp-shuffle reductions.  Reference-precision mode for testing.
@@ -110,8 +112,8 @@ struct AttKind {
 // Two addressing modes share the kernel:
 //   padded: seq_start == nullptr.  Sequence b occupies rows b*S .. b*S+S; `mask` flags valid keys.
 //   packed: rows of sequence b are seq_start[b] .. seq_start[b]+seq_len[b], all valid (mask unused).
-template <int D, int MK = 0, bool ROPE = false, int KS = ((D == 32 && MK == 0 && !ROPE) ? 32 : 64),
-          int MINB = (D == 32 ? (KS == 32 ? 4 : 3) : 2)>
+template <int D, int MK = 0, bool ROPE = false, int KS = (((D == 32 && MK == 0 && !ROPE) || D == 128) ? 32 : 64),
+          int MINB = (D == 32 ? (KS == 32 ? 4 : 3) : D == 64 ? 2 : 1)>
 __global__ void __launch_bounds__(kAttThreads, MINB)
 attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ mask,
                       const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,

@@ -151,6 +151,7 @@ cudaError_t init_kernels_for_current_device() {
     RLX_ATT_SMEM_ATTR(32, 0, true) RLX_ATT_SMEM_ATTR(64, 0, true)
     RLX_ATT_SMEM_ATTR(32, 1, false) RLX_ATT_SMEM_ATTR(64, 1, false)
     RLX_ATT_SMEM_ATTR(32, 1, true) RLX_ATT_SMEM_ATTR(64, 1, true)
+    RLX_ATT_SMEM_ATTR(128, 0, false) RLX_ATT_SMEM_ATTR(128, 0, true) RLX_ATT_SMEM_ATTR(128, 1, false) RLX_ATT_SMEM_ATTR(128, 1, true)
 #undef RLX_ATT_SMEM_ATTR
     if (dev < 64) done[dev] = true;
     return cudaSuccess;
@@ -270,7 +271,7 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     dim3 grid((S + rlx::kAttBlockM - 1) / rlx::kAttBlockM, h, B);
     const rlx::AttKind kind{window, rope_cos, rope_sin, kv_group};
     const bool rope = rope_cos != nullptr;
-    if (d != 32 && d != 64) return RLX_ERR_UNSUPPORTED;
+    if (d != 32 && d != 64 && d != 128) return RLX_ERR_UNSUPPORTED;
 #define RLX_ATT_LAUNCH(D, MK, ROPE)                                                                              \
     RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<D, MK, ROPE>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<D>), \
                            st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e, kind))
@@ -279,11 +280,16 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
         else if (!positional) RLX_ATT_LAUNCH(32, 0, true);
         else if (!rope) RLX_ATT_LAUNCH(32, 1, false);
         else RLX_ATT_LAUNCH(32, 1, true);
-    } else {
+    } else if (d == 64) {
         if (!positional && !rope) RLX_ATT_LAUNCH(64, 0, false);
         else if (!positional) RLX_ATT_LAUNCH(64, 0, true);
         else if (!rope) RLX_ATT_LAUNCH(64, 1, false);
         else RLX_ATT_LAUNCH(64, 1, true);
+    } else {
+        if (!positional && !rope) RLX_ATT_LAUNCH(128, 0, false);
+        else if (!positional) RLX_ATT_LAUNCH(128, 0, true);
+        else if (!rope) RLX_ATT_LAUNCH(128, 1, false);
+        else RLX_ATT_LAUNCH(128, 1, true);
     }
 #undef RLX_ATT_LAUNCH
     RLX_CUDA_TRY(cudaGetLastError());
@@ -1189,7 +1195,8 @@ rlx_status_t rlx_attention_kind_bf16(const void* qkv, int32_t rows, const int32_
         return RLX_ERR_INVALID_ARG;
     if (mask_kind == RLX_MASK_SLIDING_WINDOW && window < 1) return RLX_ERR_INVALID_ARG;
     if (hkv <= 0 || h % hkv != 0) return RLX_ERR_INVALID_ARG;
-    if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    if ((d != 32 && d != 64 && d != 128) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535)
+        return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
     const bool positional = mask_kind != RLX_MASK_NONE;
     const int w = mask_kind == RLX_MASK_SLIDING_WINDOW ? window : (1 << 30);   // causal: the window never cuts
@@ -1204,15 +1211,19 @@ rlx_status_t rlx_qk_rope_bf16(void* qkv, int32_t rows, const int32_t* seq_start,
         return RLX_ERR_INVALID_ARG;
     if (hkv <= 0 || h % hkv != 0) return RLX_ERR_INVALID_ARG;
     if (!aligned16(qkv) || !aligned16(rope_cos) || !aligned16(rope_sin)) return RLX_ERR_INVALID_ARG;
-    if ((d != 32 && d != 64) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535) return RLX_ERR_UNSUPPORTED;
+    if ((d != 32 && d != 64 && d != 128) || max_len > RLX_ATTENTION_KIND_MAX_LEN || B > 65535 || h > 65535)
+        return RLX_ERR_UNSUPPORTED;
     dim3 grid((max_len + rlx::kRopeRows - 1) / rlx::kRopeRows, B);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (d == 32)
         rlx::qk_rope_kernel<32><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
                                                                     rope_cos, rope_sin);
-    else
+    else if (d == 64)
         rlx::qk_rope_kernel<64><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
                                                                     rope_cos, rope_sin);
+    else
+        rlx::qk_rope_kernel<128><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
+                                                                     rope_cos, rope_sin);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }

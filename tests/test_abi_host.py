@@ -160,7 +160,7 @@ def test_attention_kind_validates_on_the_host(lib):
     assert run(cos=fake, sin=None) == 1 and run(cos=None, sin=fake) == 1   # a lone table
     assert run(cos=odd, sin=fake) == 1                     # misaligned table
     assert run(h=6, hkv=4) == 1 and run(hkv=0) == 1       # k/v heads must divide the q heads
-    assert run(d=48) == 2 and run(d=128) == 2              # head sizes other than 32 / 64
+    assert run(d=48) == 2 and run(d=256) == 2              # head sizes other than 32 / 64 / 128
     assert run(max_len=32769) == 2                         # beyond RLX_ATTENTION_KIND_MAX_LEN
 
 

@@ -130,7 +130,7 @@ def test_causal_never_reads_the_future_bitwise(rlx):
     assert torch.equal(a[:cut + 1], b[:cut + 1]) and not torch.equal(a[cut + 1:], b[cut + 1:])
 
 
-@pytest.mark.parametrize("d,h", [(32, 3), (64, 2)])
+@pytest.mark.parametrize("d,h", [(32, 3), (64, 2), (128, 2)])
 def test_qk_rope_in_place_matches_oracle(rlx, d, h):
     rng = np.random.default_rng(20 + d)
     H = h * d
@@ -168,7 +168,7 @@ def test_separate_and_in_attention_rotation_agree_bitwise(rlx, d):
     assert torch.equal(fused, split)
 
 
-@pytest.mark.parametrize("d,hq,hkv", [(64, 8, 2), (32, 6, 3), (64, 4, 1)])
+@pytest.mark.parametrize("d,hq,hkv", [(64, 8, 2), (32, 6, 3), (64, 4, 1), (128, 4, 2), (128, 2, 2)])
 @pytest.mark.parametrize("kind,window,theta", [(CAUSAL, 0, 10000.0), (SLIDING, 70, None), (NONE, 0, None)])
 def test_grouped_query_layout_matches_oracle(rlx, d, hq, hkv, kind, window, theta):
     """Fewer k/v heads than q heads: rows are [hq q heads | hkv k heads | hkv v heads]."""
@@ -201,3 +201,10 @@ def test_grouped_query_layout_matches_oracle(rlx, d, hq, hkv, kind, window, thet
         split = rlx.attention_kind_bf16(rot, i32_dev(start[:-1]), i32_dev(np.array(lengths)), max(lengths), hq, kind,
                                         window, None, num_kv_heads=hkv)
         assert np.array_equal(to_np64(split), got)
+
+
+@pytest.mark.parametrize("kind,window,theta", [(CAUSAL, 0, 10000.0), (CAUSAL, 0, None), (SLIDING, 33, 10000.0), (NONE, 0, None)])
+def test_head_dim_128(rlx, kind, window, theta):
+    """The head size of the larger decoder families: same kernel, one CTA per SM."""
+    for gain in (1.0, 3.0):
+        _run_case(rlx, [1, 17, 64, 65, 129, 300, 700], 2, 128, kind, window, theta, gain, seed=128 + kind + window)
