@@ -208,3 +208,22 @@ def test_head_dim_128(rlx, kind, window, theta):
     """The head size of the larger decoder families: same kernel, one CTA per SM."""
     for gain in (1.0, 3.0):
         _run_case(rlx, [1, 17, 64, 65, 129, 300, 700], 2, 128, kind, window, theta, gain, seed=128 + kind + window)
+
+
+def test_empty_sequences_and_a_long_one(rlx):
+    """Zero-length sequences write nothing; an 8,192-row sequence exercises 64 query tiles and, with a
+    window, the skipping of leading key blocks far from the diagonal."""
+    rng = np.random.default_rng(77)
+    h, d = 1, 32
+    H = h * d
+    lengths = [0, 8192, 0, 5]
+    total = sum(lengths)
+    qkv = rand_bf16(rng, (total, 3 * H))
+    qkv[:, :H] = round_to_bf16(qkv[:, :H] * np.float32(2.0))
+    start = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    for kind, w in ((CAUSAL, 0), (SLIDING, 300)):
+        got = to_np64(rlx.attention_kind_bf16(bf16_dev(qkv), i32_dev(start[:-1]), i32_dev(np.array(lengths)), max(lengths), h,
+                                              kind, w))
+        ref = ak.attention_packed(qkv.astype(np.float64), start[:-1], lengths, h, kind, w)
+        vmax = float(np.abs(qkv[:, 2 * H:]).max())
+        assert np.abs(got - ref).max() <= 2 * BF16_U * (vmax + np.abs(ref).max())
