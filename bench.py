@@ -125,10 +125,12 @@ def time_oracle(cfg_name: str, budget_s: float, steps: int = 1, warmup: int = 0,
     cores = usable_cores()
     oracle.set_threads(cores)
 
+    last_out = {}
+
     def run(n):
         sub = EncoderConfig(**{**cfg.__dict__, "batch": n})
         t0 = time.perf_counter()
-        oracle.encoder_forward(sub, inp.ids[:n], inp.mask[:n], inp.params, inp.layers)
+        last_out["emb"] = oracle.encoder_forward(sub, inp.ids[:n], inp.mask[:n], inp.params, inp.layers)
         return time.perf_counter() - t0
 
     run(1)  # builds/loads the library, warms caches
@@ -137,7 +139,7 @@ def time_oracle(cfg_name: str, budget_s: float, steps: int = 1, warmup: int = 0,
     for _ in range(warmup):
         run(n)
     times = [run(n) for _ in range(max(steps, 1))]
-    return {"times": times, "n": n, "cores": cores, "batch": cfg.batch}
+    return {"times": times, "n": n, "cores": cores, "batch": cfg.batch, "embeddings": last_out["emb"]}
 
 
 def run_reference_arm(args):
@@ -383,6 +385,13 @@ def run_ours(args):
 
         cb = time_oracle(args.config, budget_s=15.0, steps=1, all_valid=args.all_valid)
         cb_value = cb["n"] / cb["times"][0]
+        # the oracle's embeddings of its sample double as a parity check of this very run (rank 0's batch)
+        got = out_d[:cb["n"]].double().cpu().numpy()
+        ref = cb["embeddings"]
+        keep = mine.lengths[:cb["n"]] > 0
+        cosines = (got * ref).sum(1)[keep] / np.maximum(np.linalg.norm(got, axis=1) * np.linalg.norm(ref, axis=1), 1e-300)[keep]
+        parity = {"sequences": int(cb["n"]), "min_cosine": float(cosines.min()) if cosines.size else None,
+                  "max_abs_err": float(np.abs(got - ref).max())}
         seqs = B * world
         line = {
             "metric": METRIC, "value": seqs * args.steps / (total_ms / 1e3), "unit": "sequences/s",
@@ -404,6 +413,7 @@ def run_ours(args):
                                        f"{cb['times'][0]:.2f} s"},
             "context": {"paper_p50_ms_batch32_seq128": {"RLX-Metal": 16.6, "PyTorch-MPS": 26.74,
                                                         "hardware": "one Apple Silicon host (paper Section 8.1)"}},
+            "parity_on_sample": parity,
             "device_status": status,
             "wall_s_timed_region": wall1 - wall0,
             "gpu_busy_s": gpu_busy_s,
