@@ -38,6 +38,46 @@ __device__ __forceinline__ void ln_normalise_store(float (&v)[NV * 4], const flo
     }
 }
 
+// gamma / beta of this lane's columns, loaded once and kept in registers by kernels that normalise
+// several rows per warp
+template <int NV>
+struct LnAffine {
+    float4 g[NV], b[NV];
+    __device__ __forceinline__ void load(const float* __restrict__ gamma, const float* __restrict__ beta, int lane) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            g[i] = __ldg(reinterpret_cast<const float4*>(gamma + (i * 32 + lane) * 4));
+            b[i] = __ldg(reinterpret_cast<const float4*>(beta + (i * 32 + lane) * 4));
+        }
+    }
+};
+
+template <int NV>
+__device__ __forceinline__ void ln_normalise_store(float (&v)[NV * 4], const LnAffine<NV>& af, float eps, int lane,
+                                                   __nv_bfloat16* __restrict__ out_row) {
+    constexpr int H = NV * 128;
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV * 4; ++i) s += v[i];
+    const float mean = warp_sum(s) / (float)H;  // true division: a constant row has exactly zero deviation
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV * 4; ++i) {
+        v[i] -= mean;
+        q += v[i] * v[i];
+    }
+    const float var = warp_sum(q) / (float)H;
+    const float rstd = 1.0f / sqrtf(var + eps);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int col = (i * 32 + lane) * 4;
+        uint2 o;
+        o.x = pack_bf16(v[i * 4 + 0] * rstd * af.g[i].x + af.b[i].x, v[i * 4 + 1] * rstd * af.g[i].y + af.b[i].y);
+        o.y = pack_bf16(v[i * 4 + 2] * rstd * af.g[i].z + af.b[i].z, v[i * 4 + 3] * rstd * af.g[i].w + af.b[i].w);
+        *reinterpret_cast<uint2*>(out_row + col) = o;
+    }
+}
+
 // Sequence packing.  Valid tokens (mask != 0) are compacted so that sequence b owns the packed rows
 // seq_start[b] .. seq_start[b] + seq_len[b]; every later kernel then works on sum(len) rows instead
 // of B*S.  Exact for any 0/1 mask: positions are taken from the original index s, attention only
@@ -260,6 +300,8 @@ layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ 
 #pragma unroll
         for (int i = 0; i < NV; ++i) raw[r][i] = __ldg(reinterpret_cast<const uint2*>(row + (i * 32 + lane) * 4));
     }
+    LnAffine<NV> af;
+    if (kLnRowsPerWarp > 1) af.load(gamma, beta, lane);   // once per warp instead of once per row
 #pragma unroll
     for (int r = 0; r < kLnRowsPerWarp; ++r) {
         if (t0 + r >= rows) break;
@@ -271,7 +313,8 @@ layernorm_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ 
             v[i * 4 + 2] = bf16lo(raw[r][i].y);
             v[i * 4 + 3] = bf16hi(raw[r][i].y);
         }
-        ln_normalise_store<NV>(v, gamma, beta, eps, lane, out + (size_t)(t0 + r) * H);
+        if (kLnRowsPerWarp > 1) ln_normalise_store<NV>(v, af, eps, lane, out + (size_t)(t0 + r) * H);
+        else ln_normalise_store<NV>(v, gamma, beta, eps, lane, out + (size_t)(t0 + r) * H);
     }
 }
 
