@@ -71,8 +71,10 @@ typedef enum {
                                    normalisation per row in its epilogue from partial row statistics written by
                                    the producing GEMM; the residual adds and the pooling normalise on the fly.
                                    5 kernels per layer instead of 7; needs a larger workspace (see
-                                   rlx_encoder_workspace_bytes).  Ignored with RLX_FLAG_GEMM_SIMT; takes
-                                   precedence over RLX_FLAG_FUSED_LN / RLX_FLAG_CLUSTER_LN */
+                                   rlx_encoder_workspace_bytes).  Ignored with RLX_FLAG_GEMM_SIMT, when hidden is
+                                   not a multiple of 32 or max_seq exceeds 512; takes precedence over
+                                   RLX_FLAG_FUSED_LN / RLX_FLAG_CLUSTER_LN.  Pays for small batches (launch-bound
+                                   forwards); for large ones the separate LayerNorm kernels are faster */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */
