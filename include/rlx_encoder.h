@@ -226,6 +226,17 @@ rlx_status_t rlx_encoder_last_device_status(rlx_encoder_t *encoder, void *worksp
 int32_t rlx_encoder_kernels_per_forward(const rlx_encoder_t *encoder, int32_t batch, int32_t seq);
 
 /*
+ * Self-test of the device-side failure path (no fault is provoked): a one-thread kernel waits on a
+ * barrier that nothing signals, with the same bounded wait the GEMM and attention pipelines use but a
+ * budget of `budget_us` microseconds (1 .. 100000).  When the budget runs out the wait gives up and
+ * the kernel sets RLX_DEVSTAT_TIMEOUT in *status_word (device int32, e.g. the first word of a
+ * workspace), which rlx_encoder_last_device_status then reports as RLX_ERR_DEVICE_TIMEOUT and clears;
+ * the context stays usable.  waited_ns (device uint64, may be NULL) receives the time spent waiting.
+ */
+rlx_status_t rlx_selftest_bounded_wait(uint32_t budget_us, int32_t *status_word, uint64_t *waited_ns,
+                                       void *cuda_stream);
+
+/*
  * Per-kernel device times of the most recent forward of an encoder created with
  * RLX_FLAG_KERNEL_EVENTS (the paper's runtime exposes per-operator reports, Section 4; this is
  * the timing analogue).  Waits for that forward to finish, then writes `count` =

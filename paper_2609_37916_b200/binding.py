@@ -37,7 +37,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
 
 
@@ -334,6 +334,12 @@ def qk_rope_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, rope, st
                                     hkv, W // (num_heads + 2 * hkv), _ptr(cos), _ptr(sin), _stream(stream)),
            "rlx_qk_rope_bf16")
     return qkv
+
+
+def selftest_bounded_wait(budget_us: int, status_word: torch.Tensor, waited_ns: Optional[torch.Tensor] = None, stream=None):
+    """Runs the bounded-wait self-test kernel; status_word: int32 device tensor, waited_ns: int64 device tensor."""
+    _check(_load().rlx_selftest_bounded_wait(C.c_uint32(budget_us), _ptr(status_word), _ptr(waited_ns), _stream(stream)),
+           "rlx_selftest_bounded_wait")
 
 
 def minifloat(ebits: int, mbits: int, special: int = 0, packed4: bool = False) -> int:

@@ -93,20 +93,42 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the budget ran out or another role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t budget_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0xff) == 0) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitBudgetNs) {
+            if (global_timer_ns() - t0 > budget_ns) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetNs);
+}
+
+// Self-test of the bounded wait: one thread waits, with a caller-chosen budget, on an mbarrier that
+// nothing ever arrives on; the wait must give up, raise the abort flag and leave the time-out bit in the
+// status word exactly as the GEMM / attention pipelines do when a wait of theirs expires.
+__global__ void bounded_wait_selftest_kernel(int32_t* status, unsigned long long budget_ns, unsigned long long* waited_ns) {
+    __shared__ __align__(8) unsigned long long bar_storage;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        const uint32_t bar = smem_u32(&bar_storage);
+        abort_flag = 0;
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint64_t t0 = global_timer_ns();
+        const bool ok = mbar_wait_budget(bar, 0, &abort_flag, budget_ns);
+        const uint64_t t1 = global_timer_ns();
+        if (waited_ns) *waited_ns = t1 - t0;
+        if (!ok && abort_flag) atomicOr(status, RLX_DEVSTAT_TIMEOUT_BIT);
+    }
 }
 // ---- cluster helpers (CG = 2) ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {

@@ -1279,6 +1279,14 @@ rlx_status_t rlx_scaled_matmul_bf16(const void* A, const void* codes, const void
                        false, status, static_cast<cudaStream_t>(stream), nullptr, 0);
 }
 
+rlx_status_t rlx_selftest_bounded_wait(uint32_t budget_us, int32_t* status_word, uint64_t* waited_ns, void* stream) {
+    if (!status_word || budget_us == 0 || budget_us > 100000u) return RLX_ERR_INVALID_ARG;   // at most 100 ms
+    rlx::tc::bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        status_word, (unsigned long long)budget_us * 1000ull, reinterpret_cast<unsigned long long*>(waited_ns));
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
 void rlx_debug_set_attn_trace(void* p) { g_attn_dbg = static_cast<unsigned long long*>(p); }
 
 rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,
