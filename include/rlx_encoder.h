@@ -124,7 +124,8 @@ typedef struct {
  * Host only: validates the shape and precomputes the workspace layout.
  * Returns RLX_ERR_INVALID_ARG for null/negative fields or a wrong struct_size,
  * RLX_ERR_UNSUPPORTED when H % 128 != 0, H > 1024, H % h != 0, head_dim not in
- * {32, 64}, F % 64 != 0, or max_seq > max_pos.
+ * {32, 64}, F % 64 != 0, max_seq > max_pos, max_seq > 512 (the attention kernel's
+ * per-sequence key table) or max_batch * max_seq > 2^30.
  */
 rlx_status_t rlx_encoder_create(const rlx_encoder_config_t *config, rlx_encoder_t **out_encoder);
 
@@ -197,7 +198,8 @@ rlx_status_t rlx_encoder_forward_host(rlx_encoder_t *encoder, const int32_t *tok
  * RLX_ERR_WORKSPACE before anything is launched (at H=384, F=1536 the limit covers about 1,800
  * tokens, e.g. batch 14 x seq 128).  The call makes no cudaMalloc/cudaFree and uses no
  * allocating library routine: kernels are launched directly (no CUDA graph is built), and
- * RLX_FLAG_KERNEL_EVENTS is ignored.
+ * RLX_FLAG_KERNEL_EVENTS is ignored (no event is recorded, and the per-kernel times of an earlier
+ * rlx_encoder_forward on the same object stay as they were).
  *
  * token_ids, attention_mask, weights, out: exactly as for rlx_encoder_forward (dev pointers).
  * device_status: optional dev int32; receives this call's RLX_DEVSTAT_* bits (0 = clean).
@@ -293,7 +295,11 @@ typedef enum {
                                     grouping chosen from the problem size (the product path)      */
     RLX_GEMM_SIMT = 1,           /* plain CUDA-core tiles (bring-up / cross-check)                 */
     RLX_GEMM_TCGEN05_PAIR = 2,   /* force the CTA-pair variant (cta_group::2, 256-row tiles); N % 128 == 0 */
-    RLX_GEMM_TCGEN05_SINGLE = 3  /* force the one-CTA-per-tile variant                             */
+    RLX_GEMM_TCGEN05_SINGLE = 3, /* force the one-CTA-per-tile variant                             */
+    RLX_GEMM_TCGEN05_RESIDENT = 4 /* force the CTA-pair variant that keeps its 256 rows of A resident in
+                                    shared memory and streams only W (K <= 384, N % 128 == 0 or
+                                    N % 192 == 0); RLX_GEMM_TCGEN05 picks it by itself for such K once
+                                    there are enough 256-row blocks for every CTA pair               */
 } rlx_gemm_impl_t;
 
 /*

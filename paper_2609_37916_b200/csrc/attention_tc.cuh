@@ -91,7 +91,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t* __restrict__ seq_start,
                     const int32_t* __restrict__ seq_len, __nv_bfloat16* __restrict__ ctx, int H,
-                    float scale_log2e, int max_blocks, int32_t* status, unsigned long long* dbg) {
+                    float scale_log2e, int max_blocks, int32_t* status) {
     using SM = Smem<D>;
     pdl_launch_dependents();
     pdl_wait();
@@ -114,10 +114,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool trace = dbg != nullptr && blockIdx.x == 0 && blockIdx.y == 1 && blockIdx.z == 0 && threadIdx.x == 64;
-    int ti = 0;
-    auto stamp = [&]() { if (trace) dbg[ti++] = global_timer_ns(); };
-    stamp();
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
         for (int i = 0; i < kMaxBlocks; ++i) { mbar_init(k_full + 8 * i, 1); mbar_init(v_full + 8 * i, 1); }
@@ -137,7 +133,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    stamp();   // 1: setup done
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA: Q, then K_j and V_j
@@ -223,7 +218,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
             if (!(ok = mbar_wait(s_full, n_sfull & 1, abort_flag))) break;
             ++n_sfull;
             tc_fence_after();
-            stamp();   // S ready (pass 1)
             const int keys = min(kBlockN, len - j * kBlockN);
             for (int c0 = 0; c0 < keys; c0 += 32) {
                 uint32_t r[32];
@@ -244,7 +238,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
                 if (lane == 0) mbar_arrive(s_free);
             }
         }
-        stamp();   // pass 1 done
         const float m_scaled = m_row * scale_log2e;   // len >= 1, so m_row is finite
         float l_row = 0.f;
         // ---- pass 2: probabilities -> TMEM (bf16), row sum ----
@@ -289,13 +282,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            stamp();   // P written
             if (lane == 0) mbar_arrive(p_full);
         }
         // ---- O / sum -> bf16 -> global ----
         if (ok && (ok = mbar_wait(pv_done, n_pvdone & 1, abort_flag))) {
             tc_fence_after();
-            stamp();   // O ready
             const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
             __nv_bfloat16* orow = ctx + (size_t)(row0 + qrow) * H + head * D;
 #pragma unroll
@@ -317,8 +308,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const int32_t*
             }
         }
     }
-
-    stamp();   // stored
     // ---------------------------------------------------------------- teardown
     if (*abort_flag) {
         if (threadIdx.x == 0 && status) atomicOr(status, RLX_DEVSTAT_TIMEOUT_BIT);

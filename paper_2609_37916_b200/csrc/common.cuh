@@ -9,8 +9,6 @@
 
 namespace rlx {
 
-constexpr int kNumSMs = 148;  // B200: 2 dies x 74 SMs
-
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -5,24 +5,23 @@
 namespace rlx {
 
 // Exact-form (erf) GELU, gelu(x) = x * Phi(x), evaluated without erff:
-//   u = min(|x|, 5.5);  Phi(-u) = 2^r(u) with r a degree-7 polynomial fitted to log2 Phi(-u)
-//   (coefficients from fit_gelu_poly.py next to this file);  Phi(x) = t for x < 0, 1 - t otherwise.
-// fp32 Horner + one ex2: |error| <= 7e-7 absolute and <= 5e-6 relative against the erf form, far
-// below the bf16 rounding of the stored result.  12 issue slots instead of ~30 for erff.
+//   u = min(|x|, 5.5);  Phi(-u) = 2^r(u) with r a degree-4 polynomial fitted to log2 Phi(-u), the fit
+//   weighted by the sensitivity of the result to r (coefficients from fit_gelu_poly.py next to this
+//   file);  gelu(x) = max(x, 0) - u * 2^r(u).
+// The epilogue of a K = 384 GEMM is bound by the FP32 pipe (every output gets a handful of FP32
+// operations against 384 tensor-core MACs), so every operation counts: 8 FP32-pipe operations and one
+// ex2 per value.  |error| <= 6.2e-6 absolute against the erf form, far below the bf16 rounding of the
+// stored result.
 __device__ __forceinline__ float gelu_erf(float x) {
     const float u = fminf(fabsf(x), 5.5f);
-    float r = -1.921234571e-06f;
-    r = fmaf(r, u, 6.328849850e-05f);
-    r = fmaf(r, u, -9.434208623e-04f);
-    r = fmaf(r, u, 8.556271903e-03f);
-    r = fmaf(r, u, -5.405228212e-02f);
-    r = fmaf(r, u, -4.583817720e-01f);
-    r = fmaf(r, u, -1.151278377e+00f);
-    r = fmaf(r, u, -9.999938607e-01f);
+    float r = 3.866270650e-03f;
+    r = fmaf(r, u, -4.407931119e-02f);
+    r = fmaf(r, u, -4.680147469e-01f);
+    r = fmaf(r, u, -1.147372365e+00f);
+    r = fmaf(r, u, -1.000479579e+00f);
     float t;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(r));
-    const float phi = x < 0.f ? t : 1.0f - t;
-    return x * phi;
+    return fmaf(-u, t, fmaxf(x, 0.f));
 }
 
 // The same function on two values at once with Blackwell's packed fp32 arithmetic (fma/add/mul
@@ -52,28 +51,20 @@ __device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
     return d;
 }
 __device__ __forceinline__ void gelu_erf_x2(float& x0, float& x1) {
-    const float u0 = fminf(fabsf(x0), 5.5f), u1 = fminf(fabsf(x1), 5.5f);
-    const uint64_t u = pack_f32x2(u0, u1);
-    uint64_t r = pack_f32x2(-1.921234571e-06f, -1.921234571e-06f);
-    r = fma_f32x2(r, u, pack_f32x2(6.328849850e-05f, 6.328849850e-05f));
-    r = fma_f32x2(r, u, pack_f32x2(-9.434208623e-04f, -9.434208623e-04f));
-    r = fma_f32x2(r, u, pack_f32x2(8.556271903e-03f, 8.556271903e-03f));
-    r = fma_f32x2(r, u, pack_f32x2(-5.405228212e-02f, -5.405228212e-02f));
-    r = fma_f32x2(r, u, pack_f32x2(-4.583817720e-01f, -4.583817720e-01f));
-    r = fma_f32x2(r, u, pack_f32x2(-1.151278377e+00f, -1.151278377e+00f));
-    r = fma_f32x2(r, u, pack_f32x2(-9.999938607e-01f, -9.999938607e-01f));
+    // the polynomial runs on n = -u (odd coefficients change sign), so that the last step is the one
+    // fused operation  max(x, 0) + n * t
+    const float n0 = fmaxf(-fabsf(x0), -5.5f), n1 = fmaxf(-fabsf(x1), -5.5f);
+    const uint64_t n = pack_f32x2(n0, n1);
+    uint64_t r = pack_f32x2(3.866270650e-03f, 3.866270650e-03f);
+    r = fma_f32x2(r, n, pack_f32x2(4.407931119e-02f, 4.407931119e-02f));
+    r = fma_f32x2(r, n, pack_f32x2(-4.680147469e-01f, -4.680147469e-01f));
+    r = fma_f32x2(r, n, pack_f32x2(1.147372365e+00f, 1.147372365e+00f));
+    r = fma_f32x2(r, n, pack_f32x2(-1.000479579e+00f, -1.000479579e+00f));
     float r0, r1, t0, t1;
     unpack_f32x2(r, r0, r1);
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(r0));
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(r1));
-    // h = 0.5 - t >= 0; give it the sign of x; phi = 0.5 + h
-    const uint64_t h = fma_f32x2(pack_f32x2(t0, t1), pack_f32x2(-1.0f, -1.0f), pack_f32x2(0.5f, 0.5f));
-    float h0, h1;
-    unpack_f32x2(h, h0, h1);
-    h0 = __uint_as_float(__float_as_uint(h0) | (__float_as_uint(x0) & 0x80000000u));
-    h1 = __uint_as_float(__float_as_uint(h1) | (__float_as_uint(x1) & 0x80000000u));
-    const uint64_t phi = add_f32x2(pack_f32x2(h0, h1), pack_f32x2(0.5f, 0.5f));
-    unpack_f32x2(mul_f32x2(pack_f32x2(x0, x1), phi), x0, x1);
+    unpack_f32x2(fma_f32x2(n, pack_f32x2(t0, t1), pack_f32x2(fmaxf(x0, 0.f), fmaxf(x1, 0.f))), x0, x1);
 }
 
 }  // namespace rlx

@@ -2,45 +2,52 @@
 
 gelu(x) = x * Phi(x).  With u = min(|x|, U):  Phi(-u) = 2^r(u),  r(u) = log2 Phi(-u), which is
 smooth and nearly quadratic, so a low-degree polynomial fits it well.  The kernel evaluates r by
-Horner in fp32, takes one ex2, and uses Phi(x) = t for x < 0 and 1 - t for x >= 0.
+Horner in fp32, takes one ex2 and forms  gelu(x) = max(x, 0) - u * 2^r(u)  (for x >= 0 this is
+x - x Phi(-x) = x Phi(x); for x < 0 it is x Phi(x) directly).
 
     python fit_gelu_poly.py            # prints the coefficients and the measured error
 
-Fit: Chebyshev interpolation (near-minimax) of degree DEG on [0, U], converted to the power basis.
-Error of the resulting fp32 evaluation against the exact erf form: |gelu err| <= 7e-7 absolute,
-<= 5e-6 relative, three orders of magnitude below the bf16 rounding of the stored result.
+Fit: weighted least squares on [0, U], the weight being the sensitivity of the RESULT to an error in
+r, d gelu / d r = u 2^r ln 2 (large around |x| ~ 1, tiny in the tails where Phi(-u) vanishes), with
+Lawson re-weighting towards the minimax solution.  The epilogue is bound by the FP32 pipe (every
+output of a K = 384 GEMM gets ~8 FP32 operations against 384 tensor-core MACs), so the degree is the
+lowest whose error stays below the bf16 rounding of the stored result by a wide margin: degree 4
+gives |gelu error| <= 6.2e-6 absolute in fp32 (a uniform, unweighted fit of the same degree: 2.8e-4).
 """
 import numpy as np
-from numpy.polynomial import chebyshev as C
+from numpy.polynomial import polynomial as P
 from scipy.special import log_ndtr, ndtr
 
-U, DEG = 5.5, 7
+U, DEG = 5.5, 4
 
 
-def fit():
-    n = 400
-    x = np.cos(np.pi * (np.arange(n) + 0.5) / n)
-    u = (x + 1) * U / 2
-    c = C.chebfit(x, log_ndtr(-u) / np.log(2), DEG)
-    px = np.poly1d(C.cheb2poly(c)[::-1])
-    return px(np.poly1d([2 / U, -1])).coeffs[::-1].astype(np.float32)   # ascending powers of u
+def fit(deg=DEG, iters=60):
+    u = np.linspace(0, U, 20001)
+    target = log_ndtr(-u) / np.log(2)
+    sens = u * np.exp2(target) * np.log(2)
+    w, lw = np.maximum(sens, 1e-6), np.ones_like(u)
+    for _ in range(iters):
+        c = P.polyfit(u, target, deg, w=w * lw)
+        e = np.abs(P.polyval(u, c) - target) * sens
+        lw = lw * (1 + 4 * e / e.max())
+        lw /= lw.mean()
+    return c.astype(np.float32)   # ascending powers of u
 
 
 def check(coef):
-    u = np.linspace(0, 8, 400001).astype(np.float32)
-    uc = np.minimum(u, np.float32(U))
-    acc = np.full_like(uc, coef[-1])
+    x = np.linspace(-8, 8, 1600001).astype(np.float32)
+    u = np.minimum(np.abs(x), np.float32(U))
+    acc = np.full_like(u, coef[-1])
     for cf in coef[-2::-1]:
-        acc = (acc * uc + cf).astype(np.float32)
+        acc = (acc * u + cf).astype(np.float32)
     t = np.exp2(acc.astype(np.float64))
-    ref = ndtr(-u.astype(np.float64))
-    e_neg, e_pos = np.abs(-u * t + u * ref), np.abs(u * (1 - t) - u * (1 - ref))
-    rel = e_neg[(u > 1e-3) & (u < 5)] / (u * ref)[(u > 1e-3) & (u < 5)]
-    return max(e_neg.max(), e_pos.max()), rel.max()
+    got = np.maximum(x, 0).astype(np.float64) - u.astype(np.float64) * t
+    ref = x.astype(np.float64) * ndtr(x.astype(np.float64))
+    return np.abs(got - ref).max()
 
 
 if __name__ == "__main__":
     coef = fit()
     for i, c in enumerate(coef):
         print(f"c{i} = {float(c):.9e}f")
-    print("max abs err, max rel err (x in [-5,0)):", check(coef))
+    print("max abs err of gelu:", check(coef))

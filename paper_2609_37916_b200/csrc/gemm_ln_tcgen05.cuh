@@ -67,7 +67,6 @@ struct Params {
     int M, K;
     int32_t* status;
     const int32_t* m_ptr;            // optional device row count
-    unsigned long long* trace;       // experiments only: phase timestamps of CTA 0, epilogue warp 0
 };
 
 template <int NH>
@@ -87,6 +86,7 @@ gemm_ln_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::STAGES * C::STAGE_BYTES + kStaging + kRedBytes +
                                                       16 * C::STAGES + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* pair_ok = reinterpret_cast<volatile int*>(tmem_slot + 2);   // [kEpiWarps]: this tile's wait succeeded
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
@@ -176,11 +176,7 @@ gemm_ln_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         float* red_sq = red + 256;
         int it = 0;
         bool ok = true;
-        const bool tr = p.trace != nullptr && blockIdx.x == 0 && threadIdx.x == 64;
-        int ti = 0;
-        auto stamp = [&]() { if (tr && ti < 30) p.trace[ti++] = global_timer_ns(); };
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
-            stamp();
             const int m = tile * BLOCK_M + row;
             const bool row_ok = m < M;
             const int n0 = hf * NH;
@@ -189,9 +185,14 @@ gemm_ln_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             uint4 rq[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) rq[i] = __ldg(reinterpret_cast<const uint4*>(rrow) + i);
-            if (!mbar_wait(tfull_bar, it & 1, abort_flag)) { ok = false; break; }
+            // The two warps that share a row quadrant meet at named barriers below, so they must also
+            // give up together: each publishes whether its (bounded) wait succeeded and both leave if
+            // either one did not -- a warp that left alone would strand its partner at the barrier.
+            const bool got = mbar_wait(tfull_bar, it & 1, abort_flag);
+            if (lane == 0) pair_ok[ew] = got ? 1 : 0;
+            pair_barrier(1 + quad);
+            if (!(pair_ok[ew] & pair_ok[ew ^ 4])) { ok = false; break; }
             tc_fence_after();
-            stamp();
             const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + n0;
             uint32_t r[2][32];
             // ---- sweep 1: v = acc + bias + residual -> TMEM, partial row sum ----
@@ -229,7 +230,6 @@ gemm_ln_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 }
             }
             tmem_st_wait();
-            stamp();
             red_sum[row * 2 + hf] = sum;
             pair_barrier(1 + quad);
             const float mean = (red_sum[row * 2] + red_sum[row * 2 + 1]) / (float)N;   // true division: constant rows stay exact
@@ -247,7 +247,6 @@ gemm_ln_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 }
             }
             red_sq[row * 2 + hf] = sq;
-            stamp();
             pair_barrier(1 + quad);
             const float var = (red_sq[row * 2] + red_sq[row * 2 + 1]) / (float)N;
             const float rstd = 1.0f / sqrtf(var + p.eps);

@@ -2,19 +2,18 @@
 //
 // Structure (one persistent CTA per SM, 320 to 576 threads):
 //   warp 0      TMA producer: streams 128x64 A tiles and BLOCK_N x 64 W tiles (128-byte swizzle)
-//               through a STAGES-deep shared-memory ring guarded by full/empty mbarriers
+//               through a STAGES-deep shared-memory ring guarded by full/empty mbarriers; a stage
+//               holds one or two 64-wide k-blocks behind one barrier pair
 //   warp 1      allocates tensor memory; one elected lane issues tcgen05.mma (M=128, N=BLOCK_N,
 //               K=16 per instruction) into one of two fp32 accumulator buffers in TMEM and
 //               commits stage releases / accumulator-ready signals to mbarriers
+//               (both warps run their loops warp-uniformly; elect.sync picks the issuing lane)
 //   warps 2..   epilogue (8 to 16 warps): each warp owns one TMEM lane quadrant (32 rows) and one 64-column
-//               slab of the tile; per 32-column chunk it tcgen05.ld's the accumulator (the next chunk's load
-//               is in flight while this one is processed), adds bias, applies GELU or adds the
-//               residual in fp32, rounds to bf16, transposes the chunk through a swizzled
-//               shared-memory buffer and stores it with 16-byte stores that cover whole 64-byte row
-//               segments (a TMA store per chunk was tried: waiting for it to drain its staging buffer
-//               stalled the warp for about a microsecond per chunk).
-//               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop;
-//               a warp releases its accumulator as soon as its last tcgen05.ld has landed.
+//               slab of the tile; it tcgen05.ld's its slab into registers and hands the accumulator back
+//               at once, then per 32-column chunk adds bias, applies GELU or adds the residual in fp32,
+//               rounds to bf16, writes the chunk into its swizzled staging buffer and issues a TMA store
+//               for it (which drains while the next chunk is computed).
+//               The second accumulator buffer lets tile i's epilogue overlap tile i+1's main loop.
 // Epilogue modes (template EPI): 0 bias; 1 bias + GELU; 2 bias + residual; and the LayerNorm-folding
 // modes that let a post-LN encoder drop its LayerNorm kernels:
 //   3 / 4  the A operand is a RAW pre-LayerNorm activation y and W was pre-multiplied by gamma:
@@ -51,24 +50,36 @@ struct Cfg {
     static constexpr int A_BYTES = BLOCK_M * BLOCK_K * 2;
     static constexpr int B_ROWS = BLOCK_N / CG;                  // W rows this CTA loads per k-block
     static constexpr int B_BYTES = B_ROWS * BLOCK_K * 2;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    // epilogue: EPI_SPLIT warps share each 32-row TMEM quadrant, each taking a 64-column slab (32 for
-    // the narrowest tile); many short per-warp chains hide the TMEM / memory latencies of the epilogue
-    static constexpr int EPI_SPLIT = BLOCK_N >= 192 ? BLOCK_N / 64 : 2;
+    static constexpr int KB_BYTES = A_BYTES + B_BYTES;           // operands of one 64-wide k-block
+    // epilogue: EPI_SPLIT warps share each 32-row TMEM quadrant, each taking a 64-column slab (32 for the
+    // narrowest tile): at most 64 accumulator registers per thread leave the compiler room to interleave
+    // many independent GELU evaluations (with 128 of them live the special-function and FP32 pipes idled
+    // on dependent chains), and four warps per scheduler hide what is left.  One staging buffer per warp:
+    // the TMA store of a chunk drains while the next chunk is being computed.
+    static constexpr int EPI_SPLIT = BLOCK_N >= 128 ? BLOCK_N / 64 : 2;
     static constexpr int EPI_WARPS = 4 * EPI_SPLIT;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static constexpr int SLAB = BLOCK_N / EPI_SPLIT;
-    static constexpr int STAGING_BYTES = EPI_WARPS * kStageBufBytes;   // one transpose buffer per epilogue warp
-    static constexpr int RING_BUDGET = 222 * 1024 - STAGING_BYTES;
+    static constexpr int STAGING_BYTES = EPI_WARPS * kStageBufBytes;
+    static constexpr int BAR_BYTES = 256;
+    static constexpr int RING_BUDGET = 227 * 1024 - 1024 - BAR_BYTES - STAGING_BYTES;
+    // A stage holds KPS k-blocks behind ONE full / empty barrier pair.  A barrier wait costs the issuing
+    // thread a couple of hundred cycles whether or not the barrier is already complete (measured: 4 MMAs
+    // + wait + commit take ~430 cycles of the thread, 8 MMAs ~620), so with one k-block per wait the
+    // single MMA thread, not the tensor pipe, paces every tile narrower than 256 columns.  Two k-blocks
+    // per stage whenever three such stages still fit.
+    static constexpr int KPS = (3 * 2 * KB_BYTES <= RING_BUDGET) ? 2 : 1;
+    static constexpr int STAGE_BYTES = KPS * KB_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
     static constexpr int TMEM_COLS = (2 * BLOCK_N <= 32) ? 32 : (2 * BLOCK_N <= 64) ? 64 : (2 * BLOCK_N <= 128) ? 128
                                      : (2 * BLOCK_N <= 256) ? 256 : 512;
-    static constexpr int BAR_BYTES = 256;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + BAR_BYTES + 1024;  // +1024: manual alignment
     static_assert(BLOCK_N % 16 == 0 && BLOCK_N >= 16 && BLOCK_N <= 256, "UMMA N for M=128 / M=256");
     static_assert(CG == 1 || CG == 2, "cta_group");
     static_assert(B_BYTES % 1024 == 0, "stage tiles must stay 1024-byte aligned");
     static_assert(STAGES >= 2, "ring too shallow");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
+    static_assert(16 * STAGES + 48 <= BAR_BYTES, "barrier block");
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -111,6 +122,11 @@ __device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetNs);
 }
+// The same wait executed by all 32 lanes of a converged warp, with one outcome for the whole warp
+// (a lane that gave up takes the others with it), so that the warp stays converged afterwards.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetNs)) != 0;
+}
 
 // Self-test of the bounded wait: one thread waits, with a caller-chosen budget, on an mbarrier that
 // nothing ever arrives on; the wait must give up, raise the abort flag and leave the time-out bit in the
@@ -149,6 +165,16 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrivals that publish no memory writes of the arriving thread (handing a TMEM accumulator back after
+// tcgen05.wait::ld: the data is in registers, the tcgen05 fence orders the tensor-memory reads).  A
+// release-arrive would first wait for every earlier global store of the thread to become visible at
+// the barrier's scope -- at cluster scope that held the accumulator for thousands of cycles.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
@@ -173,6 +199,18 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
+// Global accesses of the epilogue with L1 policies: the streamed output rows must not push the few
+// lines every warp re-reads (bias, gamma, beta) out of the small L1 that is left next to ~220 KB of
+// shared memory.  (Residual rows keep the default policy: a thread reads its 64-byte piece with four
+// 16-byte loads, and only L1 allocation keeps the last three from going back to L2.)
+__device__ __forceinline__ void st_global_stream_v4(void* ptr, uint4 v) {
+    asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ float4 ld_global_keep_f4(const float* ptr) {
+    float4 v;   // not volatile: a read of read-only data, free to be scheduled early and together with its neighbours
+    asm("ld.global.nc.L1::evict_last.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr));
+    return v;
+}
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
@@ -181,6 +219,11 @@ __device__ __forceinline__ void tma_load_2d_cg2(uint32_t smem_dst, const CUtenso
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(bar_cluster) : "memory");
+}
+// L2 prefetch of one box of a tiled tensor (no shared-memory destination, no barrier)
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tmap, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
@@ -208,6 +251,21 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// True in exactly one lane of a fully converged warp.  The producer and MMA warps run their loops with
+// all 32 lanes (warp-uniform control flow and addresses) and let the elected lane issue the TMA /
+// tcgen05 instructions: measured on the MMA loop, a loop executed by a single lane under a divergent
+// branch costs the issuing thread ~110-120 cycles per tcgen05.mma, the warp-uniform form ~80.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred P;\n"
+        "elect.sync _|P, 0xFFFFFFFF;\n"
+        "selp.u32 %0, 1, 0, P;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
 template <int CG>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     if constexpr (CG == 1)
@@ -275,7 +333,10 @@ struct Params {
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
     const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
-    int debug;                       // experiments only: bit 0 = epilogue releases the accumulator without reading it
+#ifdef RLX_EXPERIMENTS
+    int debug;                       // ablation switches of the experiments build (kDbg* bits)
+    unsigned long long* trace;       // experiments build: 64 timestamp slots per CTA (or null)
+#endif
     // LayerNorm folding (EPI 3..6); unused fields stay null
     const float* cvec;               // [N] EPI 3/4: column sums of the gamma-scaled weights
     const float* dvec;               // [N] EPI 3/4: beta . W + bias
@@ -312,9 +373,243 @@ __device__ __forceinline__ void row_stats_from_partials(const float2* __restrict
     rstd = 1.0f / sqrtf((m2 + 32.f * between) / (32.f * (float)P) + eps);
 }
 
+#ifdef RLX_EXPERIMENTS
+constexpr int kDbgNoEpilogue = 1;   // epilogue warps hand the accumulator back without reading it
+constexpr int kDbgNoStore = 2;      // everything but the global stores
+constexpr int kDbgNoMma = 4;        // the MMA thread only commits (operand feed alone)
+constexpr int kDbgNoLoad = 8;       // the producer only arrives (tensor pipe alone)
+#define RLX_DBG(p, bit) (((p).debug & (bit)) != 0)
+#define RLX_TRACE(p, slot) do { if ((p).trace) (p).trace[blockIdx.x * 64 + (slot)] = global_timer_ns(); } while (0)
+#define RLX_TRACE_CLK(p, slot) do { if ((p).trace) (p).trace[blockIdx.x * 64 + (slot)] = (unsigned long long)clock64(); } while (0)
+#define RLX_CLK_DECL(name) long long name = 0
+#define RLX_CLK_ADD(name, expr) do { const long long _c0 = clock64(); expr; name += clock64() - _c0; } while (0)
+#define RLX_TRACE_VAL(p, slot, v) do { if ((p).trace) (p).trace[blockIdx.x * 64 + (slot)] = (unsigned long long)(v); } while (0)
+#else
+#define RLX_DBG(p, bit) false
+#define RLX_TRACE(p, slot) do { } while (0)
+#define RLX_TRACE_CLK(p, slot) do { } while (0)
+#define RLX_CLK_DECL(name) do { } while (0)
+#define RLX_CLK_ADD(name, expr) do { expr; } while (0)
+#define RLX_TRACE_VAL(p, slot, v) do { } while (0)
+#endif
+
+// One epilogue warp's share of one output tile: 32 rows (a TMEM lane quadrant, thread = row) x NC
+// chunks of 32 columns.  prefetch() issues the loads that do not depend on the accumulator (residual
+// rows, LayerNorm row statistics) so that their latency hides behind the main loop; drain() reads the
+// warp's accumulator slab into registers, hands the buffer back to the MMA thread, then chunk by chunk
+// applies the epilogue in fp32, rounds to bf16, writes the chunk into the warp's swizzled staging
+// buffer (thread = row, 64 bytes) and lets one lane hand it to the TMA engine as a 32 x 32
+// box.  The load/store pipe of the SM is what the epilogue runs out of first (reading the accumulator
+// and the bias already costs 64 shared-pipe wavefronts per chunk), so the stores do not go through it:
+// TMA reads the staged tile itself and writes whole lines.  Rows at or beyond the matrix's row count
+// are clipped by the tensor map; rows between a smaller device-side row count (packed batches) and the
+// end of the last tile are written with values nobody reads.
+template <int EPI, int NC>
+struct EpilogueTile {
+    static constexpr bool kRes = EPI == 2 || EPI == 5 || EPI == 6;     // a residual tile is added
+    static constexpr bool kFold = EPI == 3 || EPI == 4;                // LayerNorm folded into this GEMM's input
+    static constexpr bool kStatsIn = kFold || EPI == 6;
+    static constexpr bool kStatsOut = EPI == 5 || EPI == 6;
+    uint4 res[kRes ? NC : 1][4];
+    float ln_a = 1.f, ln_b = 0.f;   // x_norm = x * ln_a + ln_b  (ln_a = rstd, ln_b = -rstd * mu)
+
+    // The bias values of a slab (one 128-byte line per chunk) are pulled into L1 a tile ahead of their
+    // use by every lane, so that no chunk starts with an L2 round trip.
+    static __device__ __forceinline__ void prefetch_bias(const Params& p, int n0) {
+        if ((threadIdx.x & 31) < NC) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.bias + n0 + (threadIdx.x & 31) * 32));
+    }
+
+    __device__ __forceinline__ void prefetch(const Params& p, int M, int m, int n0) {
+        if (kRes && m < M) {
+            const __nv_bfloat16* rpre = p.residual + (size_t)m * p.N + n0;
+#pragma unroll
+            for (int c = 0; c < NC; ++c)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) res[c][i] = __ldg(reinterpret_cast<const uint4*>(rpre + c * 32) + i);
+        }
+        if (kStatsIn && m < M) {
+            float mu, rstd;
+            row_stats_from_partials(p.stats_in + (size_t)m * p.stats_in_p, p.stats_in_p, p.ln_eps, mu, rstd);
+            ln_a = rstd;
+            ln_b = -rstd * mu;
+        }
+    }
+
+    template <int CG>
+    __device__ __forceinline__ void release(uint32_t tempty, uint32_t cta_rank, int lane) {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            if (CG == 1) mbar_arrive_relaxed(tempty);
+            else mbar_arrive_cluster_relaxed(map_to_cta(tempty, 0));   // the leader's barrier collects both CTAs' warps
+        }
+    }
+
+    template <int CG>
+    __device__ __forceinline__ void drain(const Params& p, const CUtensorMap* tmap_out, int M, int m_row0, int n0,
+                                          uint32_t taddr, uint32_t stg, int lane, uint32_t tempty, uint32_t cta_rank,
+                                          int trace_slot = -1) {
+        const int m = m_row0 + lane;
+        const bool row_ok = m < M;
+        const uint32_t row_off = lane * 64;                 // 64-byte rows in the staging chunk
+        const uint32_t swz = (uint32_t)((lane >> 1) & 3);   // 64-byte swizzle: 16-byte chunk index ^ (row/2 % 4)
+        const float* brow = p.bias + n0;
+        if (RLX_DBG(p, kDbgNoEpilogue)) {
+            release<CG>(tempty, cta_rank, lane);
+            return;
+        }
+        if (trace_slot >= 0) RLX_TRACE_CLK(p, 56 + (trace_slot - 40) / 8);
+        // Without a residual the warp's whole slab goes to registers first, so that the accumulator
+        // buffer returns to the MMA thread after one TMEM round trip, before any of the epilogue's memory
+        // traffic.  With a residual tile held in registers there is no room for that: chunks are read one
+        // ahead and the accumulator goes back once the last one has landed.
+        constexpr bool kAllFirst = !kRes;
+        uint32_t r[kAllFirst ? NC : 2][32];
+        if constexpr (kAllFirst) {
+#pragma unroll
+            for (int c = 0; c < NC; ++c) tmem_ld_32x32(taddr + c * 32, r[c]);
+            tmem_ld_wait();
+            release<CG>(tempty, cta_rank, lane);
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c);
+                uint4 q[4];
+                compute_chunk(p, r[c], n0 + c * 32, c, m, row_ok, brow + c * 32, q);
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c + 1);
+                store_chunk(p, tmap_out, q, n0 + c * 32, m_row0, stg, lane, row_off, swz);
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c + 3);
+            }
+        } else {
+            tmem_ld_32x32(taddr, r[0]);
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                tmem_ld_wait();
+                if (c + 1 < NC) tmem_ld_32x32(taddr + (c + 1) * 32, r[(c + 1) & 1]);
+                else release<CG>(tempty, cta_rank, lane);
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c);
+                uint4 q[4];
+                compute_chunk(p, r[c & 1], n0 + c * 32, c, m, row_ok, brow + c * 32, q);
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c + 1);
+                store_chunk(p, tmap_out, q, n0 + c * 32, m_row0, stg, lane, row_off, swz);
+                if (trace_slot >= 0 && c < 2) RLX_TRACE_CLK(p, trace_slot + 4 * c + 3);
+            }
+        }
+    }
+
+    // Epilogue arithmetic of one 32-column chunk of this thread's row: acc -> bf16 pairs (16 words).
+    __device__ __forceinline__ void compute_chunk(const Params& p, const uint32_t (&acc)[32], int ncol, int c, int m,
+                                                  bool row_ok, const float* bias32, uint4 (&q)[4]) {
+        float v[32];
+        if constexpr (kFold) {
+            const float* crow = p.cvec + ncol;
+            const float* drow = p.dvec + ncol;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 c4 = __ldg(reinterpret_cast<const float4*>(crow) + i);
+                const float4 d4 = __ldg(reinterpret_cast<const float4*>(drow) + i);
+                v[4 * i + 0] = fmaf(ln_a, __uint_as_float(acc[4 * i + 0]), fmaf(ln_b, c4.x, d4.x));
+                v[4 * i + 1] = fmaf(ln_a, __uint_as_float(acc[4 * i + 1]), fmaf(ln_b, c4.y, d4.y));
+                v[4 * i + 2] = fmaf(ln_a, __uint_as_float(acc[4 * i + 2]), fmaf(ln_b, c4.z, d4.z));
+                v[4 * i + 3] = fmaf(ln_a, __uint_as_float(acc[4 * i + 3]), fmaf(ln_b, c4.w, d4.w));
+            }
+        } else {
+            float4 b4[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) b4[i] = ld_global_keep_f4(bias32 + 4 * i);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4[i].x;
+                v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b4[i].y;
+                v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b4[i].z;
+                v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b4[i].w;
+            }
+        }
+        if (EPI == 1 || EPI == 4) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
+        }
+        if ((EPI == 2 || EPI == 5) && row_ok) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 w = res[kRes ? c : 0][i];
+                v[8 * i + 0] += bf16lo(w.x); v[8 * i + 1] += bf16hi(w.x);
+                v[8 * i + 2] += bf16lo(w.y); v[8 * i + 3] += bf16hi(w.y);
+                v[8 * i + 4] += bf16lo(w.z); v[8 * i + 5] += bf16hi(w.z);
+                v[8 * i + 6] += bf16lo(w.w); v[8 * i + 7] += bf16hi(w.w);
+            }
+        }
+        if (EPI == 6 && row_ok) {
+            // residual = LN(raw residual row): (x * rstd - rstd * mu) * gamma_n + beta_n
+            const float* grow = p.ln_gamma + ncol;
+            const float* berow = p.ln_beta + ncol;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 w = res[kRes ? c : 0][i];
+                const float4 g0 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i);
+                const float4 g1 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i + 1);
+                const float4 e0 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i);
+                const float4 e1 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i + 1);
+                v[8 * i + 0] += fmaf(fmaf(bf16lo(w.x), ln_a, ln_b), g0.x, e0.x);
+                v[8 * i + 1] += fmaf(fmaf(bf16hi(w.x), ln_a, ln_b), g0.y, e0.y);
+                v[8 * i + 2] += fmaf(fmaf(bf16lo(w.y), ln_a, ln_b), g0.z, e0.z);
+                v[8 * i + 3] += fmaf(fmaf(bf16hi(w.y), ln_a, ln_b), g0.w, e0.w);
+                v[8 * i + 4] += fmaf(fmaf(bf16lo(w.z), ln_a, ln_b), g1.x, e1.x);
+                v[8 * i + 5] += fmaf(fmaf(bf16hi(w.z), ln_a, ln_b), g1.y, e1.y);
+                v[8 * i + 6] += fmaf(fmaf(bf16lo(w.w), ln_a, ln_b), g1.z, e1.z);
+                v[8 * i + 7] += fmaf(fmaf(bf16hi(w.w), ln_a, ln_b), g1.w, e1.w);
+            }
+        }
+        if (kStatsOut && row_ok) {
+            // partial statistics of this row's 32 results (two-pass inside the chunk)
+            float sm = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sm += v[i];
+            const float mean = sm * (1.0f / 32.0f);
+            float m2 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float dl = v[i] - mean;
+                m2 = fmaf(dl, dl, m2);
+            }
+            p.stats_out[(size_t)m * (p.N / 32) + ncol / 32] = make_float2(mean, m2);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            q[i].x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
+            q[i].y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+            q[i].z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+            q[i].w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+        }
+    }
+
+    // Stage one chunk in the warp's buffer (the TMA store of the previous chunk, issued a chunk's worth
+    // of arithmetic ago, must be done reading it) and hand it to the TMA engine.
+    static __device__ __forceinline__ void store_chunk(const Params& p, const CUtensorMap* tmap_out, const uint4 (&q)[4],
+                                                       int ncol, int m_row0, uint32_t stg, int lane, uint32_t row_off,
+                                                       uint32_t swz) {
+        if (lane == 0) bulk_wait_read<0>();
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) st_shared_v4(stg + row_off + (((uint32_t)i ^ swz) << 4), q[i]);
+        fence_proxy_async();   // the writes above become visible to the TMA engine
+        __syncwarp();
+        if (lane == 0 && !RLX_DBG(p, kDbgNoStore)) {
+            tma_store_2d(tmap_out, ncol, m_row0, stg);
+            bulk_commit();
+        }
+    }
+
+    // Before the warp leaves the kernel: its TMA stores must have completed (they read shared memory).
+    static __device__ __forceinline__ void finish(int lane) {
+        if (lane == 0) bulk_wait<0>();
+        __syncwarp();
+    }
+};
+
 template <int BLOCK_N, int EPI, int CG>
 __global__ void __launch_bounds__((Cfg<BLOCK_N, CG>::THREADS), 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p) {
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_out, const Params p) {
     using C = Cfg<BLOCK_N, CG>;
     constexpr int TILE_M = BLOCK_M * CG;   // rows of one output tile (per CTA pair when CG = 2)
     extern __shared__ unsigned char smem_raw[];
@@ -334,6 +629,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CG == 2) ? cluster_ctarank() : 0u;   // rank 0 leads the pair
     pdl_launch_dependents();
+    if (threadIdx.x == 0) RLX_TRACE(p, 0);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::STAGES; ++i) {
@@ -348,6 +644,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         fence_barrier_init();
         prefetch_tmap(&tmap_a);
         prefetch_tmap(&tmap_b);
+        prefetch_tmap(&tmap_out);
     }
     if (warp == 1) {
         tmem_alloc<CG>(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -360,7 +657,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const uint32_t tmem_base = *tmem_slot;
 
     // everything above is independent of the previous kernel; its outputs are read only from here on
+    if (threadIdx.x == 0) RLX_TRACE(p, 1);
     pdl_wait();
+    if (threadIdx.x == 0) RLX_TRACE(p, 2);
     int M = p.M;
     if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));   // packed activations: only sum(len) rows exist
     const int n_tiles = p.N / BLOCK_N;
@@ -370,231 +669,131 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     const int tile0 = blockIdx.x / CG, tile_step = gridDim.x / CG;   // both CTAs of a pair walk the same tiles
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // ------------------------------------------------------------ TMA producer (whole warp, one lane issues)
+        {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = tile0; tile < num_tiles && ok; tile += tile_step) {
                 const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                    const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-                    if constexpr (CG == 1) {
-                        mbar_expect_tx(full_bar + 8 * stage, C::STAGE_BYTES);
-                        tma_load_2d(sa, &tmap_a, kb * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
-                        tma_load_2d(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
-                    } else {
-                        // both CTAs' copies complete on the LEADER's full barrier, which expects all bytes
-                        const uint32_t lead_full = map_to_cta(full_bar + 8 * stage, 0);
-                        if (cta_rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * C::STAGE_BYTES);
-                        tma_load_2d_cg2(sa, &tmap_a, kb * BLOCK_K, m_blk * TILE_M + (int)cta_rank * BLOCK_M, lead_full);
-                        tma_load_2d_cg2(sb, &tmap_b, kb * BLOCK_K, n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS, lead_full);
+                for (int kb = 0; kb < num_kb; kb += C::KPS) {
+                    const int cnt = min(C::KPS, num_kb - kb);   // k-blocks in this stage
+                    if (!mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t st0 = base + stage * C::STAGE_BYTES;
+                    if (elect_one()) {
+                        if (RLX_DBG(p, kDbgNoLoad)) {
+                            if (cta_rank == 0) mbar_arrive(full_bar + 8 * stage);
+                        } else if constexpr (CG == 1) {
+                            mbar_expect_tx(full_bar + 8 * stage, cnt * C::KB_BYTES);
+                            for (int i = 0; i < cnt; ++i) {
+                                const uint32_t sa = st0 + i * C::KB_BYTES, sb = sa + C::A_BYTES;
+                                tma_load_2d(sa, &tmap_a, (kb + i) * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
+                                tma_load_2d(sb, &tmap_b, (kb + i) * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                            }
+                        } else {
+                            // both CTAs' copies complete on the LEADER's full barrier, which expects all bytes
+                            const uint32_t lead_full = map_to_cta(full_bar + 8 * stage, 0);
+                            if (cta_rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * cnt * C::KB_BYTES);
+                            for (int i = 0; i < cnt; ++i) {
+                                const uint32_t sa = st0 + i * C::KB_BYTES, sb = sa + C::A_BYTES;
+                                tma_load_2d_cg2(sa, &tmap_a, (kb + i) * BLOCK_K, m_blk * TILE_M + (int)cta_rank * BLOCK_M, lead_full);
+                                tma_load_2d_cg2(sb, &tmap_b, (kb + i) * BLOCK_K, n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS, lead_full);
+                            }
+                        }
+                        if (tile == tile0 && kb == 0) RLX_TRACE(p, 3);
                     }
+                    __syncwarp();
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
                 }
             }
+            if (lane == 0) RLX_TRACE(p, 4);
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0 && cta_rank == 0) {
+        // ------------------------------------------------------------ MMA issuer (whole warp, one lane issues)
+        if (cta_rank == 0) {
             constexpr uint32_t idesc = make_idesc(TILE_M, BLOCK_N);
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
+            if (lane == 0) { RLX_TRACE(p, 9); RLX_TRACE_CLK(p, 14); }
+            RLX_CLK_DECL(clk_full);
+            RLX_CLK_DECL(clk_tempty);
             for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
                 const int as = it & 1;
                 const uint32_t aphase = (it >> 1) & 1;
-                if (!mbar_wait(tempty_bar + 8 * as, aphase ^ 1, abort_flag)) { ok = false; break; }
+                bool got_acc;
+                RLX_CLK_ADD(clk_tempty, got_acc = mbar_wait_warp(tempty_bar + 8 * as, aphase ^ 1, abort_flag));
+                if (!got_acc) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + as * BLOCK_N;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+                for (int kb = 0; kb < num_kb; kb += C::KPS) {
+                    const int cnt = min(C::KPS, num_kb - kb);
+                    bool got_ops;
+                    RLX_CLK_ADD(clk_full, got_ops = mbar_wait_warp(full_bar + 8 * stage, phase, abort_flag));
+                    if (!got_ops) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = base + stage * C::STAGE_BYTES, sb = sa + C::A_BYTES;
-                    const uint64_t adesc = make_smem_desc(sa), bdesc = make_smem_desc(sb);
+                    const uint32_t st0 = base + stage * C::STAGE_BYTES;
+                    if (elect_one()) {
+                        if (it == 0 && kb == 0) RLX_TRACE(p, 5);
+                        if (!RLX_DBG(p, kDbgNoMma)) {
+                            for (int i = 0; i < cnt; ++i) {
+                                const uint64_t adesc = make_smem_desc(st0 + i * C::KB_BYTES);
+                                const uint64_t bdesc = make_smem_desc(st0 + i * C::KB_BYTES + C::A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                        // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
-                        umma_bf16<CG>(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                                for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                                    // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units
+                                    umma_bf16<CG>(tmem_d, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | i | k) != 0 ? 1u : 0u);
+                                }
+                            }
+                        }
+                        umma_commit<CG>(empty_bar + 8 * stage);  // stage reusable once these MMAs have read it
                     }
-                    umma_commit<CG>(empty_bar + 8 * stage);  // stage reusable once these MMAs have read it
+                    __syncwarp();
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
                 }
-                if (ok) umma_commit<CG>(tfull_bar + 8 * as);  // accumulator complete
+                if (ok && elect_one()) {
+                    umma_commit<CG>(tfull_bar + 8 * as);  // accumulator complete
+                    if (it == 0) RLX_TRACE(p, 6);
+                }
+                __syncwarp();
+            }
+            if (lane == 0) {
+                RLX_TRACE(p, 7);
+                RLX_TRACE_CLK(p, 15);
+                RLX_TRACE_VAL(p, 10, clk_full);
+                RLX_TRACE_VAL(p, 11, clk_tempty);
             }
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        constexpr int HALF_N = C::SLAB;       // columns of the tile this warp handles
-        constexpr int NC = HALF_N / 32;       // 32-column chunks per warp and tile
         const int ew = warp - 2;
         const int quad = warp & 3;            // TMEM lane quadrant this warp may read
         const int half = ew >> 2;             // which column slab of the tile
         const uint32_t stg = staging + ew * kStageBufBytes;
-        const uint32_t row_off = lane * 64;             // 64-byte rows in the staging chunk
-        const uint32_t swz = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte chunk index ^ (row/2 % 4)
         int it = 0;
         bool ok = true;
+        if (tile0 < num_tiles) EpilogueTile<EPI, C::SLAB / 32>::prefetch_bias(p, (tile0 % n_tiles) * BLOCK_N + half * C::SLAB);
         for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++it) {
             const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
+            if (tile + tile_step < num_tiles)
+                EpilogueTile<EPI, C::SLAB / 32>::prefetch_bias(p, ((tile + tile_step) % n_tiles) * BLOCK_N + half * C::SLAB);
             const int as = it & 1;
             const uint32_t aphase = (it >> 1) & 1;
             const int m_row0 = m_blk * TILE_M + (int)cta_rank * BLOCK_M + quad * 32;
-            const int m = m_row0 + lane;
-            const bool row_ok = m < M;
-            const int n0 = n_blk * BLOCK_N + half * HALF_N;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N + half * HALF_N;
-            const float* brow = p.bias + n0;
-            // residual rows of this tile are fetched before waiting for the accumulator, so their
-            // latency hides behind the main loop
-            constexpr bool kRes = EPI == 2 || EPI == 5 || EPI == 6;     // a residual tile is added
-            constexpr bool kFold = EPI == 3 || EPI == 4;                // LayerNorm folded into this GEMM's input
-            constexpr bool kStatsIn = kFold || EPI == 6;
-            constexpr bool kStatsOut = EPI == 5 || EPI == 6;
-            uint4 res[kRes ? NC : 1][4];
-            float ln_a = 1.f, ln_b = 0.f;   // x_norm = x * ln_a + ln_b  (ln_a = rstd, ln_b = -rstd * mu)
-            {
-                const int m_pre = m_blk * TILE_M + (int)cta_rank * BLOCK_M + quad * 32 + lane;
-                if (kRes && m_pre < M) {
-                    const __nv_bfloat16* rpre = p.residual + (size_t)m_pre * p.N + n_blk * BLOCK_N + half * HALF_N;
-#pragma unroll
-                    for (int c = 0; c < NC; ++c)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) res[c][i] = __ldg(reinterpret_cast<const uint4*>(rpre + c * 32) + i);
-                }
-                if (kStatsIn && m_pre < M) {
-                    float mu, rstd;
-                    row_stats_from_partials(p.stats_in + (size_t)m_pre * p.stats_in_p, p.stats_in_p, p.ln_eps, mu, rstd);
-                    ln_a = rstd;
-                    ln_b = -rstd * mu;
-                }
-            }
+            const int n0 = n_blk * BLOCK_N + half * C::SLAB;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + as * BLOCK_N + half * C::SLAB;
+            EpilogueTile<EPI, C::SLAB / 32> et;
+            et.prefetch(p, M, m_row0 + lane, n0);   // residual / row statistics: issued before the accumulator wait
             if (!mbar_wait(tfull_bar + 8 * as, aphase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            if (p.debug & 1) {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    if (CG == 1 || cta_rank == 0) mbar_arrive(tempty_bar + 8 * as);
-                    else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * as, 0));
-                }
-                continue;
-            }
-            uint32_t r[2][32];
-            tmem_ld_32x32(taddr, r[0]);
-#pragma unroll
-            for (int c = 0; c < NC; ++c) {
-                tmem_ld_wait();
-                if (c + 1 < NC) {
-                    tmem_ld_32x32(taddr + (c + 1) * 32, r[(c + 1) & 1]);
-                } else {
-                    // every accumulator value this warp needs is in registers: release the buffer
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (CG == 1 || cta_rank == 0) mbar_arrive(tempty_bar + 8 * as);
-                        else mbar_arrive_cluster(map_to_cta(tempty_bar + 8 * as, 0));
-                    }
-                }
-                const uint32_t(&acc)[32] = r[c & 1];
-                float v[32];
-                if constexpr (kFold) {
-                    const float* crow = p.cvec + n0 + c * 32;
-                    const float* drow = p.dvec + n0 + c * 32;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(crow) + i);
-                        const float4 d4 = __ldg(reinterpret_cast<const float4*>(drow) + i);
-                        v[4 * i + 0] = fmaf(ln_a, __uint_as_float(acc[4 * i + 0]), fmaf(ln_b, c4.x, d4.x));
-                        v[4 * i + 1] = fmaf(ln_a, __uint_as_float(acc[4 * i + 1]), fmaf(ln_b, c4.y, d4.y));
-                        v[4 * i + 2] = fmaf(ln_a, __uint_as_float(acc[4 * i + 2]), fmaf(ln_b, c4.z, d4.z));
-                        v[4 * i + 3] = fmaf(ln_a, __uint_as_float(acc[4 * i + 3]), fmaf(ln_b, c4.w, d4.w));
-                    }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 b4 = __ldg(reinterpret_cast<const float4*>(brow + c * 32) + i);
-                        v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4.x;
-                        v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b4.y;
-                        v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b4.z;
-                        v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b4.w;
-                    }
-                }
-                if (EPI == 1 || EPI == 4) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
-                }
-                if ((EPI == 2 || EPI == 5) && row_ok) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint4 q = res[c][i];
-                        v[8 * i + 0] += bf16lo(q.x); v[8 * i + 1] += bf16hi(q.x);
-                        v[8 * i + 2] += bf16lo(q.y); v[8 * i + 3] += bf16hi(q.y);
-                        v[8 * i + 4] += bf16lo(q.z); v[8 * i + 5] += bf16hi(q.z);
-                        v[8 * i + 6] += bf16lo(q.w); v[8 * i + 7] += bf16hi(q.w);
-                    }
-                }
-                if (EPI == 6 && row_ok) {
-                    // residual = LN(raw residual row): (x * rstd - rstd * mu) * gamma_n + beta_n
-                    const float* grow = p.ln_gamma + n0 + c * 32;
-                    const float* berow = p.ln_beta + n0 + c * 32;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint4 q = res[c][i];
-                        const float4 g0 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i);
-                        const float4 g1 = __ldg(reinterpret_cast<const float4*>(grow) + 2 * i + 1);
-                        const float4 e0 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i);
-                        const float4 e1 = __ldg(reinterpret_cast<const float4*>(berow) + 2 * i + 1);
-                        v[8 * i + 0] += fmaf(fmaf(bf16lo(q.x), ln_a, ln_b), g0.x, e0.x);
-                        v[8 * i + 1] += fmaf(fmaf(bf16hi(q.x), ln_a, ln_b), g0.y, e0.y);
-                        v[8 * i + 2] += fmaf(fmaf(bf16lo(q.y), ln_a, ln_b), g0.z, e0.z);
-                        v[8 * i + 3] += fmaf(fmaf(bf16hi(q.y), ln_a, ln_b), g0.w, e0.w);
-                        v[8 * i + 4] += fmaf(fmaf(bf16lo(q.z), ln_a, ln_b), g1.x, e1.x);
-                        v[8 * i + 5] += fmaf(fmaf(bf16hi(q.z), ln_a, ln_b), g1.y, e1.y);
-                        v[8 * i + 6] += fmaf(fmaf(bf16lo(q.w), ln_a, ln_b), g1.z, e1.z);
-                        v[8 * i + 7] += fmaf(fmaf(bf16hi(q.w), ln_a, ln_b), g1.w, e1.w);
-                    }
-                }
-                if (kStatsOut && row_ok) {
-                    // partial statistics of this row's 32 results (two-pass inside the chunk)
-                    float sm = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) sm += v[i];
-                    const float mean = sm * (1.0f / 32.0f);
-                    float m2 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float dl = v[i] - mean;
-                        m2 = fmaf(dl, dl, m2);
-                    }
-                    p.stats_out[(size_t)m * (p.N / 32) + (n0 + c * 32) / 32] = make_float2(mean, m2);
-                }
-                // transpose through this warp's staging buffer so that every store instruction writes
-                // whole 64-byte row segments (8 rows x 64 B per instruction, full sectors)
-                __syncwarp();   // the previous chunk has been read out of the buffer
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    uint4 q;
-                    q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
-                    q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
-                    q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
-                    q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-                    st_shared_v4(stg + row_off + (((uint32_t)i ^ swz) << 4), q);
-                }
-                __syncwarp();
-                if (!(p.debug & 2)) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int rr = i * 8 + (lane >> 2), cc = lane & 3;
-                        const uint4 q = ld_shared_v4(stg + rr * 64 + (((uint32_t)cc ^ (uint32_t)((rr >> 1) & 3)) << 4));
-                        if (m_row0 + rr < M)
-                            *reinterpret_cast<uint4*>(p.out + (size_t)(m_row0 + rr) * p.N + n0 + c * 32 + cc * 8) = q;
-                    }
-                }
-            }
+            if (ew == 0 && lane == 0 && it < 12) RLX_TRACE(p, 16 + it);
+            et.template drain<CG>(p, &tmap_out, M, m_row0, n0, taddr, stg, lane, tempty_bar + 8 * as, cta_rank,
+                                  (ew == 0 && lane == 0 && (it == 1 || it == 5)) ? 40 + 2 * (it - 1) : -1);
+            if (ew == 0 && lane == 0 && it < 12) RLX_TRACE(p, 28 + it);
         }
+        EpilogueTile<EPI, C::SLAB / 32>::finish(lane);
+        if (ew == 0 && lane == 0) RLX_TRACE(p, 8);
     }
 
     // ---------------------------------------------------------------- teardown
@@ -606,11 +805,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) RLX_TRACE(p, 12);
     if constexpr (CG == 2) cluster_sync_all();   // neither CTA leaves while the pair still uses its memory
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
+        if (lane == 0) RLX_TRACE(p, 13);
     }
 }
 

@@ -16,6 +16,7 @@
 #include "dequant.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
+#include "gemm_ares_tcgen05.cuh"
 #include "gemm_ln_tcgen05.cuh"
 #include "gemm_cln_tcgen05.cuh"
 #include "rowwise.cuh"
@@ -94,6 +95,31 @@ cudaError_t set_gemm_attr_all() {
 
 // Number of CTA pairs that can be resident at once (pairs must sit in one GPC), per device.
 int g_max_pairs[64] = {};
+int g_max_pairs_resident[64] = {};   // the same for the A-resident kernel (its own shared-memory footprint)
+
+// Multiprocessor count of the current device (grids of the persistent kernels are sized from it).
+constexpr int kNominalSMs = 148;   // B200; used only when no device can be queried (host-only callers)
+int sm_count_of(int dev) {
+    static int cached[64] = {};
+    if (dev < 0 || dev >= 64) return kNominalSMs;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            return kNominalSMs;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+int sm_count() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return kNominalSMs;
+    }
+    return sm_count_of(dev);
+}
 
 cudaError_t init_kernels_for_current_device() {
     static std::mutex mu;
@@ -124,7 +150,7 @@ cudaError_t init_kernels_for_current_device() {
     if ((e = (set_gemm_attr_all<256, 2>())) != cudaSuccess) return e;
     {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * rlx::kNumSMs);
+        cfg.gridDim = dim3(2 * sm_count());
         cfg.blockDim = dim3(rlx::tc::Cfg<256, 2>::THREADS);
         cfg.dynamicSmemBytes = rlx::tc::Cfg<256, 2>::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
@@ -137,6 +163,31 @@ cudaError_t init_kernels_for_current_device() {
         int n = 0;
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tc::gemm_tcgen05_kernel<256, 0, 2>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs[dev] = n;
+    }
+#define RLX_ARES_ATTR(BN, EPI)                                                                                  \
+    if ((e = cudaFuncSetAttribute(rlx::tcar::gemm_ares_tcgen05_kernel<BN, EPI>,                                \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, rlx::tcar::Cfg<BN>::SMEM_BYTES)) != \
+        cudaSuccess)                                                                                           \
+        return e;
+    RLX_ARES_ATTR(128, 0) RLX_ARES_ATTR(128, 1) RLX_ARES_ATTR(128, 2)
+    RLX_ARES_ATTR(192, 0) RLX_ARES_ATTR(192, 1) RLX_ARES_ATTR(192, 2)
+    RLX_ARES_ATTR(256, 0) RLX_ARES_ATTR(256, 1) RLX_ARES_ATTR(256, 2)
+#undef RLX_ARES_ATTR
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * sm_count());
+        cfg.blockDim = dim3(rlx::tcar::Cfg<256>::THREADS);
+        cfg.dynamicSmemBytes = rlx::tcar::Cfg<256>::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tcar::gemm_ares_tcgen05_kernel<256, 0>, &cfg)) != cudaSuccess) return e;
+        if (dev < 64) g_max_pairs_resident[dev] = n;
     }
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tca::Smem<32>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
@@ -158,7 +209,6 @@ cudaError_t init_kernels_for_current_device() {
 }
 
 // ------------------------------------------------------------------ launchers
-unsigned long long* g_attn_dbg = nullptr;   // experiments only: device buffer for in-kernel phase timestamps
 // When set, kernels are launched with the programmatic-stream-serialization attribute so that each
 // kernel's prologue overlaps its predecessor's tail (the kernels call griddepcontrol.wait before
 // they read anything a predecessor wrote).  Set by enqueue_forward around its launches.
@@ -225,7 +275,7 @@ rlx_status_t launch_layernorm(const bf16* x, const float* g, const float* b, int
                               cudaStream_t st, const int32_t* rows_ptr = nullptr) {
     // rows per warp: as many as still leave ~4 CTAs for every SM (static row bound T), so that large
     // problems run as about one full wave of fat CTAs and small ones still cover all SMs
-    const int want_ctas = 4 * rlx::kNumSMs;
+    const int want_ctas = 4 * sm_count();
     const int rpw = (T >= want_ctas * rlx::kRowWarps * 4) ? 4 : 1;   // 8 rows per warp measured slower
     const int rows_per_cta = rlx::kRowWarps * rpw;
     const int grid = (T + rows_per_cta - 1) / rows_per_cta, thr = rlx::kRowWarps * 32;
@@ -309,10 +359,10 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
     const int nblk = (S + rlx::tca::kBlockN - 1) / rlx::tca::kBlockN;   // K/V tiles held in shared memory
     if (d == 32)
         RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, grid, rlx::tca::kThreads, rlx::tca::Smem<32>::bytes(nblk), st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status, g_attn_dbg));
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status));
     else if (d == 64)
         RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, grid, rlx::tca::kThreads, rlx::tca::Smem<64>::bytes(nblk), st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status, g_attn_dbg));
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status));
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
@@ -321,46 +371,52 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
 
 struct TileChoice { int bn; int cg; };
 
+// Tuning overrides: compiled in only with -DRLX_EXPERIMENTS (rlx_experiment_set); constants otherwise.
+#ifdef RLX_EXPERIMENTS
+int g_exp_cg = 0, g_exp_bn = 0, g_exp_debug = 0, g_exp_resident = 0;
+unsigned long long* g_exp_trace = nullptr;
+#else
+constexpr int g_exp_cg = 0, g_exp_resident = 0;
+#endif
+
 // Tile shape for an [M, N] output.  CTA pairs (cg = 2, 256-row tiles, each CTA loading half of the
 // W tile) are used when there are enough tiles to keep every pair busy for a few rounds; smaller
 // problems keep one CTA per 128-row tile and shrink BLOCK_N until every SM has work.
 TileChoice pick_tile(int M, int N, int K, int want_cg = 0) {
-    static const int env_cg = getenv("RLX_GEMM_CG") ? atoi(getenv("RLX_GEMM_CG")) : 0;   // tuning knobs
-    const int force_cg = want_cg ? want_cg : env_cg;
-    static const int force_bn = getenv("RLX_GEMM_BN") ? atoi(getenv("RLX_GEMM_BN")) : 0;
+    const int force_cg = want_cg ? want_cg : g_exp_cg;
     int dev = 0;
     cudaGetDevice(&dev);
     const int pairs = (dev >= 0 && dev < 64) ? g_max_pairs[dev] : 0;
+#ifdef RLX_EXPERIMENTS
+    if (g_exp_bn && N % g_exp_bn == 0 && (g_exp_bn == 64 || g_exp_bn == 128 || g_exp_bn == 192 || g_exp_bn == 256))
+        return {g_exp_bn, (force_cg == 2 && g_exp_bn >= 128) ? 2 : 1};
+#endif
     // pairs pay off once a tile's main loop is long enough to amortise the cross-CTA handshakes
     // (K >= 1536, or K >= 768 with a wide output) and every pair gets at least two tiles
     if (force_cg != 1 && pairs > 0 && (force_cg == 2 || K >= 1536 || (K >= 768 && N >= 1536))) {
         const int m_tiles2 = (M + 255) / 256;
         const int cand2[3] = {256, 192, 128};
-        for (int i = 0; i < 3; ++i) {
-            if (force_bn && cand2[i] != force_bn) continue;
+        for (int i = 0; i < 3; ++i)
             if (N % cand2[i] == 0 && (force_cg == 2 || m_tiles2 * (N / cand2[i]) >= 2 * pairs)) return {cand2[i], 2};
-        }
     }
     const int m_tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
     const int cand[4] = {256, 192, 128, 64};
-    if (force_bn && N % force_bn == 0 && (force_bn == 64 || force_bn == 128 || force_bn == 192 || force_bn == 256))
-        return {force_bn, 1};
     // largest tile that still gives every SM work; otherwise the smallest that divides N
     for (int i = 0; i < 4; ++i)
-        if (N % cand[i] == 0 && m_tiles * (N / cand[i]) >= rlx::kNumSMs) return {cand[i], 1};
+        if (N % cand[i] == 0 && m_tiles * (N / cand[i]) >= sm_count()) return {cand[i], 1};
     for (int i = 3; i >= 0; --i)
         if (N % cand[i] == 0) return {cand[i], 1};
     return {0, 1};
 }
 
 template <int BN, int CG>
-rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const rlx::tc::Params& p, int epi,
-                               cudaStream_t st) {
+rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                               const rlx::tc::Params& p, int epi, cudaStream_t st) {
     const int tile_m = rlx::tc::BLOCK_M * CG;
     const int tiles = ((p.M + tile_m - 1) / tile_m) * (p.N / BN);
     int dev = 0;
     cudaGetDevice(&dev);
-    const int slots = CG == 1 ? rlx::kNumSMs : ((dev >= 0 && dev < 64) ? g_max_pairs[dev] : 1);
+    const int slots = CG == 1 ? sm_count() : ((dev >= 0 && dev < 64) ? g_max_pairs[dev] : 1);
     const int grid = CG * (tiles < slots ? tiles : slots);
     const int smem = rlx::tc::Cfg<BN, CG>::SMEM_BYTES;
     struct ClusterScope {
@@ -368,17 +424,59 @@ rlx_status_t launch_gemm_tc_bn(const CUtensorMap& ta, const CUtensorMap& tb, con
         ~ClusterScope() { g_cluster_x = 1; }
     } scope(CG);
     switch (epi) {
-        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 3: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 3, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 4: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 4, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 5: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 5, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
-        case 6: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 6, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, p)); break;
+        case 0: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 0, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 1: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 1, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 2: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 2, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 3: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 3, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 4: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 4, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 5: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 5, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
+        case 6: RLX_CUDA_TRY(launch_ex(rlx::tc::gemm_tcgen05_kernel<BN, 6, CG>, grid, rlx::tc::Cfg<BN, CG>::THREADS, smem, st, ta, tb, to, p)); break;
         default: return RLX_ERR_INVALID_ARG;
     }
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
+}
+
+// A-resident CTA-pair GEMM (short contractions): grid = 2 x min(work units, resident pairs).
+template <int BN>
+rlx_status_t launch_gemm_resident_bn(const CUtensorMap& ta, const CUtensorMap& tb, const CUtensorMap& to,
+                                     const rlx::tc::Params& p, int epi, cudaStream_t st) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int pairs = (dev >= 0 && dev < 64) ? g_max_pairs_resident[dev] : 0;
+    if (pairs <= 0) return RLX_ERR_UNSUPPORTED;
+    const int m_blocks = (p.M + rlx::tcar::kPairRows - 1) / rlx::tcar::kPairRows;
+    const int units = m_blocks * (p.N / BN);   // the finest split the kernel may choose
+    const int grid = 2 * (units < pairs ? units : pairs);
+    const int smem = rlx::tcar::Cfg<BN>::SMEM_BYTES, thr = rlx::tcar::Cfg<BN>::THREADS;
+    struct ClusterScope {
+        explicit ClusterScope(int x) { g_cluster_x = x; }
+        ~ClusterScope() { g_cluster_x = 1; }
+    } scope(2);
+    switch (epi) {
+        case 0: RLX_CUDA_TRY(launch_ex(rlx::tcar::gemm_ares_tcgen05_kernel<BN, 0>, grid, thr, smem, st, ta, tb, to, p)); break;
+        case 1: RLX_CUDA_TRY(launch_ex(rlx::tcar::gemm_ares_tcgen05_kernel<BN, 1>, grid, thr, smem, st, ta, tb, to, p)); break;
+        case 2: RLX_CUDA_TRY(launch_ex(rlx::tcar::gemm_ares_tcgen05_kernel<BN, 2>, grid, thr, smem, st, ta, tb, to, p)); break;
+        default: return RLX_ERR_INVALID_ARG;
+    }
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+// Tile width of the A-resident kernel for an [M, N] x K problem, or 0 when it does not apply: K must
+// fit the resident block, N must split into 256-, 192- or 128-wide tiles, and (unless forced) there must
+// be enough 256-row blocks to give every CTA pair one -- smaller problems keep 128-row tiles per CTA.
+int pick_resident_bn(int M, int N, int K, int epi, bool forced) {
+    if (epi > 2 || K > rlx::tcar::kMaxKB * rlx::tc::BLOCK_K) return 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int pairs = (dev >= 0 && dev < 64) ? g_max_pairs_resident[dev] : 0;
+    if (pairs <= 0) return 0;
+    if (!forced && (M + rlx::tcar::kPairRows - 1) / rlx::tcar::kPairRows < pairs) return 0;
+    const int cand[3] = {256, 192, 128};
+    for (int i = 0; i < 3; ++i)
+        if (N % cand[i] == 0) return cand[i];
+    return 0;
 }
 
 // Extra operands of the LayerNorm-folding epilogues (EPI 3..6 of the tcgen05 GEMM).
@@ -408,14 +506,34 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
         RLX_CUDA_TRY(cudaGetLastError());
         return RLX_OK;
     }
+    if (K % 8 != 0) return RLX_ERR_UNSUPPORTED;
+    rlx::tc::Params p{};
+    p.bias = bias; p.residual = residual; p.out = out; p.M = M; p.N = N; p.K = K; p.status = status; p.m_ptr = m_ptr;
+#ifdef RLX_EXPERIMENTS
+    p.debug = g_exp_debug;
+    p.trace = g_exp_trace;
+#endif
+    CUtensorMap ta, tb, to;
+    if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
+    // output chunks: 32 x 32 bf16 boxes with the 64-byte swizzle of the epilogue's staging buffers
+    if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
+    // want_cg == 3: the A-resident CTA-pair kernel, forced; 0: chosen when the problem is large enough
+    if (want_cg == 3 || (want_cg == 0 && g_exp_resident >= 0)) {
+        const int rbn = pick_resident_bn(M, N, K, epi, want_cg == 3 || g_exp_resident > 0);
+        if (rbn == 0 && want_cg == 3) return RLX_ERR_UNSUPPORTED;
+        if (rbn != 0) {
+            if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(rbn / 2))) return RLX_ERR_CUDA;
+            switch (rbn) {
+                case 128: return launch_gemm_resident_bn<128>(ta, tb, to, p, epi, st);
+                case 192: return launch_gemm_resident_bn<192>(ta, tb, to, p, epi, st);
+                case 256: return launch_gemm_resident_bn<256>(ta, tb, to, p, epi, st);
+            }
+        }
+    }
     const TileChoice tc = pick_tile(M, N, K, want_cg);
     const int bn = tc.bn;
-    if (bn == 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
-    CUtensorMap ta, tb;
-    if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
+    if (bn == 0) return RLX_ERR_UNSUPPORTED;
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / tc.cg))) return RLX_ERR_CUDA;
-    static const int dbg = getenv("RLX_GEMM_DEBUG") ? atoi(getenv("RLX_GEMM_DEBUG")) : 0;
-    rlx::tc::Params p{bias, residual, out, M, N, K, status, m_ptr, dbg};
     if (epi >= 3) {
         if (!lf || N % 32 != 0) return RLX_ERR_INVALID_ARG;
         p.cvec = lf->cvec; p.dvec = lf->dvec; p.stats_in = lf->stats_in; p.stats_in_p = lf->stats_in_p;
@@ -423,17 +541,17 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     }
     if (tc.cg == 2) {
         switch (bn) {
-            case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, p, epi, st);
-            case 192: return launch_gemm_tc_bn<192, 2>(ta, tb, p, epi, st);
-            case 256: return launch_gemm_tc_bn<256, 2>(ta, tb, p, epi, st);
+            case 128: return launch_gemm_tc_bn<128, 2>(ta, tb, to, p, epi, st);
+            case 192: return launch_gemm_tc_bn<192, 2>(ta, tb, to, p, epi, st);
+            case 256: return launch_gemm_tc_bn<256, 2>(ta, tb, to, p, epi, st);
         }
         return RLX_ERR_UNSUPPORTED;
     }
     switch (bn) {
-        case 64: return launch_gemm_tc_bn<64, 1>(ta, tb, p, epi, st);
-        case 128: return launch_gemm_tc_bn<128, 1>(ta, tb, p, epi, st);
-        case 192: return launch_gemm_tc_bn<192, 1>(ta, tb, p, epi, st);
-        case 256: return launch_gemm_tc_bn<256, 1>(ta, tb, p, epi, st);
+        case 64: return launch_gemm_tc_bn<64, 1>(ta, tb, to, p, epi, st);
+        case 128: return launch_gemm_tc_bn<128, 1>(ta, tb, to, p, epi, st);
+        case 192: return launch_gemm_tc_bn<192, 1>(ta, tb, to, p, epi, st);
+        case 256: return launch_gemm_tc_bn<256, 1>(ta, tb, to, p, epi, st);
     }
     return RLX_ERR_UNSUPPORTED;
 }
@@ -447,9 +565,9 @@ rlx_status_t launch_gemm_ln(const bf16* A, const bf16* W, const float* bias, con
     CUtensorMap ta, tb;
     if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
     if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)nh)) return RLX_ERR_CUDA;
-    rlx::tcln::Params p{bias, residual, gamma, beta, out, eps, M, K, status, m_ptr, g_attn_dbg};
+    rlx::tcln::Params p{bias, residual, gamma, beta, out, eps, M, K, status, m_ptr};
     const int tiles = (M + rlx::tc::BLOCK_M - 1) / rlx::tc::BLOCK_M;
-    const int grid = tiles < rlx::kNumSMs ? tiles : rlx::kNumSMs;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
     switch (nh) {
         case 128: RLX_CUDA_TRY(launch_ex(rlx::tcln::gemm_ln_tcgen05_kernel<128>, grid, rlx::tcln::kThreads, rlx::tcln::Cfg<128>::SMEM_BYTES, st, ta, tb, p)); break;
         case 192: RLX_CUDA_TRY(launch_ex(rlx::tcln::gemm_ln_tcgen05_kernel<192>, grid, rlx::tcln::kThreads, rlx::tcln::Cfg<192>::SMEM_BYTES, st, ta, tb, p)); break;
@@ -474,7 +592,7 @@ rlx_status_t launch_gemm_cln_bn(const bf16* A, const bf16* W, const rlx::tccl::P
     if (dev < 0 || dev >= 64) return RLX_ERR_UNSUPPORTED;
     if (max_clusters[dev][nranks] == 0) {
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(nranks * rlx::kNumSMs);
+        cfg.gridDim = dim3(nranks * sm_count());
         cfg.blockDim = dim3(rlx::tccl::Cfg<BN>::THREADS);
         cfg.dynamicSmemBytes = rlx::tccl::Cfg<BN>::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
@@ -508,7 +626,7 @@ int pick_cln_block_n(int M, int N) {
     int fallback = 0;
     for (int i = 0; i < 3; ++i) {
         if (N % cand[i] != 0 || N / cand[i] > rlx::tccl::kMaxCluster) continue;
-        if (m_tiles * (N / cand[i]) >= rlx::kNumSMs) return cand[i];
+        if (m_tiles * (N / cand[i]) >= sm_count()) return cand[i];
         fallback = cand[i];   // keeps the narrowest admissible slab
     }
     return fallback;
@@ -584,7 +702,7 @@ Arena plan_arena(int B, int S, int H, int F, int L = 0, bool fold = false) {
 bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
     if ((c.flags & RLX_FLAG_GEMM_SIMT) || !(c.flags & RLX_FLAG_FUSED_LN)) return false;
     if (c.hidden != 256 && c.hidden != 384 && c.hidden != 512) return false;
-    return (long long)B * S >= 128ll * rlx::kNumSMs;
+    return (long long)B * S >= 128ll * sm_count_of(c.device);
 }
 
 // RLX_FLAG_CLUSTER_LN: LayerNorm folded into the out-proj / FFN-down GEMMs with cluster-wide row
@@ -647,7 +765,7 @@ void drop_graphs(rlx_encoder* e) {
 // The kernel sequence of one forward, enqueued on `st` (eagerly or under stream capture).
 rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
                              const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st,
-                             bool capturing) {
+                             bool capturing, bool with_events = true) {
     const rlx_encoder_config_t& c = e->cfg;
     const int H = c.hidden, F = c.ffn, T = B * S, h = c.num_heads, d = e->head_dim;
     const bool simt = (c.flags & RLX_FLAG_GEMM_SIMT) != 0;
@@ -668,8 +786,9 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     // With RLX_FLAG_KERNEL_EVENTS an event is recorded between consecutive kernels; under stream
     // capture the records become event-record nodes of the graph, so replays time each kernel on
     // the device without any host launch gap.
+    const bool timing = with_events && !e->events.empty();
     auto mark = [&]() -> rlx_status_t {
-        if (e->events.empty()) return RLX_OK;
+        if (!timing) return RLX_OK;
         RLX_CUDA_TRY(cudaEventRecordWithFlags(e->events[ev++], st,
                                               capturing ? cudaEventRecordExternal : cudaEventRecordDefault));
         return RLX_OK;
@@ -681,7 +800,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     struct PdlScope {
         explicit PdlScope(bool on) { g_pdl_launch = on; }
         ~PdlScope() { g_pdl_launch = false; }
-    } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && e->events.empty());
+    } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && !timing);
     // side branch (captured graphs only): prefetch the Linear weights into L2 when they all fit
     bool forked = false;
     if (capturing && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH) && !fold) {   // the fold pass reads the weights anyway
@@ -702,7 +821,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
             }
             RLX_CUDA_TRY(cudaEventRecord(e->fork_event, st));
             RLX_CUDA_TRY(cudaStreamWaitEvent(e->side_stream, e->fork_event, 0));
-            rlx::prefetch_l2_kernel<<<rlx::kNumSMs, 32, 0, e->side_stream>>>(pf);
+            rlx::prefetch_l2_kernel<<<sm_count(), 32, 0, e->side_stream>>>(pf);
             RLX_CUDA_TRY(cudaGetLastError());
             RLX_CUDA_TRY(cudaEventRecord(e->join_event, e->side_stream));
             forked = true;
@@ -1092,7 +1211,9 @@ rlx_status_t rlx_encoder_forward_static(rlx_encoder_t* e, const int32_t* ids, co
     // the arena keeps the previous call's bytes: the status word is the only part read before it is
     // written, so it alone is cleared; every activation row is rewritten by the kernels below
     RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status, 0, sizeof(int32_t), st));
-    s = enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);  // direct launches: no graph objects
+    // direct launches: no graph objects; and no event records even when an ordinary forward of this
+    // object created its per-kernel events (they stay those of that forward)
+    s = enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false, false);
     if (s != RLX_OK) return s;
     if (device_status)
         RLX_CUDA_TRY(cudaMemcpyAsync(device_status, ws + a.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
@@ -1134,11 +1255,13 @@ rlx_status_t rlx_gemm_bf16(const void* A, const void* W, const float* bias, cons
         return RLX_ERR_INVALID_ARG;
     if (N % 64 != 0 || K % 8 != 0) return RLX_ERR_UNSUPPORTED;
     if (impl != RLX_GEMM_TCGEN05 && impl != RLX_GEMM_SIMT && impl != RLX_GEMM_TCGEN05_PAIR &&
-        impl != RLX_GEMM_TCGEN05_SINGLE)
+        impl != RLX_GEMM_TCGEN05_SINGLE && impl != RLX_GEMM_TCGEN05_RESIDENT)
         return RLX_ERR_INVALID_ARG;
     if (impl == RLX_GEMM_TCGEN05_PAIR && N % 128 != 0 && N % 192 != 0) return RLX_ERR_UNSUPPORTED;
+    if (impl == RLX_GEMM_TCGEN05_RESIDENT && (K > 384 || (N % 128 != 0 && N % 192 != 0))) return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
-    const int want_cg = impl == RLX_GEMM_TCGEN05_PAIR ? 2 : impl == RLX_GEMM_TCGEN05_SINGLE ? 1 : 0;
+    const int want_cg = impl == RLX_GEMM_TCGEN05_PAIR ? 2 : impl == RLX_GEMM_TCGEN05_SINGLE ? 1
+                        : impl == RLX_GEMM_TCGEN05_RESIDENT ? 3 : 0;
     return launch_gemm((const bf16*)A, (const bf16*)W, bias, (const bf16*)residual, (int)epi, M, N, K, (bf16*)out,
                        impl == RLX_GEMM_SIMT, status, static_cast<cudaStream_t>(stream), nullptr, want_cg);
 }
@@ -1253,7 +1376,7 @@ rlx_status_t rlx_dequant_block_scaled_bf16(const void* codes, const void* scales
     if (K % 32 != 0) return RLX_ERR_UNSUPPORTED;
     const long long tasks = (long long)N * (K / rlx::kDequantElemsPerThread);
     const int blocks = (int)std::min<long long>((tasks + rlx::kDequantThreads - 1) / rlx::kDequantThreads,
-                                                (long long)rlx::kNumSMs * 16);
+                                                (long long)sm_count() * 16);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (packed4)
         rlx::dequant_block_scaled_kernel<true><<<blocks, rlx::kDequantThreads, 0, st>>>(
@@ -1287,8 +1410,6 @@ rlx_status_t rlx_selftest_bounded_wait(uint32_t budget_us, int32_t* status_word,
     return RLX_OK;
 }
 
-void rlx_debug_set_attn_trace(void* p) { g_attn_dbg = static_cast<unsigned long long*>(p); }
-
 rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B, int32_t S, int32_t h, int32_t d,
                                float* ctx, void* stream) {
     if (!qkv || !mask || !ctx || B <= 0 || S <= 0 || h <= 0) return RLX_ERR_INVALID_ARG;
@@ -1311,5 +1432,25 @@ rlx_status_t rlx_pool_l2norm(const void* x, const int32_t* mask, int32_t B, int3
     if (!aligned16(x)) return RLX_ERR_INVALID_ARG;
     return launch_pool((const bf16*)x, mask, B, S, H, out, static_cast<cudaStream_t>(stream));
 }
+
+#ifdef RLX_EXPERIMENTS
+// Experiments build only (not declared in the header): 0 = CTA grouping, 1 = tile width, 2 = ablation bits
+// of the GEMM kernels, 3 = A-resident kernel (-1 off, 0 automatic, 1 whenever it applies).
+void rlx_experiment_set(int key, int value) {
+    switch (key) {
+        case 0: g_exp_cg = value; break;
+        case 1: g_exp_bn = value; break;
+        case 2: g_exp_debug = value; break;
+        case 3: g_exp_resident = value; break;
+    }
+}
+void rlx_experiment_trace(void* buf) { g_exp_trace = static_cast<unsigned long long*>(buf); }
+int rlx_experiment_pairs(int resident) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (init_kernels_for_current_device() != cudaSuccess) return -1;
+    return resident ? g_max_pairs_resident[dev] : g_max_pairs[dev];
+}
+#endif
 
 }  // extern "C"

@@ -125,17 +125,27 @@ def test_pack_sequences_is_bit_exact(rlx, B, S, holes):
 
 # ------------------------------------------------------------------ GEMM
 GEMM_SHAPES = [(128, 64, 64), (16, 1152, 384), (300, 384, 384), (257, 1536, 384), (1000, 384, 1536),
-               (129, 768, 768), (4096, 192, 72), (2048, 2304, 768)]
+               (129, 768, 768), (4096, 192, 72), (2048, 2304, 768), (9000, 1152, 384), (40000, 384, 384)]
+GEMM_IMPLS = [0, 1, 2, 3, 4]
+GEMM_IMPL_IDS = ["tcgen05", "simt", "tcgen05_pair", "tcgen05_single", "tcgen05_resident"]
 
 
-@pytest.mark.parametrize("impl", [0, 1, 2, 3], ids=["tcgen05", "simt", "tcgen05_pair", "tcgen05_single"])
+def _impl_applies(impl, N, K):
+    if impl == 2:
+        return N % 128 == 0          # CTA-pair tiles
+    if impl == 4:
+        return K <= 384 and (N % 128 == 0 or N % 192 == 0)   # A-resident CTA-pair kernel
+    return True
+
+
+@pytest.mark.parametrize("impl", GEMM_IMPLS, ids=GEMM_IMPL_IDS)
 def test_gemm_small_integers_is_bit_exact(rlx, impl):
     """Operands are small integers (exact in bf16, sums exact in fp32): any layout, descriptor or
     indexing mistake shows up as a wrong integer, with no tolerance to hide behind."""
     rng = np.random.default_rng(11)
     for (M, N, K) in [(128, 64, 64), (128, 128, 128), (200, 192, 384), (384, 256, 136), (130, 384, 1536),
-                      (700, 1152, 384)]:
-        if impl == 2 and N % 128:
+                      (700, 1152, 384), (5000, 1536, 320)]:
+        if not _impl_applies(impl, N, K):
             continue
         a = rng.integers(-1, 2, size=(M, K)).astype(np.float32)
         w = rng.integers(-1, 2, size=(N, K)).astype(np.float32)
@@ -148,13 +158,13 @@ def test_gemm_small_integers_is_bit_exact(rlx, impl):
         assert np.array_equal(got, ref), (M, N, K, np.abs(got - ref).max())
 
 
-@pytest.mark.parametrize("impl", [0, 1, 2, 3], ids=["tcgen05", "simt", "tcgen05_pair", "tcgen05_single"])
+@pytest.mark.parametrize("impl", GEMM_IMPLS, ids=GEMM_IMPL_IDS)
 @pytest.mark.parametrize("epi", [0, 1, 2], ids=["bias", "gelu", "residual"])
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
 def test_gemm_matches_oracle_linear(rlx, shape, epi, impl):
     M, N, K = shape
-    if impl == 2 and N % 128:
-        pytest.skip("CTA-pair tiles need N % 128 == 0")
+    if not _impl_applies(impl, N, K):
+        pytest.skip("tile shape of this variant does not divide the problem")
     if impl == 1 and M * N * K > 2e9:
         pytest.skip("bring-up GEMM: large case covered by the tensor-core path")
     rng = np.random.default_rng(M + N + K + epi)
