@@ -159,22 +159,29 @@ gemm_ares_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                             // that its loads, one unit later, do not pay an HBM round trip on the critical path
                             if (load_a && unit + pairs < units) {
                                 const int next_m = (unit + pairs) / n_groups;
-                                for (int i = 0; i < cnt; ++i)
-                                    tma_prefetch_2d(&tmap_a, (kb + i) * BLOCK_K, next_m * kPairRows + (int)cta_rank * BLOCK_M);
+                                const int nrow = next_m * kPairRows + (int)cta_rank * BLOCK_M;
+                                if (p.kblock_maps) tma_prefetch_3d(&tmap_a, 0, nrow, kb);
+                                else for (int i = 0; i < cnt; ++i) tma_prefetch_2d(&tmap_a, (kb + i) * BLOCK_K, nrow);
                             }
                             // both CTAs' copies complete on the LEADER's full barrier, which expects all bytes
                             const uint32_t lead_full = map_to_cta(full_bar + 8 * stage, 0);
                             if (RLX_DBG(p, kDbgNoLoad)) {
                                 if (cta_rank == 0) mbar_arrive(full_bar + 8 * stage);
                             } else {
+                                const bool k3 = p.kblock_maps != 0;   // one 3-D load per operand and stage
+                                const int nkb = k3 ? C::KPS : cnt;
                                 if (cta_rank == 0)
-                                    mbar_expect_tx(full_bar + 8 * stage, 2 * cnt * (C::B_BYTES + (load_a ? C::A_BYTES : 0)));
-                                for (int i = 0; i < cnt; ++i) {
-                                    if (load_a)
-                                        tma_load_2d_cg2(a_smem + (kb + i) * C::A_BYTES, &tmap_a, (kb + i) * BLOCK_K,
-                                                        m_blk * kPairRows + (int)cta_rank * BLOCK_M, lead_full);
-                                    tma_load_2d_cg2(sb + i * C::B_BYTES, &tmap_b, (kb + i) * BLOCK_K,
-                                                    n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS, lead_full);
+                                    mbar_expect_tx(full_bar + 8 * stage, 2 * nkb * (C::B_BYTES + (load_a ? C::A_BYTES : 0)));
+                                const int arow = m_blk * kPairRows + (int)cta_rank * BLOCK_M;
+                                const int brow = n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS;
+                                if (k3) {
+                                    if (load_a) tma_load_3d_cg2(a_smem + kb * C::A_BYTES, &tmap_a, 0, arow, kb, lead_full);
+                                    tma_load_3d_cg2(sb, &tmap_b, 0, brow, kb, lead_full);
+                                } else {
+                                    for (int i = 0; i < cnt; ++i) {
+                                        if (load_a) tma_load_2d_cg2(a_smem + (kb + i) * C::A_BYTES, &tmap_a, (kb + i) * BLOCK_K, arow, lead_full);
+                                        tma_load_2d_cg2(sb + i * C::B_BYTES, &tmap_b, (kb + i) * BLOCK_K, brow, lead_full);
+                                    }
                                 }
                             }
                             if (uit == 0 && j == 0 && kb == 0) RLX_TRACE(p, 3);

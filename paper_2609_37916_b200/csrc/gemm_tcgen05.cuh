@@ -63,12 +63,20 @@ struct Cfg {
     static constexpr int STAGING_BYTES = EPI_WARPS * kStageBufBytes;
     static constexpr int BAR_BYTES = 256;
     static constexpr int RING_BUDGET = 227 * 1024 - 1024 - BAR_BYTES - STAGING_BYTES;
-    // A stage holds KPS k-blocks behind ONE full / empty barrier pair.  A barrier wait costs the issuing
+    // A stage holds KPS k-blocks behind ONE full / empty barrier pair.  A barrier round costs the issuing
     // thread a couple of hundred cycles whether or not the barrier is already complete (measured: 4 MMAs
-    // + wait + commit take ~430 cycles of the thread, 8 MMAs ~620), so with one k-block per wait the
-    // single MMA thread, not the tensor pipe, paces every tile narrower than 256 columns.  Two k-blocks
-    // per stage whenever three such stages still fit.
-    static constexpr int KPS = (3 * 2 * KB_BYTES <= RING_BUDGET) ? 2 : 1;
+    // + wait + commit take ~430 cycles of the thread, 8 MMAs ~620), so with one k-block per round the
+    // single MMA thread, not the tensor pipe, paces every tile narrower than 256 columns (384 tensor
+    // cycles per k-block at N = 192).  Such tiles take two k-blocks per stage when four stages still
+    // fit; 256-wide tiles (512 tensor cycles per k-block) keep one, which buys ring depth: what the
+    // ring can hide is (STAGES - 1) stages of tensor time, and the operands come from L2 or HBM.
+#ifndef RLX_KPS_MIN_STAGES
+#define RLX_KPS_MIN_STAGES 4
+#endif
+#ifndef RLX_KPS_MAX_BN
+#define RLX_KPS_MAX_BN 192
+#endif
+    static constexpr int KPS = (BLOCK_N <= RLX_KPS_MAX_BN && RLX_KPS_MIN_STAGES * 2 * KB_BYTES <= RING_BUDGET) ? 2 : 1;
     static constexpr int STAGE_BYTES = KPS * KB_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
     static constexpr int TMEM_COLS = (2 * BLOCK_N <= 32) ? 32 : (2 * BLOCK_N <= 64) ? 64 : (2 * BLOCK_N <= 128) ? 128
@@ -214,6 +222,18 @@ __device__ __forceinline__ float4 ld_global_keep_f4(const float* ptr) {
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+// 3-D forms: operand viewed as [k-block][row][64 columns]; the box covers several k-blocks, which land
+// one after the other as complete 128-byte-swizzled tiles
+__device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap* tmap, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_cg2(uint32_t smem_dst, const CUtensorMap* tmap, int x, int y, int z, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z), "r"(bar_cluster) : "memory");
+}
 // CG = 2 form: the mbarrier may live in the peer CTA (cluster address); the data lands in this CTA
 __device__ __forceinline__ void tma_load_2d_cg2(uint32_t smem_dst, const CUtensorMap* tmap, int x, int y, uint32_t bar_cluster) {
     asm volatile(
@@ -224,6 +244,10 @@ __device__ __forceinline__ void tma_load_2d_cg2(uint32_t smem_dst, const CUtenso
 __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tmap, int x, int y) {
     asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
                  ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* tmap, int x, int y, int z) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];"
+                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
@@ -333,6 +357,8 @@ struct Params {
     int M, N, K;
     int32_t* status;                 // device status word (may be null)
     const int32_t* m_ptr;            // optional device row count: rows >= *m_ptr are not computed
+    int kblock_maps;                 // the operand tensor maps are 3-D views [K/64][rows][64]: one TMA load brings a
+                                     // whole stage's k-blocks of an operand (needs K % 64 == 0); else 2-D, one per k-block
 #ifdef RLX_EXPERIMENTS
     int debug;                       // ablation switches of the experiments build (kDbg* bits)
     unsigned long long* trace;       // experiments build: 64 timestamp slots per CTA (or null)
@@ -679,25 +705,39 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 for (int kb = 0; kb < num_kb; kb += C::KPS) {
                     const int cnt = min(C::KPS, num_kb - kb);   // k-blocks in this stage
                     if (!mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
-                    const uint32_t st0 = base + stage * C::STAGE_BYTES;
+                    const uint32_t st0 = base + stage * C::STAGE_BYTES;   // [A k-blocks][W k-blocks]
+                    const uint32_t sb0 = st0 + C::KPS * C::A_BYTES;
                     if (elect_one()) {
+                        // 3-D maps: one load per operand brings all KPS k-blocks (a k-block past the end of K
+                        // arrives as zeros and still counts its bytes)
+                        const bool k3 = p.kblock_maps != 0;
+                        const int nbytes = k3 ? C::KPS * C::KB_BYTES : cnt * C::KB_BYTES;
                         if (RLX_DBG(p, kDbgNoLoad)) {
                             if (cta_rank == 0) mbar_arrive(full_bar + 8 * stage);
                         } else if constexpr (CG == 1) {
-                            mbar_expect_tx(full_bar + 8 * stage, cnt * C::KB_BYTES);
-                            for (int i = 0; i < cnt; ++i) {
-                                const uint32_t sa = st0 + i * C::KB_BYTES, sb = sa + C::A_BYTES;
-                                tma_load_2d(sa, &tmap_a, (kb + i) * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
-                                tma_load_2d(sb, &tmap_b, (kb + i) * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                            mbar_expect_tx(full_bar + 8 * stage, nbytes);
+                            if (k3) {
+                                tma_load_3d(st0, &tmap_a, 0, m_blk * BLOCK_M, kb, full_bar + 8 * stage);
+                                tma_load_3d(sb0, &tmap_b, 0, n_blk * BLOCK_N, kb, full_bar + 8 * stage);
+                            } else {
+                                for (int i = 0; i < cnt; ++i) {
+                                    tma_load_2d(st0 + i * C::A_BYTES, &tmap_a, (kb + i) * BLOCK_K, m_blk * BLOCK_M, full_bar + 8 * stage);
+                                    tma_load_2d(sb0 + i * C::B_BYTES, &tmap_b, (kb + i) * BLOCK_K, n_blk * BLOCK_N, full_bar + 8 * stage);
+                                }
                             }
                         } else {
                             // both CTAs' copies complete on the LEADER's full barrier, which expects all bytes
                             const uint32_t lead_full = map_to_cta(full_bar + 8 * stage, 0);
-                            if (cta_rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * cnt * C::KB_BYTES);
-                            for (int i = 0; i < cnt; ++i) {
-                                const uint32_t sa = st0 + i * C::KB_BYTES, sb = sa + C::A_BYTES;
-                                tma_load_2d_cg2(sa, &tmap_a, (kb + i) * BLOCK_K, m_blk * TILE_M + (int)cta_rank * BLOCK_M, lead_full);
-                                tma_load_2d_cg2(sb, &tmap_b, (kb + i) * BLOCK_K, n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS, lead_full);
+                            if (cta_rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * nbytes);
+                            const int arow = m_blk * TILE_M + (int)cta_rank * BLOCK_M, brow = n_blk * BLOCK_N + (int)cta_rank * C::B_ROWS;
+                            if (k3) {
+                                tma_load_3d_cg2(st0, &tmap_a, 0, arow, kb, lead_full);
+                                tma_load_3d_cg2(sb0, &tmap_b, 0, brow, kb, lead_full);
+                            } else {
+                                for (int i = 0; i < cnt; ++i) {
+                                    tma_load_2d_cg2(st0 + i * C::A_BYTES, &tmap_a, (kb + i) * BLOCK_K, arow, lead_full);
+                                    tma_load_2d_cg2(sb0 + i * C::B_BYTES, &tmap_b, (kb + i) * BLOCK_K, brow, lead_full);
+                                }
                             }
                         }
                         if (tile == tile0 && kb == 0) RLX_TRACE(p, 3);
@@ -738,8 +778,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                         if (it == 0 && kb == 0) RLX_TRACE(p, 5);
                         if (!RLX_DBG(p, kDbgNoMma)) {
                             for (int i = 0; i < cnt; ++i) {
-                                const uint64_t adesc = make_smem_desc(st0 + i * C::KB_BYTES);
-                                const uint64_t bdesc = make_smem_desc(st0 + i * C::KB_BYTES + C::A_BYTES);
+                                const uint64_t adesc = make_smem_desc(st0 + i * C::A_BYTES);
+                                const uint64_t bdesc = make_smem_desc(st0 + C::KPS * C::A_BYTES + i * C::B_BYTES);
 #pragma unroll
                                 for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                                     // advancing 16 bf16 = 32 bytes along K inside the swizzle row: +2 in 16-byte units

@@ -75,6 +75,33 @@ bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
     return r == CUDA_SUCCESS;
 }
 
+// The same matrix viewed as [k-block][row][64 columns] (cols % 64 == 0): a box of `kps` k-blocks x
+// box_rows rows lands in shared memory as kps complete 128-byte-swizzled operand tiles, one after the
+// other, so one TMA instruction feeds a whole multi-k-block pipeline stage.
+bool make_tmap_kblocks(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t kps) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn || cols % rlx::tc::BLOCK_K != 0) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)rlx::tc::BLOCK_K, rows, cols / rlx::tc::BLOCK_K};
+    cuuint64_t strides[2] = {cols * sizeof(bf16), rlx::tc::BLOCK_K * sizeof(bf16)};
+    cuuint32_t box[3] = {(cuuint32_t)rlx::tc::BLOCK_K, box_rows, kps};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Operand maps of a GEMM whose pipeline stages hold `kps` k-blocks: the k-block view when it exists
+// (K % 64 == 0, kps > 1), else the plain 2-D maps with one load per k-block.  Returns the kblock_maps flag.
+int make_operand_tmaps(CUtensorMap* ta, CUtensorMap* tb, const void* A, const void* W, uint64_t M, uint64_t N, uint64_t K,
+                       uint32_t a_rows, uint32_t b_rows, int kps) {
+    if (kps > 1 && K % rlx::tc::BLOCK_K == 0 && make_tmap_kblocks(ta, A, M, K, a_rows, (uint32_t)kps) &&
+        make_tmap_kblocks(tb, W, N, K, b_rows, (uint32_t)kps))
+        return 1;
+    if (!make_tmap(ta, A, M, K, a_rows) || !make_tmap(tb, W, N, K, b_rows)) return -1;
+    return 0;
+}
+
 // ------------------------------------------------------------------ one-time kernel attributes
 template <int BN, int EPI, int CG>
 cudaError_t set_gemm_attr() {
@@ -514,7 +541,6 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     p.trace = g_exp_trace;
 #endif
     CUtensorMap ta, tb, to;
-    if (!make_tmap(&ta, A, (uint64_t)M, (uint64_t)K, rlx::tc::BLOCK_M)) return RLX_ERR_CUDA;
     // output chunks: 32 x 32 bf16 boxes with the 64-byte swizzle of the epilogue's staging buffers
     if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
     // want_cg == 3: the A-resident CTA-pair kernel, forced; 0: chosen when the problem is large enough
@@ -522,7 +548,9 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
         const int rbn = pick_resident_bn(M, N, K, epi, want_cg == 3 || g_exp_resident > 0);
         if (rbn == 0 && want_cg == 3) return RLX_ERR_UNSUPPORTED;
         if (rbn != 0) {
-            if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(rbn / 2))) return RLX_ERR_CUDA;
+            p.kblock_maps = make_operand_tmaps(&ta, &tb, A, W, (uint64_t)M, (uint64_t)N, (uint64_t)K, rlx::tc::BLOCK_M,
+                                               (uint32_t)(rbn / 2), rlx::tcar::Cfg<128>::KPS);
+            if (p.kblock_maps < 0) return RLX_ERR_CUDA;
             switch (rbn) {
                 case 128: return launch_gemm_resident_bn<128>(ta, tb, to, p, epi, st);
                 case 192: return launch_gemm_resident_bn<192>(ta, tb, to, p, epi, st);
@@ -533,7 +561,19 @@ rlx_status_t launch_gemm(const bf16* A, const bf16* W, const float* bias, const 
     const TileChoice tc = pick_tile(M, N, K, want_cg);
     const int bn = tc.bn;
     if (bn == 0) return RLX_ERR_UNSUPPORTED;
-    if (!make_tmap(&tb, W, (uint64_t)N, (uint64_t)K, (uint32_t)(bn / tc.cg))) return RLX_ERR_CUDA;
+    int kps = 1;
+    switch (bn * 10 + tc.cg) {
+        case 641: kps = rlx::tc::Cfg<64, 1>::KPS; break;
+        case 1281: kps = rlx::tc::Cfg<128, 1>::KPS; break;
+        case 1921: kps = rlx::tc::Cfg<192, 1>::KPS; break;
+        case 2561: kps = rlx::tc::Cfg<256, 1>::KPS; break;
+        case 1282: kps = rlx::tc::Cfg<128, 2>::KPS; break;
+        case 1922: kps = rlx::tc::Cfg<192, 2>::KPS; break;
+        case 2562: kps = rlx::tc::Cfg<256, 2>::KPS; break;
+    }
+    p.kblock_maps = make_operand_tmaps(&ta, &tb, A, W, (uint64_t)M, (uint64_t)N, (uint64_t)K, rlx::tc::BLOCK_M,
+                                       (uint32_t)(bn / tc.cg), kps);
+    if (p.kblock_maps < 0) return RLX_ERR_CUDA;
     if (epi >= 3) {
         if (!lf || N % 32 != 0) return RLX_ERR_INVALID_ARG;
         p.cvec = lf->cvec; p.dvec = lf->dvec; p.stats_in = lf->stats_in; p.stats_in_p = lf->stats_in_p;
