@@ -125,7 +125,8 @@ typedef struct {
  * Returns RLX_ERR_INVALID_ARG for null/negative fields or a wrong struct_size,
  * RLX_ERR_UNSUPPORTED when H % 128 != 0, H > 1024, H % h != 0, head_dim not in
  * {32, 64}, F % 64 != 0, max_seq > max_pos, max_seq > 512 (the attention kernel's
- * per-sequence key table) or max_batch * max_seq > 2^30.
+ * per-sequence key table), max_batch > 65535 (one grid row per sequence) or
+ * max_batch * max_seq > 2^30.
  */
 rlx_status_t rlx_encoder_create(const rlx_encoder_config_t *config, rlx_encoder_t **out_encoder);
 
@@ -391,6 +392,18 @@ rlx_status_t rlx_attention_kind_bf16(const void *qkv_bf16, int32_t rows, const i
                                      int32_t num_heads, int32_t num_kv_heads, int32_t head_dim, int32_t mask_kind,
                                      int32_t window, const float *rope_cos, const float *rope_sin,
                                      void *ctx_bf16, void *cuda_stream);
+
+/*
+ * Tables for the rotary embedding of rlx_attention_kind_bf16 / rlx_qk_rope_bf16 (Section 3.2 names the
+ * fused QK-RoPE region; the angle convention is the one of the decoder families of the paper's model
+ * zoo): rope_cos[pos, j] = cos(pos * theta^(-2j/head_dim)), rope_sin likewise, for pos < max_len and
+ * j < head_dim/2.  Angles and functions are evaluated in fp64 on the device and stored as fp32.
+ * rope_cos / rope_sin: device fp32 [max_len, head_dim/2], 16-byte aligned, the caller's.  theta > 0
+ * (10000 in the usual models).  RLX_ERR_UNSUPPORTED for head sizes other than 32 / 64 / 128 or
+ * max_len > RLX_ATTENTION_KIND_MAX_LEN.  Asynchronous on cuda_stream.
+ */
+rlx_status_t rlx_rope_tables(int32_t max_len, int32_t head_dim, double theta, float *rope_cos, float *rope_sin,
+                             void *cuda_stream);
 
 /*
  * The fused QK-RoPE region of Section 3.2 on its own: rotates the q and the k column blocks of the

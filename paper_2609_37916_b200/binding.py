@@ -37,7 +37,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
 
 
@@ -298,13 +298,14 @@ MASK_NONE, MASK_CAUSAL, MASK_SLIDING_WINDOW = 0, 1, 2
 ATTENTION_KIND_MAX_LEN = 32768
 
 
-def rope_tables(max_len: int, head_dim: int, theta: float = 10000.0, device="cuda"):
-    """cos / sin of position * theta^(-2j/head_dim) as fp32 device tables [max_len, head_dim/2] (the
-    constant inputs rlx_attention_kind_bf16 takes; angles are formed in fp64 on the host)."""
-    j = torch.arange(head_dim // 2, dtype=torch.float64)
-    ang = torch.arange(max_len, dtype=torch.float64)[:, None] * torch.pow(torch.tensor(theta, dtype=torch.float64),
-                                                                         -2.0 * j / head_dim)[None, :]
-    return ang.cos().float().contiguous().to(device), ang.sin().float().contiguous().to(device)
+def rope_tables(max_len: int, head_dim: int, theta: float = 10000.0, device="cuda", stream=None):
+    """rlx_rope_tables: cos / sin of position * theta^(-2j/head_dim) as fp32 device tables
+    [max_len, head_dim/2] (the constant inputs rlx_attention_kind_bf16 takes), built by the library."""
+    cos = torch.empty((max_len, head_dim // 2), dtype=torch.float32, device=device)
+    sin = torch.empty_like(cos)
+    _check(_load().rlx_rope_tables(max_len, head_dim, C.c_double(theta), _ptr(cos), _ptr(sin), _stream(stream)),
+           "rlx_rope_tables")
+    return cos, sin
 
 
 def attention_kind_bf16(qkv, seq_start, seq_len, max_len: int, num_heads: int, mask_kind: int, window: int = 0,

@@ -1106,7 +1106,7 @@ rlx_status_t rlx_encoder_create(const rlx_encoder_config_t* c, rlx_encoder_t** o
     const int d = c->hidden / c->num_heads;
     if ((d != 32 && d != 64) || c->ffn % 64 != 0 || c->max_seq > c->max_pos || c->max_seq > 512)
         return RLX_ERR_UNSUPPORTED;
-    if ((long long)c->max_batch * c->max_seq > (1ll << 30)) return RLX_ERR_UNSUPPORTED;
+    if ((long long)c->max_batch * c->max_seq > (1ll << 30) || c->max_batch > 65535) return RLX_ERR_UNSUPPORTED;
     rlx_encoder* e = new (std::nothrow) rlx_encoder();
     if (!e) return RLX_ERR_INVALID_ARG;
     e->cfg = *c;
@@ -1387,6 +1387,18 @@ rlx_status_t rlx_qk_rope_bf16(void* qkv, int32_t rows, const int32_t* seq_start,
     else
         rlx::qk_rope_kernel<128><<<grid, rlx::kRopeThreads, 0, st>>>((bf16*)qkv, seq_start, seq_len, h + hkv, (h + 2 * hkv) * d,
                                                                      rope_cos, rope_sin);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t rlx_rope_tables(int32_t max_len, int32_t head_dim, double theta, float* rope_cos, float* rope_sin,
+                             void* stream) {
+    if (!rope_cos || !rope_sin || max_len <= 0 || !(theta > 0.0)) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(rope_cos) || !aligned16(rope_sin)) return RLX_ERR_INVALID_ARG;
+    if ((head_dim != 32 && head_dim != 64 && head_dim != 128) || max_len > RLX_ATTENTION_KIND_MAX_LEN) return RLX_ERR_UNSUPPORTED;
+    const long long n = (long long)max_len * (head_dim / 2);
+    rlx::rope_tables_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        rope_cos, rope_sin, max_len, head_dim / 2, theta);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }

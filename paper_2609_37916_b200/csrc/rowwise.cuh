@@ -213,6 +213,20 @@ qk_rope_kernel(__nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ seq_
     }
 }
 
+// cos / sin tables of the rotary embedding: entry [pos, j] = cos / sin(pos * theta^(-2j/D)), j < D/2.
+// The angle is formed in fp64 (position times an fp64 power) and the functions are evaluated in fp64,
+// so that the fp32 table entries are correctly rounded up to the last bit or so for every position.
+__global__ void __launch_bounds__(256)
+rope_tables_kernel(float* __restrict__ cos_tab, float* __restrict__ sin_tab, int max_len, int half_dim, double theta) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (long long)max_len * half_dim) return;
+    const int pos = (int)(i / half_dim), j = (int)(i % half_dim);
+    const double freq = pow(theta, -(double)j / (double)half_dim);   // theta^(-2j/D), D = 2 * half_dim
+    const double ang = (double)pos * freq;
+    cos_tab[i] = (float)cos(ang);
+    sin_tab[i] = (float)sin(ang);
+}
+
 // The same search done by a whole warp (p warp-uniform): every round samples 32 evenly spaced entries
 // of the remaining range and a ballot picks the sub-range, so 256 sequences take two dependent loads
 // instead of eight.
