@@ -700,11 +700,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = tile0; tile < num_tiles && ok; tile += tile_step) {
+            int pit = 0;
+            for (int tile = tile0; tile < num_tiles && ok; tile += tile_step, ++pit) {
                 const int m_blk = tile / n_tiles, n_blk = tile % n_tiles;
                 for (int kb = 0; kb < num_kb; kb += C::KPS) {
                     const int cnt = min(C::KPS, num_kb - kb);   // k-blocks in this stage
+                    if (pit == 2 && kb == 0 && lane == 0) RLX_TRACE_CLK(p, 58);   // about to wait for a free stage
                     if (!mbar_wait_warp(empty_bar + 8 * stage, phase ^ 1, abort_flag)) { ok = false; break; }
+                    if (pit == 2 && kb == 0 && lane == 0) RLX_TRACE_CLK(p, 59);   // stage free: loads issued now
                     const uint32_t st0 = base + stage * C::STAGE_BYTES;   // [A k-blocks][W k-blocks]
                     const uint32_t sb0 = st0 + C::KPS * C::A_BYTES;
                     if (elect_one()) {
@@ -770,8 +773,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                 for (int kb = 0; kb < num_kb; kb += C::KPS) {
                     const int cnt = min(C::KPS, num_kb - kb);
                     bool got_ops;
+                    if (it == 2 && kb == 0 && lane == 0) RLX_TRACE_CLK(p, 60);            // MMA thread starts waiting for that stage
                     RLX_CLK_ADD(clk_full, got_ops = mbar_wait_warp(full_bar + 8 * stage, phase, abort_flag));
                     if (!got_ops) { ok = false; break; }
+                    if (it == 2 && kb == 0 && lane == 0) RLX_TRACE_CLK(p, 61);            // operands landed
                     tc_fence_after();
                     const uint32_t st0 = base + stage * C::STAGE_BYTES;
                     if (elect_one()) {

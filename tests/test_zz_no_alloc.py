@@ -69,3 +69,35 @@ def test_static_arena_rejects_sizes_beyond_its_limit_and_flags_bad_ids(rlx):
     torch.cuda.synchronize()
     assert int(status.item()) == 0       # the status word does not leak from the previous call
     enc.close()
+
+
+def test_static_forward_allocates_nothing_and_leaves_kernel_times_alone(rlx):
+    """The static call on an encoder that records per-kernel events: device free memory does not move
+    across the call (cudaMemGetInfo before and after, both after a warm call so that lazily loaded
+    modules are in), the result is the ordinary entry point's bit for bit, and the per-kernel times
+    of the last instrumented forward stay as they were (the static path records no events)."""
+    inp = make_inputs(CONFIGS["c1"], batch=4, seq=64, num_layers=2, lengths=[64, 9, 33, 20])
+    B, S, H = inp.cfg.batch, inp.cfg.seq, inp.cfg.hidden
+    w = rlx.upload_weights(inp.params, inp.layers)
+    enc = rlx.Encoder.from_config(inp.cfg, max_batch=B, max_seq=S, flags=rlx.binding.FLAG_KERNEL_EVENTS)
+    ids, mask = i32_dev(inp.ids), i32_dev(inp.mask)
+    want = torch.empty((B, H), dtype=torch.float32, device="cuda")
+    got = torch.empty_like(want)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = enc.alloc_workspace(B, S)
+    enc.forward(ids, mask, w, want, ws)
+    torch.cuda.synchronize()
+    times = enc.kernel_times(B, S)
+    assert len(times) == enc.kernels_per_forward(B, S) and all(t > 0 for t in times)
+    enc.forward_static(ids, mask, w, got, device_status=status)      # warm call
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        enc.forward_static(ids, mask, w, got, device_status=status)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert int(status.item()) == 0
+    assert np.array_equal(to_np64(got), to_np64(want))
+    assert enc.kernel_times(B, S) == times
+    enc.close()
