@@ -217,9 +217,9 @@ cudaError_t init_kernels_for_current_device() {
         if (dev < 64) g_max_pairs_resident[dev] = n;
     }
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tca::Smem<32>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
+                                  rlx::tca::Smem<32>::BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tca::Smem<64>::bytes(rlx::tca::kMaxBlocks))) != cudaSuccess) return e;
+                                  rlx::tca::Smem<64>::BYTES)) != cudaSuccess) return e;
 #define RLX_ATT_SMEM_ATTR(D, MK, ROPE)                                                                       \
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<D, MK, ROPE>,                                  \
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(rlx::AttSmem<D>))) != \
@@ -373,23 +373,31 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     return RLX_OK;
 }
 
+__device__ unsigned int g_attn_ticket_standalone;   // work-item counter of rlx_attention_packed_bf16's own launches
+
 // Packed-sequence attention on tcgen05 (the product path): qkv is the packed [rows, 3H] projection.
 rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_start, const int32_t* seq_len, int B,
-                                 int S, int h, int d, bf16* ctx, int32_t* status, cudaStream_t st) {
+                                 int S, int h, int d, bf16* ctx, unsigned int* ticket, int32_t* status, cudaStream_t st) {
     const int H = h * d;
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)d);
     CUtensorMap tq;
     if (!make_tmap(&tq, qkv, (uint64_t)rows, (uint64_t)3 * H, rlx::tca::kBlockN, (uint32_t)d,
                    d == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B))
         return RLX_ERR_CUDA;
-    dim3 grid((S + rlx::tca::kBlockM - 1) / rlx::tca::kBlockM, h, B);
-    const int nblk = (S + rlx::tca::kBlockN - 1) / rlx::tca::kBlockN;   // K/V tiles held in shared memory
+    // persistent: two CTAs per SM walk the (sequence, query tile, head) list with a fixed stride
+    const int qtiles = (S + rlx::tca::kBlockM - 1) / rlx::tca::kBlockM;
+    const long long n_cand = (long long)B * qtiles * h;
+#ifdef RLX_ATTN_ONE_PER_SM
+    const int grid = (int)std::min<long long>(n_cand, 1LL * sm_count());
+#else
+    const int grid = (int)std::min<long long>(n_cand, 2LL * sm_count());
+#endif
     if (d == 32)
-        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, grid, rlx::tca::kThreads, rlx::tca::Smem<32>::bytes(nblk), st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status));
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<32>, dim3(grid), rlx::tca::kThreads, rlx::tca::Smem<32>::BYTES, st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, B, qtiles, ticket, status));
     else if (d == 64)
-        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, grid, rlx::tca::kThreads, rlx::tca::Smem<64>::bytes(nblk), st,
-                               tq, seq_start, seq_len, ctx, H, scale_log2e, nblk, status));
+        RLX_CUDA_TRY(launch_ex(rlx::tca::attention_tc_kernel<64>, dim3(grid), rlx::tca::kThreads, rlx::tca::Smem<64>::BYTES, st,
+                               tq, seq_start, seq_len, ctx, H, scale_log2e, B, qtiles, ticket, status));
     else
         return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(cudaGetLastError());
@@ -694,6 +702,7 @@ struct Arena {
     size_t stats_y, stats_z, fold, fold_layer, f_wqkv, f_w1, f_cqkv, f_dqkv, f_c1, f_d1;
 };
 constexpr size_t kTicketOffset = 64;   // packing ticket counter inside the 256-byte status block
+constexpr size_t kAttnTicketOffset = 128;   // work-item counter of the attention kernel, same block
 
 Arena plan_arena(int B, int S, int H, int F, int L = 0, bool fold = false) {
     const size_t T = (size_t)B * S;
@@ -872,8 +881,9 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
         int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
         int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
-        // the ticket must be zero when the packing kernel starts, whatever the workspace held before
-        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, sizeof(unsigned int), st));
+        // the tickets must be zero when their kernels start, whatever the workspace held before (each
+        // kernel leaves its own at zero again)
+        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, kAttnTicketOffset - kTicketOffset + sizeof(unsigned int), st));
         RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
                             reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
         pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
@@ -946,7 +956,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
                 RLX_TRY(launch_gemm(z, (const bf16*)(fb + a.f_wqkv), lw.bqkv, nullptr, 3, T, 3 * H, H, qkv, false, status, st, rows, 0, &lf));
             }
             if (pack && (c.flags & RLX_FLAG_ATTN_TCGEN05))
-                RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx, status, st));
+                RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx,
+                                            reinterpret_cast<unsigned int*>(ws + a.status + kAttnTicketOffset), status, st));
             else
                 RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
             // y = ctx Wo^T + bo + (l == 0 ? x : LN2_{l-1}(z)); partial statistics of y
@@ -985,7 +996,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         const rlx_layer_weights_t& lw = w->layers[l];
         RLX_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H, H, qkv, simt, status, st, rows));
         if (pack && (c.flags & RLX_FLAG_ATTN_TCGEN05))
-            RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx, status, st));
+            RLX_TRY(launch_attention_tc(qkv, T, pk.seq_start, pk.seq_len, B, S, h, d, ctx,
+                                            reinterpret_cast<unsigned int*>(ws + a.status + kAttnTicketOffset), status, st));
         else
             RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
         if (fuse_ln) {
@@ -1341,7 +1353,13 @@ rlx_status_t rlx_attention_packed_bf16(const void* qkv, int32_t rows, const int3
     RLX_CUDA_TRY(init_kernels_for_current_device());
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (impl == 0)
-        return launch_attention_tc((const bf16*)qkv, rows, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, status, st);
+        {
+        // the kernel-level call owns no workspace: its work-item counter is a word inside the library
+        // (zero between launches; calls on different streams of one device must therefore not overlap)
+        unsigned int* ticket = nullptr;
+        RLX_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&ticket), g_attn_ticket_standalone));
+        return launch_attention_tc((const bf16*)qkv, rows, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, ticket, status, st);
+    }
     if (impl == 1)
         return launch_attention_bf16((const bf16*)qkv, nullptr, seq_start, seq_len, B, max_len, h, d, (bf16*)ctx, st);
     return RLX_ERR_INVALID_ARG;

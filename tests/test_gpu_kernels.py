@@ -312,6 +312,43 @@ def test_attention_packed_matches_oracle(rlx, lengths, h, d, gain, impl):
     assert np.array_equal(got[total:], np.zeros((rows - total, H)))
 
 
+@pytest.mark.parametrize("impl", [0, 1], ids=["tcgen05", "mma_sync"])
+@pytest.mark.parametrize("trend", ["rising", "falling", "spike_last"])
+def test_attention_packed_row_maximum_moves_between_key_blocks(rlx, trend, impl):
+    """Logits whose level changes by far more than 2^8 from one 64-key block to the next: a running
+    maximum that is only corrected when it is exceeded by a margin has to take the correction path
+    (rising, spike in the last block) or live with probabilities that underflow (falling)."""
+    h, d = 2, 32
+    H = h * d
+    lengths = [300, 512, 70]
+    total = sum(lengths)
+    rng = np.random.default_rng(len(trend))
+    qkv = rand_bf16(rng, (total, 3 * H))
+    start = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int32)
+    for b, n in enumerate(lengths):
+        pos = np.arange(n)
+        blk = pos // 64
+        level = {"rising": blk * 14.0, "falling": -blk * 14.0,
+                 "spike_last": np.where(pos >= n - 3, 40.0, 0.0)}[trend]
+        # q = (1, 0, ...) * sqrt(d) makes the logit equal to k's first component
+        q = np.zeros((n, H), np.float32)
+        q[:, 0::d] = np.sqrt(d)
+        k = qkv[start[b]:start[b] + n, H:2 * H].copy()
+        k[:, 0::d] = round_to_bf16((level + rng.normal(size=n)).astype(np.float32))[:, None]
+        qkv[start[b]:start[b] + n, :H] = round_to_bf16(q)
+        qkv[start[b]:start[b] + n, H:2 * H] = k
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.attention_packed_bf16(bf16_dev(qkv), i32_dev(start[:-1]), i32_dev(np.array(lengths)),
+                                            max(lengths), h, impl=impl, status=status))
+    assert int(status.item()) == 0
+    vmax = np.abs(qkv[:, 2 * H:]).max()
+    for b, n in enumerate(lengths):
+        seq = qkv[start[b]:start[b] + n].astype(np.float64)[None]
+        ref = oracle.attention(seq, np.ones((1, n), np.int32), h)[0]
+        err = np.abs(got[start[b]:start[b] + n] - ref).max()
+        assert np.isfinite(err) and err <= 2 * BF16_U * (vmax + np.abs(ref).max()), (b, n, err)
+
+
 def test_attention_adversarial_logits(rlx):
     """One dominant key (+30), all-equal logits, and logits so negative that exp underflows."""
     h, d, S = 1, 32, 64
