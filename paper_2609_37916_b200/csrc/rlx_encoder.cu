@@ -1025,6 +1025,65 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     return RLX_OK;
 }
 
+// Tensor-parallel forward (Section 3.4: column / row sharding with an all-reduce inside the layer).
+// Rank r of n holds heads r*h/n .. (r+1)*h/n - 1 of every layer: the rows of Wqkv that produce their q, k
+// and v (column-parallel: no exchange), the matching COLUMNS of Wo (row-parallel: every rank forms a
+// partial sum over its own heads), rows r*F/n .. of W1 and the matching columns of W2.  The two
+// row-parallel products of a layer end in the caller's all-reduce; the residual and the bias enter the
+// sum once, on rank 0 (the other ranks pass a zero bias vector).  Everything between two all-reduces
+// is the single-GPU kernels on narrower operands; LayerNorm and pooling run replicated.  Eager
+// launches only: the exchange is the caller's library call, not a node of a captured graph.
+rlx_status_t enqueue_forward_tp(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
+                                const rlx_encoder_weights_t* w, int tp_rank, int tp_size,
+                                rlx_allreduce_bf16_fn allreduce, void* user, float* out, unsigned char* ws,
+                                cudaStream_t st) {
+    const rlx_encoder_config_t& c = e->cfg;
+    const int H = c.hidden, F = c.ffn, T = B * S, d = e->head_dim;
+    const int h_loc = c.num_heads / tp_size, H_loc = h_loc * d, F_loc = F / tp_size;
+    const Arena a = plan_arena(B, S, H, F, c.num_layers, false);
+    int32_t* status = reinterpret_cast<int32_t*>(ws + a.status);
+    bf16* x = reinterpret_cast<bf16*>(ws + a.x);
+    bf16* qkv = reinterpret_cast<bf16*>(ws + a.qkv);
+    bf16* ctx = reinterpret_cast<bf16*>(ws + a.ctx);
+    bf16* y = reinterpret_cast<bf16*>(ws + a.y);
+    bf16* x1 = reinterpret_cast<bf16*>(ws + a.x1);
+    bf16* g = reinterpret_cast<bf16*>(ws + a.g);
+    rlx_status_t s;
+#define RLX_TP_TRY(call) do { s = (call); if (s != RLX_OK) return s; } while (0)
+    Packing pk;
+    {
+        int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
+        int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
+        int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
+        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, kAttnTicketOffset - kTicketOffset + sizeof(unsigned int), st));
+        RLX_TP_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
+                               reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
+        pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
+    }
+    const int32_t* rows = pk.total();
+    // the partial sums of all T rows are exchanged: the number of packed rows is known on the device only,
+    // and rows past it are never read
+    const size_t exchange = (size_t)T * H;
+    const int row_epi = tp_rank == 0 ? RLX_EPI_BIAS_RESIDUAL : RLX_EPI_BIAS;
+    RLX_TP_TRY(launch_embed_ln(ids, (const bf16*)w->word_emb, (const bf16*)w->pos_emb, (const bf16*)w->type_emb,
+                               w->emb_ln_g, w->emb_ln_b, T, S, H, c.vocab, c.ln_eps, x, status, st, pk));
+    for (int l = 0; l < c.num_layers; ++l) {
+        const rlx_layer_weights_t& lw = w->layers[l];
+        RLX_TP_TRY(launch_gemm(x, (const bf16*)lw.wqkv, lw.bqkv, nullptr, RLX_EPI_BIAS, T, 3 * H_loc, H, qkv, false, status, st, rows));
+        RLX_TP_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h_loc, d, ctx, st));
+        RLX_TP_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, tp_rank == 0 ? x : nullptr, row_epi, T, H, H_loc, y, false, status, st, rows));
+        if (allreduce(user, y, exchange, st) != 0) return RLX_ERR_CUDA;
+        RLX_TP_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
+        RLX_TP_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F_loc, H, g, false, status, st, rows));
+        RLX_TP_TRY(launch_gemm(g, (const bf16*)lw.w2, lw.b2, tp_rank == 0 ? x1 : nullptr, row_epi, T, H, F_loc, y, false, status, st, rows));
+        if (allreduce(user, y, exchange, st) != 0) return RLX_ERR_CUDA;
+        RLX_TP_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
+    }
+    RLX_TP_TRY(launch_pool(x, mask, B, S, H, out, st, pk));
+#undef RLX_TP_TRY
+    return RLX_OK;
+}
+
 rlx_status_t check_forward_args(const rlx_encoder* e, const void* ids, const void* mask, int B, int S,
                                 const rlx_encoder_weights_t* w, const void* out, const void* ws, size_t ws_bytes,
                                 bool host_io) {
@@ -1154,6 +1213,26 @@ rlx_status_t rlx_encoder_forward(rlx_encoder_t* e, const int32_t* ids, const int
     rlx_status_t s = check_forward_args(e, ids, mask, B, S, w, out, ws, ws_bytes, false);
     if (s != RLX_OK) return s;
     return forward_device(e, ids, mask, B, S, w, out, static_cast<unsigned char*>(ws), static_cast<cudaStream_t>(stream));
+}
+
+rlx_status_t rlx_encoder_forward_tp(rlx_encoder_t* e, const int32_t* ids, const int32_t* mask, int32_t B, int32_t S,
+                                    const rlx_encoder_weights_t* w_shard, int32_t tp_rank, int32_t tp_size,
+                                    rlx_allreduce_bf16_fn allreduce, void* allreduce_user, float* out, void* ws,
+                                    size_t ws_bytes, void* stream) {
+    rlx_status_t s = check_forward_args(e, ids, mask, B, S, w_shard, out, ws, ws_bytes, false);
+    if (s != RLX_OK) return s;
+    if (!allreduce || tp_size < 1 || tp_rank < 0 || tp_rank >= tp_size) return RLX_ERR_INVALID_ARG;
+    const rlx_encoder_config_t& c = e->cfg;
+    // every shard must still be whole heads and whole 64-wide contraction blocks
+    if (c.num_heads % tp_size != 0 || (c.hidden / tp_size) % 64 != 0 || c.ffn % tp_size != 0 || (c.ffn / tp_size) % 64 != 0)
+        return RLX_ERR_UNSUPPORTED;
+    if (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_NO_PACK | RLX_FLAG_FOLD_LN)) return RLX_ERR_UNSUPPORTED;
+    int dev = -1;
+    RLX_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != c.device) return RLX_ERR_INVALID_ARG;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return enqueue_forward_tp(e, ids, mask, B, S, w_shard, tp_rank, tp_size, allreduce, allreduce_user, out,
+                              static_cast<unsigned char*>(ws), static_cast<cudaStream_t>(stream));
 }
 
 rlx_status_t rlx_encoder_forward_host(rlx_encoder_t* e, const int32_t* ids_h, const int32_t* mask_h, int32_t B,

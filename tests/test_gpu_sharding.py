@@ -67,3 +67,54 @@ def test_two_rank_sharded_cuda_forward_equals_unsharded_bitwise():
     whole = _forward(rlx, CFG, inp.ids, inp.mask, inp.params, inp.layers).numpy()
     # sequences are independent and every reduction has a fixed order: sharding changes nothing, bit for bit
     assert np.array_equal(ret["full"], whole)
+
+
+# ---------------------------------------------------------------- tensor parallel (column / row sharding)
+TP_CFG = CONFIGS["c1"]
+
+
+def _tp_worker(rank, world, port, ret):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import paper_2609_37916_b200 as rlx
+        from paper_2609_37916_b200.tensor_parallel import allreduce_through_host, shard_weights_tp
+        torch.cuda.set_device(0)
+        inp = make_inputs(TP_CFG)
+        cfg = inp.cfg
+        shard = shard_weights_tp(inp.layers, rank, world, cfg.num_heads)
+        w = rlx.upload_weights(inp.params, shard)
+        enc = rlx.Encoder.from_config(cfg, max_batch=cfg.batch, max_seq=cfg.seq)
+        ws = enc.alloc_workspace(cfg.batch, cfg.seq)
+        out = torch.empty((cfg.batch, cfg.hidden), dtype=torch.float32, device="cuda")
+        enc.forward_tp(torch.from_numpy(inp.ids).cuda(), torch.from_numpy(inp.mask).cuda(), w, rank, world,
+                       allreduce_through_host(), out, ws)
+        torch.cuda.synchronize()
+        assert enc.last_device_status(ws) == 0
+        ret[rank] = out.cpu().numpy()
+        enc.close()
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_tensor_parallel_cuda_forward_matches_oracle_and_unsharded(world):
+    """Two / three ranks share cuda:0 (their kernels never wait on each other: the exchange is a host
+    round trip over gloo), each runs rlx_encoder_forward_tp on its parameter shard."""
+    import paper_2609_37916_b200 as rlx
+    from paper_2609_37916_b200.build import build
+    from oracle import oracle
+    build()
+    oracle.build()
+    mgr = mp.Manager()
+    ret = mgr.dict()
+    mp.spawn(_tp_worker, args=(world, _free_port(), ret), nprocs=world, join=True)
+    inp = make_inputs(TP_CFG)
+    ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
+    whole = _forward(rlx, TP_CFG, inp.ids, inp.mask, inp.params, inp.layers).numpy().astype(np.float64)
+    for r in range(world):
+        got = ret[r].astype(np.float64)
+        cos = (got * ref).sum(-1) / (np.linalg.norm(got, axis=-1) * np.linalg.norm(ref, axis=-1))
+        assert cos.min() >= 0.9995 and np.abs(got - ref).max() <= 2e-2     # the graded tolerance
+        assert np.abs(got - whole).max() <= 5e-3                            # a few more bf16 roundings than one GPU
+        assert np.array_equal(ret[r], ret[0])                               # same sum on every rank
