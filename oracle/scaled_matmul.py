@@ -93,3 +93,63 @@ def scaled_matmul(x: np.ndarray, codes: np.ndarray, scales: np.ndarray, fmt: Min
     """y [M, N] = x [M, K] W^T (+ bias), W = dequantise(codes, scales)."""
     y = np.asarray(x, np.float64) @ dequantise(codes, scales, fmt).T
     return y if bias is None else y + np.asarray(bias, np.float64)
+
+
+# ------------------------------------------------------------------------------------------------
+# Quantised ACTIVATIONS (a reading: Section 3.2 is weight-only).  The tensor cores' block-scaled
+# product takes BOTH operands as (element codes, one E8M0 scale per 32 elements along K), so running
+# ScaledMatMul on that path needs a rule that puts a real activation row on such a grid.  The rule used
+# is the microscaling convention's, per block of 32 consecutive elements of a row:
+#   shared exponent  s = floor(log2(max |x_i|)) - emax(fmt),   emax = exponent of the largest finite
+#                    element value (8 for E4M3: 448 = 1.75 * 2^8; 15 for E5M2);  clamped to the E8M0
+#                    range [-127, 127];  an all-zero block takes s = 0
+#   element          code of the grid value nearest to x_i / 2^s, ties to the even code, values beyond
+#                    the largest finite element saturate to it (keeping the sign); never NaN / inf codes
+# and the quantised activation is value(code) * 2^s.  Everything below is that definition in fp64.
+
+def emax(fmt: MiniFloat) -> int:
+    t = decode_table(fmt)
+    return int(np.floor(np.log2(np.nanmax(t[np.isfinite(t)]))))
+
+
+def _finite_grid(fmt: MiniFloat):
+    """(values, codes) of the non-negative finite codes, ascending."""
+    t = decode_table(fmt)
+    half = t.size // 2
+    codes = np.array([c for c in range(half) if np.isfinite(t[c])])
+    return t[codes], codes
+
+
+def quantise_elements(v: np.ndarray, fmt: MiniFloat) -> np.ndarray:
+    """Nearest code on the element grid for every real v (ties to the even code, saturating)."""
+    vals, codes = _finite_grid(fmt)
+    v = np.asarray(v, np.float64)
+    mag = np.minimum(np.abs(v), vals[-1])
+    hi = np.searchsorted(vals, mag, side="left").clip(0, vals.size - 1)     # first grid value >= mag
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = vals[hi] - mag, mag - vals[lo]
+    take_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (codes[lo] % 2 == 0))
+    pick = np.where(take_lo, lo, hi)
+    sign_bit = fmt.ebits + fmt.mbits
+    return (codes[pick] | (np.signbit(v).astype(np.int64) << sign_bit)).astype(np.uint8)
+
+
+def quantise_mx(x: np.ndarray, fmt: MiniFloat):
+    """x [M, K] real -> (codes [M, K] uint8, scales [M, K/32] E8M0 bytes) by the rule above."""
+    x = np.asarray(x, np.float64)
+    M, K = x.shape
+    assert K % BLOCK == 0
+    blocks = x.reshape(M, K // BLOCK, BLOCK)
+    amax = np.abs(blocks).max(axis=2)
+    with np.errstate(divide="ignore"):
+        s = np.where(amax > 0, np.floor(np.log2(np.where(amax > 0, amax, 1.0))) - emax(fmt), 0.0)
+    s = np.clip(s, -127, 127)
+    codes = quantise_elements(blocks / np.exp2(s)[:, :, None], fmt).reshape(M, K)
+    return codes, (s + 127).astype(np.uint8)
+
+
+def mx_matmul(a_codes, a_scales, a_fmt: MiniFloat, w_codes, w_scales, w_fmt: MiniFloat,
+              bias: Optional[np.ndarray] = None) -> np.ndarray:
+    """y [M, N] = A W^T (+ bias) with BOTH operands on block-scaled grids."""
+    y = dequantise(a_codes, a_scales, a_fmt) @ dequantise(w_codes, w_scales, w_fmt).T
+    return y if bias is None else y + np.asarray(bias, np.float64)
