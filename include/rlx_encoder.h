@@ -485,6 +485,32 @@ rlx_status_t rlx_scaled_matmul_bf16(const void *A, const void *codes, const void
                                     int32_t M, int32_t N, int32_t K, void *w_scratch_bf16, void *out,
                                     int32_t *status, void *cuda_stream);
 
+/*
+ * ScaledMatMul on the tensor cores' own block-scaled path (tcgen05.mma kind::mxf8f6f4 with block
+ * scaling: the instruction takes 8-bit element codes for BOTH operands and applies the two E8M0 scales
+ * of every 32-wide k-group itself).  Section 3.2 quantises weights only; to use this path the
+ * activations have to be put on a block-scaled grid too, which is a reading, not the paper's method:
+ *   rlx_quantise_mx   x bf16 [M,K] -> codes [M,K] bytes + scales [M,K/32] E8M0 bytes by the microscaling
+ *                     rule: per block of 32 along K, shared exponent s = floor(log2 max|x|) - emax
+ *                     (emax = 8 for E4M3, 15 for E5M2; clamped to [-127,127]; 0 for an all-zero block),
+ *                     element = code nearest to x / 2^s, ties to the even code, saturating at the largest
+ *                     finite element; never a NaN or infinity code.  Bit-exact against that definition.
+ *   rlx_mx_matmul_bf16  out bf16 [M,N] = A W^T (+ bias), A given as (a_codes [M,K], a_scales [M,K/32]),
+ *                     W as (w_codes [N,K], w_scales [N,K/32]); products are exact, accumulation is the
+ *                     tensor core's fp32.  Scales of 255 (NaN) are the caller's responsibility.
+ * format: RLX_FMT_FP8_E4M3 or RLX_FMT_FP8_E5M2, chosen per operand (RLX_ERR_UNSUPPORTED otherwise: the
+ * 6- and 4-bit grids go through rlx_dequant_block_scaled_bf16).  rlx_mx_matmul_bf16 needs K % 128 == 0
+ * and N % 128 == 0 (RLX_ERR_UNSUPPORTED).  All pointers device, 16-byte aligned; bias f32 [N] or NULL;
+ * status: optional device word that receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.
+ * Asynchronous on cuda_stream; nothing is allocated.
+ */
+rlx_status_t rlx_quantise_mx(const void *x_bf16, int32_t M, int32_t K, int32_t format, void *codes,
+                             void *scales_e8m0, void *cuda_stream);
+rlx_status_t rlx_mx_matmul_bf16(const void *a_codes, const void *a_scales_e8m0, int32_t a_format,
+                                const void *w_codes, const void *w_scales_e8m0, int32_t w_format,
+                                const float *bias, int32_t M, int32_t N, int32_t K, void *out_bf16,
+                                int32_t *status, void *cuda_stream);
+
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
 rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,
                              int32_t seq, int32_t hidden, float *out, void *cuda_stream);

@@ -18,6 +18,8 @@ from .binding import (  # noqa: F401
     gemm_bf16,
     gemm_residual_layernorm_bf16,
     layernorm,
+    mx_matmul_bf16,
+    quantise_mx,
     pack_sequences,
     lib_path,
     pool_l2norm,

@@ -37,7 +37,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_tp", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_quantise_mx", "rlx_mx_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
 
 
@@ -402,6 +402,27 @@ def scaled_matmul_bf16(a, codes, scales, fmt: int, bias, residual=None, epilogue
     _check(_load().rlx_scaled_matmul_bf16(_ptr(a), _ptr(codes), _ptr(scales), fmt, _ptr(bias), _ptr(residual), epilogue,
                                           M, N, K, _ptr(w), _ptr(out), _ptr(status), _stream(stream)),
            "rlx_scaled_matmul_bf16")
+    return out
+
+
+def quantise_mx(x, fmt: int, stream=None):
+    """rlx_quantise_mx: x bf16 [M,K] -> (codes uint8 [M,K], scales uint8 [M,K/32])."""
+    M, K = x.shape
+    codes = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    scales = torch.empty((M, K // 32), dtype=torch.uint8, device=x.device)
+    _check(_load().rlx_quantise_mx(_ptr(x), M, K, fmt, _ptr(codes), _ptr(scales), _stream(stream)), "rlx_quantise_mx")
+    return codes, scales
+
+
+def mx_matmul_bf16(a_codes, a_scales, a_fmt: int, w_codes, w_scales, w_fmt: int, bias=None, out=None, status=None,
+                   stream=None):
+    """rlx_mx_matmul_bf16: out bf16 [M,N] = A W^T (+ bias), both operands block-scaled FP8."""
+    M, K = a_codes.shape
+    N = w_codes.shape[0]
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=a_codes.device) if out is None else out
+    _check(_load().rlx_mx_matmul_bf16(_ptr(a_codes), _ptr(a_scales), a_fmt, _ptr(w_codes), _ptr(w_scales), w_fmt,
+                                      _ptr(bias), M, N, K, _ptr(out), _ptr(status), _stream(stream)),
+           "rlx_mx_matmul_bf16")
     return out
 
 

@@ -13,6 +13,7 @@
 #include "../../include/rlx_encoder.h"
 #include "attention.cuh"
 #include "attention_tc.cuh"
+#include "gemm_mx_tcgen05.cuh"
 #include "dequant.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
@@ -71,6 +72,20 @@ bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// Row-major matrix of BYTES (8-bit element codes), 128-byte swizzle, box = box_rows x 128 bytes.
+bool make_tmap_u8(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -216,6 +231,8 @@ cudaError_t init_kernels_for_current_device() {
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tcar::gemm_ares_tcgen05_kernel<256, 0>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs_resident[dev] = n;
     }
+    if ((e = cudaFuncSetAttribute(rlx::tcmx::gemm_mx_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcmx::kSmemBytes)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tca::Smem<32>::BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1570,6 +1587,55 @@ rlx_status_t rlx_attention_f32(const float* qkv, const int32_t* mask, int32_t B,
         rlx::attention_f32_kernel<32><<<grid, rlx::kAttF32Warps * 32, 0, st>>>(qkv, mask, ctx, S, h * d, scale);
     else
         rlx::attention_f32_kernel<64><<<grid, rlx::kAttF32Warps * 32, 0, st>>>(qkv, mask, ctx, S, h * d, scale);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+// element format of the block-scaled tensor-core path: only the two 8-bit grids
+static int mx_element_format(int32_t format) {
+    if (format == RLX_FMT_FP8_E4M3) return rlx::tcmx::kFmtE4M3;
+    if (format == RLX_FMT_FP8_E5M2) return rlx::tcmx::kFmtE5M2;
+    return -1;
+}
+
+rlx_status_t rlx_quantise_mx(const void* x_bf16, int32_t M, int32_t K, int32_t format, void* codes, void* scales,
+                             void* stream) {
+    if (!x_bf16 || !codes || !scales || M <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(x_bf16) || !aligned16(codes)) return RLX_ERR_INVALID_ARG;
+    const int fmt = mx_element_format(format);
+    if (fmt < 0 || K % 32 != 0) return RLX_ERR_UNSUPPORTED;
+    const long long blocks = (long long)M * (K / 32);
+    const unsigned grid = (unsigned)((blocks + rlx::tcmx::kQuantThreads - 1) / rlx::tcmx::kQuantThreads);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (fmt == rlx::tcmx::kFmtE5M2)
+        rlx::tcmx::quantise_mx_kernel<true><<<grid, rlx::tcmx::kQuantThreads, 0, st>>>((const bf16*)x_bf16, (uint8_t*)codes, (uint8_t*)scales, blocks);
+    else
+        rlx::tcmx::quantise_mx_kernel<false><<<grid, rlx::tcmx::kQuantThreads, 0, st>>>((const bf16*)x_bf16, (uint8_t*)codes, (uint8_t*)scales, blocks);
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+rlx_status_t rlx_mx_matmul_bf16(const void* a_codes, const void* a_scales, int32_t a_format, const void* w_codes,
+                                const void* w_scales, int32_t w_format, const float* bias, int32_t M, int32_t N,
+                                int32_t K, void* out, int32_t* status, void* stream) {
+    if (!a_codes || !a_scales || !w_codes || !w_scales || !out || M <= 0 || N <= 0 || K <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(a_codes) || !aligned16(w_codes) || !aligned16(a_scales) || !aligned16(w_scales) || !aligned16(out) ||
+        (bias && !aligned16(bias)))
+        return RLX_ERR_INVALID_ARG;
+    const int af = mx_element_format(a_format), wf = mx_element_format(w_format);
+    if (af < 0 || wf < 0 || K % rlx::tcmx::kBlockK != 0 || N % rlx::tcmx::kTileN != 0) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    CUtensorMap ta, tw;
+    if (!make_tmap_u8(&ta, a_codes, (uint64_t)M, (uint64_t)K, rlx::tcmx::kTileM) ||
+        !make_tmap_u8(&tw, w_codes, (uint64_t)N, (uint64_t)K, rlx::tcmx::kTileN))
+        return RLX_ERR_CUDA;
+    rlx::tcmx::MxParams p;
+    p.sfa = (const uint8_t*)a_scales; p.sfw = (const uint8_t*)w_scales; p.bias = bias; p.out = (bf16*)out;
+    p.M = M; p.N = N; p.K = K; p.a_fmt = af; p.w_fmt = wf; p.status = status;
+    const long long tiles = (long long)((M + rlx::tcmx::kTileM - 1) / rlx::tcmx::kTileM) * (N / rlx::tcmx::kTileN);
+    if (tiles > 0x7fffffffLL) return RLX_ERR_UNSUPPORTED;
+    rlx::tcmx::gemm_mx_tcgen05_kernel<<<(unsigned)tiles, rlx::tcmx::kThreads, rlx::tcmx::kSmemBytes,
+                                        static_cast<cudaStream_t>(stream)>>>(ta, tw, p);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }

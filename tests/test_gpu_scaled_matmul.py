@@ -122,3 +122,110 @@ def test_scaled_matmul_is_bit_exact_when_sums_are_exact(rlx):
                                  _fmt_word(rlx, "fp4_e2m1"), f32_dev(zero))
     ref = osm.scaled_matmul(x.astype(np.float64), codes, scales, f)
     _assert_same_bits(got, round_to_bf16(ref.astype(np.float32)))
+
+
+# ---------------------------------------------------------------- block-scaled tensor-core path (both operands FP8)
+MX_FORMATS = {"fp8_e4m3": osm.E4M3, "fp8_e5m2": osm.E5M2}
+
+
+def _mx_word(rlx, name):
+    f = MX_FORMATS[name]
+    return rlx.binding.minifloat(f.ebits, f.mbits, SPECIAL[f.special], False)
+
+
+def _u8_dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.uint8)).cuda()
+
+
+@pytest.mark.parametrize("name", sorted(MX_FORMATS))
+def test_quantise_mx_is_bit_exact_against_the_definition(rlx, name):
+    """Codes and scale bytes are integer decisions: every one must equal the oracle's (the inputs are bf16,
+    the scaling is by exact powers of two, and the rounding rule is round-to-nearest-even on both sides)."""
+    fmt = MX_FORMATS[name]
+    rng = np.random.default_rng(5)
+    M, K = 77, 384
+    x = rng.standard_normal((M, K)).astype(np.float32) * np.exp2(rng.integers(-30, 30, size=(M, K // 32))).repeat(32, axis=1).astype(np.float32)
+    x[3, 64:96] = 0.0                                      # all-zero block
+    x[5, 0] = 3.0e38                                       # top of the range: shared exponent clamps at 127
+    x[6, :32] = 1e-38                                      # bottom: bf16 subnormal neighbourhood
+    x[7, :32] = np.linspace(0.9, 1.1, 32) * 256.0          # block maximum just past a binade edge
+    x[8, :32] = 255.0
+    x[8, 5] = 256.0
+    # every tie of the element grid: midpoints between neighbouring E4M3 / E5M2 values, block maximum 256 or 2^15
+    t = osm.decode_table(fmt)
+    pos = np.sort(t[: t.size // 2][np.isfinite(t[: t.size // 2])])
+    mids = (pos[:-1] + pos[1:]) / 2
+    top = 2.0 ** osm.emax(fmt)
+    for r, chunk in enumerate(np.array_split(mids, 8)):
+        row = np.zeros(K, np.float32)
+        row[:32] = top
+        row[32:32 + chunk.size] = chunk[:K - 32]
+        row[0] = top
+        for b in range(1, K // 32):
+            row[b * 32] = top                               # shared exponent 0 in every block
+        x[10 + r] = row
+    x = round_to_bf16(x)
+    codes, scales = rlx.quantise_mx(bf16_dev(x), _mx_word(rlx, name))
+    want_codes, want_scales = osm.quantise_mx(x.astype(np.float64), fmt)
+    assert np.array_equal(scales.cpu().numpy(), want_scales)
+    assert np.array_equal(codes.cpu().numpy(), want_codes)
+
+
+def test_mx_matmul_places_every_scale_byte_and_operand_where_the_definition_says(rlx):
+    """Exact cases that fail if a scale byte reaches the wrong row, column or k-group, or an operand tile is
+    transposed: all elements 1.0 with a different power-of-two scale per (row, k-group) and per (column,
+    k-group); then integer-valued elements with unit scales (integer arithmetic, exact in fp32)."""
+    M, N, K = 300, 256, 1024          # ragged rows, two column tiles, 8 stages of k: every ring wraps
+    rng = np.random.default_rng(6)
+    one = 0x38                          # 1.0 in E4M3
+    a_codes = np.full((M, K), one, np.uint8)
+    w_codes = np.full((N, K), one, np.uint8)
+    a_scales = (127 + rng.integers(-3, 4, size=(M, K // 32))).astype(np.uint8)
+    w_scales = (127 + rng.integers(-3, 4, size=(N, K // 32))).astype(np.uint8)
+    word = _mx_word(rlx, "fp8_e4m3")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.mx_matmul_bf16(_u8_dev(a_codes), _u8_dev(a_scales), word, _u8_dev(w_codes), _u8_dev(w_scales), word,
+                                     status=status))
+    assert int(status.item()) == 0
+    want = osm.mx_matmul(a_codes, a_scales, osm.E4M3, w_codes, w_scales, osm.E4M3)
+    assert np.array_equal(got, round_to_bf16(want.astype(np.float32)).astype(np.float64))   # sums of 32 * 2^e: exact
+    # integers in [-4, 4] (E4M3 holds them exactly), unit scales: |sum| <= 16 * 1024, exact in fp32; bf16 rounds once
+    ai = rng.integers(-4, 5, size=(M, K))
+    wi = rng.integers(-4, 5, size=(N, K))
+    ac = osm.quantise_elements(ai.astype(np.float64), osm.E4M3)
+    wc = osm.quantise_elements(wi.astype(np.float64), osm.E4M3)
+    ones = np.full((M, K // 32), 127, np.uint8)
+    bias = rng.integers(-8, 9, size=N).astype(np.float32)
+    got = to_np64(rlx.mx_matmul_bf16(_u8_dev(ac), _u8_dev(ones), word, _u8_dev(wc), _u8_dev(ones[:N]), word,
+                                     bias=f32_dev(bias)))
+    exact = (ai @ wi.T + bias).astype(np.float32)
+    assert np.array_equal(got, round_to_bf16(exact).astype(np.float64))
+
+
+@pytest.mark.parametrize("a_name,w_name", [("fp8_e4m3", "fp8_e4m3"), ("fp8_e4m3", "fp8_e5m2"), ("fp8_e5m2", "fp8_e4m3")])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (517, 384, 384), (2000, 1536, 384), (1000, 384, 1536)])
+def test_quantise_then_mx_matmul_matches_oracle(rlx, a_name, w_name, M, N, K):
+    """The whole path on encoder-shaped operands: activations quantised on the GPU (bit-exact, previous test),
+    weights quantised by the oracle's rule on the host, product on the block-scaled tensor-core path,
+    compared with the fp64 product of the two dequantised operands.  Products are exact; the error is fp32
+    accumulation (K terms, relative 2^-24 each against the sum of magnitudes) plus the bf16 store."""
+    rng = np.random.default_rng(M + N + K)
+    x = rand_bf16(rng, (M, K))
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    a_codes, a_scales = rlx.quantise_mx(bf16_dev(x), _mx_word(rlx, a_name))
+    w_codes, w_scales = osm.quantise_mx(w.astype(np.float64), MX_FORMATS[w_name])
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.mx_matmul_bf16(a_codes, a_scales, _mx_word(rlx, a_name), _u8_dev(w_codes), _u8_dev(w_scales),
+                                     _mx_word(rlx, w_name), bias=f32_dev(bias), status=status))
+    assert int(status.item()) == 0
+    A = osm.dequantise(a_codes.cpu().numpy(), a_scales.cpu().numpy(), MX_FORMATS[a_name])
+    W = osm.dequantise(w_codes, w_scales, MX_FORMATS[w_name])
+    ref = A @ W.T + bias
+    mag = np.abs(A) @ np.abs(W).T + np.abs(bias)
+    half_ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(ref), 1e-300))) - 8)     # bf16: 8 significant bits
+    assert np.all(np.abs(got - ref) <= half_ulp + K * 2.0 ** -23 * mag + 1e-30)
+    # and the quantised product stays close to the unquantised one: the point of the format
+    full = x.astype(np.float64) @ w.astype(np.float64).T + bias
+    rel = np.linalg.norm(got - full) / np.linalg.norm(full)
+    assert rel < (0.04 if "e5m2" not in (a_name + w_name) else 0.08)
