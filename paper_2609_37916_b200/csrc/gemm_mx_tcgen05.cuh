@@ -22,7 +22,9 @@
 //                      warps writes the same 32 x 4 words into its own quarter with one tcgen05.st (and the
 //                      same again for the 128 columns of W).  After the last stage the same warps read the
 //                      fp32 accumulator (thread = row), add the bias, round to bf16 and store.
-//  TMEM: 128 accumulator columns + 4 scale slots of 8 columns = 160 -> 256 allocated, two CTAs per SM,
+//  One mbarrier per stage collects the TMA bytes AND the four scale warps' arrivals, and one commit per
+//  stage frees operands and scale slot together: the issuing thread pays for every barrier round.
+//  TMEM: 128 accumulator columns + 3 scale slots of 8 columns = 152 -> 256 allocated, two CTAs per SM,
 //  which is what overlaps one tile's epilogue with another's main loop.
 // All mbarrier waits are bounded; on expiry the CTA sets the status bit and leaves.
 #pragma once
@@ -39,9 +41,8 @@ constexpr int kThreads = 192;
 constexpr int kTileM = 128, kTileN = 128;
 constexpr int kBlockK = 128;            // 8-bit elements per stage row = 128 bytes = one swizzle row
 constexpr int kStages = 3;              // 3 x 32 KB: two CTAs fit an SM
-constexpr int kSfSlots = 4;
 constexpr int kTmemCols = 256;
-constexpr int kColSf = kTileN;          // scale slots behind the accumulator
+constexpr int kColSf = kTileN;          // one scale slot (8 columns) per stage, behind the accumulator
 constexpr int kOperandBytes = kTileM * kBlockK;
 constexpr int kSmemBytes = kStages * 2 * kOperandBytes + 256 + 1024;
 
@@ -87,9 +88,8 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* gbase = smem_raw + (base - raw);
     const uint32_t bars = base + kStages * 2 * kOperandBytes;
-    const uint32_t full = bars, empty = full + 8 * kStages, sf_full = empty + 8 * kStages, sf_empty = sf_full + 8 * kSfSlots;
-    const uint32_t acc_full = sf_empty + 8 * kSfSlots;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + kStages * 2 * kOperandBytes + 8 * (2 * kStages + 2 * kSfSlots + 1));
+    const uint32_t full = bars, empty = full + 8 * kStages, acc_full = empty + 8 * kStages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + kStages * 2 * kOperandBytes + 8 * (2 * kStages + 1));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -99,8 +99,8 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     const int sf_ld = p.K / 32;   // scale bytes per row
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }
-        for (int i = 0; i < kSfSlots; ++i) { mbar_init(sf_full + 8 * i, 4); mbar_init(sf_empty + 8 * i, 1); }
+        // full: the TMA lane's expect_tx arrival + one arrival per scale warp
+        for (int i = 0; i < kStages; ++i) { mbar_init(full + 8 * i, 5); mbar_init(empty + 8 * i, 1); }
         mbar_init(acc_full, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -128,23 +128,23 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int st = kb % kStages, slot = kb % kSfSlots;
-                if (!(ok = mbar_wait(full + 8 * st, (kb / kStages) & 1, abort_flag))) break;
-                if (!(ok = mbar_wait(sf_full + 8 * slot, (kb / kSfSlots) & 1, abort_flag))) break;
-                tc_fence_after();
+        // warp-uniform loop, one elected lane issues (cheaper per instruction than a lone lane under a branch)
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int st = kb % kStages;
+            if (!(ok = mbar_wait_warp(full + 8 * st, (kb / kStages) & 1, abort_flag))) break;
+            tc_fence_after();
+            if (elect_one()) {
                 const uint64_t adesc = make_smem_desc(base + st * 2 * kOperandBytes);
                 const uint64_t bdesc = make_smem_desc(base + st * 2 * kOperandBytes + kOperandBytes);
-                const uint32_t sfa = tmem + kColSf + slot * 8, sfb = sfa + 4;
+                const uint32_t sfa = tmem + kColSf + st * 8, sfb = sfa + 4;
 #pragma unroll
                 for (int k = 0; k < kBlockK / 32; ++k)   // 32 bytes of k per instruction: descriptor start + 2
                     umma_mx(tmem, adesc + 2 * k, bdesc + 2 * k, idesc_mx(p.a_fmt, p.w_fmt, k), sfa, sfb, (kb | k) != 0 ? 1u : 0u);
                 umma_commit<1>(empty + 8 * st);
-                umma_commit<1>(sf_empty + 8 * slot);
+                if (kb == nkb - 1) umma_commit<1>(acc_full);
             }
-            if (ok) umma_commit<1>(acc_full);
+            __syncwarp();
         }
     } else {
         // ------------------------------------------------------------ scale feed, then epilogue
@@ -152,7 +152,7 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int slot = kb % kSfSlots, use = kb / kSfSlots;
+            const int slot = kb % kStages, use = kb / kStages;
             uint32_t w[8];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -161,13 +161,13 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
                 w[c] = ar < p.M ? __ldg(reinterpret_cast<const uint32_t*>(p.sfa + (size_t)ar * sf_ld) + kb) : 0x7F7F7F7Fu;
                 w[4 + c] = __ldg(reinterpret_cast<const uint32_t*>(p.sfw + (size_t)wr * sf_ld) + kb);
             }
-            if (use >= 1 && !(ok = mbar_wait(sf_empty + 8 * slot, (use - 1) & 1, abort_flag))) break;
+            if (use >= 1 && !(ok = mbar_wait(empty + 8 * slot, (use - 1) & 1, abort_flag))) break;
             tc_fence_after();
             tmem_st_32x8(lane_addr + kColSf + slot * 8, w);
             tmem_st_wait_all();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(sf_full + 8 * slot);
+            if (lane == 0) mbar_arrive(full + 8 * slot);
         }
         if (ok && (ok = mbar_wait(acc_full, 0, abort_flag))) {
             tc_fence_after();
