@@ -159,7 +159,9 @@ size_t rlx_encoder_workspace_bytes(const rlx_encoder_t *encoder, int32_t batch, 
  * out             dev f32 [batch, H]; a sequence with no valid position yields zeros
  * workspace       dev, 256-byte aligned, >= rlx_encoder_workspace_bytes(batch, seq);
  *                 scratch: contents are overwritten by every call.  Its first 256 bytes hold the
- *                 sticky device status word: zero them once before the first call
+ *                 sticky device status word and two work counters that every forward leaves at
+ *                 zero: zero these 256 bytes once before the first call, and again after a call
+ *                 that reported RLX_ERR_DEVICE_TIMEOUT (a forward that gave up may leave a counter set)
  *
  * config->device must be the current CUDA device (RLX_ERR_INVALID_ARG otherwise).
  * Asynchronous on cuda_stream.  Unless RLX_FLAG_NO_GRAPH is set the kernel

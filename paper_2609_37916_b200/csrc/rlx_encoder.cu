@@ -898,9 +898,8 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
         int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
         int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
-        // the tickets must be zero when their kernels start, whatever the workspace held before (each
-        // kernel leaves its own at zero again)
-        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, kAttnTicketOffset - kTicketOffset + sizeof(unsigned int), st));
+        // The tickets live in the status block, which the caller zeroes once before the first call; each
+        // kernel leaves its own at zero again, so no memset node sits in front of the first kernel.
         RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
                             reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
         pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
@@ -1072,7 +1071,6 @@ rlx_status_t enqueue_forward_tp(const rlx_encoder* e, const int32_t* ids, const 
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
         int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
         int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
-        RLX_CUDA_TRY(cudaMemsetAsync(ws + a.status + kTicketOffset, 0, kAttnTicketOffset - kTicketOffset + sizeof(unsigned int), st));
         RLX_TP_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
                                reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
         pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
