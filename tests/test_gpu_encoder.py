@@ -100,6 +100,39 @@ def test_large_config_sampled_sequences_match_oracle(rlx, name, sample, flags):
     check(got[sample], ref, inp.lengths[sample])
 
 
+def test_host_call_pinned_and_pageable_buffers_and_new_contents_between_calls(rlx):
+    """rlx_encoder_forward_host with pinned and with pageable host buffers: both give the device call's
+    bits, and a second call on the same buffers (the cached graph is replayed) reads what they hold at
+    that moment."""
+    a = make_inputs(CONFIGS["c1"], num_layers=2)
+    c = a.cfg
+    w = rlx.upload_weights(a.params, a.layers)
+    enc = rlx.Encoder.from_config(c, max_batch=c.batch, max_seq=c.seq)
+    ws = enc.alloc_workspace(c.batch, c.seq)
+    want = torch.empty((c.batch, c.hidden), dtype=torch.float32, device="cuda")
+
+    def device_result(ids, mask):
+        enc.forward(i32_dev(ids), i32_dev(mask), w, want, ws)
+        torch.cuda.synchronize()
+        return want.cpu().numpy().copy()
+
+    second_ids, second_mask = a.ids[::-1].copy(), a.mask[::-1].copy()   # the batch in reverse order
+    for pinned in (True, False):
+        ids = torch.from_numpy(a.ids.copy())
+        mask = torch.from_numpy(a.mask.copy())
+        out = torch.empty((c.batch, c.hidden), dtype=torch.float32)
+        if pinned:
+            ids, mask, out = ids.pin_memory(), mask.pin_memory(), out.pin_memory()
+        enc.forward_host(ids, mask, w, out, ws)
+        assert np.array_equal(out.numpy(), device_result(a.ids, a.mask))
+        ids.copy_(torch.from_numpy(second_ids))       # same buffers, new contents: the cached graph is replayed
+        mask.copy_(torch.from_numpy(second_mask))
+        enc.forward_host(ids, mask, w, out, ws)
+        assert np.array_equal(out.numpy(), device_result(second_ids, second_mask))
+    assert enc.last_device_status(ws) == 0
+    enc.close()
+
+
 @pytest.mark.parametrize("name", ["c3", "c4"])
 def test_large_config_every_sequence_matches_oracle(rlx, name):
     """The two large configurations in the benchmark's launch configuration, EVERY sequence compared
