@@ -74,7 +74,10 @@ typedef enum {
                                    rlx_encoder_workspace_bytes).  Ignored with RLX_FLAG_GEMM_SIMT, when hidden is
                                    not a multiple of 32 or max_seq exceeds 512; takes precedence over
                                    RLX_FLAG_FUSED_LN / RLX_FLAG_CLUSTER_LN.  Pays for small batches (launch-bound
-                                   forwards); for large ones the separate LayerNorm kernels are faster */
+                                   forwards); for large ones the separate LayerNorm kernels are faster.  Chosen
+                                   AUTOMATICALLY for calls with batch*seq <= 4096 unless one of the other two
+                                   fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
+#define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */

@@ -62,13 +62,13 @@ def check(got, ref, lengths, tight=True):
 
 
 @pytest.mark.parametrize("name", ["c0", "c1", "c2"])
-@pytest.mark.parametrize("mode", ["graph", "eager", "padded", "attn_tcgen05", "cluster_ln", "fold_ln", "fold_ln_eager",
-                                  "fold_ln_padded", "simt_gemm", "host_io"])
+@pytest.mark.parametrize("mode", ["graph", "eager", "padded", "separate_ln", "separate_ln_eager", "attn_tcgen05", "cluster_ln",
+                                  "fold_ln", "fold_ln_eager", "fold_ln_padded", "simt_gemm", "host_io"])
 def test_full_config_matches_oracle(rlx, name, mode):
     if mode == "simt_gemm" and name == "c2":
         pytest.skip("bring-up GEMM is covered on c0/c1")
     inp = make_inputs(CONFIGS[name])
-    flags = {"graph": 0, "eager": 1, "padded": 8, "attn_tcgen05": 0x20, "cluster_ln": 0x80, "fold_ln": 0x200,
+    flags = {"graph": 0, "eager": 1, "padded": 8, "separate_ln": 0x400, "separate_ln_eager": 0x401, "attn_tcgen05": 0x20, "cluster_ln": 0x80, "fold_ln": 0x200,
              "fold_ln_eager": 0x201, "fold_ln_padded": 0x208, "simt_gemm": 1 | 2, "host_io": 0}[mode]
     got, status = run_gpu(rlx, inp, flags=flags, host_io=(mode == "host_io"))
     assert status == 0
@@ -83,7 +83,7 @@ def test_c0_matches_stored_golden(rlx):
     check(got, want.reshape(1, -1), inp.lengths)
 
 
-@pytest.mark.parametrize("flags", [0, 0x20, 0x40, 0x80, 0x200], ids=["default", "attn_tcgen05", "whole_row_ln", "cluster_ln", "fold_ln"])
+@pytest.mark.parametrize("flags", [0, 0x400, 0x20, 0x40, 0x80, 0x200], ids=["default", "separate_ln", "attn_tcgen05", "whole_row_ln", "cluster_ln", "fold_ln"])
 @pytest.mark.parametrize("name,sample", [("c3", [0, 1, 100, 255]), ("c4", [0, 63])])
 def test_large_config_sampled_sequences_match_oracle(rlx, name, sample, flags):
     """Full-size run in the benchmark's launch configuration; the oracle recomputes a sample of the
@@ -205,7 +205,7 @@ def test_random_small_problems_match_oracle(rlx, seed):
     assert status == 0
     check(base, ref, inp.lengths, tight=(seed % 4 != 0))
     assert np.array_equal(base[inp.lengths == 0], np.zeros_like(base[inp.lengths == 0]))
-    for flags in (0x10, 0x100, 1, 0x20, 0x80, 8, 0x200, 0x201):   # no PDL, no prefetch, eager, tcgen05 attn, cluster LN, padded, folded LN (graph / eager)
+    for flags in (0x10, 0x100, 1, 0x400, 0x401, 0x420, 0x20, 0x80, 8, 0x408, 0x200, 0x201):   # no PDL, no prefetch, eager, tcgen05 attn, cluster LN, padded, folded LN (graph / eager)
         other, status = run_gpu(rlx, inp, weights=w, flags=flags)
         assert status == 0
         if flags in (0x10, 0x100, 1):
