@@ -78,6 +78,12 @@ typedef enum {
                                    AUTOMATICALLY for calls with batch*seq <= 4096 unless one of the other two
                                    fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
 #define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
+#define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
+                                   about that size, one after the other through the same workspace, so that every
+                                   kernel's input is still in L2 when its consumer starts.  Results are bit for bit
+                                   those of the unchunked call; rlx_encoder_kernels_per_forward still reports the
+                                   kernels of ONE sub-batch.  Ignored with RLX_FLAG_KERNEL_EVENTS, for a single
+                                   sequence, or when seq is not a multiple of 4 */
 
 typedef struct {
     uint32_t struct_size; /* sizeof(rlx_encoder_config_t), for versioning */

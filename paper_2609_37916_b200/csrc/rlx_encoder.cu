@@ -804,6 +804,8 @@ int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool fused = uses_fold_ln(c, B, S) || uses_fused_ln(c, B, S) || uses_cluster_ln(c);
     return 2 + (fused ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
 }
+bool uses_chunks(const rlx_encoder_config_t& c, int B, int S);
+int chunk_batch(int B, int S);
 
 struct GraphEntry {
     int B, S;
@@ -1056,6 +1058,33 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     return RLX_OK;
 }
 
+// Token-chunk scheduling (RLX_FLAG_CHUNKED): sequences are independent, so a large batch can run as
+// several sub-batches one after the other through the SAME workspace, each small enough that a kernel's
+// input is still in the 126 MB L2 when its consumer starts.  Same kernels on fewer rows: the result is bit
+// for bit the unchunked one.  The price is launches (chunks x kernels per forward) and shorter grids.
+constexpr long long kChunkTokens = 16384;   // padded tokens per sub-batch
+bool uses_chunks(const rlx_encoder_config_t& c, int B, int S) {
+    return (c.flags & RLX_FLAG_CHUNKED) && !(c.flags & RLX_FLAG_KERNEL_EVENTS) && S % 4 == 0 &&
+           (long long)B * S > kChunkTokens && B > 1;
+}
+int chunk_batch(int B, int S) {
+    const long long n_chunks = ((long long)B * S + kChunkTokens - 1) / kChunkTokens;
+    return (int)((B + n_chunks - 1) / n_chunks);
+}
+rlx_status_t enqueue_forward_any(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
+                                 const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st,
+                                 bool capturing, bool with_events = true) {
+    if (!uses_chunks(e->cfg, B, S)) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, capturing, with_events);
+    const int bc = chunk_batch(B, S);
+    for (int b0 = 0; b0 < B; b0 += bc) {
+        const int nb = std::min(bc, B - b0);
+        rlx_status_t s = enqueue_forward(e, ids + (size_t)b0 * S, mask + (size_t)b0 * S, nb, S, w,
+                                         out + (size_t)b0 * e->cfg.hidden, ws, st, capturing, false);
+        if (s != RLX_OK) return s;
+    }
+    return RLX_OK;
+}
+
 // Tensor-parallel forward (Section 3.4: column / row sharding with an all-reduce inside the layer).
 // Rank r of n holds heads r*h/n .. (r+1)*h/n - 1 of every layer: the rows of Wqkv that produce their q, k
 // and v (column-parallel: no exchange), the matching COLUMNS of Wo (row-parallel: every rank forms a
@@ -1147,7 +1176,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
         for (auto& evt : e->events) RLX_CUDA_TRY(cudaEventCreate(&evt));
     }
     e->last_kernels = kernels_in_forward(e->cfg, B, S);
-    if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, false);
+    if (e->cfg.flags & RLX_FLAG_NO_GRAPH) return enqueue_forward_any(e, ids, mask, B, S, w, out, ws, st, false);
 
     if (!same_weights(e, w)) {
         drop_graphs(e);
@@ -1171,7 +1200,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
         RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->fold_event, cudaEventDisableTiming));
     }
     RLX_CUDA_TRY(cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal));
-    rlx_status_t s = enqueue_forward(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream, true);
+    rlx_status_t s = enqueue_forward_any(e, ids, mask, B, S, &e->weights, out, ws, e->capture_stream, true);
     cudaError_t ce = cudaStreamEndCapture(e->capture_stream, &graph);
     if (s != RLX_OK) {
         if (graph) cudaGraphDestroy(graph);

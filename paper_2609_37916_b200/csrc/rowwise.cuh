@@ -96,6 +96,9 @@ pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* _
     __shared__ int warp_cnt[kPackThreads / 32];
     __shared__ int is_last;
     pdl_launch_dependents();
+    // the tables written here may still be read by the kernels of the previous forward (or sub-batch) on the
+    // same workspace when this launch is a programmatic dependent of its last kernel
+    pdl_wait();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int running = 0;
     for (int base = 0; base < S; base += kPackThreads) {

@@ -133,6 +133,21 @@ def test_host_call_pinned_and_pageable_buffers_and_new_contents_between_calls(rl
     enc.close()
 
 
+@pytest.mark.parametrize("flags", [0x800, 0x801], ids=["graph", "eager"])
+def test_token_chunk_scheduling_is_bitwise_the_unchunked_forward(rlx, flags):
+    """RLX_FLAG_CHUNKED: 200 sequences x 128 positions (25,600 padded tokens) run as two sub-batches through the
+    same workspace; same kernels on fewer rows, so every bit must agree with the single-pass forward."""
+    inp = make_inputs(CONFIGS["c2"], batch=200, num_layers=2)
+    w = rlx.upload_weights(inp.params, inp.layers)
+    whole, status = run_gpu(rlx, inp, weights=w, flags=flags & 1)
+    assert status == 0
+    parts, status = run_gpu(rlx, inp, weights=w, flags=flags)
+    assert status == 0
+    assert np.array_equal(whole, parts)
+    again, status = run_gpu(rlx, inp, weights=w, flags=flags)      # a second call on a fresh encoder: same bits
+    assert status == 0 and np.array_equal(again, parts)
+
+
 @pytest.mark.parametrize("name", ["c3", "c4"])
 def test_large_config_every_sequence_matches_oracle(rlx, name):
     """The two large configurations in the benchmark's launch configuration, EVERY sequence compared
