@@ -390,8 +390,13 @@ rlx_status_t rlx_attention_f32(const float *qkv_f32, const int32_t *attention_ma
  * The same attention on PACKED rows (what the forward runs after sequence packing): qkv holds
  * `rows` rows of [q | k | v]; sequence b owns rows seq_start[b] .. seq_start[b] + seq_len[b], all
  * valid, seq_len[b] <= max_len <= 512; ctx uses the same row numbering.  impl 0: tcgen05/TMEM
- * kernel (TMA-fed, S and P in tensor memory, one thread per query row in the softmax);
- * impl 1: warp-level mma.sync kernel.  Rows outside every sequence are not written.
+ * kernel (persistent, TMA-fed, one pass over the keys, S and P in tensor memory, one thread per
+ * query row in the softmax); impl 1: warp-level mma.sync kernel (what rlx_encoder_forward runs
+ * unless RLX_FLAG_ATTN_TCGEN05 is set).  Rows outside every sequence are not written.
+ * impl 0 hands its work items out through a counter word inside the library (zero between
+ * launches): two impl-0 calls must not run concurrently on one device (calls ordered on one stream,
+ * or otherwise serialised, are fine).  status: optional device word, receives RLX_DEVSTAT_TIMEOUT
+ * if a bounded wait of impl 0 ran out.
  */
 rlx_status_t rlx_attention_packed_bf16(const void *qkv_bf16, int32_t rows, const int32_t *seq_start,
                                        const int32_t *seq_len, int32_t batch, int32_t max_len,
