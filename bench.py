@@ -503,7 +503,7 @@ def run_ours(args):
             "config": workload_config(args.config, {"valid_lengths": f"all {cfg.seq} (--all-valid)"} if args.all_valid else None),
             "e2e": {"value": seqs * args.steps / (e2e_total / 1e3), "unit": "sequences/s", "p50_ms": e2e_p50,
                     "h2d_bytes_per_step": 2 * B * S * 4, "d2h_bytes_per_step": B * H * 4,
-                    "timing": "host wall clock around rlx_encoder_forward_host (copies + forward + sync)"},
+                    "timing": "host wall clock around rlx_encoder_forward_host with pinned host buffers: the kernels read ids / mask from, and write the embeddings to, host memory over the bus (no separate copy operations), then the stream is synchronised"},
             # main chain + the side-branch weight prefetch kernel (models whose Linear weights fit in L2)
             "gpu_launches": args.steps * (run.n_kernels + (1 if cfg.num_layers * 24 * cfg.hidden * cfg.hidden <= (48 << 20)
                                                            and cfg.ffn == 4 * cfg.hidden else 0)),

@@ -215,11 +215,15 @@ rlx_status_t rlx_encoder_forward_tp(rlx_encoder_t *encoder, const int32_t *token
                                     float *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
- * Same computation with HOST inputs and output (the end-to-end path): copies
- * ids and mask host->device into the workspace staging area, runs the forward,
- * copies the embeddings device->host and synchronises the stream before
- * returning.  token_ids / attention_mask / out are host pointers (pinned memory
- * makes the copies asynchronous); weights and workspace are as above.
+ * Same computation with HOST inputs and output (the end-to-end path), synchronous: returns after the
+ * stream has been synchronised and `out_host` holds the embeddings.  token_ids / attention_mask / out
+ * are host pointers; weights and workspace are as above.
+ *   pinned (page-locked, mapped) buffers, 16-byte aligned: no copy operations at all -- the first
+ *     kernels read ids and mask from host memory over the bus and the pooling kernel writes the
+ *     embeddings there (each copy operation would cost several microseconds of engine latency in
+ *     stream order; the bytes crossing the bus are the same);
+ *   pageable buffers: ids and mask are copied into the workspace staging area, the forward runs on
+ *     those, and the embeddings are copied back.
  */
 rlx_status_t rlx_encoder_forward_host(rlx_encoder_t *encoder, const int32_t *token_ids_host,
                                       const int32_t *attention_mask_host, int32_t batch,
