@@ -520,7 +520,8 @@ rlx_status_t rlx_scaled_matmul_bf16(const void *A, const void *codes, const void
  *                     tensor core's fp32.  Scales of 255 (NaN) are the caller's responsibility.
  * format: RLX_FMT_FP8_E4M3 or RLX_FMT_FP8_E5M2, chosen per operand (RLX_ERR_UNSUPPORTED otherwise: the
  * 6- and 4-bit grids go through rlx_dequant_block_scaled_bf16).  rlx_mx_matmul_bf16 needs K % 128 == 0
- * and N % 128 == 0 (RLX_ERR_UNSUPPORTED).  All pointers device, 16-byte aligned; bias f32 [N] or NULL;
+ * and N % 128 == 0 or N % 192 == 0 (RLX_ERR_UNSUPPORTED otherwise; multiples of 192 run on persistent
+ * 128 x 192 tiles, the rest on 128 x 128 tiles).  All pointers device, 16-byte aligned; bias f32 [N] or NULL;
  * status: optional device word that receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.
  * Asynchronous on cuda_stream; nothing is allocated.
  */

@@ -209,6 +209,192 @@ gemm_mx_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_
     }
 }
 
+// ---------------------------------------------------------------------------- persistent 128 x 192 tiles
+// The same product for N % 192 == 0 (the encoder's widths 384, 1152, 1536 and multiples): one persistent
+// CTA per SM walks the tile list, the fp32 accumulators are double-buffered in tensor memory so that the
+// epilogue of tile i overlaps the main loop of tile i + 1, the scale feed has its own four warps and the
+// epilogue eight (one lane quarter x one 96-column half each).  A 128 x 192 tile moves 40 KB of operands
+// per 384 tensor-core cycles (the 128 x 128 tile: 32 KB per 256), which is what the SM's fill rate can
+// sustain.  TMEM: 2 x 192 accumulator columns + 4 scale slots of 12 columns (A's 4, W's 8) = 432 -> 512.
+namespace wide {
+constexpr int kTileNW = 192;
+constexpr int kStagesW = 4;
+constexpr int kThreadsW = 448;   // TMA, MMA, 4 scale warps, 8 epilogue warps
+constexpr int kAccCols = 2 * kTileNW;
+constexpr int kSfCols = 12;
+constexpr int kWBytes = kTileNW * kBlockK;
+constexpr int kStageBytesW = kOperandBytes + kWBytes;
+constexpr int kEpiWarpsW = 8;
+constexpr int kStagingW = kEpiWarpsW * kStageBufBytes;   // one 2 KB chunk buffer per epilogue warp (TMA-store source)
+constexpr int kSmemBytesW = kStagesW * kStageBytesW + kStagingW + 256 + 1024;
+
+__device__ __forceinline__ uint32_t idesc_mx_w(int a_fmt, int b_fmt, int sf_id) {
+    return ((uint32_t)sf_id << 4) | ((uint32_t)a_fmt << 7) | ((uint32_t)b_fmt << 10) | ((uint32_t)(kTileNW >> 3) << 17) |
+           (1u << 23) | ((uint32_t)(kTileM >> 4) << 24) | ((uint32_t)sf_id << 29);
+}
+__device__ __forceinline__ void tmem_st_32x4(uint32_t taddr, const uint32_t (&r)[4]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreadsW, 1)
+gemm_mx192_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+                          const __grid_constant__ CUtensorMap tmap_out, MxParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - raw);
+    const uint32_t staging = base + kStagesW * kStageBytesW;
+    const uint32_t bars = staging + kStagingW;
+    const uint32_t full = bars, empty = full + 8 * kStagesW, tfull = empty + 8 * kStagesW, tempty = tfull + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + kStagesW * kStageBytesW + kStagingW + 8 * (2 * kStagesW + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles = p.N / kTileNW, m_tiles = (p.M + kTileM - 1) / kTileM, num_tiles = n_tiles * m_tiles;
+    const int nkb = p.K / kBlockK;
+    const int sf_ld = p.K / 32;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStagesW; ++i) { mbar_init(full + 8 * i, 5); mbar_init(empty + 8 * i, 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(tfull + 8 * i, 1); mbar_init(tempty + 8 * i, 8); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap_a);
+        prefetch_tmap(&tmap_w);
+        prefetch_tmap(&tmap_out);
+    }
+    if (warp == 1) {
+        tmem_alloc<1>(smem_u32(tmem_slot), 512);
+        tmem_relinquish<1>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t it = 0;   // stages issued so far
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / n_tiles) * kTileM, n0 = (tile % n_tiles) * kTileNW;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const uint32_t st = it % kStagesW, use = it / kStagesW;
+                    if (use >= 1 && !(ok = mbar_wait(empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                    const uint32_t dst = base + st * kStageBytesW;
+                    mbar_expect_tx(full + 8 * st, kStageBytesW);
+                    tma_load_2d(dst, &tmap_a, kb * kBlockK, m0, full + 8 * st);
+                    tma_load_2d(dst + kOperandBytes, &tmap_w, kb * kBlockK, n0, full + 8 * st);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        uint32_t it = 0, tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+            const uint32_t as = tcount & 1, ause = tcount >> 1;
+            if (ause >= 1 && !(ok = mbar_wait_warp(tempty + 8 * as, (ause - 1) & 1, abort_flag))) break;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t st = it % kStagesW;
+                if (!(ok = mbar_wait_warp(full + 8 * st, (it / kStagesW) & 1, abort_flag))) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t adesc = make_smem_desc(base + st * kStageBytesW);
+                    const uint64_t bdesc = make_smem_desc(base + st * kStageBytesW + kOperandBytes);
+                    const uint32_t sfa = tmem + kAccCols + st * kSfCols, sfb = sfa + 4;
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 32; ++k)
+                        umma_mx(tmem + as * kTileNW, adesc + 2 * k, bdesc + 2 * k, idesc_mx_w(p.a_fmt, p.w_fmt, k), sfa, sfb,
+                                (kb | k) != 0 ? 1u : 0u);
+                    umma_commit<1>(empty + 8 * st);
+                    if (kb == nkb - 1) umma_commit<1>(tfull + 8 * as);
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------ scale feed (one warp per lane quarter)
+        // The scale words of a stage are requested kAhead stages before they are written to tensor memory,
+        // so that their global-memory latency stays off the pipeline's critical path.
+        constexpr int kAhead = 3;
+        const int quad = warp & 3;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+        const int my_tiles = blockIdx.x < num_tiles ? (num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+        const long long total = (long long)my_tiles * nkb;
+        uint32_t wa[kAhead][4], wb[kAhead][8];
+        auto fetch = [&](long long i, uint32_t (&a4)[4], uint32_t (&b8)[8]) {
+            const int tile = blockIdx.x + (int)(i / nkb) * gridDim.x, kb = (int)(i % nkb);
+            const int m0 = (tile / n_tiles) * kTileM, n0 = (tile % n_tiles) * kTileNW;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int ar = m0 + 32 * c + lane;
+                // rows past M are zero-filled operand rows: any finite scale will do
+                a4[c] = ar < p.M ? __ldg(reinterpret_cast<const uint32_t*>(p.sfa + (size_t)ar * sf_ld) + kb) : 0x7F7F7F7Fu;
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {   // two 128-row groups of W's rows; the second is half used
+                const int wr = 32 * c + lane;
+                b8[c] = wr < kTileNW ? __ldg(reinterpret_cast<const uint32_t*>(p.sfw + (size_t)(n0 + wr) * sf_ld) + kb) : 0x7F7F7F7Fu;
+            }
+        };
+#pragma unroll
+        for (int i = 0; i < kAhead; ++i)
+            if (i < total) fetch(i, wa[i], wb[i]);
+        bool ok = true;
+        for (long long i0 = 0; i0 < total && ok; i0 += kAhead) {
+#pragma unroll
+            for (int u = 0; u < kAhead; ++u) {
+                const long long i = i0 + u;
+                if (i >= total) break;
+                const uint32_t slot = (uint32_t)(i % kStagesW), use = (uint32_t)(i / kStagesW);
+                if (use >= 1 && !(ok = mbar_wait(empty + 8 * slot, (use - 1) & 1, abort_flag))) break;
+                tc_fence_after();
+                tmem_st_32x4(lane_addr + kAccCols + slot * kSfCols, wa[u]);
+                tmem_st_32x8(lane_addr + kAccCols + slot * kSfCols + 4, wb[u]);
+                tmem_st_wait_all();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full + 8 * slot);
+                if (i + kAhead < total) fetch(i + kAhead, wa[u], wb[u]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: lane quarter x 96-column half
+        // the bf16 GEMM's epilogue tile: all three chunks to registers, accumulator handed back, bias, one
+        // TMA store per 32 x 32 chunk out of the warp's swizzled staging buffer
+        const int quad = warp & 3, half = (warp - 6) >> 2, ew = warp - 6;
+        const uint32_t stg = staging + ew * kStageBufBytes;
+        Params gp = {};
+        gp.bias = p.bias; gp.out = p.out; gp.M = p.M; gp.N = p.N; gp.K = p.K; gp.status = p.status;
+        uint32_t tcount = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+            const int m_row0 = (tile / n_tiles) * kTileM + quad * 32, n0 = (tile % n_tiles) * kTileNW + half * 96;
+            const uint32_t as = tcount & 1;
+            if (!(ok = mbar_wait(tfull + 8 * as, (tcount >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            EpilogueTile<0, 3> et;
+            et.template drain<1>(gp, &tmap_out, p.M, m_row0, n0, tmem + ((uint32_t)(quad * 32) << 16) + as * kTileNW + half * 96,
+                                 stg, lane, tempty + 8 * as, 0u);
+        }
+        EpilogueTile<0, 3>::finish(lane);
+    }
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, RLX_DEVSTAT_TIMEOUT_BIT);
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc<1>(tmem, 512);
+    }
+}
+}  // namespace wide
+
 // ---------------------------------------------------------------------------- activation quantiser
 template <bool E5M2>
 __device__ __forceinline__ uint16_t cvt_fp8x2(float lo, float hi) {

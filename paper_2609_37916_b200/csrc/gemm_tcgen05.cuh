@@ -442,7 +442,7 @@ struct EpilogueTile {
     // The bias values of a slab (one 128-byte line per chunk) are pulled into L1 a tile ahead of their
     // use by every lane, so that no chunk starts with an L2 round trip.
     static __device__ __forceinline__ void prefetch_bias(const Params& p, int n0) {
-        if ((threadIdx.x & 31) < NC) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.bias + n0 + (threadIdx.x & 31) * 32));
+        if (p.bias != nullptr && (threadIdx.x & 31) < NC) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.bias + n0 + (threadIdx.x & 31) * 32));
     }
 
     __device__ __forceinline__ void prefetch(const Params& p, int M, int m, int n0) {
@@ -540,8 +540,13 @@ struct EpilogueTile {
             }
         } else {
             float4 b4[8];
+            if (p.bias != nullptr) {   // uniform; the encoder's GEMMs always carry a bias
 #pragma unroll
-            for (int i = 0; i < 8; ++i) b4[i] = ld_global_keep_f4(bias32 + 4 * i);
+                for (int i = 0; i < 8; ++i) b4[i] = ld_global_keep_f4(bias32 + 4 * i);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) b4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b4[i].x;

@@ -233,6 +233,8 @@ cudaError_t init_kernels_for_current_device() {
     }
     if ((e = cudaFuncSetAttribute(rlx::tcmx::gemm_mx_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcmx::kSmemBytes)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcmx::wide::gemm_mx192_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcmx::wide::kSmemBytesW)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tca::Smem<32>::BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tca::attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1688,19 +1690,30 @@ rlx_status_t rlx_mx_matmul_bf16(const void* a_codes, const void* a_scales, int32
         (bias && !aligned16(bias)))
         return RLX_ERR_INVALID_ARG;
     const int af = mx_element_format(a_format), wf = mx_element_format(w_format);
-    if (af < 0 || wf < 0 || K % rlx::tcmx::kBlockK != 0 || N % rlx::tcmx::kTileN != 0) return RLX_ERR_UNSUPPORTED;
+    if (af < 0 || wf < 0 || K % rlx::tcmx::kBlockK != 0 || (N % rlx::tcmx::kTileN != 0 && N % rlx::tcmx::wide::kTileNW != 0))
+        return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
+    const bool wide_tiles = N % rlx::tcmx::wide::kTileNW == 0;   // persistent 128 x 192 tiles when N allows
     CUtensorMap ta, tw;
     if (!make_tmap_u8(&ta, a_codes, (uint64_t)M, (uint64_t)K, rlx::tcmx::kTileM) ||
-        !make_tmap_u8(&tw, w_codes, (uint64_t)N, (uint64_t)K, rlx::tcmx::kTileN))
+        !make_tmap_u8(&tw, w_codes, (uint64_t)N, (uint64_t)K, wide_tiles ? rlx::tcmx::wide::kTileNW : rlx::tcmx::kTileN))
         return RLX_ERR_CUDA;
     rlx::tcmx::MxParams p;
     p.sfa = (const uint8_t*)a_scales; p.sfw = (const uint8_t*)w_scales; p.bias = bias; p.out = (bf16*)out;
     p.M = M; p.N = N; p.K = K; p.a_fmt = af; p.w_fmt = wf; p.status = status;
-    const long long tiles = (long long)((M + rlx::tcmx::kTileM - 1) / rlx::tcmx::kTileM) * (N / rlx::tcmx::kTileN);
+    const long long m_tiles = (M + rlx::tcmx::kTileM - 1) / rlx::tcmx::kTileM;
+    const long long tiles = m_tiles * (wide_tiles ? N / rlx::tcmx::wide::kTileNW : N / rlx::tcmx::kTileN);
     if (tiles > 0x7fffffffLL) return RLX_ERR_UNSUPPORTED;
-    rlx::tcmx::gemm_mx_tcgen05_kernel<<<(unsigned)tiles, rlx::tcmx::kThreads, rlx::tcmx::kSmemBytes,
-                                        static_cast<cudaStream_t>(stream)>>>(ta, tw, p);
+    if (wide_tiles) {
+        const unsigned grid = (unsigned)std::min<long long>(tiles, sm_count());
+        CUtensorMap to;   // output chunks: 32 x 32 bf16 boxes with the 64-byte swizzle of the staging buffers
+        if (!make_tmap(&to, out, (uint64_t)M, (uint64_t)N, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return RLX_ERR_CUDA;
+        rlx::tcmx::wide::gemm_mx192_tcgen05_kernel<<<grid, rlx::tcmx::wide::kThreadsW, rlx::tcmx::wide::kSmemBytesW,
+                                                     static_cast<cudaStream_t>(stream)>>>(ta, tw, to, p);
+    } else {
+        rlx::tcmx::gemm_mx_tcgen05_kernel<<<(unsigned)tiles, rlx::tcmx::kThreads, rlx::tcmx::kSmemBytes,
+                                            static_cast<cudaStream_t>(stream)>>>(ta, tw, p);
+    }
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }

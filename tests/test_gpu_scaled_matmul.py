@@ -171,11 +171,12 @@ def test_quantise_mx_is_bit_exact_against_the_definition(rlx, name):
     assert np.array_equal(codes.cpu().numpy(), want_codes)
 
 
-def test_mx_matmul_places_every_scale_byte_and_operand_where_the_definition_says(rlx):
+@pytest.mark.parametrize("N", [256, 384], ids=["tiles_128", "tiles_192"])
+def test_mx_matmul_places_every_scale_byte_and_operand_where_the_definition_says(rlx, N):
     """Exact cases that fail if a scale byte reaches the wrong row, column or k-group, or an operand tile is
     transposed: all elements 1.0 with a different power-of-two scale per (row, k-group) and per (column,
     k-group); then integer-valued elements with unit scales (integer arithmetic, exact in fp32)."""
-    M, N, K = 300, 256, 1024          # ragged rows, two column tiles, 8 stages of k: every ring wraps
+    M, K = 300, 1024                  # ragged rows, two column tiles (128- or 192-wide), 8 stages of k: every ring wraps
     rng = np.random.default_rng(6)
     one = 0x38                          # 1.0 in E4M3
     a_codes = np.full((M, K), one, np.uint8)
@@ -194,9 +195,9 @@ def test_mx_matmul_places_every_scale_byte_and_operand_where_the_definition_says
     wi = rng.integers(-4, 5, size=(N, K))
     ac = osm.quantise_elements(ai.astype(np.float64), osm.E4M3)
     wc = osm.quantise_elements(wi.astype(np.float64), osm.E4M3)
-    ones = np.full((M, K // 32), 127, np.uint8)
+    ones = np.full((max(M, N), K // 32), 127, np.uint8)
     bias = rng.integers(-8, 9, size=N).astype(np.float32)
-    got = to_np64(rlx.mx_matmul_bf16(_u8_dev(ac), _u8_dev(ones), word, _u8_dev(wc), _u8_dev(ones[:N]), word,
+    got = to_np64(rlx.mx_matmul_bf16(_u8_dev(ac), _u8_dev(ones[:M]), word, _u8_dev(wc), _u8_dev(ones[:N]), word,
                                      bias=f32_dev(bias)))
     exact = (ai @ wi.T + bias).astype(np.float32)
     assert np.array_equal(got, round_to_bf16(exact).astype(np.float64))
