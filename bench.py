@@ -689,6 +689,86 @@ def run_qk_rope(args):
     print(json.dumps(line), flush=True)
 
 
+def run_mx_matmul(args):
+    """`--op mx_matmul`: the block-scaled tensor-core path (both operands FP8 E4M3 with E8M0 scales per 32) on the
+    encoder's three projection shapes at the roofline configuration's row count and on a large square problem;
+    the activation quantiser is timed alone.  The JSON line's value / roofline are the FFN-down shape's."""
+    import torch
+    import paper_2609_37916_b200 as rlx
+    from oracle import scaled_matmul as osm
+
+    torch.cuda.set_device(0)
+    word = rlx.binding.FMT_FP8_E4M3
+    g = torch.Generator(device="cuda").manual_seed(5)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    peaks, peak_kind = load_peaks()
+    fp8_peak = 2.0 * peaks["bf16_tflops"]
+    sampler = ClockSampler(0)
+    sampler.start()
+    shapes = [("qkv", 36736, 1152, 384), ("ffn_up", 36736, 1536, 384), ("ffn_down", 36736, 384, 1536), ("square", 8192, 8192, 8192)]
+    rows = {}
+    first = True
+    for name, M, N, K in shapes:
+        x = torch.randn(M, K, device="cuda", generator=g).to(torch.bfloat16)
+        w = (torch.randn(N, K, device="cuda", generator=g) * 0.05).to(torch.bfloat16)
+        bias = torch.randn(N, device="cuda", generator=g)
+        a_codes, a_scales = rlx.quantise_mx(x, word)
+        w_codes, w_scales = rlx.quantise_mx(w, word)      # weights through the same rule (bit-exact against the oracle's)
+        out = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+
+        def timed(fn):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            return e0, e1
+
+        mm = lambda: rlx.mx_matmul_bf16(a_codes, a_scales, word, w_codes, w_scales, word, bias=bias, out=out)
+        qz = lambda: rlx.quantise_mx(x, word)
+        for _ in range(max(args.warmup, 3)):
+            timed(mm)
+            timed(qz)
+        torch.cuda.synchronize()
+        if first:
+            sampler.active.set()
+        ev = [timed(mm) for _ in range(args.steps)]
+        evq = [timed(qz) for _ in range(args.steps)]
+        torch.cuda.synchronize()
+        ms = statistics.median(a.elapsed_time(b) for a, b in ev)
+        msq = statistics.median(a.elapsed_time(b) for a, b in evq)
+        tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+        hbm_floor_us = (M * K + N * K + (M + N) * K / 32 + 2.0 * M * N) / (peaks["hbm_gbs"] * 1e9) * 1e6
+        rows[name] = {"M": M, "N": N, "K": K, "p50_us": ms * 1e3, "tflops": tf, "frac_of_fp8_peak": tf / fp8_peak,
+                      "hbm_floor_us": hbm_floor_us, "tensor_floor_us": 2.0 * M * N * K / (fp8_peak * 1e12) * 1e6,
+                      "quantise_p50_us": msq * 1e3, "quantise_gbs": M * K * (2 + 1 + 1 / 32) / (msq * 1e-3) / 1e9}
+        if name == "ffn_down":
+            m0 = 64     # parity of the timed launch's output on a sample, against the fp64 product of the dequantised operands
+            ref = osm.mx_matmul(a_codes[:m0].cpu().numpy(), a_scales[:m0].cpu().numpy(), osm.E4M3, w_codes.cpu().numpy(),
+                                w_scales.cpu().numpy(), osm.E4M3, bias.cpu().numpy().astype(np.float64))
+            got = out[:m0].float().cpu().numpy().astype(np.float64)
+            rows[name]["max_err_over_max_ref"] = float(np.abs(got - ref).max() / np.abs(ref).max())
+        first = False
+    sampler.active.clear()
+    sampler.stop()
+    r = rows["ffn_down"]
+    line = {
+        "metric": "block-scaled FP8 matmul tokens/s (p50 reported alongside)", "op": "mx_matmul",
+        "value": r["M"] / (r["p50_us"] * 1e-6), "unit": "tokens/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": r["p50_us"] * 1e-3, "p50_ms": r["p50_us"] * 1e-3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3 x fp8_e4m3 -> f32 accumulate -> bf16",
+        "data": "synthetic",
+        "config": {"workload": "M=36736 tokens, N=384, K=1536 (FFN-down shape), both operands FP8 E4M3 with E8M0 scales per 32; "
+                               "the other shapes are in `shapes`", "l2": "256 MiB flush write between steps"},
+        "gpu_launches": args.steps, "clocks": sampler.summary(),
+        "roofline": {"kernel": "gemm_mx192_tcgen05_kernel", "bound": "tensor", "achieved": r["tflops"], "peak": fp8_peak,
+                     "unit": "TFLOP/s", "frac": r["frac_of_fp8_peak"], "traffic": None,
+                     "peak_source": peak_kind + "; FP8 peak taken as 2 x the measured bf16 figure (no FP8 peak measured)"},
+        "e2e": None, "cpu_baseline": None, "shapes": rows,
+    }
+    print(json.dumps(line))
+
+
 def run_scaled_matmul(args):
     """`--op scaled_matmul`: one step = rlx_scaled_matmul_bf16 (block-scaled minifloat weights dequantised
     to bf16, then the tcgen05 GEMM with bias) at the BERT-base FFN-up shape over 32,768 tokens; the
@@ -786,7 +866,7 @@ def main():
     ap.add_argument("--all-valid", action="store_true", help="encoder op: every sequence has the full length")
     ap.add_argument("--no-c3", action="store_true", help="encoder op, default workload: skip the roofline_c3 block")
     ap.add_argument("--c3-steps", type=int, default=20, help="timed steps of the roofline_c3 block")
-    ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope", "scaled_matmul"])
+    ap.add_argument("--op", default="encoder", choices=["encoder", "attention_kind", "qk_rope", "scaled_matmul", "mx_matmul"])
     ap.add_argument("--fmt", default="fp8_e4m3", choices=["fp8_e4m3", "fp4_e2m1"])
     ap.add_argument("--mask", default="causal", choices=["none", "causal", "sliding"])
     ap.add_argument("--window", type=int, default=512)
@@ -798,7 +878,8 @@ def main():
     if args.op != "encoder":
         if args.impl != "ours" or args.gpus != 1:
             raise SystemExit(f"--op {args.op} runs on one GPU with --impl ours")
-        {"attention_kind": run_attention_kind, "qk_rope": run_qk_rope, "scaled_matmul": run_scaled_matmul}[args.op](args)
+        {"attention_kind": run_attention_kind, "qk_rope": run_qk_rope, "scaled_matmul": run_scaled_matmul,
+         "mx_matmul": run_mx_matmul}[args.op](args)
         return
     if args.impl == "reference":
         run_reference_arm(args)

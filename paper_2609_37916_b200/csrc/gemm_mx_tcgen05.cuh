@@ -1,6 +1,7 @@
 // Block-scaled FP8 product on the tensor cores' own block-scaled path (the Blackwell half of
 // ScaledMatMul): out[M,N] = A W^T (+ bias) with BOTH operands given as (8-bit element codes, one E8M0
-// scale byte per 32 consecutive k).  Two kernels:
+// scale byte per 32 consecutive k).  Three kernels (the product has a 128 x 128-tile form, described
+// first, and a persistent 128 x 192-tile form further down for widths that are multiples of 192):
 //
 //  quantise_mx_kernel      bf16 activations -> (codes, scales) by the microscaling rule: per block of 32,
 //                          shared exponent floor(log2 max|x|) - emax(format), elements rounded to the
