@@ -243,7 +243,8 @@ rlx_status_t rlx_encoder_forward_host(rlx_encoder_t *encoder, const int32_t *tok
  * image, so every GPU that loads the library gives up that much memory until the process exits.
  * A (batch, seq) whose rlx_encoder_workspace_bytes exceeds the limit is rejected with
  * RLX_ERR_WORKSPACE before anything is launched (at H=384, F=1536 the limit covers about 1,800
- * tokens, e.g. batch 14 x seq 128).  The call makes no cudaMalloc/cudaFree and uses no
+ * tokens, e.g. batch 14 x seq 128; the call always runs the 7-kernel layer unless RLX_FLAG_FOLD_LN is set,
+ * because the folded form's weight copies would not fit).  The call makes no cudaMalloc/cudaFree and uses no
  * allocating library routine: kernels are launched directly (no CUDA graph is built), and
  * RLX_FLAG_KERNEL_EVENTS is ignored (no event is recorded, and the per-kernel times of an earlier
  * rlx_encoder_forward on the same object stay as they were).

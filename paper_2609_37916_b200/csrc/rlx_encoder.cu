@@ -793,12 +793,15 @@ bool uses_cluster_ln(const rlx_encoder_config_t& c) {
 // near 3 k VALID tokens -- 32 x 128 with every position valid loses 4 % -- but only the padded size is
 // known on the host; at 256 x 256 the folded form loses 10 %).
 constexpr int kAutoFoldMaxTokens = 4096;
+// Set for the duration of a call that runs out of the built-in arena: the folded form needs room for a
+// gamma-scaled copy of every Linear weight (12 MB at H = 384), which that arena does not have.
+thread_local bool g_no_auto_fold = false;
 bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S) {
     const bool can = !(c.flags & RLX_FLAG_GEMM_SIMT) && c.hidden % 32 == 0 && c.max_seq <= rlx::kPoolMaxRows;
     if (!can) return false;
     if (c.flags & RLX_FLAG_FOLD_LN) return true;
     const bool other_fusion = (c.flags & (RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN)) != 0;
-    return !(c.flags & RLX_FLAG_NO_AUTO_FOLD) && !other_fusion && (long long)B * S <= kAutoFoldMaxTokens;
+    return !g_no_auto_fold && !(c.flags & RLX_FLAG_NO_AUTO_FOLD) && !other_fusion && (long long)B * S <= kAutoFoldMaxTokens;
 }
 
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
@@ -1413,6 +1416,10 @@ rlx_status_t rlx_encoder_forward_static(rlx_encoder_t* e, const int32_t* ids, co
     rlx_status_t s = check_forward_args(e, ids, mask, B, S, w, out, reinterpret_cast<void*>(uintptr_t(256)),
                                         ~size_t(0), false);
     if (s != RLX_OK) return s;
+    struct NoAutoFold {
+        NoAutoFold() { g_no_auto_fold = true; }
+        ~NoAutoFold() { g_no_auto_fold = false; }
+    } no_auto_fold;   // the 7-kernel layer unless RLX_FLAG_FOLD_LN asks for the folded one
     const Arena a = plan_arena(B, S, e->cfg.hidden, e->cfg.ffn, e->cfg.num_layers, uses_fold_ln(e->cfg, B, S));
     if (a.total > (size_t)RLX_STATIC_WORKSPACE_BYTES) return RLX_ERR_WORKSPACE;  // beyond the built-in arena
     cudaStream_t st = static_cast<cudaStream_t>(stream);

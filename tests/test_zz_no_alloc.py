@@ -26,7 +26,9 @@ def test_static_arena_forward_matches_workspace_forward_twice(rlx):
     first = make_inputs(CONFIGS["c1"], batch=3, seq=96, num_layers=2, lengths=[96, 17, 50])
     second = make_inputs(CONFIGS["c1"], batch=2, seq=128, num_layers=2, lengths=[5, 128], weights=False)
     w = rlx.upload_weights(first.params, first.layers)
-    enc = rlx.Encoder.from_config(first.cfg, max_batch=4, max_seq=128)
+    # the built-in arena has no room for the folded-LayerNorm weights, so the static call always runs the
+    # 7-kernel layer: the ordinary forward it is compared with is told to do the same
+    enc = rlx.Encoder.from_config(first.cfg, max_batch=4, max_seq=128, flags=rlx.binding.FLAG_NO_AUTO_FOLD)
     for inp in (first, second):     # second call: other shape, arena still holds the first call's bytes
         B, S, H = inp.cfg.batch, inp.cfg.seq, inp.cfg.hidden
         assert enc.workspace_bytes(B, S) <= rlx.binding.STATIC_WORKSPACE_BYTES
@@ -79,7 +81,7 @@ def test_static_forward_allocates_nothing_and_leaves_kernel_times_alone(rlx):
     inp = make_inputs(CONFIGS["c1"], batch=4, seq=64, num_layers=2, lengths=[64, 9, 33, 20])
     B, S, H = inp.cfg.batch, inp.cfg.seq, inp.cfg.hidden
     w = rlx.upload_weights(inp.params, inp.layers)
-    enc = rlx.Encoder.from_config(inp.cfg, max_batch=B, max_seq=S, flags=rlx.binding.FLAG_KERNEL_EVENTS)
+    enc = rlx.Encoder.from_config(inp.cfg, max_batch=B, max_seq=S, flags=rlx.binding.FLAG_KERNEL_EVENTS | rlx.binding.FLAG_NO_AUTO_FOLD)
     ids, mask = i32_dev(inp.ids), i32_dev(inp.mask)
     want = torch.empty((B, H), dtype=torch.float32, device="cuda")
     got = torch.empty_like(want)
