@@ -201,8 +201,11 @@ def workload_config(name: str, extra=None):
 
 
 # ---------------------------------------------------------------------------- roofline bookkeeping
-def kernel_classes(num_layers: int, fused_ln: bool):
+def kernel_classes(num_layers: int, fused_ln: bool, fused_ffn: bool = False):
     per_layer = [k for k in KERNEL_CLASSES if not (fused_ln and k in ("ln1", "ln2"))]
+    if fused_ffn:   # FFN-up, GELU and FFN-down are one kernel
+        per_layer = [k for k in per_layer if k != "gemm_ffn2"]
+        per_layer[per_layer.index("gemm_ffn1")] = "ffn_fused"
     names = ["pack", "embed_ln"]
     for _ in range(num_layers):
         names += per_layer
@@ -226,6 +229,8 @@ def algorithmic_work(cls: str, c, lengths):
         return "tensor", 2.0 * T * H * H, "flop"
     if cls in ("gemm_ffn1", "gemm_ffn2"):
         return "tensor", 2.0 * T * F * H, "flop"
+    if cls == "ffn_fused":
+        return "tensor", 4.0 * T * F * H, "flop"
     if cls == "attention":
         # at head_dim 32/64 the softmax exponentials (one per query-key pair and head), not the
         # QK^T / PV flops, are the scarce resource: 128..256 flops per exp against a tensor : MUFU
@@ -250,6 +255,8 @@ def gemm_bytes(cls: str, c, T: int):
         return T * (H + H + H) * 2.0 + H * H * 2.0
     if cls == "gemm_ffn1":
         return T * (H + F) * 2.0 + F * H * 2.0
+    if cls == "ffn_fused":
+        return T * (H + H) * 2.0 + 2.0 * F * H * 2.0   # the hidden activation never leaves the chip
     return T * (F + H + H) * 2.0 + F * H * 2.0   # gemm_ffn2
 
 
@@ -317,7 +324,9 @@ class EncoderRun:
         self.out_h = torch.empty((B, H), dtype=torch.float32).pin_memory()
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         self.n_kernels = self.enc.kernels_per_forward(B, S)
-        self.names = kernel_classes(cfg.num_layers, fused_ln=(self.n_kernels == 3 + 5 * cfg.num_layers))
+        per_layer = (self.n_kernels - 3) // cfg.num_layers
+        fused_ffn = bool(args.flags & 0x1000) and per_layer in (4, 6)
+        self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer + (1 if fused_ffn else 0) == 5), fused_ffn=fused_ffn)
         assert len(self.names) == self.n_kernels
 
     def step_device(self, e, w):

@@ -78,6 +78,9 @@ typedef enum {
                                    AUTOMATICALLY for calls with batch*seq <= 4096 unless one of the other two
                                    fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
 #define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
+#define RLX_FLAG_FUSED_FFN 0x1000u /* FFN-up, GELU and FFN-down in ONE kernel per layer (the F-wide activation never
+                                      reaches global memory); hidden 256 or 384, F % 64 == 0; ignored together with the
+                                      LayerNorm fusion flags, the bring-up GEMM, or where the folded layer is chosen */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
                                    kernel's input is still in L2 when its consumer starts.  Results are bit for bit
@@ -531,6 +534,19 @@ rlx_status_t rlx_quantise_mx(const void *x_bf16, int32_t M, int32_t K, int32_t f
 rlx_status_t rlx_mx_matmul_bf16(const void *a_codes, const void *a_scales_e8m0, int32_t a_format,
                                 const void *w_codes, const void *w_scales_e8m0, int32_t w_format,
                                 const float *bias, int32_t M, int32_t N, int32_t K, void *out_bf16,
+                                int32_t *status, void *cuda_stream);
+
+/*
+ * The feed-forward block of a layer in one kernel (Section 3.2, operator fusion):
+ *   out = gelu(x W1^T + b1) W2^T + b2 + x        erf GELU; x is the block's input AND its residual.
+ * x, out: device bf16 [M, H]; w1: bf16 [F, H]; w2: bf16 [H, F]; b1: f32 [F]; b2: f32 [H]; all 16-byte aligned.
+ * The F-wide activation is produced and consumed in 64-column chunks on the chip (tensor memory ->
+ * registers -> shared memory) and rounded to bf16 once, as in the two-kernel form; fp32 accumulation.
+ * H in {256, 384}, F % 64 == 0 (RLX_ERR_UNSUPPORTED otherwise).  status: optional device word that
+ * receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.  Asynchronous on cuda_stream.
+ */
+rlx_status_t rlx_ffn_fused_bf16(const void *x_bf16, const void *w1_bf16, const float *b1, const void *w2_bf16,
+                                const float *b2, int32_t M, int32_t H, int32_t F, void *out_bf16,
                                 int32_t *status, void *cuda_stream);
 
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     attention_packed_bf16,
     dequant_block_scaled_bf16,
     embed_layernorm,
+    ffn_fused_bf16,
     gemm_bf16,
     gemm_residual_layernorm_bf16,
     layernorm,

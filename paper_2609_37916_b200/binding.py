@@ -31,6 +31,7 @@ FLAG_NO_PREFETCH = 0x100
 FLAG_FOLD_LN = 0x200
 FLAG_NO_AUTO_FOLD = 0x400
 FLAG_CHUNKED = 0x800
+FLAG_FUSED_FFN = 0x1000
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_PAIR, GEMM_TCGEN05_SINGLE, GEMM_TCGEN05_RESIDENT = 0, 1, 2, 3, 4
 STATIC_WORKSPACE_BYTES = 16 << 20
@@ -39,7 +40,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_tp", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_quantise_mx", "rlx_mx_matmul_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_quantise_mx", "rlx_mx_matmul_bf16", "rlx_ffn_fused_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
 
 
@@ -404,6 +405,16 @@ def scaled_matmul_bf16(a, codes, scales, fmt: int, bias, residual=None, epilogue
     _check(_load().rlx_scaled_matmul_bf16(_ptr(a), _ptr(codes), _ptr(scales), fmt, _ptr(bias), _ptr(residual), epilogue,
                                           M, N, K, _ptr(w), _ptr(out), _ptr(status), _stream(stream)),
            "rlx_scaled_matmul_bf16")
+    return out
+
+
+def ffn_fused_bf16(x, w1, b1, w2, b2, out=None, status=None, stream=None):
+    """rlx_ffn_fused_bf16: out [M,H] = gelu(x w1^T + b1) w2^T + b2 + x in one kernel."""
+    M, H = x.shape
+    F = w1.shape[0]
+    out = torch.empty((M, H), dtype=torch.bfloat16, device=x.device) if out is None else out
+    _check(_load().rlx_ffn_fused_bf16(_ptr(x), _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2), M, H, F, _ptr(out), _ptr(status),
+                                      _stream(stream)), "rlx_ffn_fused_bf16")
     return out
 
 

@@ -1,0 +1,304 @@
+// Feed-forward block in one kernel:  out = gelu(X W1^T + b1) W2^T + b2 + X   (X = the LayerNorm output that
+// is both the block's input and its residual; W1 [F, H], W2 [H, F]; erf GELU).  The F-wide hidden activation
+// never reaches global memory: it is produced and consumed in chunks of 64 columns.
+//
+// A CTA pair (tcgen05 cta_group::2, M = 256) owns a block of 256 rows at a time:
+//   X block    resident in shared memory for the whole block (H/64 swizzled k-block tiles per CTA); it is the
+//              A operand of every first product and, at the end, the residual (read from shared memory)
+//   chunk c    S_c = X W1[64c .. 64c+63, :]^T            M = 256, N = 64, K = H       -> TMEM (two S buffers)
+//              G_c = bf16(gelu(S_c + b1))                 epilogue warps: TMEM -> registers -> shared memory,
+//                                                         written in the K-major 128-byte-swizzled layout the
+//                                                         tensor core reads (two G buffers of one k-block)
+//              O  += G_c W2[:, 64c .. 64c+63]^T           M = 256, N = H (two instructions of H/2), K = 64
+//   end        out = O + b2 + X  -> bf16 -> 16-byte stores of whole 64-byte row segments (no staging: the
+//              shared memory is full, and a buffer shared with G would need an unbounded barrier between warps)
+// The MMA thread issues S_{c+1} before O += G_c ..., so the tensor core works on the next chunk's first
+// product while the epilogue warps turn S_c into G_c.  W1 / W2 chunks stream through two-stage rings, each
+// CTA loading its half of the rows.  TMEM: O (H columns) + 2 x 64 columns of S = 512 at H = 384.
+// Rounding points are those of the two-kernel form (G rounded to bf16 once, fp32 accumulation in the same
+// k order), so the results agree with it to the last bit wherever the accumulation order is the same.
+// All mbarrier waits are bounded; on expiry the CTA sets the status bit and leaves.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+#include "epilogue.cuh"
+#include "gemm_tcgen05.cuh"
+
+namespace rlx {
+namespace tcff {
+
+using namespace rlx::tc;
+
+constexpr int kPairRows = 256;
+constexpr int kChunk = 64;          // hidden columns per chunk = one k-block of the second product
+constexpr int kEpiWarps = 8;        // per CTA: lane quarter x column half of a 64-column S chunk
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+
+template <int HID>
+struct Cfg {
+    static_assert(HID % 128 == 0 && HID <= 384, "hidden size");
+    static constexpr int KB1 = HID / BLOCK_K;                       // k-blocks of the first product
+    static constexpr int X_BYTES = KB1 * BLOCK_M * 128;             // this CTA's 128 rows of X
+    static constexpr int W1_ROWS = kChunk / 2;                      // this CTA's half of a chunk's W1 rows
+    static constexpr int W1_STAGE = KB1 * W1_ROWS * 128;
+    static constexpr int W2_ROWS = HID / 4;                         // per instruction (N = HID/2), this CTA's half
+    static constexpr int W2_STAGE = 2 * W2_ROWS * 128;              // two instructions' halves, one k-block
+    static constexpr int G_BYTES = BLOCK_M * 128;                   // one k-block tile of G
+    static constexpr int X_OFF = 0, W1_OFF = X_BYTES, W2_OFF = W1_OFF + 2 * W1_STAGE, G_OFF = W2_OFF + 2 * W2_STAGE;
+    static constexpr int BAR_OFF = G_OFF + 2 * G_BYTES;
+    static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+    static constexpr int COL_S = HID;                               // S buffers behind O
+    static constexpr int TMEM_COLS = 512;
+    static_assert(HID + 2 * kChunk <= 512, "tensor memory");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory");
+};
+
+struct FfnParams {
+    const float* b1;            // [F]
+    const float* b2;            // [H]
+    __nv_bfloat16* out;         // [M, H]
+    int M, F;
+    const int32_t* m_ptr;       // optional device row count
+    int32_t* status;
+};
+
+// byte offset of 16-byte chunk j of row r in a K-major tile of 128-byte rows with the 128-byte swizzle
+__device__ __forceinline__ uint32_t sw128(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
+
+template <int HID>
+__global__ void __launch_bounds__(kThreads, 1)
+ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
+                         const __grid_constant__ CUtensorMap tmap_w2, const FfnParams p) {
+    using C = Cfg<HID>;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* gbase = smem_raw + (base - raw);
+    const uint32_t xs = base + C::X_OFF, w1s = base + C::W1_OFF, w2s = base + C::W2_OFF, gs = base + C::G_OFF;
+    const uint32_t bars = base + C::BAR_OFF;
+    // leader-side barriers that both CTAs' TMA / warps arrive on: x_full, w1_full[2], w2_full[2], s_empty[2],
+    // g_full[2], o_empty.  Per-CTA barriers (multicast commits / own warps): x_empty, w1_empty[2], w2_empty[2],
+    // s_full[2], g_empty[2], o_full.
+    const uint32_t x_full = bars, w1_full = x_full + 8, w2_full = w1_full + 16, s_empty = w2_full + 16, g_full = s_empty + 16;
+    const uint32_t o_empty = g_full + 16, x_empty = o_empty + 8, w1_empty = x_empty + 8, w2_empty = w1_empty + 16;
+    const uint32_t s_full = w2_empty + 16, g_empty = s_full + 16, o_full = g_empty + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 20);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = cluster_ctarank();
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        mbar_init(x_full, 1);
+        mbar_init(o_empty, 2 * kEpiWarps);
+        mbar_init(x_empty, 1 + kEpiWarps);      // the last first-product commit + this CTA's residual readers
+        mbar_init(o_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(w1_full + 8 * i, 1); mbar_init(w2_full + 8 * i, 1);
+            mbar_init(w1_empty + 8 * i, 1); mbar_init(w2_empty + 8 * i, 1);
+            mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, 2 * kEpiWarps);
+            mbar_init(g_full + 8 * i, 2 * kEpiWarps); mbar_init(g_empty + 8 * i, 1);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w1); prefetch_tmap(&tmap_w2);
+    }
+    if (warp == 1) {
+        tmem_alloc<2>(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish<2>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    pdl_wait();
+    int M = p.M;
+    if (p.m_ptr != nullptr) M = min(M, __ldg(p.m_ptr));
+    const int blocks = (M + kPairRows - 1) / kPairRows;
+    const int pairs = gridDim.x / 2, pair0 = blockIdx.x / 2;
+    const int n_chunks = p.F / kChunk;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t nb = 0, cc = 0;   // blocks and chunks done so far
+            for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+                if (nb >= 1 && !(ok = mbar_wait(x_empty, (nb - 1) & 1, abort_flag))) break;
+                const uint32_t lead_x = map_to_cta(x_full, 0);
+                if (cta_rank == 0) mbar_expect_tx(x_full, 2 * C::X_BYTES);
+                const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
+                for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d_cg2(xs + kb * BLOCK_M * 128, &tmap_x, kb * BLOCK_K, xrow, lead_x);
+                for (int c = 0; c < n_chunks; ++c, ++cc) {
+                    const uint32_t st = cc & 1, use = cc >> 1;
+                    if (use >= 1 && !(ok = mbar_wait(w1_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                    const uint32_t lead1 = map_to_cta(w1_full + 8 * st, 0);
+                    if (cta_rank == 0) mbar_expect_tx(w1_full + 8 * st, 2 * C::W1_STAGE);
+                    for (int kb = 0; kb < C::KB1; ++kb)
+                        tma_load_2d_cg2(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128, &tmap_w1, kb * BLOCK_K,
+                                        c * kChunk + (int)cta_rank * C::W1_ROWS, lead1);
+                    if (use >= 1 && !(ok = mbar_wait(w2_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                    const uint32_t lead2 = map_to_cta(w2_full + 8 * st, 0);
+                    if (cta_rank == 0) mbar_expect_tx(w2_full + 8 * st, 2 * C::W2_STAGE);
+                    for (int i = 0; i < 2; ++i)   // instruction i covers output columns i*HID/2 .., this CTA feeds its half of them
+                        tma_load_2d_cg2(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128, &tmap_w2, c * kChunk,
+                                        i * (HID / 2) + (int)cta_rank * C::W2_ROWS, lead2);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA, one lane)
+        if (cta_rank == 0 && lane == 0) {
+            constexpr uint32_t id1 = make_idesc(kPairRows, kChunk), id2 = make_idesc(kPairRows, HID / 2);
+            bool ok = true;
+            uint32_t nb = 0, cc = 0;
+            auto first_product = [&](uint32_t q) -> bool {   // S_q: q counts chunks of all blocks
+                const uint32_t st = q & 1, use = q >> 1;
+                if (!mbar_wait(w1_full + 8 * st, use & 1, abort_flag)) return false;
+                if (use >= 1 && !mbar_wait(s_empty + 8 * st, (use - 1) & 1, abort_flag)) return false;
+                tc_fence_after();
+                for (int kb = 0; kb < C::KB1; ++kb) {
+                    const uint64_t adesc = make_smem_desc(xs + kb * BLOCK_M * 128);
+                    const uint64_t bdesc = make_smem_desc(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_bf16<2>(tmem + C::COL_S + st * kChunk, adesc + 2 * k, bdesc + 2 * k, id1, (kb | k) != 0 ? 1u : 0u);
+                }
+                umma_commit<2>(w1_empty + 8 * st);
+                umma_commit<2>(s_full + 8 * st);
+                return true;
+            };
+            for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+                if (!(ok = mbar_wait(x_full, nb & 1, abort_flag))) break;
+                if (!(ok = first_product(cc))) break;
+                for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
+                    if (c + 1 < n_chunks) {
+                        if (!(ok = first_product(cc + 1))) break;
+                    } else {
+                        umma_commit<2>(x_empty);   // the block's last read of X by the tensor core
+                    }
+                    const uint32_t st = cc & 1, use = cc >> 1;
+                    if (!(ok = mbar_wait(g_full + 8 * st, use & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait(w2_full + 8 * st, use & 1, abort_flag))) break;
+                    // first accumulation of the block overwrites O: the previous block's rows must have been read
+                    if (c == 0 && nb >= 1 && !(ok = mbar_wait(o_empty, (nb - 1) & 1, abort_flag))) break;
+                    tc_fence_after();
+                    const uint64_t adesc = make_smem_desc(gs + st * C::G_BYTES);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        const uint64_t bdesc = make_smem_desc(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128);
+#pragma unroll
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            umma_bf16<2>(tmem + i * (HID / 2), adesc + 2 * k, bdesc + 2 * k, id2, (c | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit<2>(w2_empty + 8 * st);
+                    umma_commit<2>(g_empty + 8 * st);
+                    if (c == n_chunks - 1) umma_commit<2>(o_full);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps (both CTAs)
+        const int ew = warp - 2, quad = warp & 3, half = ew >> 2;
+        const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+        const int r = quad * 32 + lane;                      // this thread's row within the CTA's 128
+            const uint32_t lead_s_empty = map_to_cta(s_empty, 0), lead_g_full = map_to_cta(g_full, 0), lead_o_empty = map_to_cta(o_empty, 0);
+        bool ok = true;
+        uint32_t nb = 0, cc = 0;
+        for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+            for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
+                const uint32_t st = cc & 1, use = cc >> 1;
+                if (!(ok = mbar_wait(s_full + 8 * st, use & 1, abort_flag))) break;
+                tc_fence_after();
+                uint32_t acc[32];
+                tmem_ld_32x32(lane_addr + C::COL_S + st * kChunk + half * 32, acc);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster_relaxed(lead_s_empty + 8 * st);   // S buffer back to the MMA thread
+                const float* b1 = p.b1 + c * kChunk + half * 32;
+                float v[32];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 b = __ldg(reinterpret_cast<const float4*>(b1) + i);
+                    v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b.x;
+                    v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b.y;
+                    v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b.z;
+                    v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b.w;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
+                // the G buffer is free once the second product of two chunks ago has read it
+                if (use >= 1 && !(ok = mbar_wait(g_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 q;
+                    q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]); q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+                    q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]); q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+                    st_shared_v4(gs + st * C::G_BYTES + sw128(r, half * 4 + i), q);
+                }
+                fence_proxy_async();     // generic-proxy writes -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(lead_g_full + 8 * st);   // release: orders the stores above
+            }
+            if (!ok) break;
+            // ---- end of the block: out = O + b2 + X ----
+            if (!(ok = mbar_wait(o_full, nb & 1, abort_flag))) break;
+            tc_fence_after();
+            const int row = blk * kPairRows + (int)cta_rank * BLOCK_M + r;
+            constexpr int kChunksPerWarp = HID / 64;   // this warp's column half = HID/2 columns = HID/64 chunks of 32
+#pragma unroll 1
+            for (int ch = 0; ch < kChunksPerWarp; ++ch) {
+                const int col0 = half * (HID / 2) + ch * 32;
+                uint32_t acc[32];
+                tmem_ld_32x32(lane_addr + col0, acc);
+                tmem_ld_wait();
+                if (ch == kChunksPerWarp - 1) {   // last read of O by this warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
+                }
+                const float* b2 = p.b2 + col0;
+                const int kb = col0 / 64, j0 = (col0 % 64) / 8;    // residual: X's k-block tile kb, 16-byte chunks j0 .. j0+3
+                uint4 q[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 x = ld_shared_v4(xs + kb * BLOCK_M * 128 + sw128(r, j0 + i));
+                    const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
+                    const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
+                    q[i].x = pack_bf16(__uint_as_float(acc[8 * i + 0]) + ba.x + bf16lo(x.x), __uint_as_float(acc[8 * i + 1]) + ba.y + bf16hi(x.x));
+                    q[i].y = pack_bf16(__uint_as_float(acc[8 * i + 2]) + ba.z + bf16lo(x.y), __uint_as_float(acc[8 * i + 3]) + ba.w + bf16hi(x.y));
+                    q[i].z = pack_bf16(__uint_as_float(acc[8 * i + 4]) + bb.x + bf16lo(x.z), __uint_as_float(acc[8 * i + 5]) + bb.y + bf16hi(x.z));
+                    q[i].w = pack_bf16(__uint_as_float(acc[8 * i + 6]) + bb.z + bf16lo(x.w), __uint_as_float(acc[8 * i + 7]) + bb.w + bf16hi(x.w));
+                }
+                if (row < p.M) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)row * HID + col0);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dst[i] = q[i];
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_empty);   // this warp's residual reads of X are done
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicOr(p.status, RLX_DEVSTAT_TIMEOUT_BIT);
+        const uint64_t t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc<2>(tmem, C::TMEM_COLS);
+    }
+}
+
+}  // namespace tcff
+}  // namespace rlx

@@ -14,6 +14,7 @@
 #include "attention.cuh"
 #include "attention_tc.cuh"
 #include "gemm_mx_tcgen05.cuh"
+#include "gemm_ffn_tcgen05.cuh"
 #include "dequant.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tcgen05.cuh"
@@ -231,6 +232,10 @@ cudaError_t init_kernels_for_current_device() {
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tcar::gemm_ares_tcgen05_kernel<256, 0>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs_resident[dev] = n;
     }
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcff::Cfg<384>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tcmx::gemm_mx_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcmx::kSmemBytes)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tcmx::wide::gemm_mx192_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -419,6 +424,35 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
                                tq, seq_start, seq_len, ctx, H, scale_log2e, B, qtiles, ticket, status));
     else
         return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(cudaGetLastError());
+    return RLX_OK;
+}
+
+// Feed-forward block in one kernel (hidden 256 or 384, F % 64 == 0): out = gelu(x W1^T + b1) W2^T + b2 + x.
+bool ffn_fused_supported(int H, int F) { return (H == 256 || H == 384) && F % 64 == 0 && F >= 64; }
+rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, const bf16* w2, const float* b2, int M, int H,
+                              int F, bf16* out, int32_t* status, cudaStream_t st, const int32_t* rows_ptr) {
+    if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
+    CUtensorMap tx, t1, t2;
+    if (!make_tmap(&tx, x, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M) ||
+        !make_tmap(&t1, w1, (uint64_t)F, (uint64_t)H, H == 384 ? rlx::tcff::Cfg<384>::W1_ROWS : rlx::tcff::Cfg<256>::W1_ROWS) ||
+        !make_tmap(&t2, w2, (uint64_t)H, (uint64_t)F, H == 384 ? rlx::tcff::Cfg<384>::W2_ROWS : rlx::tcff::Cfg<256>::W2_ROWS))
+        return RLX_ERR_CUDA;
+    rlx::tcff::FfnParams p;
+    p.b1 = b1; p.b2 = b2; p.out = out; p.M = M; p.F = F; p.m_ptr = rows_ptr; p.status = status;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int pairs_max = (dev >= 0 && dev < 64 && g_max_pairs_resident[dev] > 0) ? g_max_pairs_resident[dev] : sm_count() / 2;
+    const int blocks = (M + rlx::tcff::kPairRows - 1) / rlx::tcff::kPairRows;
+    const int grid = 2 * std::min(blocks, pairs_max);
+    struct ClusterScope {
+        ClusterScope() { g_cluster_x = 2; }
+        ~ClusterScope() { g_cluster_x = 1; }
+    } scope;
+    if (H == 384)
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, p));
+    else
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, p));
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -779,6 +813,14 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
     return (long long)B * S >= 128ll * sm_count_of(c.device);
 }
 
+// RLX_FLAG_FUSED_FFN: FFN-up, GELU and FFN-down in one kernel (needs the plain 7-kernel layer around it).
+bool ffn_fused_supported(int H, int F);
+bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S);
+bool uses_fused_ffn(const rlx_encoder_config_t& c, int B, int S) {
+    if (!(c.flags & RLX_FLAG_FUSED_FFN) || (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN))) return false;
+    return ffn_fused_supported(c.hidden, c.ffn) && !uses_fold_ln(c, B, S);
+}
+
 // RLX_FLAG_CLUSTER_LN: LayerNorm folded into the out-proj / FFN-down GEMMs with cluster-wide row
 // statistics.  Opt-in: the two exchanges per tile cost about what the separate LayerNorm kernel costs.
 bool uses_cluster_ln(const rlx_encoder_config_t& c) {
@@ -807,7 +849,7 @@ bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S) {
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
     const bool fused = uses_fold_ln(c, B, S) || uses_fused_ln(c, B, S) || uses_cluster_ln(c);
-    return 2 + (fused ? 5 : 7) * c.num_layers + (pack ? 1 : 0);
+    return 2 + ((fused ? 5 : 7) - (uses_fused_ffn(c, B, S) ? 1 : 0)) * c.num_layers + (pack ? 1 : 0);
 }
 bool uses_chunks(const rlx_encoder_config_t& c, int B, int S);
 int chunk_batch(int B, int S);
@@ -929,6 +971,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     const int32_t* rows = pk.total();
     const bool fuse_ln = !fold && uses_fused_ln(c, B, S);
     const bool fuse_cln = !fold && !fuse_ln && uses_cluster_ln(c);
+    const bool fuse_ffn = uses_fused_ffn(c, B, S);
     if (fold) {
         // ---- LayerNorm folded into the GEMMs: 5 kernels per layer, no LayerNorm kernel ----
         // gamma-scaled weights and their c / d vectors, rebuilt inside every forward (weights may change
@@ -1045,6 +1088,12 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         } else {
             RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
             RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
+        }
+        if (fuse_ffn) {
+            // the whole feed-forward block in one kernel: the F-wide activation stays on the chip
+            RLX_TRY(launch_ffn_fused(x1, (const bf16*)lw.w1, lw.b1, (const bf16*)lw.w2, lw.b2, T, H, F, y, status, st, rows));
+            RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
+            continue;
         }
         RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
         if (fuse_ln) {
@@ -1723,6 +1772,17 @@ rlx_status_t rlx_mx_matmul_bf16(const void* a_codes, const void* a_scales, int32
     }
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
+}
+
+rlx_status_t rlx_ffn_fused_bf16(const void* x, const void* w1, const float* b1, const void* w2, const float* b2,
+                                int32_t M, int32_t H, int32_t F, void* out, int32_t* status, void* stream) {
+    if (!x || !w1 || !b1 || !w2 || !b2 || !out || M <= 0 || H <= 0 || F <= 0) return RLX_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w1) || !aligned16(b1) || !aligned16(w2) || !aligned16(b2) || !aligned16(out))
+        return RLX_ERR_INVALID_ARG;
+    if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    return launch_ffn_fused((const bf16*)x, (const bf16*)w1, b1, (const bf16*)w2, b2, M, H, F, (bf16*)out, status,
+                            static_cast<cudaStream_t>(stream), nullptr);
 }
 
 rlx_status_t rlx_pool_l2norm(const void* x, const int32_t* mask, int32_t B, int32_t S, int32_t H, float* out,

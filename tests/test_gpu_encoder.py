@@ -326,3 +326,19 @@ def test_graph_cache_reuse_and_new_inputs(rlx):
     ref3 = oracle.encoder_forward(c, ids2, inp.mask, other.params, other.layers)
     check(to_np64(out), ref3, inp.lengths)
     enc.close()
+
+
+@pytest.mark.parametrize("flags", [0x1400, 0x1401], ids=["graph", "eager"])
+def test_fused_ffn_forward_is_bitwise_the_two_kernel_forward(rlx, flags):
+    """RLX_FLAG_FUSED_FFN: FFN-up, GELU and FFN-down of every layer in one kernel.  Same rounding points and
+    the same k order as the two-kernel form, so the embeddings agree bit for bit with the plain 7-kernel
+    layer (0x400 keeps LayerNorm folding out of both)."""
+    inp = make_inputs(CONFIGS["c2"])
+    w = rlx.upload_weights(inp.params, inp.layers)
+    plain, status = run_gpu(rlx, inp, weights=w, flags=0x400 | (flags & 1))
+    assert status == 0
+    fused, status = run_gpu(rlx, inp, weights=w, flags=flags)
+    assert status == 0
+    assert np.array_equal(plain, fused)
+    ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
+    check(fused, ref, inp.lengths)
