@@ -79,7 +79,7 @@ typedef enum {
                                    fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
 #define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
 #define RLX_FLAG_FUSED_FFN 0x1000u /* FFN-up, GELU and FFN-down in ONE kernel per layer (the F-wide activation never
-                                      reaches global memory); hidden 256 or 384, F % 64 == 0; ignored together with the
+                                      reaches global memory); hidden 256 or 384, F % 128 == 0; ignored together with the
                                       LayerNorm fusion flags, the bring-up GEMM, or where the folded layer is chosen */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
@@ -542,7 +542,7 @@ rlx_status_t rlx_mx_matmul_bf16(const void *a_codes, const void *a_scales_e8m0, 
  * x, out: device bf16 [M, H]; w1: bf16 [F, H]; w2: bf16 [H, F]; b1: f32 [F]; b2: f32 [H]; all 16-byte aligned.
  * The F-wide activation is produced and consumed in 64-column chunks on the chip (tensor memory ->
  * registers -> shared memory) and rounded to bf16 once, as in the two-kernel form; fp32 accumulation.
- * H in {256, 384}, F % 64 == 0 (RLX_ERR_UNSUPPORTED otherwise).  status: optional device word that
+ * H in {256, 384}, F % 128 == 0 (RLX_ERR_UNSUPPORTED otherwise).  status: optional device word that
  * receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.  Asynchronous on cuda_stream.
  */
 rlx_status_t rlx_ffn_fused_bf16(const void *x_bf16, const void *w1_bf16, const float *b1, const void *w2_bf16,

@@ -10,11 +10,16 @@
 //                                                         written in the K-major 128-byte-swizzled layout the
 //                                                         tensor core reads (two G buffers of one k-block)
 //              O  += G_c W2[:, 64c .. 64c+63]^T           M = 256, N = H (two instructions of H/2), K = 64
-//   end        out = O + b2 + X  -> bf16 -> 16-byte stores of whole 64-byte row segments (no staging: the
-//              shared memory is full, and a buffer shared with G would need an unbounded barrier between warps)
-// The MMA thread issues S_{c+1} before O += G_c ..., so the tensor core works on the next chunk's first
-// product while the epilogue warps turn S_c into G_c.  W1 / W2 chunks stream through two-stage rings, each
-// CTA loading its half of the rows.  TMEM: O (H columns) + 2 x 64 columns of S = 512 at H = 384.
+//   end        out = O + b2 + X  -> bf16, written back over the X tile slots the residual was read from, and
+//              stored from there with one TMA store per warp and 64-column tile (the shared memory is full,
+//              the X tiles are the only staging room and already have the store's layout)
+// Roles (per CTA): warp 0 loads X and the W1 chunks, another warp the W2 chunks (so a late W2 slot never holds
+// back W1); in the leader CTA two warps issue the first products (even / odd chunks) and a third the second
+// products -- a thread pays ~100 cycles per tcgen05.mma, and one thread for a chunk's 32 instructions paced the
+// kernel; eight epilogue warps turn S_c into G_c in a software pipeline that overlaps the barrier probes and
+// the tensor-memory load of S_{c+1} with the GELU arithmetic of S_c.  W1 / W2 chunks stream through
+// two-stage rings, each CTA loading its half of the rows.  TMEM: O (H columns) + 2 x 64 columns of S = 512
+// at H = 384.
 // Rounding points are those of the two-kernel form (G rounded to bf16 once, fp32 accumulation in the same
 // k order), so the results agree with it to the last bit wherever the accumulation order is the same.
 // All mbarrier waits are bounded; on expiry the CTA sets the status bit and leaves.
@@ -32,7 +37,7 @@ using namespace rlx::tc;
 constexpr int kPairRows = 256;
 constexpr int kChunk = 64;          // hidden columns per chunk = one k-block of the second product
 constexpr int kEpiWarps = 8;        // per CTA: lane quarter x column half of a 64-column S chunk
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kThreads = 64 + 32 * kEpiWarps + 96;   // TMA, first products (even chunks), epilogue warps, second products, first products (odd chunks), W2 loads
 
 template <int HID>
 struct Cfg {
@@ -68,7 +73,7 @@ __device__ __forceinline__ uint32_t sw128(int r, int j) { return (uint32_t)(r * 
 template <int HID>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
-                         const __grid_constant__ CUtensorMap tmap_w2, const FfnParams p) {
+                         const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out, const FfnParams p) {
     using C = Cfg<HID>;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -91,7 +96,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     if (threadIdx.x == 0) {
         mbar_init(x_full, 1);
         mbar_init(o_empty, 2 * kEpiWarps);
-        mbar_init(x_empty, 1 + kEpiWarps);      // the last first-product commit + this CTA's residual readers
+        mbar_init(x_empty, 2 + kEpiWarps);      // both first-product warps' last commits + this CTA's epilogue warps
         mbar_init(o_full, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(w1_full + 8 * i, 1); mbar_init(w2_full + 8 * i, 1);
@@ -101,7 +106,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         }
         *abort_flag = 0;
         fence_barrier_init();
-        prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w1); prefetch_tmap(&tmap_w2);
+        prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w1); prefetch_tmap(&tmap_w2); prefetch_tmap(&tmap_out);
     }
     if (warp == 1) {
         tmem_alloc<2>(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -121,7 +126,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     const int n_chunks = p.F / kChunk;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer (both CTAs)
+        // ------------------------------------------------------------ TMA producer of X and the W1 chunks (both CTAs)
         if (lane == 0) {
             bool ok = true;
             uint32_t nb = 0, cc = 0;   // blocks and chunks done so far
@@ -139,6 +144,19 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                     for (int kb = 0; kb < C::KB1; ++kb)
                         tma_load_2d_cg2(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128, &tmap_w1, kb * BLOCK_K,
                                         c * kChunk + (int)cta_rank * C::W1_ROWS, lead1);
+                }
+            }
+        }
+    } else if (warp == 4 + kEpiWarps) {
+        // ------------------------------------------------------------ TMA producer of the W2 chunks (both CTAs)
+        // A thread of its own: behind the W1 loads in one thread, a W2 slot that frees late (its second
+        // product waits for the epilogue warps) would hold back the next chunk's W1 tiles as well.
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t cc = 0;
+            for (int blk = pair0; blk < blocks && ok; blk += pairs) {
+                for (int c = 0; c < n_chunks; ++c, ++cc) {
+                    const uint32_t st = cc & 1, use = cc >> 1;
                     if (use >= 1 && !(ok = mbar_wait(w2_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
                     const uint32_t lead2 = map_to_cta(w2_full + 8 * st, 0);
                     if (cta_rank == 0) mbar_expect_tx(w2_full + 8 * st, 2 * C::W2_STAGE);
@@ -148,54 +166,71 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer (leader CTA, one lane)
-        if (cta_rank == 0 && lane == 0) {
-            constexpr uint32_t id1 = make_idesc(kPairRows, kChunk), id2 = make_idesc(kPairRows, HID / 2);
+    } else if (warp == 1 || warp == 3 + kEpiWarps) {
+        // ------------------------------------------------------------ first products S_c = X W1_c^T (leader CTA)
+        // Three issuing warps in all: a thread pays ~80-110 cycles per tcgen05.mma and ~230 per barrier round,
+        // and a chunk is 24 + 8 instructions, so one thread for everything was the kernel's limiter.  The
+        // first products alternate between two warps by chunk parity (warp 1: even chunks into S buffer 0,
+        // a second warp: odd chunks into S buffer 1; F is a multiple of 128, so the parity of a chunk is
+        // the parity of its ring slot in every block); a third warp issues the second products.  Whole-warp
+        // loops, one elected lane issues.
+        if (cta_rank == 0) {
+            constexpr uint32_t id1 = make_idesc(kPairRows, kChunk);
+            const uint32_t st = warp == 1 ? 0u : 1u;
+            bool ok = true;
+            uint32_t nb = 0;
+            for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+                if (!(ok = mbar_wait_warp(x_full, nb & 1, abort_flag))) break;
+                for (int c = st; c < n_chunks && ok; c += 2) {
+                    const uint32_t use = (nb * n_chunks + c) >> 1;
+                    if (!(ok = mbar_wait_warp(w1_full + 8 * st, use & 1, abort_flag))) break;
+                    if (use >= 1 && !(ok = mbar_wait_warp(s_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+                        for (int kb = 0; kb < C::KB1; ++kb) {
+                            const uint64_t adesc = make_smem_desc(xs + kb * BLOCK_M * 128);
+                            const uint64_t bdesc = make_smem_desc(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128);
+#pragma unroll
+                            for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                                umma_bf16<2>(tmem + C::COL_S + st * kChunk, adesc + 2 * k, bdesc + 2 * k, id1, (kb | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit<2>(w1_empty + 8 * st);
+                        umma_commit<2>(s_full + 8 * st);
+                        // this warp's last read of X in the block; the barrier counts both first-product warps
+                        if (c + 2 >= n_chunks) umma_commit<2>(x_empty);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+    } else if (warp == 2 + kEpiWarps) {
+        // ------------------------------------------------------------ second products O += G_c W2_c^T (leader CTA)
+        if (cta_rank == 0) {
+            constexpr uint32_t id2 = make_idesc(kPairRows, HID / 2);
             bool ok = true;
             uint32_t nb = 0, cc = 0;
-            auto first_product = [&](uint32_t q) -> bool {   // S_q: q counts chunks of all blocks
-                const uint32_t st = q & 1, use = q >> 1;
-                if (!mbar_wait(w1_full + 8 * st, use & 1, abort_flag)) return false;
-                if (use >= 1 && !mbar_wait(s_empty + 8 * st, (use - 1) & 1, abort_flag)) return false;
-                tc_fence_after();
-                for (int kb = 0; kb < C::KB1; ++kb) {
-                    const uint64_t adesc = make_smem_desc(xs + kb * BLOCK_M * 128);
-                    const uint64_t bdesc = make_smem_desc(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128);
-#pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_bf16<2>(tmem + C::COL_S + st * kChunk, adesc + 2 * k, bdesc + 2 * k, id1, (kb | k) != 0 ? 1u : 0u);
-                }
-                umma_commit<2>(w1_empty + 8 * st);
-                umma_commit<2>(s_full + 8 * st);
-                return true;
-            };
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                if (!(ok = mbar_wait(x_full, nb & 1, abort_flag))) break;
-                if (!(ok = first_product(cc))) break;
                 for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
-                    if (c + 1 < n_chunks) {
-                        if (!(ok = first_product(cc + 1))) break;
-                    } else {
-                        umma_commit<2>(x_empty);   // the block's last read of X by the tensor core
-                    }
                     const uint32_t st = cc & 1, use = cc >> 1;
-                    if (!(ok = mbar_wait(g_full + 8 * st, use & 1, abort_flag))) break;
-                    if (!(ok = mbar_wait(w2_full + 8 * st, use & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait_warp(w2_full + 8 * st, use & 1, abort_flag))) break;
                     // first accumulation of the block overwrites O: the previous block's rows must have been read
-                    if (c == 0 && nb >= 1 && !(ok = mbar_wait(o_empty, (nb - 1) & 1, abort_flag))) break;
+                    if (c == 0 && nb >= 1 && !(ok = mbar_wait_warp(o_empty, (nb - 1) & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait_warp(g_full + 8 * st, use & 1, abort_flag))) break;
                     tc_fence_after();
-                    const uint64_t adesc = make_smem_desc(gs + st * C::G_BYTES);
+                    if (elect_one()) {
+                        const uint64_t adesc = make_smem_desc(gs + st * C::G_BYTES);
 #pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const uint64_t bdesc = make_smem_desc(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128);
+                        for (int i = 0; i < 2; ++i) {
+                            const uint64_t bdesc = make_smem_desc(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128);
 #pragma unroll
-                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                            umma_bf16<2>(tmem + i * (HID / 2), adesc + 2 * k, bdesc + 2 * k, id2, (c | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                                umma_bf16<2>(tmem + i * (HID / 2), adesc + 2 * k, bdesc + 2 * k, id2, (c | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit<2>(w2_empty + 8 * st);
+                        umma_commit<2>(g_empty + 8 * st);
+                        if (c == n_chunks - 1) umma_commit<2>(o_full);
                     }
-                    umma_commit<2>(w2_empty + 8 * st);
-                    umma_commit<2>(g_empty + 8 * st);
-                    if (c == n_chunks - 1) umma_commit<2>(o_full);
+                    __syncwarp();
                 }
             }
         }
@@ -208,16 +243,26 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         bool ok = true;
         uint32_t nb = 0, cc = 0;
         for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-            for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
+            // Software pipeline over the chunks: the registers hold S_c when an iteration starts; the probe of
+            // S_{c+1}'s barrier, the tensor-memory load of S_{c+1} and the probe of the G buffer's barrier are
+            // issued between the halves of the GELU arithmetic, so their round trips (150-250 cycles each)
+            // overlap it instead of adding to the chain  S ready -> G ready  that paces the whole kernel.
+            uint32_t acc[32];
+            {
                 const uint32_t st = cc & 1, use = cc >> 1;
                 if (!(ok = mbar_wait(s_full + 8 * st, use & 1, abort_flag))) break;
                 tc_fence_after();
-                uint32_t acc[32];
                 tmem_ld_32x32(lane_addr + C::COL_S + st * kChunk + half * 32, acc);
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster_relaxed(lead_s_empty + 8 * st);   // S buffer back to the MMA thread
+            }
+            for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
+                const uint32_t st = cc & 1, use = cc >> 1;
+                const bool more = c + 1 < n_chunks;
+                const uint32_t nst = st ^ 1, nuse = (cc + 1) >> 1;
+                const bool s_ready = more && mbar_test_wait(s_full + 8 * nst, nuse & 1);
                 const float* b1 = p.b1 + c * kChunk + half * 32;
                 float v[32];
 #pragma unroll
@@ -229,58 +274,87 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                     v[4 * i + 3] = __uint_as_float(acc[4 * i + 3]) + b.w;
                 }
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
+                for (int i = 0; i < 16; i += 2) gelu_erf_x2(v[i], v[i + 1]);
+                if (more) {
+                    if (!s_ready && !(ok = mbar_wait(s_full + 8 * nst, nuse & 1, abort_flag))) break;
+                    tc_fence_after();
+                    tmem_ld_32x32(lane_addr + C::COL_S + nst * kChunk + half * 32, acc);   // lands during the second half
+                }
                 // the G buffer is free once the second product of two chunks ago has read it
-                if (use >= 1 && !(ok = mbar_wait(g_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                const bool g_ready = use < 1 || mbar_test_wait(g_empty + 8 * st, (use - 1) & 1);
+#pragma unroll
+                for (int i = 16; i < 32; i += 2) gelu_erf_x2(v[i], v[i + 1]);
+                uint4 q[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    uint4 q;
-                    q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]); q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
-                    q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]); q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-                    st_shared_v4(gs + st * C::G_BYTES + sw128(r, half * 4 + i), q);
+                    q[i].x = pack_bf16(v[8 * i + 0], v[8 * i + 1]); q[i].y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+                    q[i].z = pack_bf16(v[8 * i + 4], v[8 * i + 5]); q[i].w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
                 }
+                if (!g_ready && !(ok = mbar_wait(g_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) st_shared_v4(gs + st * C::G_BYTES + sw128(r, half * 4 + i), q[i]);
                 fence_proxy_async();     // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(lead_g_full + 8 * st);   // release: orders the stores above
+                if (lane == 0) mbar_arrive_cluster_release_cta(lead_g_full + 8 * st);
+                if (more) {
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster_relaxed(lead_s_empty + 8 * nst);
+                }
             }
             if (!ok) break;
             // ---- end of the block: out = O + b2 + X ----
             if (!(ok = mbar_wait(o_full, nb & 1, abort_flag))) break;
             tc_fence_after();
-            const int row = blk * kPairRows + (int)cta_rank * BLOCK_M + r;
-            constexpr int kChunksPerWarp = HID / 64;   // this warp's column half = HID/2 columns = HID/64 chunks of 32
+            // The resident X tiles serve twice more: each thread reads its residual values from them and writes
+            // the finished bf16 outputs back to the same 16-byte slots (same rows, same swizzle), and the warp
+            // then stores its 32-row slice of a 64-column tile with one TMA store -- the tile's layout in shared
+            // memory is the one the TMA load produced, so the store map has the load map's geometry.
+            const int row0 = blk * kPairRows + (int)cta_rank * BLOCK_M + quad * 32;
+            constexpr int kTilesPerWarp = HID / 128;   // this warp's column half = HID/2 columns = HID/128 tiles of 64
 #pragma unroll 1
-            for (int ch = 0; ch < kChunksPerWarp; ++ch) {
-                const int col0 = half * (HID / 2) + ch * 32;
-                uint32_t acc[32];
-                tmem_ld_32x32(lane_addr + col0, acc);
-                tmem_ld_wait();
-                if (ch == kChunksPerWarp - 1) {   // last read of O by this warp
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
-                }
-                const float* b2 = p.b2 + col0;
-                const int kb = col0 / 64, j0 = (col0 % 64) / 8;    // residual: X's k-block tile kb, 16-byte chunks j0 .. j0+3
-                uint4 q[4];
+            for (int t = 0; t < kTilesPerWarp; ++t) {
+                const int kb = half * kTilesPerWarp + t;
+                const uint32_t tile = xs + kb * BLOCK_M * 128;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 x = ld_shared_v4(xs + kb * BLOCK_M * 128 + sw128(r, j0 + i));
-                    const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
-                    const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
-                    q[i].x = pack_bf16(__uint_as_float(acc[8 * i + 0]) + ba.x + bf16lo(x.x), __uint_as_float(acc[8 * i + 1]) + ba.y + bf16hi(x.x));
-                    q[i].y = pack_bf16(__uint_as_float(acc[8 * i + 2]) + ba.z + bf16lo(x.y), __uint_as_float(acc[8 * i + 3]) + ba.w + bf16hi(x.y));
-                    q[i].z = pack_bf16(__uint_as_float(acc[8 * i + 4]) + bb.x + bf16lo(x.z), __uint_as_float(acc[8 * i + 5]) + bb.y + bf16hi(x.z));
-                    q[i].w = pack_bf16(__uint_as_float(acc[8 * i + 6]) + bb.z + bf16lo(x.w), __uint_as_float(acc[8 * i + 7]) + bb.w + bf16hi(x.w));
-                }
-                if (row < p.M) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)row * HID + col0);
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int col0 = kb * 64 + hh * 32;
+                    uint32_t acc[32];
+                    tmem_ld_32x32(lane_addr + col0, acc);
+                    tmem_ld_wait();
+                    if (t == kTilesPerWarp - 1 && hh == 1) {   // last read of O by this warp
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
+                    }
+                    const float* b2 = p.b2 + col0;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) dst[i] = q[i];
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t slot = tile + sw128(r, hh * 4 + i);
+                        const uint4 x = ld_shared_v4(slot);
+                        const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
+                        const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
+                        uint4 q;
+                        q.x = pack_bf16(__uint_as_float(acc[8 * i + 0]) + ba.x + bf16lo(x.x), __uint_as_float(acc[8 * i + 1]) + ba.y + bf16hi(x.x));
+                        q.y = pack_bf16(__uint_as_float(acc[8 * i + 2]) + ba.z + bf16lo(x.y), __uint_as_float(acc[8 * i + 3]) + ba.w + bf16hi(x.y));
+                        q.z = pack_bf16(__uint_as_float(acc[8 * i + 4]) + bb.x + bf16lo(x.z), __uint_as_float(acc[8 * i + 5]) + bb.y + bf16hi(x.z));
+                        q.w = pack_bf16(__uint_as_float(acc[8 * i + 6]) + bb.z + bf16lo(x.w), __uint_as_float(acc[8 * i + 7]) + bb.w + bf16hi(x.w));
+                        st_shared_v4(slot, q);
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(&tmap_out, kb * 64, row0, tile + quad * 32 * 128);   // rows past the matrix are clipped
+                    bulk_commit();
                 }
             }
+            if (lane == 0) {
+                bulk_wait_read<0>();      // the stores have read their slices: X may be overwritten
+                mbar_arrive(x_empty);
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(x_empty);   // this warp's residual reads of X are done
         }
     }
 

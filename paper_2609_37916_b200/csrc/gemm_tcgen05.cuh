@@ -111,6 +111,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Non-blocking probe (try_wait may suspend the thread for a while; this one never does): issued early,
+// its result is consumed after independent work, which hides the round trip to the barrier.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false when the budget ran out or another role already aborted.
 __device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t budget_ns) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -182,6 +195,13 @@ __device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
 }
 __device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Arrival on another CTA's barrier that publishes only shared-memory stores of the arriving warp which a
+// fence.proxy.async has already made visible to the async proxy (an operand tile written from registers
+// for the tensor core of this same SM).  Release at CTA scope: the cluster-scope form also waits for the
+// thread's global traffic and costs over a thousand cycles per arrival.
+__device__ __forceinline__ void mbar_arrive_cluster_release_cta(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cta.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

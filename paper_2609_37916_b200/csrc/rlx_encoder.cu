@@ -429,12 +429,12 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
 }
 
 // Feed-forward block in one kernel (hidden 256 or 384, F % 64 == 0): out = gelu(x W1^T + b1) W2^T + b2 + x.
-bool ffn_fused_supported(int H, int F) { return (H == 256 || H == 384) && F % 64 == 0 && F >= 64; }
+bool ffn_fused_supported(int H, int F) { return (H == 256 || H == 384) && F % 128 == 0 && F >= 128; }
 rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, const bf16* w2, const float* b2, int M, int H,
                               int F, bf16* out, int32_t* status, cudaStream_t st, const int32_t* rows_ptr) {
     if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
-    CUtensorMap tx, t1, t2;
-    if (!make_tmap(&tx, x, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M) ||
+    CUtensorMap tx, t1, t2, to;
+    if (!make_tmap(&tx, x, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M) || !make_tmap(&to, out, (uint64_t)M, (uint64_t)H, 32) ||
         !make_tmap(&t1, w1, (uint64_t)F, (uint64_t)H, H == 384 ? rlx::tcff::Cfg<384>::W1_ROWS : rlx::tcff::Cfg<256>::W1_ROWS) ||
         !make_tmap(&t2, w2, (uint64_t)H, (uint64_t)F, H == 384 ? rlx::tcff::Cfg<384>::W2_ROWS : rlx::tcff::Cfg<256>::W2_ROWS))
         return RLX_ERR_CUDA;
@@ -450,9 +450,9 @@ rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, co
         ~ClusterScope() { g_cluster_x = 1; }
     } scope;
     if (H == 384)
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, p));
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
     else
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, p));
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
