@@ -325,7 +325,7 @@ class EncoderRun:
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         self.n_kernels = self.enc.kernels_per_forward(B, S)
         per_layer = (self.n_kernels - 3) // cfg.num_layers
-        fused_ffn = bool(args.flags & 0x1000) and per_layer in (4, 6)
+        fused_ffn = per_layer in (4, 6)   # 7 = plain layer, 5 = LayerNorm fused into the GEMMs, one less with the one-kernel feed-forward block
         self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer + (1 if fused_ffn else 0) == 5), fused_ffn=fused_ffn)
         assert len(self.names) == self.n_kernels
 

@@ -79,8 +79,13 @@ typedef enum {
                                    fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
 #define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
 #define RLX_FLAG_FUSED_FFN 0x1000u /* FFN-up, GELU and FFN-down in ONE kernel per layer (the F-wide activation never
-                                      reaches global memory); hidden 256 or 384, F % 128 == 0; ignored together with the
-                                      LayerNorm fusion flags, the bring-up GEMM, or where the folded layer is chosen */
+                                      reaches global memory) at every batch size; hidden 256 or 384, F % 128 == 0;
+                                      ignored together with the LayerNorm fusion flags, the bring-up GEMM, or where
+                                      the folded layer is chosen.  Without this flag the one-kernel form is chosen
+                                      AUTOMATICALLY for calls with batch*seq >= 16384 (it works in blocks of 256
+                                      rows per CTA pair and needs about a wave of them to beat the two GEMMs);
+                                      results are bit for bit those of the two-kernel form */
+#define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep FFN-up and FFN-down as two GEMM kernels at every batch size */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
                                    kernel's input is still in L2 when its consumer starts.  Results are bit for bit

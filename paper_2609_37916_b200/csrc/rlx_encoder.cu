@@ -813,11 +813,16 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
     return (long long)B * S >= 128ll * sm_count_of(c.device);
 }
 
-// RLX_FLAG_FUSED_FFN: FFN-up, GELU and FFN-down in one kernel (needs the plain 7-kernel layer around it).
+// FFN-up, GELU and FFN-down in one kernel (needs the plain 7-kernel layer around it).  The kernel works in
+// blocks of 256 rows, one per CTA pair, so it needs about a wave of blocks to beat the two GEMMs: forced by
+// RLX_FLAG_FUSED_FFN at any size, chosen by itself from 16384 padded tokens on (the number of valid tokens
+// is known only on the device), never with RLX_FLAG_NO_FUSED_FFN.
+constexpr long long kAutoFusedFfnMinTokens = 16384;
 bool ffn_fused_supported(int H, int F);
 bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S);
 bool uses_fused_ffn(const rlx_encoder_config_t& c, int B, int S) {
-    if (!(c.flags & RLX_FLAG_FUSED_FFN) || (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN))) return false;
+    if (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN | RLX_FLAG_NO_FUSED_FFN)) return false;
+    if (!(c.flags & RLX_FLAG_FUSED_FFN) && (long long)B * S < kAutoFusedFfnMinTokens) return false;
     return ffn_fused_supported(c.hidden, c.ffn) && !uses_fold_ln(c, B, S);
 }
 

@@ -342,3 +342,22 @@ def test_fused_ffn_forward_is_bitwise_the_two_kernel_forward(rlx, flags):
     assert np.array_equal(plain, fused)
     ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
     check(fused, ref, inp.lengths)
+
+
+def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
+    """Without a flag the one-kernel feed-forward block takes over at batch*seq >= 16384; RLX_FLAG_NO_FUSED_FFN
+    (0x2000) keeps the two GEMMs.  Same embeddings bit for bit, one kernel less per layer."""
+    inp = make_inputs(CONFIGS["c2"], batch=130, num_layers=2)
+    w = rlx.upload_weights(inp.params, inp.layers)
+    auto, status = run_gpu(rlx, inp, weights=w, flags=0)
+    assert status == 0
+    two, status = run_gpu(rlx, inp, weights=w, flags=0x2000)
+    assert status == 0
+    assert np.array_equal(auto, two)
+    c = inp.cfg
+    assert c.batch * c.seq >= 16384
+    a = rlx.Encoder.from_config(c, flags=0, max_batch=c.batch, max_seq=c.seq)
+    b = rlx.Encoder.from_config(c, flags=0x2000, max_batch=c.batch, max_seq=c.seq)
+    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == c.num_layers
+    assert a.kernels_per_forward(127, 128) == b.kernels_per_forward(127, 128)
+    a.close(); b.close()
