@@ -203,8 +203,8 @@ def workload_config(name: str, extra=None):
 # ---------------------------------------------------------------------------- roofline bookkeeping
 def kernel_classes(num_layers: int, fused_ln: bool, fused_ffn: bool = False):
     per_layer = [k for k in KERNEL_CLASSES if not (fused_ln and k in ("ln1", "ln2"))]
-    if fused_ffn:   # FFN-up, GELU and FFN-down are one kernel
-        per_layer = [k for k in per_layer if k != "gemm_ffn2"]
+    if fused_ffn:   # FFN-up, GELU, FFN-down and the second LayerNorm are one kernel
+        per_layer = [k for k in per_layer if k not in ("gemm_ffn2", "ln2")]
         per_layer[per_layer.index("gemm_ffn1")] = "ffn_fused"
     names = ["pack", "embed_ln"]
     for _ in range(num_layers):
@@ -325,8 +325,11 @@ class EncoderRun:
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         self.n_kernels = self.enc.kernels_per_forward(B, S)
         per_layer = (self.n_kernels - 3) // cfg.num_layers
-        fused_ffn = per_layer in (4, 6)   # 7 = plain layer, 5 = LayerNorm fused into the GEMMs, one less with the one-kernel feed-forward block
-        self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer + (1 if fused_ffn else 0) == 5), fused_ffn=fused_ffn)
+        # 7 = plain layer; 5 = either both LayerNorms fused into the GEMMs (a flag, or the library's own choice for
+        # batch*seq <= 4096) or the one-kernel feed-forward block with the second LayerNorm (a flag, or from 16384 on)
+        ln_flags = args.flags & (0x40 | 0x80 | 0x200)
+        fused_ffn = per_layer == 5 and not ln_flags and not (args.flags & 0x2000) and (B * S > 4096 or bool(args.flags & 0x400)) and (bool(args.flags & 0x1000) or B * S >= 16384)
+        self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer == 5 and not fused_ffn), fused_ffn=fused_ffn)
         assert len(self.names) == self.n_kernels
 
     def step_device(self, e, w):

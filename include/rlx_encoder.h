@@ -84,7 +84,8 @@ typedef enum {
                                       the folded layer is chosen.  Without this flag the one-kernel form is chosen
                                       AUTOMATICALLY for calls with batch*seq >= 16384 (it works in blocks of 256
                                       rows per CTA pair and needs about a wave of them to beat the two GEMMs);
-                                      results are bit for bit those of the two-kernel form */
+                                      the kernel also applies the layer's second LayerNorm (on the
+                                      unrounded sums), so a layer is 5 kernels */
 #define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep FFN-up and FFN-down as two GEMM kernels at every batch size */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
@@ -543,7 +544,10 @@ rlx_status_t rlx_mx_matmul_bf16(const void *a_codes, const void *a_scales_e8m0, 
 
 /*
  * The feed-forward block of a layer in one kernel (Section 3.2, operator fusion):
- *   out = gelu(x W1^T + b1) W2^T + b2 + x        erf GELU; x is the block's input AND its residual.
+ *   v   = gelu(x W1^T + b1) W2^T + b2 + x        erf GELU; x is the block's input AND its residual
+ *   out = v                                       ln_gamma == NULL
+ *   out = LayerNorm(v; ln_gamma, ln_beta, ln_eps) otherwise (biased variance over the H columns, computed on the
+ *                                                 unrounded fp32 v; ln_gamma and ln_beta f32 [H], both or neither)
  * x, out: device bf16 [M, H]; w1: bf16 [F, H]; w2: bf16 [H, F]; b1: f32 [F]; b2: f32 [H]; all 16-byte aligned.
  * The F-wide activation is produced and consumed in 64-column chunks on the chip (tensor memory ->
  * registers -> shared memory) and rounded to bf16 once, as in the two-kernel form; fp32 accumulation.
@@ -551,7 +555,8 @@ rlx_status_t rlx_mx_matmul_bf16(const void *a_codes, const void *a_scales_e8m0, 
  * receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.  Asynchronous on cuda_stream.
  */
 rlx_status_t rlx_ffn_fused_bf16(const void *x_bf16, const void *w1_bf16, const float *b1, const void *w2_bf16,
-                                const float *b2, int32_t M, int32_t H, int32_t F, void *out_bf16,
+                                const float *b2, const float *ln_gamma, const float *ln_beta, float ln_eps,
+                                int32_t M, int32_t H, int32_t F, void *out_bf16,
                                 int32_t *status, void *cuda_stream);
 
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */

@@ -409,12 +409,14 @@ def scaled_matmul_bf16(a, codes, scales, fmt: int, bias, residual=None, epilogue
     return out
 
 
-def ffn_fused_bf16(x, w1, b1, w2, b2, out=None, status=None, stream=None):
-    """rlx_ffn_fused_bf16: out [M,H] = gelu(x w1^T + b1) w2^T + b2 + x in one kernel."""
+def ffn_fused_bf16(x, w1, b1, w2, b2, ln_gamma=None, ln_beta=None, ln_eps=0.0, out=None, status=None, stream=None):
+    """rlx_ffn_fused_bf16: out [M,H] = gelu(x w1^T + b1) w2^T + b2 + x in one kernel, through LayerNorm when
+    ln_gamma / ln_beta are given."""
     M, H = x.shape
     F = w1.shape[0]
     out = torch.empty((M, H), dtype=torch.bfloat16, device=x.device) if out is None else out
-    _check(_load().rlx_ffn_fused_bf16(_ptr(x), _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2), M, H, F, _ptr(out), _ptr(status),
+    _check(_load().rlx_ffn_fused_bf16(_ptr(x), _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2), _ptr(ln_gamma), _ptr(ln_beta),
+                                      C.c_float(ln_eps), M, H, F, _ptr(out), _ptr(status),
                                       _stream(stream)), "rlx_ffn_fused_bf16")
     return out
 

@@ -64,13 +64,30 @@ struct FfnParams {
     __nv_bfloat16* out;         // [M, H]
     int M, F;
     const int32_t* m_ptr;       // optional device row count
+    const float* ln_gamma;      // [H]  LayerNorm over the rows of the result (kernel variant LN only)
+    const float* ln_beta;       // [H]
+    float ln_eps;
     int32_t* status;
 };
 
 // byte offset of 16-byte chunk j of row r in a K-major tile of 128-byte rows with the 128-byte swizzle
 __device__ __forceinline__ uint32_t sw128(int r, int j) { return (uint32_t)(r * 128 + ((j ^ (r & 7)) << 4)); }
 
-template <int HID>
+// v[j] = accumulator + bias + residual for eight consecutive columns (x: the eight bf16 residual values)
+__device__ __forceinline__ void residual_row8(const uint32_t* acc, const uint4& x, const float4& ba, const float4& bb, float* v) {
+    v[0] = __uint_as_float(acc[0]) + ba.x + bf16lo(x.x); v[1] = __uint_as_float(acc[1]) + ba.y + bf16hi(x.x);
+    v[2] = __uint_as_float(acc[2]) + ba.z + bf16lo(x.y); v[3] = __uint_as_float(acc[3]) + ba.w + bf16hi(x.y);
+    v[4] = __uint_as_float(acc[4]) + bb.x + bf16lo(x.z); v[5] = __uint_as_float(acc[5]) + bb.y + bf16hi(x.z);
+    v[6] = __uint_as_float(acc[6]) + bb.z + bf16lo(x.w); v[7] = __uint_as_float(acc[7]) + bb.w + bf16hi(x.w);
+}
+__device__ __forceinline__ void st_shared_f32x2(uint32_t addr, float a, float b) {
+    asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void ld_shared_f32x2(uint32_t addr, float& a, float& b) {
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
+}
+
+template <int HID, bool LN>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
                          const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out, const FfnParams p) {
@@ -87,7 +104,8 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     const uint32_t x_full = bars, w1_full = x_full + 8, w2_full = w1_full + 16, s_empty = w2_full + 16, g_full = s_empty + 16;
     const uint32_t o_empty = g_full + 16, x_empty = o_empty + 8, w1_empty = x_empty + 8, w2_empty = w1_empty + 16;
     const uint32_t s_full = w2_empty + 16, g_empty = s_full + 16, o_full = g_empty + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 20);
+    const uint32_t ln_bar = o_full + 8;   // [4] per lane quarter: the two column halves' row sums are in shared memory
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 24);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,6 +116,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         mbar_init(o_empty, 2 * kEpiWarps);
         mbar_init(x_empty, 2 + kEpiWarps);      // both first-product warps' last commits + this CTA's epilogue warps
         mbar_init(o_full, 1);
+        for (int i = 0; i < 4; ++i) mbar_init(ln_bar + 8 * i, 2);
         for (int i = 0; i < 2; ++i) {
             mbar_init(w1_full + 8 * i, 1); mbar_init(w2_full + 8 * i, 1);
             mbar_init(w1_empty + 8 * i, 1); mbar_init(w2_empty + 8 * i, 1);
@@ -313,6 +332,58 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             // memory is the one the TMA load produced, so the store map has the load map's geometry.
             const int row0 = blk * kPairRows + (int)cta_rank * BLOCK_M + quad * 32;
             constexpr int kTilesPerWarp = HID / 128;   // this warp's column half = HID/2 columns = HID/128 tiles of 64
+            // LN variant: the row then goes through LayerNorm before it is rounded.  A row's H values sit with two
+            // threads (same lane quarter and lane, the two column halves): a first pass over O and X sums v and
+            // v^2 per thread, the pair swaps its sums through shared memory (the first G buffer, idle until the
+            // next block's first chunk, which cannot start before every warp here has released X), and the
+            // second pass recomputes v and normalises it.  Tensor memory is read twice; nothing else moves.
+            float ln_a = 1.f, ln_c = 0.f;    // y = (v * ln_a + ln_c) * gamma + beta
+            if constexpr (LN) {
+                // sums of (v - pivot) and (v - pivot)^2 with the thread's first value as the pivot: no cancellation
+                // when a row's mean is large against its spread
+                float sum = 0.f, sq = 0.f, pivot = 0.f;
+                bool have_pivot = false;
+#pragma unroll 1
+                for (int t = 0; t < kTilesPerWarp; ++t) {
+                    const int kb = half * kTilesPerWarp + t;
+                    const uint32_t tile = xs + kb * BLOCK_M * 128;
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int col0 = kb * 64 + hh * 32;
+                        uint32_t acc[32];
+                        tmem_ld_32x32(lane_addr + col0, acc);
+                        tmem_ld_wait();
+                        const float* b2 = p.b2 + col0;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 x = ld_shared_v4(tile + sw128(r, hh * 4 + i));
+                            const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
+                            const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
+                            float v[8];
+                            residual_row8(acc + 8 * i, x, ba, bb, v);
+#pragma unroll
+                            if (!have_pivot) { pivot = v[0]; have_pivot = true; }
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) { const float dv = v[j] - pivot; sum += dv; sq = fmaf(dv, dv, sq); }
+                        }
+                    }
+                }
+                // this thread's half row: mean and sum of squared deviations; the halves combine pairwise
+                constexpr float kHalf = (float)(HID / 2);
+                const float my_mean = pivot + sum * (1.f / kHalf);
+                const float my_m2 = fmaxf(sq - sum * sum * (1.f / kHalf), 0.f);
+                st_shared_f32x2(gs + (uint32_t)((half * BLOCK_M + r) * 8), my_mean, my_m2);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ln_bar + 8 * quad);
+                if (!(ok = mbar_wait(ln_bar + 8 * quad, nb & 1, abort_flag))) break;
+                float o_mean, o_m2;
+                ld_shared_f32x2(gs + (uint32_t)(((half ^ 1) * BLOCK_M + r) * 8), o_mean, o_m2);
+                const float mean = 0.5f * (my_mean + o_mean);
+                const float dm = my_mean - o_mean;
+                const float var = (my_m2 + o_m2 + dm * dm * (0.5f * kHalf)) * (1.f / HID);
+                ln_a = rsqrtf(var + p.ln_eps);
+                ln_c = -mean * ln_a;
+            }
 #pragma unroll 1
             for (int t = 0; t < kTilesPerWarp; ++t) {
                 const int kb = half * kTilesPerWarp + t;
@@ -335,11 +406,20 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                         const uint4 x = ld_shared_v4(slot);
                         const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
                         const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
+                        float v[8];
+                        residual_row8(acc + 8 * i, x, ba, bb, v);
+                        if constexpr (LN) {
+                            const float4 ga = __ldg(reinterpret_cast<const float4*>(p.ln_gamma + col0) + 2 * i);
+                            const float4 gb = __ldg(reinterpret_cast<const float4*>(p.ln_gamma + col0) + 2 * i + 1);
+                            const float4 ea = __ldg(reinterpret_cast<const float4*>(p.ln_beta + col0) + 2 * i);
+                            const float4 eb = __ldg(reinterpret_cast<const float4*>(p.ln_beta + col0) + 2 * i + 1);
+                            v[0] = fmaf(fmaf(v[0], ln_a, ln_c), ga.x, ea.x); v[1] = fmaf(fmaf(v[1], ln_a, ln_c), ga.y, ea.y);
+                            v[2] = fmaf(fmaf(v[2], ln_a, ln_c), ga.z, ea.z); v[3] = fmaf(fmaf(v[3], ln_a, ln_c), ga.w, ea.w);
+                            v[4] = fmaf(fmaf(v[4], ln_a, ln_c), gb.x, eb.x); v[5] = fmaf(fmaf(v[5], ln_a, ln_c), gb.y, eb.y);
+                            v[6] = fmaf(fmaf(v[6], ln_a, ln_c), gb.z, eb.z); v[7] = fmaf(fmaf(v[7], ln_a, ln_c), gb.w, eb.w);
+                        }
                         uint4 q;
-                        q.x = pack_bf16(__uint_as_float(acc[8 * i + 0]) + ba.x + bf16lo(x.x), __uint_as_float(acc[8 * i + 1]) + ba.y + bf16hi(x.x));
-                        q.y = pack_bf16(__uint_as_float(acc[8 * i + 2]) + ba.z + bf16lo(x.y), __uint_as_float(acc[8 * i + 3]) + ba.w + bf16hi(x.y));
-                        q.z = pack_bf16(__uint_as_float(acc[8 * i + 4]) + bb.x + bf16lo(x.z), __uint_as_float(acc[8 * i + 5]) + bb.y + bf16hi(x.z));
-                        q.w = pack_bf16(__uint_as_float(acc[8 * i + 6]) + bb.z + bf16lo(x.w), __uint_as_float(acc[8 * i + 7]) + bb.w + bf16hi(x.w));
+                        q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]); q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
                         st_shared_v4(slot, q);
                     }
                 }

@@ -232,9 +232,13 @@ cudaError_t init_kernels_for_current_device() {
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tcar::gemm_ares_tcgen05_kernel<256, 0>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs_resident[dev] = n;
     }
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcff::Cfg<384>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  rlx::tcff::Cfg<384>::SMEM_BYTES)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tcmx::gemm_mx_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcmx::kSmemBytes)) != cudaSuccess) return e;
@@ -431,7 +435,8 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
 // Feed-forward block in one kernel (hidden 256 or 384, F % 64 == 0): out = gelu(x W1^T + b1) W2^T + b2 + x.
 bool ffn_fused_supported(int H, int F) { return (H == 256 || H == 384) && F % 128 == 0 && F >= 128; }
 rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, const bf16* w2, const float* b2, int M, int H,
-                              int F, bf16* out, int32_t* status, cudaStream_t st, const int32_t* rows_ptr) {
+                              int F, bf16* out, int32_t* status, cudaStream_t st, const int32_t* rows_ptr,
+                              const float* ln_gamma = nullptr, const float* ln_beta = nullptr, float ln_eps = 0.f) {
     if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
     CUtensorMap tx, t1, t2, to;
     if (!make_tmap(&tx, x, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M) || !make_tmap(&to, out, (uint64_t)M, (uint64_t)H, 32) ||
@@ -440,6 +445,8 @@ rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, co
         return RLX_ERR_CUDA;
     rlx::tcff::FfnParams p;
     p.b1 = b1; p.b2 = b2; p.out = out; p.M = M; p.F = F; p.m_ptr = rows_ptr; p.status = status;
+    p.ln_gamma = ln_gamma; p.ln_beta = ln_beta; p.ln_eps = ln_eps;
+    const bool ln = ln_gamma != nullptr;
     int dev = 0;
     cudaGetDevice(&dev);
     const int pairs_max = (dev >= 0 && dev < 64 && g_max_pairs_resident[dev] > 0) ? g_max_pairs_resident[dev] : sm_count() / 2;
@@ -449,10 +456,14 @@ rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, co
         ClusterScope() { g_cluster_x = 2; }
         ~ClusterScope() { g_cluster_x = 1; }
     } scope;
-    if (H == 384)
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
+    if (H == 384 && ln)
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384, true>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
+    else if (H == 384)
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384, false>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
+    else if (ln)
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256, true>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
     else
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
+        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256, false>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -854,7 +865,7 @@ bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S) {
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
     const bool fused = uses_fold_ln(c, B, S) || uses_fused_ln(c, B, S) || uses_cluster_ln(c);
-    return 2 + ((fused ? 5 : 7) - (uses_fused_ffn(c, B, S) ? 1 : 0)) * c.num_layers + (pack ? 1 : 0);
+    return 2 + ((fused ? 5 : 7) - (uses_fused_ffn(c, B, S) ? 2 : 0)) * c.num_layers + (pack ? 1 : 0);
 }
 bool uses_chunks(const rlx_encoder_config_t& c, int B, int S);
 int chunk_batch(int B, int S);
@@ -1096,8 +1107,9 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         }
         if (fuse_ffn) {
             // the whole feed-forward block in one kernel: the F-wide activation stays on the chip
-            RLX_TRY(launch_ffn_fused(x1, (const bf16*)lw.w1, lw.b1, (const bf16*)lw.w2, lw.b2, T, H, F, y, status, st, rows));
-            RLX_TRY(launch_layernorm(y, lw.ln2_g, lw.ln2_b, T, H, c.ln_eps, x, st, rows));
+            // and the layer's second LayerNorm in its epilogue, on the unrounded sums
+            RLX_TRY(launch_ffn_fused(x1, (const bf16*)lw.w1, lw.b1, (const bf16*)lw.w2, lw.b2, T, H, F, x, status, st, rows,
+                                     lw.ln2_g, lw.ln2_b, c.ln_eps));
             continue;
         }
         RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
@@ -1780,14 +1792,17 @@ rlx_status_t rlx_mx_matmul_bf16(const void* a_codes, const void* a_scales, int32
 }
 
 rlx_status_t rlx_ffn_fused_bf16(const void* x, const void* w1, const float* b1, const void* w2, const float* b2,
+                                const float* ln_gamma, const float* ln_beta, float ln_eps,
                                 int32_t M, int32_t H, int32_t F, void* out, int32_t* status, void* stream) {
     if (!x || !w1 || !b1 || !w2 || !b2 || !out || M <= 0 || H <= 0 || F <= 0) return RLX_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(w1) || !aligned16(b1) || !aligned16(w2) || !aligned16(b2) || !aligned16(out))
         return RLX_ERR_INVALID_ARG;
+    if ((ln_gamma == nullptr) != (ln_beta == nullptr) || !aligned16(ln_gamma) || !aligned16(ln_beta)) return RLX_ERR_INVALID_ARG;
+    if (ln_gamma && !(ln_eps > 0.f)) return RLX_ERR_INVALID_ARG;
     if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
     RLX_CUDA_TRY(init_kernels_for_current_device());
     return launch_ffn_fused((const bf16*)x, (const bf16*)w1, b1, (const bf16*)w2, b2, M, H, F, (bf16*)out, status,
-                            static_cast<cudaStream_t>(stream), nullptr);
+                            static_cast<cudaStream_t>(stream), nullptr, ln_gamma, ln_beta, ln_eps);
 }
 
 rlx_status_t rlx_pool_l2norm(const void* x, const int32_t* mask, int32_t B, int32_t S, int32_t H, float* out,

@@ -329,35 +329,39 @@ def test_graph_cache_reuse_and_new_inputs(rlx):
 
 
 @pytest.mark.parametrize("flags", [0x1400, 0x1401], ids=["graph", "eager"])
-def test_fused_ffn_forward_is_bitwise_the_two_kernel_forward(rlx, flags):
-    """RLX_FLAG_FUSED_FFN: FFN-up, GELU and FFN-down of every layer in one kernel.  Same rounding points and
-    the same k order as the two-kernel form, so the embeddings agree bit for bit with the plain 7-kernel
-    layer (0x400 keeps LayerNorm folding out of both)."""
+def test_fused_ffn_forward_against_the_two_kernel_forward(rlx, flags):
+    """RLX_FLAG_FUSED_FFN: FFN-up, GELU, FFN-down and the second LayerNorm of every layer in one kernel.  The
+    feed-forward part has the rounding points and the k order of the two-kernel form; the LayerNorm works on
+    the unrounded sums (one bf16 rounding fewer per layer), so the embeddings differ from the plain 7-kernel
+    layer's by rounding noise only (0x400 keeps LayerNorm folding out of both)."""
     inp = make_inputs(CONFIGS["c2"])
     w = rlx.upload_weights(inp.params, inp.layers)
     plain, status = run_gpu(rlx, inp, weights=w, flags=0x400 | (flags & 1))
     assert status == 0
     fused, status = run_gpu(rlx, inp, weights=w, flags=flags)
     assert status == 0
-    assert np.array_equal(plain, fused)
+    assert np.abs(plain - fused).max() <= 2e-3
     ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
     check(fused, ref, inp.lengths)
 
 
 def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
-    """Without a flag the one-kernel feed-forward block takes over at batch*seq >= 16384; RLX_FLAG_NO_FUSED_FFN
-    (0x2000) keeps the two GEMMs.  Same embeddings bit for bit, one kernel less per layer."""
+    """Without a flag the one-kernel feed-forward block (with the second LayerNorm) takes over at batch*seq >=
+    16384; RLX_FLAG_NO_FUSED_FFN (0x2000) keeps the two GEMMs and the LayerNorm kernel.  Two kernels less per
+    layer, embeddings equal up to rounding noise."""
     inp = make_inputs(CONFIGS["c2"], batch=130, num_layers=2)
     w = rlx.upload_weights(inp.params, inp.layers)
     auto, status = run_gpu(rlx, inp, weights=w, flags=0)
     assert status == 0
     two, status = run_gpu(rlx, inp, weights=w, flags=0x2000)
     assert status == 0
-    assert np.array_equal(auto, two)
+    assert np.abs(auto - two).max() <= 2e-3
+    ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
+    check(auto, ref, inp.lengths)
     c = inp.cfg
     assert c.batch * c.seq >= 16384
     a = rlx.Encoder.from_config(c, flags=0, max_batch=c.batch, max_seq=c.seq)
     b = rlx.Encoder.from_config(c, flags=0x2000, max_batch=c.batch, max_seq=c.seq)
-    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == c.num_layers
+    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == 2 * c.num_layers
     assert a.kernels_per_forward(127, 128) == b.kernels_per_forward(127, 128)
     a.close(); b.close()

@@ -208,6 +208,28 @@ def test_ffn_fused_matches_oracle(rlx, M, H, F):
     two = rlx.gemm_bf16(rlx.gemm_bf16(bf16_dev(x), bf16_dev(w1), f32_dev(b1), epilogue=1), bf16_dev(w2), f32_dev(b2),
                         residual=bf16_dev(x), epilogue=2)
     assert np.array_equal(to_np64(two), got)
+    # the LayerNorm variant normalises the unrounded sums
+    gamma = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    got_ln = to_np64(rlx.ffn_fused_bf16(bf16_dev(x), bf16_dev(w1), f32_dev(b1), bf16_dev(w2), f32_dev(b2), f32_dev(gamma),
+                                        f32_dev(beta), 1e-12, status=status))
+    assert int(status.item()) == 0
+    assert_close_bf16_out(got_ln, oracle.layernorm(ref, gamma, beta, 1e-12), extra_abs=1e-2)
+
+
+def test_ffn_fused_layernorm_rows_with_a_large_mean(rlx):
+    """Rows whose mean is 200 times their spread: the row statistics are kept as deviations from a pivot, so the
+    variance does not cancel.  Zero weights make the pre-LayerNorm row exactly x + b2."""
+    M, H, F = 300, 384, 256
+    rng = np.random.default_rng(5)
+    x = round_to_bf16((100.0 + 0.5 * rng.standard_normal((M, H))).astype(np.float32))
+    zeros = lambda *s: np.zeros(s, np.float32)
+    gamma = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    got = to_np64(rlx.ffn_fused_bf16(bf16_dev(x), bf16_dev(zeros(F, H)), f32_dev(zeros(F)), bf16_dev(zeros(H, F)),
+                                     f32_dev(zeros(H)), f32_dev(gamma), f32_dev(beta), 1e-12))
+    ref = oracle.layernorm(x.astype(np.float64), gamma, beta, 1e-12)
+    assert_close_bf16_out(got, ref, extra_abs=1e-4)
 
 
 @pytest.mark.parametrize("impl", [0, 1], ids=["cluster", "whole_row"])
