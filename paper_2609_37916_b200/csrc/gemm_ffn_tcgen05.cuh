@@ -51,7 +51,8 @@ struct Cfg {
     static constexpr int G_BYTES = BLOCK_M * 128;                   // one k-block tile of G
     static constexpr int X_OFF = 0, W1_OFF = X_BYTES, W2_OFF = W1_OFF + 2 * W1_STAGE, G_OFF = W2_OFF + 2 * W2_STAGE;
     static constexpr int BAR_OFF = G_OFF + 2 * G_BYTES;
-    static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+    static constexpr int B1_OFF = BAR_OFF + 256;                    // per epilogue warp: the 32 bias values of its chunk half
+    static constexpr int SMEM_BYTES = B1_OFF + kEpiWarps * 128 + 1024;
     static constexpr int COL_S = HID;                               // S buffers behind O
     static constexpr int TMEM_COLS = 512;
     static_assert(HID + 2 * kChunk <= 512, "tensor memory");
@@ -79,6 +80,29 @@ __device__ __forceinline__ void residual_row8(const uint32_t* acc, const uint4& 
     v[2] = __uint_as_float(acc[2]) + ba.z + bf16lo(x.y); v[3] = __uint_as_float(acc[3]) + ba.w + bf16hi(x.y);
     v[4] = __uint_as_float(acc[4]) + bb.x + bf16lo(x.z); v[5] = __uint_as_float(acc[5]) + bb.y + bf16hi(x.z);
     v[6] = __uint_as_float(acc[6]) + bb.z + bf16lo(x.w); v[7] = __uint_as_float(acc[7]) + bb.w + bf16hi(x.w);
+}
+// the same as four packed pairs (Blackwell's f32x2 arithmetic: one issue slot per pair)
+__device__ __forceinline__ void residual_row8_x2(const uint32_t* acc, const uint4& x, const float4& ba, const float4& bb, uint64_t* v) {
+    v[0] = add_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[0]), __uint_as_float(acc[1])), pack_f32x2(ba.x, ba.y)), pack_f32x2(bf16lo(x.x), bf16hi(x.x)));
+    v[1] = add_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[2]), __uint_as_float(acc[3])), pack_f32x2(ba.z, ba.w)), pack_f32x2(bf16lo(x.y), bf16hi(x.y)));
+    v[2] = add_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[4]), __uint_as_float(acc[5])), pack_f32x2(bb.x, bb.y)), pack_f32x2(bf16lo(x.z), bf16hi(x.z)));
+    v[3] = add_f32x2(add_f32x2(pack_f32x2(__uint_as_float(acc[6]), __uint_as_float(acc[7])), pack_f32x2(bb.z, bb.w)), pack_f32x2(bf16lo(x.w), bf16hi(x.w)));
+}
+__device__ __forceinline__ uint32_t pack_bf16_pair(uint64_t v) {
+    float lo, hi;
+    unpack_f32x2(v, lo, hi);
+    return pack_bf16(lo, hi);
+}
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float a) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(a) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_f32x4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_shared_f32x4(uint32_t addr, const float4& v) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 __device__ __forceinline__ void st_shared_f32x2(uint32_t addr, float a, float b) {
     asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(a), "f"(b) : "memory");
@@ -258,6 +282,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         const int ew = warp - 2, quad = warp & 3, half = ew >> 2;
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const int r = quad * 32 + lane;                      // this thread's row within the CTA's 128
+        const uint32_t b1_slot = base + C::B1_OFF + ew * 128;
             const uint32_t lead_s_empty = map_to_cta(s_empty, 0), lead_g_full = map_to_cta(g_full, 0), lead_o_empty = map_to_cta(o_empty, 0);
         bool ok = true;
         uint32_t nb = 0, cc = 0;
@@ -267,6 +292,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             // issued between the halves of the GELU arithmetic, so their round trips (150-250 cycles each)
             // overlap it instead of adding to the chain  S ready -> G ready  that paces the whole kernel.
             uint32_t acc[32];
+            float b1_next = __ldg(p.b1 + half * 32 + lane);
             {
                 const uint32_t st = cc & 1, use = cc >> 1;
                 if (!(ok = mbar_wait(s_full + 8 * st, use & 1, abort_flag))) break;
@@ -282,11 +308,15 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                 const bool more = c + 1 < n_chunks;
                 const uint32_t nst = st ^ 1, nuse = (cc + 1) >> 1;
                 const bool s_ready = more && mbar_test_wait(s_full + 8 * nst, nuse & 1);
-                const float* b1 = p.b1 + c * kChunk + half * 32;
+                // this warp's 32 bias values: one coalesced load (issued an iteration ahead), then broadcast reads
+                // from the warp's slot -- 8 same-address 16-byte global loads per thread cost hundreds of cycles
+                st_shared_f32(b1_slot + 4 * lane, b1_next);
+                __syncwarp();
+                if (more) b1_next = __ldg(p.b1 + (c + 1) * kChunk + half * 32 + lane);
                 float v[32];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
-                    const float4 b = __ldg(reinterpret_cast<const float4*>(b1) + i);
+                    const float4 b = ld_shared_f32x4(b1_slot + 16 * i);
                     v[4 * i + 0] = __uint_as_float(acc[4 * i + 0]) + b.x;
                     v[4 * i + 1] = __uint_as_float(acc[4 * i + 1]) + b.y;
                     v[4 * i + 2] = __uint_as_float(acc[4 * i + 2]) + b.z;
@@ -337,36 +367,75 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             // v^2 per thread, the pair swaps its sums through shared memory (the first G buffer, idle until the
             // next block's first chunk, which cannot start before every warp here has released X), and the
             // second pass recomputes v and normalises it.  Tensor memory is read twice; nothing else moves.
+            // Both passes walk the warp's column half in chunks of 32 columns with the tensor-memory load of the
+            // next chunk in flight while the current one is worked on (two register buffers).
+            constexpr int kColChunks = 2 * kTilesPerWarp;
+            static_assert(kColChunks % 2 == 0, "chunk pairs");
+            // b2 (and gamma, beta) of the warp's column half go to a private copy in the idle G buffers first
+            // (behind the 2 KB the row sums are swapped through): every thread needs every value, and broadcast
+            // reads from shared memory are several times cheaper than same-address global loads.
+            constexpr int kParamVecs = LN ? 3 : 1, kHalfCols = HID / 2;
+            const uint32_t par = gs + 2048 + ew * (3 * kHalfCols * 4);
+            static_assert(2048 + kEpiWarps * 3 * kHalfCols * 4 <= 2 * C::G_BYTES, "parameter copies fit in the G buffers");
+            for (int idx = lane; idx < kParamVecs * (kHalfCols / 4); idx += 32) {
+                const int a = idx / (kHalfCols / 4), w4 = idx - a * (kHalfCols / 4);
+                const float* src = (a == 0 ? p.b2 : a == 1 ? p.ln_gamma : p.ln_beta) + half * kHalfCols;
+                st_shared_f32x4(par + (a * kHalfCols + w4 * 4) * 4, __ldg(reinterpret_cast<const float4*>(src) + w4));
+            }
+            __syncwarp();
+            const auto param4 = [&](int a, int col0, int i4) {   // 4 values of vector a at columns col0 + 4*i4 ..
+                return ld_shared_f32x4(par + (a * kHalfCols + (col0 - half * kHalfCols) + 4 * i4) * 4);
+            };
+            const auto chunk_col = [&](int cidx) { return (half * kTilesPerWarp + (cidx >> 1)) * 64 + (cidx & 1) * 32; };
             float ln_a = 1.f, ln_c = 0.f;    // y = (v * ln_a + ln_c) * gamma + beta
             if constexpr (LN) {
                 // sums of (v - pivot) and (v - pivot)^2 with the thread's first value as the pivot: no cancellation
                 // when a row's mean is large against its spread
-                float sum = 0.f, sq = 0.f, pivot = 0.f;
+                uint64_t sum2 = pack_f32x2(0.f, 0.f), sq2 = sum2, npivot2 = sum2;
+                float pivot = 0.f;
                 bool have_pivot = false;
-#pragma unroll 1
-                for (int t = 0; t < kTilesPerWarp; ++t) {
-                    const int kb = half * kTilesPerWarp + t;
-                    const uint32_t tile = xs + kb * BLOCK_M * 128;
+                const auto stats_chunk = [&](const uint32_t* acc, int cidx) {
+                    const int col0 = chunk_col(cidx);
+                    const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        const int col0 = kb * 64 + hh * 32;
-                        uint32_t acc[32];
-                        tmem_ld_32x32(lane_addr + col0, acc);
-                        tmem_ld_wait();
-                        const float* b2 = p.b2 + col0;
+                    for (int i = 0; i < 4; ++i) {
+                        const uint4 x = ld_shared_v4(tile + sw128(r, (cidx & 1) * 4 + i));
+                        const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
+                        uint64_t v[4];
+                        residual_row8_x2(acc + 8 * i, x, ba, bb, v);
+                        if (!have_pivot) {
+                            float hi;
+                            unpack_f32x2(v[0], pivot, hi);
+                            npivot2 = pack_f32x2(-pivot, -pivot);
+                            have_pivot = true;
+                        }
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint4 x = ld_shared_v4(tile + sw128(r, hh * 4 + i));
-                            const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
-                            const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
-                            float v[8];
-                            residual_row8(acc + 8 * i, x, ba, bb, v);
-#pragma unroll
-                            if (!have_pivot) { pivot = v[0]; have_pivot = true; }
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) { const float dv = v[j] - pivot; sum += dv; sq = fmaf(dv, dv, sq); }
+                        for (int j = 0; j < 4; ++j) {
+                            const uint64_t dv = add_f32x2(v[j], npivot2);
+                            sum2 = add_f32x2(sum2, dv);
+                            sq2 = fma_f32x2(dv, dv, sq2);
                         }
                     }
+                };
+                {
+                    uint32_t acc_a[32], acc_b[32];
+                    tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
+#pragma unroll 1
+                    for (int cidx = 0; cidx < kColChunks; cidx += 2) {
+                        tmem_ld_wait();
+                        tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
+                        stats_chunk(acc_a, cidx);
+                        tmem_ld_wait();
+                        if (cidx + 2 < kColChunks) tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
+                        stats_chunk(acc_b, cidx + 1);
+                    }
+                }
+                float sum, sq;
+                {
+                    float a0, a1, q0, q1;
+                    unpack_f32x2(sum2, a0, a1);
+                    unpack_f32x2(sq2, q0, q1);
+                    sum = a0 + a1; sq = q0 + q1;
                 }
                 // this thread's half row: mean and sum of squared deviations; the halves combine pairwise
                 constexpr float kHalf = (float)(HID / 2);
@@ -384,50 +453,55 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                 ln_a = rsqrtf(var + p.ln_eps);
                 ln_c = -mean * ln_a;
             }
-#pragma unroll 1
-            for (int t = 0; t < kTilesPerWarp; ++t) {
-                const int kb = half * kTilesPerWarp + t;
-                const uint32_t tile = xs + kb * BLOCK_M * 128;
+            const uint64_t ln_a2 = pack_f32x2(ln_a, ln_a), ln_c2 = pack_f32x2(ln_c, ln_c);
+            const auto out_chunk = [&](const uint32_t* acc, int cidx) {
+                const int col0 = chunk_col(cidx);
+                const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int col0 = kb * 64 + hh * 32;
-                    uint32_t acc[32];
-                    tmem_ld_32x32(lane_addr + col0, acc);
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t slot = tile + sw128(r, (cidx & 1) * 4 + i);
+                    const uint4 x = ld_shared_v4(slot);
+                    const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
+                    uint64_t v[4];
+                    residual_row8_x2(acc + 8 * i, x, ba, bb, v);
+                    if constexpr (LN) {
+                        const float4 ga = param4(1, col0, 2 * i), gb = param4(1, col0, 2 * i + 1);
+                        const float4 ea = param4(2, col0, 2 * i), eb = param4(2, col0, 2 * i + 1);
+                        v[0] = fma_f32x2(fma_f32x2(v[0], ln_a2, ln_c2), pack_f32x2(ga.x, ga.y), pack_f32x2(ea.x, ea.y));
+                        v[1] = fma_f32x2(fma_f32x2(v[1], ln_a2, ln_c2), pack_f32x2(ga.z, ga.w), pack_f32x2(ea.z, ea.w));
+                        v[2] = fma_f32x2(fma_f32x2(v[2], ln_a2, ln_c2), pack_f32x2(gb.x, gb.y), pack_f32x2(eb.x, eb.y));
+                        v[3] = fma_f32x2(fma_f32x2(v[3], ln_a2, ln_c2), pack_f32x2(gb.z, gb.w), pack_f32x2(eb.z, eb.w));
+                    }
+                    uint4 q;
+                    q.x = pack_bf16_pair(v[0]); q.y = pack_bf16_pair(v[1]); q.z = pack_bf16_pair(v[2]); q.w = pack_bf16_pair(v[3]);
+                    st_shared_v4(slot, q);
+                }
+                if (cidx & 1) {   // the warp's slice of this 64-column tile is complete
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmap_out, (col0 >> 6) * 64, row0, tile + quad * 32 * 128);   // rows past the matrix are clipped
+                        bulk_commit();
+                    }
+                }
+            };
+            {
+                uint32_t acc_a[32], acc_b[32];
+                tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
+#pragma unroll 1
+                for (int cidx = 0; cidx < kColChunks; cidx += 2) {
                     tmem_ld_wait();
-                    if (t == kTilesPerWarp - 1 && hh == 1) {   // last read of O by this warp
+                    tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
+                    out_chunk(acc_a, cidx);
+                    tmem_ld_wait();
+                    if (cidx + 2 < kColChunks) {
+                        tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
+                    } else {   // last read of O by this warp
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
                     }
-                    const float* b2 = p.b2 + col0;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint32_t slot = tile + sw128(r, hh * 4 + i);
-                        const uint4 x = ld_shared_v4(slot);
-                        const float4 ba = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i);
-                        const float4 bb = __ldg(reinterpret_cast<const float4*>(b2) + 2 * i + 1);
-                        float v[8];
-                        residual_row8(acc + 8 * i, x, ba, bb, v);
-                        if constexpr (LN) {
-                            const float4 ga = __ldg(reinterpret_cast<const float4*>(p.ln_gamma + col0) + 2 * i);
-                            const float4 gb = __ldg(reinterpret_cast<const float4*>(p.ln_gamma + col0) + 2 * i + 1);
-                            const float4 ea = __ldg(reinterpret_cast<const float4*>(p.ln_beta + col0) + 2 * i);
-                            const float4 eb = __ldg(reinterpret_cast<const float4*>(p.ln_beta + col0) + 2 * i + 1);
-                            v[0] = fmaf(fmaf(v[0], ln_a, ln_c), ga.x, ea.x); v[1] = fmaf(fmaf(v[1], ln_a, ln_c), ga.y, ea.y);
-                            v[2] = fmaf(fmaf(v[2], ln_a, ln_c), ga.z, ea.z); v[3] = fmaf(fmaf(v[3], ln_a, ln_c), ga.w, ea.w);
-                            v[4] = fmaf(fmaf(v[4], ln_a, ln_c), gb.x, eb.x); v[5] = fmaf(fmaf(v[5], ln_a, ln_c), gb.y, eb.y);
-                            v[6] = fmaf(fmaf(v[6], ln_a, ln_c), gb.z, eb.z); v[7] = fmaf(fmaf(v[7], ln_a, ln_c), gb.w, eb.w);
-                        }
-                        uint4 q;
-                        q.x = pack_bf16(v[0], v[1]); q.y = pack_bf16(v[2], v[3]); q.z = pack_bf16(v[4], v[5]); q.w = pack_bf16(v[6], v[7]);
-                        st_shared_v4(slot, q);
-                    }
-                }
-                fence_proxy_async();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_2d(&tmap_out, kb * 64, row0, tile + quad * 32 * 128);   // rows past the matrix are clipped
-                    bulk_commit();
+                    out_chunk(acc_b, cidx + 1);
                 }
             }
             if (lane == 0) {
