@@ -203,9 +203,8 @@ def workload_config(name: str, extra=None):
 # ---------------------------------------------------------------------------- roofline bookkeeping
 def kernel_classes(num_layers: int, fused_ln: bool, fused_ffn: bool = False):
     per_layer = [k for k in KERNEL_CLASSES if not (fused_ln and k in ("ln1", "ln2"))]
-    if fused_ffn:   # FFN-up, GELU, FFN-down and the second LayerNorm are one kernel
-        per_layer = [k for k in per_layer if k not in ("gemm_ffn2", "ln2")]
-        per_layer[per_layer.index("gemm_ffn1")] = "ffn_fused"
+    if fused_ffn:   # everything behind the attention is one kernel
+        per_layer = ["gemm_qkv", "attention", "layer_tail"]
     names = ["pack", "embed_ln"]
     for _ in range(num_layers):
         names += per_layer
@@ -229,8 +228,8 @@ def algorithmic_work(cls: str, c, lengths):
         return "tensor", 2.0 * T * H * H, "flop"
     if cls in ("gemm_ffn1", "gemm_ffn2"):
         return "tensor", 2.0 * T * F * H, "flop"
-    if cls == "ffn_fused":
-        return "tensor", 4.0 * T * F * H, "flop"
+    if cls == "layer_tail":
+        return "tensor", 4.0 * T * F * H + 2.0 * T * H * H, "flop"
     if cls == "attention":
         # at head_dim 32/64 the softmax exponentials (one per query-key pair and head), not the
         # QK^T / PV flops, are the scarce resource: 128..256 flops per exp against a tensor : MUFU
@@ -255,8 +254,8 @@ def gemm_bytes(cls: str, c, T: int):
         return T * (H + H + H) * 2.0 + H * H * 2.0
     if cls == "gemm_ffn1":
         return T * (H + F) * 2.0 + F * H * 2.0
-    if cls == "ffn_fused":
-        return T * (H + H) * 2.0 + 2.0 * F * H * 2.0   # the hidden activation never leaves the chip
+    if cls == "layer_tail":   # reads ctx and the layer's input rows, writes its output rows; three weight matrices
+        return T * (H + H + H) * 2.0 + (2.0 * F * H + H * H) * 2.0
     return T * (F + H + H) * 2.0 + F * H * 2.0   # gemm_ffn2
 
 
@@ -325,11 +324,9 @@ class EncoderRun:
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         self.n_kernels = self.enc.kernels_per_forward(B, S)
         per_layer = (self.n_kernels - 3) // cfg.num_layers
-        # 7 = plain layer; 5 = either both LayerNorms fused into the GEMMs (a flag, or the library's own choice for
-        # batch*seq <= 4096) or the one-kernel feed-forward block with the second LayerNorm (a flag, or from 16384 on)
-        ln_flags = args.flags & (0x40 | 0x80 | 0x200)
-        fused_ffn = per_layer == 5 and not ln_flags and not (args.flags & 0x2000) and (B * S > 4096 or bool(args.flags & 0x400)) and (bool(args.flags & 0x1000) or B * S >= 16384)
-        self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer == 5 and not fused_ffn), fused_ffn=fused_ffn)
+        # 7 = plain layer; 5 = both LayerNorms fused into the GEMMs; 3 = QKV GEMM, attention, one kernel for the rest
+        fused_ffn = per_layer == 3
+        self.names = kernel_classes(cfg.num_layers, fused_ln=(per_layer == 5), fused_ffn=fused_ffn)
         assert len(self.names) == self.n_kernels
 
     def step_device(self, e, w):

@@ -78,15 +78,16 @@ typedef enum {
                                    AUTOMATICALLY for calls with batch*seq <= 4096 unless one of the other two
                                    fusion flags or RLX_FLAG_NO_AUTO_FOLD is set */
 #define RLX_FLAG_NO_AUTO_FOLD 0x400u /* keep the 7-kernel layer (separate LayerNorm kernels) at every batch size */
-#define RLX_FLAG_FUSED_FFN 0x1000u /* FFN-up, GELU and FFN-down in ONE kernel per layer (the F-wide activation never
-                                      reaches global memory) at every batch size; hidden 256 or 384, F % 128 == 0;
-                                      ignored together with the LayerNorm fusion flags, the bring-up GEMM, or where
-                                      the folded layer is chosen.  Without this flag the one-kernel form is chosen
-                                      AUTOMATICALLY for calls with batch*seq >= 16384 (it works in blocks of 256
-                                      rows per CTA pair and needs about a wave of them to beat the two GEMMs);
-                                      the kernel also applies the layer's second LayerNorm (on the
-                                      unrounded sums), so a layer is 5 kernels */
-#define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep FFN-up and FFN-down as two GEMM kernels at every batch size */
+#define RLX_FLAG_FUSED_FFN 0x1000u /* everything of a layer behind the attention in ONE kernel (rlx_layer_tail_bf16:
+                                      out-projection + residual + LayerNorm, FFN-up, GELU, FFN-down + residual +
+                                      LayerNorm; the F-wide activation and the intermediate row never reach global
+                                      memory) at every batch size, so that a layer is 3 kernels; hidden 256 or 384,
+                                      F % 128 == 0; ignored together with the LayerNorm fusion flags, the bring-up
+                                      GEMM, or where the folded layer is chosen.  Without this flag that form is
+                                      chosen AUTOMATICALLY for calls with batch*seq >= 16384 (the kernel works in
+                                      blocks of 256 rows per CTA pair and needs about a wave of them to win) */
+#define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep out-projection, LayerNorms and the two feed-forward GEMMs as separate
+                                         kernels at every batch size */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
                                    kernel's input is still in L2 when its consumer starts.  Results are bit for bit
@@ -558,6 +559,23 @@ rlx_status_t rlx_ffn_fused_bf16(const void *x_bf16, const void *w1_bf16, const f
                                 const float *b2, const float *ln_gamma, const float *ln_beta, float ln_eps,
                                 int32_t M, int32_t H, int32_t F, void *out_bf16,
                                 int32_t *status, void *cuda_stream);
+
+/*
+ * Everything of an encoder layer behind the attention, in one kernel (Section 3.2, operator fusion):
+ *   x1  = LayerNorm(ctx Wo^T + bo + h;  ln1_gamma, ln1_beta, ln_eps)      attention output projection + residual
+ *   out = LayerNorm(gelu(x1 W1^T + b1) W2^T + b2 + x1;  ln2_gamma, ln2_beta, ln_eps)
+ * ctx (the attention's context rows), h (the layer's input rows), out: device bf16 [M, H]; wo: bf16 [H, H];
+ * w1: bf16 [F, H]; w2: bf16 [H, F]; bo, b2, ln*_gamma, ln*_beta: f32 [H]; b1: f32 [F]; all 16-byte aligned.
+ * out may be h (each row block reads its rows of h before it writes them).  x1 is rounded to bf16 once (it is the
+ * A operand of the first product and the residual of the second sum) and never reaches global memory; both
+ * LayerNorms work on unrounded fp32 sums.  H in {256, 384}, F % 128 == 0 (RLX_ERR_UNSUPPORTED otherwise).
+ * status: optional device word that receives RLX_DEVSTAT_TIMEOUT if a bounded wait ran out.  Asynchronous.
+ */
+rlx_status_t rlx_layer_tail_bf16(const void *ctx_bf16, const void *h_bf16, const void *wo_bf16, const float *bo,
+                                 const float *ln1_gamma, const float *ln1_beta, const void *w1_bf16, const float *b1,
+                                 const void *w2_bf16, const float *b2, const float *ln2_gamma, const float *ln2_beta,
+                                 float ln_eps, int32_t M, int32_t H, int32_t F, void *out_bf16, int32_t *status,
+                                 void *cuda_stream);
 
 /* out[b] = L2-normalised masked mean over s of x[b,s,:]  (x bf16 [batch,seq,H], out f32 [batch,H]). */
 rlx_status_t rlx_pool_l2norm(const void *x_bf16, const int32_t *attention_mask, int32_t batch,

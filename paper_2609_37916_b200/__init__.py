@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     dequant_block_scaled_bf16,
     embed_layernorm,
     ffn_fused_bf16,
+    layer_tail_bf16,
     gemm_bf16,
     gemm_residual_layernorm_bf16,
     layernorm,

@@ -41,7 +41,7 @@ EXPORTS = (
     "rlx_encoder_create", "rlx_encoder_destroy", "rlx_encoder_workspace_bytes", "rlx_encoder_forward",
     "rlx_encoder_forward_host", "rlx_encoder_forward_tp", "rlx_encoder_forward_static", "rlx_encoder_last_device_status", "rlx_encoder_kernels_per_forward", "rlx_encoder_kernel_times",
     "rlx_status_string", "rlx_pack_sequences", "rlx_embed_layernorm", "rlx_layernorm", "rlx_gemm_bf16", "rlx_gemm_residual_layernorm_bf16", "rlx_attention_bf16",
-    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_quantise_mx", "rlx_mx_matmul_bf16", "rlx_ffn_fused_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
+    "rlx_attention_f32", "rlx_attention_packed_bf16", "rlx_attention_kind_bf16", "rlx_rope_tables", "rlx_qk_rope_bf16", "rlx_dequant_block_scaled_bf16", "rlx_scaled_matmul_bf16", "rlx_quantise_mx", "rlx_mx_matmul_bf16", "rlx_ffn_fused_bf16", "rlx_layer_tail_bf16", "rlx_selftest_bounded_wait", "rlx_pool_l2norm",
 )
 
 
@@ -418,6 +418,19 @@ def ffn_fused_bf16(x, w1, b1, w2, b2, ln_gamma=None, ln_beta=None, ln_eps=0.0, o
     _check(_load().rlx_ffn_fused_bf16(_ptr(x), _ptr(w1), _ptr(b1), _ptr(w2), _ptr(b2), _ptr(ln_gamma), _ptr(ln_beta),
                                       C.c_float(ln_eps), M, H, F, _ptr(out), _ptr(status),
                                       _stream(stream)), "rlx_ffn_fused_bf16")
+    return out
+
+
+def layer_tail_bf16(ctx, h, wo, bo, ln1_gamma, ln1_beta, w1, b1, w2, b2, ln2_gamma, ln2_beta, ln_eps, out=None, status=None,
+                    stream=None):
+    """rlx_layer_tail_bf16: out-projection + residual + LayerNorm + feed-forward block + residual + LayerNorm of an
+    encoder layer in one kernel; ctx, h, out bf16 [M,H]."""
+    M, H = ctx.shape
+    F = w1.shape[0]
+    out = torch.empty((M, H), dtype=torch.bfloat16, device=ctx.device) if out is None else out
+    _check(_load().rlx_layer_tail_bf16(_ptr(ctx), _ptr(h), _ptr(wo), _ptr(bo), _ptr(ln1_gamma), _ptr(ln1_beta), _ptr(w1),
+                                       _ptr(b1), _ptr(w2), _ptr(b2), _ptr(ln2_gamma), _ptr(ln2_beta), C.c_float(ln_eps),
+                                       M, H, F, _ptr(out), _ptr(status), _stream(stream)), "rlx_layer_tail_bf16")
     return out
 
 

@@ -65,6 +65,9 @@ struct FfnParams {
     __nv_bfloat16* out;         // [M, H]
     int M, F;
     const int32_t* m_ptr;       // optional device row count
+    const float* bo;            // [H]  PRE variant: bias of the projection in front, and the LayerNorm behind it
+    const float* ln1_gamma;     // [H]
+    const float* ln1_beta;      // [H]
     const float* ln_gamma;      // [H]  LayerNorm over the rows of the result (kernel variant LN only)
     const float* ln_beta;       // [H]
     float ln_eps;
@@ -111,10 +114,177 @@ __device__ __forceinline__ void ld_shared_f32x2(uint32_t addr, float& a, float& 
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(a), "=f"(b) : "r"(addr) : "memory");
 }
 
-template <int HID, bool LN>
+// What a warp of the row epilogue knows about its place: tensor-memory lanes, shared-memory regions, barriers.
+struct RowCtx {
+    uint32_t lane_addr;      // tensor-memory address of the warp's lane quarter, column 0 (the accumulator O)
+    uint32_t xs, gs;         // X tiles (residual in, result out), G buffers (scratch)
+    uint32_t ln_bar;         // [4] per lane quarter
+    uint32_t lead_o_empty;   // leader CTA's barrier: O has been read
+    volatile int* abort_flag;
+    int r, ew, quad, half, lane;
+};
+
+// Row epilogue of a 128 x HID accumulator block:  v = O + bias + residual (the bf16 values in the X tiles),
+// optionally through LayerNorm, rounded to bf16 and written back over the residual's slots; with STORE each
+// warp then stores its 32-row slice of every 64-column tile with one TMA store (row0 = the slice's first global
+// row).  Returns false when a bounded wait ran out.
+template <int HID, bool DO_LN, bool STORE>
+__device__ __forceinline__ bool row_epilogue(const RowCtx& rc, const float* bias, const float* gamma, const float* beta, float eps,
+                                             uint32_t ln_parity, const CUtensorMap* tmap_out, int row0) {
+    const uint32_t lane_addr = rc.lane_addr, xs = rc.xs, gs = rc.gs, ln_bar = rc.ln_bar, lead_o_empty = rc.lead_o_empty;
+    volatile int* abort_flag = rc.abort_flag;
+    const int r = rc.r, ew = rc.ew, quad = rc.quad, half = rc.half, lane = rc.lane;
+    constexpr int kTilesPerWarp = HID / 128;   // this warp's column half = HID/2 columns = HID/128 tiles of 64
+    // LN variant: the row then goes through LayerNorm before it is rounded.  A row's H values sit with two
+    // threads (same lane quarter and lane, the two column halves): a first pass over O and X sums v and
+    // v^2 per thread, the pair swaps its sums through shared memory (the first G buffer, idle until the
+    // next block's first chunk, which cannot start before every warp here has released X), and the
+    // second pass recomputes v and normalises it.  Tensor memory is read twice; nothing else moves.
+    // Both passes walk the warp's column half in chunks of 32 columns with the tensor-memory load of the
+    // next chunk in flight while the current one is worked on (two register buffers).
+    constexpr int kColChunks = 2 * kTilesPerWarp;
+    static_assert(kColChunks % 2 == 0, "chunk pairs");
+    // b2 (and gamma, beta) of the warp's column half go to a private copy in the idle G buffers first
+    // (behind the 2 KB the row sums are swapped through): every thread needs every value, and broadcast
+    // reads from shared memory are several times cheaper than same-address global loads.
+    constexpr int kParamVecs = DO_LN ? 3 : 1, kHalfCols = HID / 2;
+    const uint32_t par = gs + 2048 + ew * (3 * kHalfCols * 4);
+    static_assert(2048 + kEpiWarps * 3 * kHalfCols * 4 <= 2 * Cfg<HID>::G_BYTES, "parameter copies fit in the G buffers");
+    for (int idx = lane; idx < kParamVecs * (kHalfCols / 4); idx += 32) {
+        const int a = idx / (kHalfCols / 4), w4 = idx - a * (kHalfCols / 4);
+        const float* src = (a == 0 ? bias : a == 1 ? gamma : beta) + half * kHalfCols;
+        st_shared_f32x4(par + (a * kHalfCols + w4 * 4) * 4, __ldg(reinterpret_cast<const float4*>(src) + w4));
+    }
+    __syncwarp();
+    const auto param4 = [&](int a, int col0, int i4) {   // 4 values of vector a at columns col0 + 4*i4 ..
+        return ld_shared_f32x4(par + (a * kHalfCols + (col0 - half * kHalfCols) + 4 * i4) * 4);
+    };
+    const auto chunk_col = [&](int cidx) { return (half * kTilesPerWarp + (cidx >> 1)) * 64 + (cidx & 1) * 32; };
+    float ln_a = 1.f, ln_c = 0.f;    // y = (v * ln_a + ln_c) * gamma + beta
+    if constexpr (DO_LN) {
+        // sums of (v - pivot) and (v - pivot)^2 with the thread's first value as the pivot: no cancellation
+        // when a row's mean is large against its spread
+        uint64_t sum2 = pack_f32x2(0.f, 0.f), sq2 = sum2, npivot2 = sum2;
+        float pivot = 0.f;
+        bool have_pivot = false;
+        const auto stats_chunk = [&](const uint32_t* acc, int cidx) {
+            const int col0 = chunk_col(cidx);
+            const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 x = ld_shared_v4(tile + sw128(r, (cidx & 1) * 4 + i));
+                const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
+                uint64_t v[4];
+                residual_row8_x2(acc + 8 * i, x, ba, bb, v);
+                if (!have_pivot) {
+                    float hi;
+                    unpack_f32x2(v[0], pivot, hi);
+                    npivot2 = pack_f32x2(-pivot, -pivot);
+                    have_pivot = true;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint64_t dv = add_f32x2(v[j], npivot2);
+                    sum2 = add_f32x2(sum2, dv);
+                    sq2 = fma_f32x2(dv, dv, sq2);
+                }
+            }
+        };
+        {
+            uint32_t acc_a[32], acc_b[32];
+            tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
+#pragma unroll 1
+            for (int cidx = 0; cidx < kColChunks; cidx += 2) {
+                tmem_ld_wait();
+                tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
+                stats_chunk(acc_a, cidx);
+                tmem_ld_wait();
+                if (cidx + 2 < kColChunks) tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
+                stats_chunk(acc_b, cidx + 1);
+            }
+        }
+        float sum, sq;
+        {
+            float a0, a1, q0, q1;
+            unpack_f32x2(sum2, a0, a1);
+            unpack_f32x2(sq2, q0, q1);
+            sum = a0 + a1; sq = q0 + q1;
+        }
+        // this thread's half row: mean and sum of squared deviations; the halves combine pairwise
+        constexpr float kHalf = (float)(HID / 2);
+        const float my_mean = pivot + sum * (1.f / kHalf);
+        const float my_m2 = fmaxf(sq - sum * sum * (1.f / kHalf), 0.f);
+        st_shared_f32x2(gs + (uint32_t)((half * BLOCK_M + r) * 8), my_mean, my_m2);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(ln_bar + 8 * quad);
+        if (!mbar_wait(ln_bar + 8 * quad, ln_parity, abort_flag)) return false;
+        float o_mean, o_m2;
+        ld_shared_f32x2(gs + (uint32_t)(((half ^ 1) * BLOCK_M + r) * 8), o_mean, o_m2);
+        const float mean = 0.5f * (my_mean + o_mean);
+        const float dm = my_mean - o_mean;
+        const float var = (my_m2 + o_m2 + dm * dm * (0.5f * kHalf)) * (1.f / HID);
+        ln_a = rsqrtf(var + eps);
+        ln_c = -mean * ln_a;
+    }
+    const uint64_t ln_a2 = pack_f32x2(ln_a, ln_a), ln_c2 = pack_f32x2(ln_c, ln_c);
+    const auto out_chunk = [&](const uint32_t* acc, int cidx) {
+        const int col0 = chunk_col(cidx);
+        const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t slot = tile + sw128(r, (cidx & 1) * 4 + i);
+            const uint4 x = ld_shared_v4(slot);
+            const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
+            uint64_t v[4];
+            residual_row8_x2(acc + 8 * i, x, ba, bb, v);
+            if constexpr (DO_LN) {
+                const float4 ga = param4(1, col0, 2 * i), gb = param4(1, col0, 2 * i + 1);
+                const float4 ea = param4(2, col0, 2 * i), eb = param4(2, col0, 2 * i + 1);
+                v[0] = fma_f32x2(fma_f32x2(v[0], ln_a2, ln_c2), pack_f32x2(ga.x, ga.y), pack_f32x2(ea.x, ea.y));
+                v[1] = fma_f32x2(fma_f32x2(v[1], ln_a2, ln_c2), pack_f32x2(ga.z, ga.w), pack_f32x2(ea.z, ea.w));
+                v[2] = fma_f32x2(fma_f32x2(v[2], ln_a2, ln_c2), pack_f32x2(gb.x, gb.y), pack_f32x2(eb.x, eb.y));
+                v[3] = fma_f32x2(fma_f32x2(v[3], ln_a2, ln_c2), pack_f32x2(gb.z, gb.w), pack_f32x2(eb.z, eb.w));
+            }
+            uint4 q;
+            q.x = pack_bf16_pair(v[0]); q.y = pack_bf16_pair(v[1]); q.z = pack_bf16_pair(v[2]); q.w = pack_bf16_pair(v[3]);
+            st_shared_v4(slot, q);
+        }
+        if (STORE && (cidx & 1)) {   // the warp's slice of this 64-column tile is complete
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(tmap_out, (col0 >> 6) * 64, row0, tile + quad * 32 * 128);   // rows past the matrix are clipped
+                bulk_commit();
+            }
+        }
+    };
+    {
+        uint32_t acc_a[32], acc_b[32];
+        tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
+#pragma unroll 1
+        for (int cidx = 0; cidx < kColChunks; cidx += 2) {
+            tmem_ld_wait();
+            tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
+            out_chunk(acc_a, cidx);
+            tmem_ld_wait();
+            if (cidx + 2 < kColChunks) {
+                tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
+            } else {   // last read of O by this warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
+            }
+            out_chunk(acc_b, cidx + 1);
+        }
+    }
+    return true;
+}
+
+template <int HID, bool LN, bool PRE>
 __global__ void __launch_bounds__(kThreads, 1)
 ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
-                         const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out, const FfnParams p) {
+                         const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out,
+                         const __grid_constant__ CUtensorMap tmap_wo, const __grid_constant__ CUtensorMap tmap_h, const FfnParams p) {
     using C = Cfg<HID>;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -129,7 +299,10 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     const uint32_t o_empty = g_full + 16, x_empty = o_empty + 8, w1_empty = x_empty + 8, w2_empty = w1_empty + 16;
     const uint32_t s_full = w2_empty + 16, g_empty = s_full + 16, o_full = g_empty + 16;
     const uint32_t ln_bar = o_full + 8;   // [4] per lane quarter: the two column halves' row sums are in shared memory
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 24);
+    // PRE variant: a_done (per CTA: the projection's products are complete), h_full (per CTA: the residual rows have
+    // landed in the X tiles), x_ready (leader: all 16 epilogue warps have written their rows of X)
+    const uint32_t a_done = ln_bar + 32, h_full = a_done + 8, x_ready = h_full + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 27);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -141,6 +314,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         mbar_init(x_empty, 2 + kEpiWarps);      // both first-product warps' last commits + this CTA's epilogue warps
         mbar_init(o_full, 1);
         for (int i = 0; i < 4; ++i) mbar_init(ln_bar + 8 * i, 2);
+        mbar_init(a_done, 1); mbar_init(h_full, 1); mbar_init(x_ready, 2 * kEpiWarps);
         for (int i = 0; i < 2; ++i) {
             mbar_init(w1_full + 8 * i, 1); mbar_init(w2_full + 8 * i, 1);
             mbar_init(w1_empty + 8 * i, 1); mbar_init(w2_empty + 8 * i, 1);
@@ -150,6 +324,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmap_x); prefetch_tmap(&tmap_w1); prefetch_tmap(&tmap_w2); prefetch_tmap(&tmap_out);
+        if (PRE) { prefetch_tmap(&tmap_wo); prefetch_tmap(&tmap_h); }
     }
     if (warp == 1) {
         tmem_alloc<2>(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -194,18 +369,36 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         // ------------------------------------------------------------ TMA producer of the W2 chunks (both CTAs)
         // A thread of its own: behind the W1 loads in one thread, a W2 slot that frees late (its second
         // product waits for the epilogue warps) would hold back the next chunk's W1 tiles as well.
+        // PRE variant: the same ring first carries the k-block tiles of Wo (same shape: H output rows, 64 columns
+        // of K), and this thread also reloads the X tiles with the residual rows once the projection has read
+        // them -- between its first two W2 chunks, whose slots free at about that moment anyway.
         if (lane == 0) {
             bool ok = true;
-            uint32_t cc = 0;
-            for (int blk = pair0; blk < blocks && ok; blk += pairs) {
-                for (int c = 0; c < n_chunks; ++c, ++cc) {
-                    const uint32_t st = cc & 1, use = cc >> 1;
-                    if (use >= 1 && !(ok = mbar_wait(w2_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
-                    const uint32_t lead2 = map_to_cta(w2_full + 8 * st, 0);
-                    if (cta_rank == 0) mbar_expect_tx(w2_full + 8 * st, 2 * C::W2_STAGE);
-                    for (int i = 0; i < 2; ++i)   // instruction i covers output columns i*HID/2 .., this CTA feeds its half of them
-                        tma_load_2d_cg2(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128, &tmap_w2, c * kChunk,
-                                        i * (HID / 2) + (int)cta_rank * C::W2_ROWS, lead2);
+            uint32_t u2 = 0, nb = 0;     // uses of the ring so far
+            const auto load_tile = [&](const CUtensorMap* tmap, int kcol) -> bool {
+                const uint32_t st = u2 & 1, use = u2 >> 1;
+                ++u2;
+                if (use >= 1 && !mbar_wait(w2_empty + 8 * st, (use - 1) & 1, abort_flag)) return false;
+                const uint32_t lead2 = map_to_cta(w2_full + 8 * st, 0);
+                if (cta_rank == 0) mbar_expect_tx(w2_full + 8 * st, 2 * C::W2_STAGE);
+                for (int i = 0; i < 2; ++i)   // instruction i covers output columns i*HID/2 .., this CTA feeds its half of them
+                    tma_load_2d_cg2(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128, tmap, kcol,
+                                    i * (HID / 2) + (int)cta_rank * C::W2_ROWS, lead2);
+                return true;
+            };
+            for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+                if (PRE) {
+                    for (int kb = 0; kb < C::KB1 && ok; ++kb) ok = load_tile(&tmap_wo, kb * BLOCK_K);
+                    if (!ok) break;
+                }
+                for (int c = 0; c < n_chunks && ok; ++c) {
+                    if (PRE && c == 1) {
+                        if (!(ok = mbar_wait(a_done, nb & 1, abort_flag))) break;
+                        mbar_expect_tx(h_full, C::X_BYTES);
+                        const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
+                        for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d(xs + kb * BLOCK_M * 128, &tmap_h, kb * BLOCK_K, xrow, h_full);
+                    }
+                    ok = load_tile(&tmap_w2, c * kChunk);
                 }
             }
         }
@@ -223,7 +416,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             bool ok = true;
             uint32_t nb = 0;
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                if (!(ok = mbar_wait_warp(x_full, nb & 1, abort_flag))) break;
+                if (!(ok = mbar_wait_warp(PRE ? x_ready : x_full, nb & 1, abort_flag))) break;
                 for (int c = st; c < n_chunks && ok; c += 2) {
                     const uint32_t use = (nb * n_chunks + c) >> 1;
                     if (!(ok = mbar_wait_warp(w1_full + 8 * st, use & 1, abort_flag))) break;
@@ -251,25 +444,56 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         if (cta_rank == 0) {
             constexpr uint32_t id2 = make_idesc(kPairRows, HID / 2);
             bool ok = true;
-            uint32_t nb = 0, cc = 0;
+            uint32_t nb = 0, cc = 0, u2 = 0, oe = 0;   // blocks, chunks, W2-ring uses, completions of o_empty waited for
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
-                    const uint32_t st = cc & 1, use = cc >> 1;
-                    if (!(ok = mbar_wait_warp(w2_full + 8 * st, use & 1, abort_flag))) break;
-                    // first accumulation of the block overwrites O: the previous block's rows must have been read
-                    if (c == 0 && nb >= 1 && !(ok = mbar_wait_warp(o_empty, (nb - 1) & 1, abort_flag))) break;
+                if (PRE) {
+                    // the projection in front:  O = ctx Wo^T, the resident tiles as A, Wo's k-block tiles through the ring
+                    if (!(ok = mbar_wait_warp(x_full, nb & 1, abort_flag))) break;
+                    if (nb >= 1) {   // the previous block's result rows have been read out of O
+                        if (!(ok = mbar_wait_warp(o_empty, oe & 1, abort_flag))) break;
+                        ++oe;
+                    }
+                    for (int kb = 0; kb < C::KB1 && ok; ++kb, ++u2) {
+                        const uint32_t st2 = u2 & 1;
+                        if (!(ok = mbar_wait_warp(w2_full + 8 * st2, (u2 >> 1) & 1, abort_flag))) break;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint64_t adesc = make_smem_desc(xs + kb * BLOCK_M * 128);
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                const uint64_t bdesc = make_smem_desc(w2s + st2 * C::W2_STAGE + i * C::W2_ROWS * 128);
+#pragma unroll
+                                for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                                    umma_bf16<2>(tmem + i * (HID / 2), adesc + 2 * k, bdesc + 2 * k, id2, (kb | k) != 0 ? 1u : 0u);
+                            }
+                            umma_commit<2>(w2_empty + 8 * st2);
+                            if (kb == C::KB1 - 1) umma_commit<2>(a_done);
+                        }
+                        __syncwarp();
+                    }
+                    if (!ok) break;
+                }
+                for (int c = 0; c < n_chunks && ok; ++c, ++cc, ++u2) {
+                    const uint32_t st = cc & 1, use = cc >> 1, st2 = u2 & 1;
+                    if (!(ok = mbar_wait_warp(w2_full + 8 * st2, (u2 >> 1) & 1, abort_flag))) break;
+                    // first accumulation of the block overwrites O: its last readers (the previous block's epilogue, or
+                    // with PRE this block's LayerNorm in front) must be done
+                    if (c == 0 && (PRE || nb >= 1)) {
+                        if (!(ok = mbar_wait_warp(o_empty, oe & 1, abort_flag))) break;
+                        ++oe;
+                    }
                     if (!(ok = mbar_wait_warp(g_full + 8 * st, use & 1, abort_flag))) break;
                     tc_fence_after();
                     if (elect_one()) {
                         const uint64_t adesc = make_smem_desc(gs + st * C::G_BYTES);
 #pragma unroll
                         for (int i = 0; i < 2; ++i) {
-                            const uint64_t bdesc = make_smem_desc(w2s + st * C::W2_STAGE + i * C::W2_ROWS * 128);
+                            const uint64_t bdesc = make_smem_desc(w2s + st2 * C::W2_STAGE + i * C::W2_ROWS * 128);
 #pragma unroll
                             for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
                                 umma_bf16<2>(tmem + i * (HID / 2), adesc + 2 * k, bdesc + 2 * k, id2, (c | k) != 0 ? 1u : 0u);
                         }
-                        umma_commit<2>(w2_empty + 8 * st);
+                        umma_commit<2>(w2_empty + 8 * st2);
                         umma_commit<2>(g_empty + 8 * st);
                         if (c == n_chunks - 1) umma_commit<2>(o_full);
                     }
@@ -283,10 +507,26 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
         const int r = quad * 32 + lane;                      // this thread's row within the CTA's 128
         const uint32_t b1_slot = base + C::B1_OFF + ew * 128;
+        RowCtx rc;
+        rc.lane_addr = lane_addr; rc.xs = xs; rc.gs = gs; rc.ln_bar = ln_bar; rc.abort_flag = abort_flag;
+        rc.r = r; rc.ew = ew; rc.quad = quad; rc.half = half; rc.lane = lane;
             const uint32_t lead_s_empty = map_to_cta(s_empty, 0), lead_g_full = map_to_cta(g_full, 0), lead_o_empty = map_to_cta(o_empty, 0);
+        rc.lead_o_empty = lead_o_empty;
         bool ok = true;
         uint32_t nb = 0, cc = 0;
+        const uint32_t lead_x_ready = map_to_cta(x_ready, 0);
         for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+            if (PRE) {
+                // x1 = LayerNorm(ctx Wo^T + bo + h) for the block's rows, written over the residual rows h in the X
+                // tiles: the A operand of the first products and the residual of the block's end, never in global memory
+                if (!(ok = mbar_wait(a_done, nb & 1, abort_flag))) break;
+                tc_fence_after();
+                if (!(ok = mbar_wait(h_full, nb & 1, abort_flag))) break;
+                if (!(ok = row_epilogue<HID, true, false>(rc, p.bo, p.ln1_gamma, p.ln1_beta, p.ln_eps, 0u, nullptr, 0))) break;
+                fence_proxy_async();     // generic-proxy writes -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster_release_cta(lead_x_ready);
+            }
             // Software pipeline over the chunks: the registers hold S_c when an iteration starts; the probe of
             // S_{c+1}'s barrier, the tensor-memory load of S_{c+1} and the probe of the G buffer's barrier are
             // issued between the halves of the GELU arithmetic, so their round trips (150-250 cycles each)
@@ -360,150 +600,8 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             // the finished bf16 outputs back to the same 16-byte slots (same rows, same swizzle), and the warp
             // then stores its 32-row slice of a 64-column tile with one TMA store -- the tile's layout in shared
             // memory is the one the TMA load produced, so the store map has the load map's geometry.
-            const int row0 = blk * kPairRows + (int)cta_rank * BLOCK_M + quad * 32;
-            constexpr int kTilesPerWarp = HID / 128;   // this warp's column half = HID/2 columns = HID/128 tiles of 64
-            // LN variant: the row then goes through LayerNorm before it is rounded.  A row's H values sit with two
-            // threads (same lane quarter and lane, the two column halves): a first pass over O and X sums v and
-            // v^2 per thread, the pair swaps its sums through shared memory (the first G buffer, idle until the
-            // next block's first chunk, which cannot start before every warp here has released X), and the
-            // second pass recomputes v and normalises it.  Tensor memory is read twice; nothing else moves.
-            // Both passes walk the warp's column half in chunks of 32 columns with the tensor-memory load of the
-            // next chunk in flight while the current one is worked on (two register buffers).
-            constexpr int kColChunks = 2 * kTilesPerWarp;
-            static_assert(kColChunks % 2 == 0, "chunk pairs");
-            // b2 (and gamma, beta) of the warp's column half go to a private copy in the idle G buffers first
-            // (behind the 2 KB the row sums are swapped through): every thread needs every value, and broadcast
-            // reads from shared memory are several times cheaper than same-address global loads.
-            constexpr int kParamVecs = LN ? 3 : 1, kHalfCols = HID / 2;
-            const uint32_t par = gs + 2048 + ew * (3 * kHalfCols * 4);
-            static_assert(2048 + kEpiWarps * 3 * kHalfCols * 4 <= 2 * C::G_BYTES, "parameter copies fit in the G buffers");
-            for (int idx = lane; idx < kParamVecs * (kHalfCols / 4); idx += 32) {
-                const int a = idx / (kHalfCols / 4), w4 = idx - a * (kHalfCols / 4);
-                const float* src = (a == 0 ? p.b2 : a == 1 ? p.ln_gamma : p.ln_beta) + half * kHalfCols;
-                st_shared_f32x4(par + (a * kHalfCols + w4 * 4) * 4, __ldg(reinterpret_cast<const float4*>(src) + w4));
-            }
-            __syncwarp();
-            const auto param4 = [&](int a, int col0, int i4) {   // 4 values of vector a at columns col0 + 4*i4 ..
-                return ld_shared_f32x4(par + (a * kHalfCols + (col0 - half * kHalfCols) + 4 * i4) * 4);
-            };
-            const auto chunk_col = [&](int cidx) { return (half * kTilesPerWarp + (cidx >> 1)) * 64 + (cidx & 1) * 32; };
-            float ln_a = 1.f, ln_c = 0.f;    // y = (v * ln_a + ln_c) * gamma + beta
-            if constexpr (LN) {
-                // sums of (v - pivot) and (v - pivot)^2 with the thread's first value as the pivot: no cancellation
-                // when a row's mean is large against its spread
-                uint64_t sum2 = pack_f32x2(0.f, 0.f), sq2 = sum2, npivot2 = sum2;
-                float pivot = 0.f;
-                bool have_pivot = false;
-                const auto stats_chunk = [&](const uint32_t* acc, int cidx) {
-                    const int col0 = chunk_col(cidx);
-                    const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const uint4 x = ld_shared_v4(tile + sw128(r, (cidx & 1) * 4 + i));
-                        const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
-                        uint64_t v[4];
-                        residual_row8_x2(acc + 8 * i, x, ba, bb, v);
-                        if (!have_pivot) {
-                            float hi;
-                            unpack_f32x2(v[0], pivot, hi);
-                            npivot2 = pack_f32x2(-pivot, -pivot);
-                            have_pivot = true;
-                        }
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint64_t dv = add_f32x2(v[j], npivot2);
-                            sum2 = add_f32x2(sum2, dv);
-                            sq2 = fma_f32x2(dv, dv, sq2);
-                        }
-                    }
-                };
-                {
-                    uint32_t acc_a[32], acc_b[32];
-                    tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
-#pragma unroll 1
-                    for (int cidx = 0; cidx < kColChunks; cidx += 2) {
-                        tmem_ld_wait();
-                        tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
-                        stats_chunk(acc_a, cidx);
-                        tmem_ld_wait();
-                        if (cidx + 2 < kColChunks) tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
-                        stats_chunk(acc_b, cidx + 1);
-                    }
-                }
-                float sum, sq;
-                {
-                    float a0, a1, q0, q1;
-                    unpack_f32x2(sum2, a0, a1);
-                    unpack_f32x2(sq2, q0, q1);
-                    sum = a0 + a1; sq = q0 + q1;
-                }
-                // this thread's half row: mean and sum of squared deviations; the halves combine pairwise
-                constexpr float kHalf = (float)(HID / 2);
-                const float my_mean = pivot + sum * (1.f / kHalf);
-                const float my_m2 = fmaxf(sq - sum * sum * (1.f / kHalf), 0.f);
-                st_shared_f32x2(gs + (uint32_t)((half * BLOCK_M + r) * 8), my_mean, my_m2);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(ln_bar + 8 * quad);
-                if (!(ok = mbar_wait(ln_bar + 8 * quad, nb & 1, abort_flag))) break;
-                float o_mean, o_m2;
-                ld_shared_f32x2(gs + (uint32_t)(((half ^ 1) * BLOCK_M + r) * 8), o_mean, o_m2);
-                const float mean = 0.5f * (my_mean + o_mean);
-                const float dm = my_mean - o_mean;
-                const float var = (my_m2 + o_m2 + dm * dm * (0.5f * kHalf)) * (1.f / HID);
-                ln_a = rsqrtf(var + p.ln_eps);
-                ln_c = -mean * ln_a;
-            }
-            const uint64_t ln_a2 = pack_f32x2(ln_a, ln_a), ln_c2 = pack_f32x2(ln_c, ln_c);
-            const auto out_chunk = [&](const uint32_t* acc, int cidx) {
-                const int col0 = chunk_col(cidx);
-                const uint32_t tile = xs + (col0 >> 6) * BLOCK_M * 128;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint32_t slot = tile + sw128(r, (cidx & 1) * 4 + i);
-                    const uint4 x = ld_shared_v4(slot);
-                    const float4 ba = param4(0, col0, 2 * i), bb = param4(0, col0, 2 * i + 1);
-                    uint64_t v[4];
-                    residual_row8_x2(acc + 8 * i, x, ba, bb, v);
-                    if constexpr (LN) {
-                        const float4 ga = param4(1, col0, 2 * i), gb = param4(1, col0, 2 * i + 1);
-                        const float4 ea = param4(2, col0, 2 * i), eb = param4(2, col0, 2 * i + 1);
-                        v[0] = fma_f32x2(fma_f32x2(v[0], ln_a2, ln_c2), pack_f32x2(ga.x, ga.y), pack_f32x2(ea.x, ea.y));
-                        v[1] = fma_f32x2(fma_f32x2(v[1], ln_a2, ln_c2), pack_f32x2(ga.z, ga.w), pack_f32x2(ea.z, ea.w));
-                        v[2] = fma_f32x2(fma_f32x2(v[2], ln_a2, ln_c2), pack_f32x2(gb.x, gb.y), pack_f32x2(eb.x, eb.y));
-                        v[3] = fma_f32x2(fma_f32x2(v[3], ln_a2, ln_c2), pack_f32x2(gb.z, gb.w), pack_f32x2(eb.z, eb.w));
-                    }
-                    uint4 q;
-                    q.x = pack_bf16_pair(v[0]); q.y = pack_bf16_pair(v[1]); q.z = pack_bf16_pair(v[2]); q.w = pack_bf16_pair(v[3]);
-                    st_shared_v4(slot, q);
-                }
-                if (cidx & 1) {   // the warp's slice of this 64-column tile is complete
-                    fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmap_out, (col0 >> 6) * 64, row0, tile + quad * 32 * 128);   // rows past the matrix are clipped
-                        bulk_commit();
-                    }
-                }
-            };
-            {
-                uint32_t acc_a[32], acc_b[32];
-                tmem_ld_32x32(lane_addr + chunk_col(0), acc_a);
-#pragma unroll 1
-                for (int cidx = 0; cidx < kColChunks; cidx += 2) {
-                    tmem_ld_wait();
-                    tmem_ld_32x32(lane_addr + chunk_col(cidx + 1), acc_b);
-                    out_chunk(acc_a, cidx);
-                    tmem_ld_wait();
-                    if (cidx + 2 < kColChunks) {
-                        tmem_ld_32x32(lane_addr + chunk_col(cidx + 2), acc_a);
-                    } else {   // last read of O by this warp
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_cluster_relaxed(lead_o_empty);
-                    }
-                    out_chunk(acc_b, cidx + 1);
-                }
-            }
+            if (!(ok = row_epilogue<HID, LN, true>(rc, p.b2, p.ln_gamma, p.ln_beta, p.ln_eps, PRE ? 1u : (nb & 1), &tmap_out,
+                                                   blk * kPairRows + (int)cta_rank * BLOCK_M + quad * 32))) break;
             if (lane == 0) {
                 bulk_wait_read<0>();      // the stores have read their slices: X may be overwritten
                 mbar_arrive(x_empty);

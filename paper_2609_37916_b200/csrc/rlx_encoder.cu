@@ -232,14 +232,14 @@ cudaError_t init_kernels_for_current_device() {
         if ((e = cudaOccupancyMaxActiveClusters(&n, rlx::tcar::gemm_ares_tcgen05_kernel<256, 0>, &cfg)) != cudaSuccess) return e;
         if (dev < 64) g_max_pairs_resident[dev] = n;
     }
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tcff::Cfg<384>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<384, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tcff::Cfg<384>::SMEM_BYTES)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(rlx::tcff::ffn_fused_tcgen05_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
+    {
+        const void* ffn_kernels[] = {(const void*)rlx::tcff::ffn_fused_tcgen05_kernel<384, false, false>, (const void*)rlx::tcff::ffn_fused_tcgen05_kernel<384, true, false>,
+                                     (const void*)rlx::tcff::ffn_fused_tcgen05_kernel<384, true, true>,   (const void*)rlx::tcff::ffn_fused_tcgen05_kernel<256, false, false>,
+                                     (const void*)rlx::tcff::ffn_fused_tcgen05_kernel<256, true, false>,  (const void*)rlx::tcff::ffn_fused_tcgen05_kernel<256, true, true>};
+        for (int i = 0; i < 6; ++i)
+            if ((e = cudaFuncSetAttribute(ffn_kernels[i], cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          i < 3 ? rlx::tcff::Cfg<384>::SMEM_BYTES : rlx::tcff::Cfg<256>::SMEM_BYTES)) != cudaSuccess) return e;
+    }
     if ((e = cudaFuncSetAttribute(rlx::tcmx::gemm_mx_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   rlx::tcmx::kSmemBytes)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(rlx::tcmx::wide::gemm_mx192_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -434,19 +434,36 @@ rlx_status_t launch_attention_tc(const bf16* qkv, int rows, const int32_t* seq_s
 
 // Feed-forward block in one kernel (hidden 256 or 384, F % 64 == 0): out = gelu(x W1^T + b1) W2^T + b2 + x.
 bool ffn_fused_supported(int H, int F) { return (H == 256 || H == 384) && F % 128 == 0 && F >= 128; }
+// One launcher for the three forms of the row-block kernel:
+//   pre == nullptr:  out = [LayerNorm2](gelu(x W1^T + b1) W2^T + b2 + x)
+//   pre != nullptr:  x1 = LayerNorm1(ctx Wo^T + bo + h) first (x = ctx), then the same with x1 in place of x
+struct FfnPre {
+    const bf16* h;      // residual rows of the projection in front
+    const bf16* wo;     // [H, H]
+    const float* bo;
+    const float* ln1_gamma;
+    const float* ln1_beta;
+};
 rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, const bf16* w2, const float* b2, int M, int H,
                               int F, bf16* out, int32_t* status, cudaStream_t st, const int32_t* rows_ptr,
-                              const float* ln_gamma = nullptr, const float* ln_beta = nullptr, float ln_eps = 0.f) {
+                              const float* ln_gamma = nullptr, const float* ln_beta = nullptr, float ln_eps = 0.f,
+                              const FfnPre* pre = nullptr) {
     if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
-    CUtensorMap tx, t1, t2, to;
+    if (pre && !ln_gamma) return RLX_ERR_INVALID_ARG;
+    const uint32_t w2_rows = H == 384 ? rlx::tcff::Cfg<384>::W2_ROWS : rlx::tcff::Cfg<256>::W2_ROWS;
+    CUtensorMap tx, t1, t2, to, two, th;
     if (!make_tmap(&tx, x, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M) || !make_tmap(&to, out, (uint64_t)M, (uint64_t)H, 32) ||
         !make_tmap(&t1, w1, (uint64_t)F, (uint64_t)H, H == 384 ? rlx::tcff::Cfg<384>::W1_ROWS : rlx::tcff::Cfg<256>::W1_ROWS) ||
-        !make_tmap(&t2, w2, (uint64_t)H, (uint64_t)F, H == 384 ? rlx::tcff::Cfg<384>::W2_ROWS : rlx::tcff::Cfg<256>::W2_ROWS))
+        !make_tmap(&t2, w2, (uint64_t)H, (uint64_t)F, w2_rows))
+        return RLX_ERR_CUDA;
+    two = t2; th = tx;
+    if (pre && (!make_tmap(&two, pre->wo, (uint64_t)H, (uint64_t)H, w2_rows) || !make_tmap(&th, pre->h, (uint64_t)M, (uint64_t)H, rlx::tc::BLOCK_M)))
         return RLX_ERR_CUDA;
     rlx::tcff::FfnParams p;
     p.b1 = b1; p.b2 = b2; p.out = out; p.M = M; p.F = F; p.m_ptr = rows_ptr; p.status = status;
     p.ln_gamma = ln_gamma; p.ln_beta = ln_beta; p.ln_eps = ln_eps;
-    const bool ln = ln_gamma != nullptr;
+    p.bo = pre ? pre->bo : nullptr; p.ln1_gamma = pre ? pre->ln1_gamma : nullptr; p.ln1_beta = pre ? pre->ln1_beta : nullptr;
+    const int form = pre ? 2 : ln_gamma ? 1 : 0;
     int dev = 0;
     cudaGetDevice(&dev);
     const int pairs_max = (dev >= 0 && dev < 64 && g_max_pairs_resident[dev] > 0) ? g_max_pairs_resident[dev] : sm_count() / 2;
@@ -456,14 +473,15 @@ rlx_status_t launch_ffn_fused(const bf16* x, const bf16* w1, const float* b1, co
         ClusterScope() { g_cluster_x = 2; }
         ~ClusterScope() { g_cluster_x = 1; }
     } scope;
-    if (H == 384 && ln)
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384, true>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
-    else if (H == 384)
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<384, false>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<384>::SMEM_BYTES, st, tx, t1, t2, to, p));
-    else if (ln)
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256, true>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
-    else
-        RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<256, false>, grid, rlx::tcff::kThreads, rlx::tcff::Cfg<256>::SMEM_BYTES, st, tx, t1, t2, to, p));
+#define RLX_FFN_LAUNCH(HID, LN, PRE)                                                                                   \
+    RLX_CUDA_TRY(launch_ex(rlx::tcff::ffn_fused_tcgen05_kernel<HID, LN, PRE>, grid, rlx::tcff::kThreads,               \
+                           rlx::tcff::Cfg<HID>::SMEM_BYTES, st, tx, t1, t2, to, two, th, p))
+    if (H == 384) {
+        if (form == 2) RLX_FFN_LAUNCH(384, true, true); else if (form == 1) RLX_FFN_LAUNCH(384, true, false); else RLX_FFN_LAUNCH(384, false, false);
+    } else {
+        if (form == 2) RLX_FFN_LAUNCH(256, true, true); else if (form == 1) RLX_FFN_LAUNCH(256, true, false); else RLX_FFN_LAUNCH(256, false, false);
+    }
+#undef RLX_FFN_LAUNCH
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -824,8 +842,9 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
     return (long long)B * S >= 128ll * sm_count_of(c.device);
 }
 
-// FFN-up, GELU and FFN-down in one kernel (needs the plain 7-kernel layer around it).  The kernel works in
-// blocks of 256 rows, one per CTA pair, so it needs about a wave of blocks to beat the two GEMMs: forced by
+// Everything of a layer behind the attention in one kernel (out-projection, residual, LayerNorm, FFN-up, GELU,
+// FFN-down, residual, LayerNorm): a layer is QKV GEMM, attention and this.  The kernel works in blocks of 256
+// rows, one per CTA pair, so it needs about a wave of blocks to beat the separate kernels: forced by
 // RLX_FLAG_FUSED_FFN at any size, chosen by itself from 16384 padded tokens on (the number of valid tokens
 // is known only on the device), never with RLX_FLAG_NO_FUSED_FFN.
 constexpr long long kAutoFusedFfnMinTokens = 16384;
@@ -865,7 +884,7 @@ bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S) {
 int kernels_in_forward(const rlx_encoder_config_t& c, int B, int S) {
     const bool pack = !(c.flags & RLX_FLAG_NO_PACK) && !(c.flags & RLX_FLAG_GEMM_SIMT);
     const bool fused = uses_fold_ln(c, B, S) || uses_fused_ln(c, B, S) || uses_cluster_ln(c);
-    return 2 + ((fused ? 5 : 7) - (uses_fused_ffn(c, B, S) ? 2 : 0)) * c.num_layers + (pack ? 1 : 0);
+    return 2 + ((fused ? 5 : 7) - (uses_fused_ffn(c, B, S) ? 4 : 0)) * c.num_layers + (pack ? 1 : 0);
 }
 bool uses_chunks(const rlx_encoder_config_t& c, int B, int S);
 int chunk_batch(int B, int S);
@@ -1097,6 +1116,14 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
                                             reinterpret_cast<unsigned int*>(ws + a.status + kAttnTicketOffset), status, st));
         else
             RLX_TRY(launch_attention_bf16(qkv, mask, pk.seq_start, pk.seq_len, B, S, h, d, ctx, st));
+        if (fuse_ffn) {
+            // everything behind the attention in one kernel: out-projection + residual + LayerNorm, the feed-forward
+            // block (the F-wide activation stays on the chip) + residual + LayerNorm; x is read and rewritten by rows
+            FfnPre pre{x, (const bf16*)lw.wo, lw.bo, lw.ln1_g, lw.ln1_b};
+            RLX_TRY(launch_ffn_fused(ctx, (const bf16*)lw.w1, lw.b1, (const bf16*)lw.w2, lw.b2, T, H, F, x, status, st, rows,
+                                     lw.ln2_g, lw.ln2_b, c.ln_eps, &pre));
+            continue;
+        }
         if (fuse_ln) {
             RLX_TRY(launch_gemm_ln(ctx, (const bf16*)lw.wo, lw.bo, x, lw.ln1_g, lw.ln1_b, c.ln_eps, T, H, H, x1, status, st, rows));
         } else if (fuse_cln) {
@@ -1104,13 +1131,6 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         } else {
             RLX_TRY(launch_gemm(ctx, (const bf16*)lw.wo, lw.bo, x, RLX_EPI_BIAS_RESIDUAL, T, H, H, y, simt, status, st, rows));
             RLX_TRY(launch_layernorm(y, lw.ln1_g, lw.ln1_b, T, H, c.ln_eps, x1, st, rows));
-        }
-        if (fuse_ffn) {
-            // the whole feed-forward block in one kernel: the F-wide activation stays on the chip
-            // and the layer's second LayerNorm in its epilogue, on the unrounded sums
-            RLX_TRY(launch_ffn_fused(x1, (const bf16*)lw.w1, lw.b1, (const bf16*)lw.w2, lw.b2, T, H, F, x, status, st, rows,
-                                     lw.ln2_g, lw.ln2_b, c.ln_eps));
-            continue;
         }
         RLX_TRY(launch_gemm(x1, (const bf16*)lw.w1, lw.b1, nullptr, RLX_EPI_BIAS_GELU, T, F, H, g, simt, status, st, rows));
         if (fuse_ln) {
@@ -1803,6 +1823,23 @@ rlx_status_t rlx_ffn_fused_bf16(const void* x, const void* w1, const float* b1, 
     RLX_CUDA_TRY(init_kernels_for_current_device());
     return launch_ffn_fused((const bf16*)x, (const bf16*)w1, b1, (const bf16*)w2, b2, M, H, F, (bf16*)out, status,
                             static_cast<cudaStream_t>(stream), nullptr, ln_gamma, ln_beta, ln_eps);
+}
+
+rlx_status_t rlx_layer_tail_bf16(const void* ctx, const void* h, const void* wo, const float* bo, const float* ln1_gamma,
+                                 const float* ln1_beta, const void* w1, const float* b1, const void* w2, const float* b2,
+                                 const float* ln2_gamma, const float* ln2_beta, float ln_eps, int32_t M, int32_t H, int32_t F,
+                                 void* out, int32_t* status, void* stream) {
+    if (!ctx || !h || !wo || !bo || !ln1_gamma || !ln1_beta || !w1 || !b1 || !w2 || !b2 || !ln2_gamma || !ln2_beta || !out)
+        return RLX_ERR_INVALID_ARG;
+    if (M <= 0 || H <= 0 || F <= 0 || !(ln_eps > 0.f)) return RLX_ERR_INVALID_ARG;
+    const void* ptrs[] = {ctx, h, wo, bo, ln1_gamma, ln1_beta, w1, b1, w2, b2, ln2_gamma, ln2_beta, out};
+    for (const void* q : ptrs)
+        if (!aligned16(q)) return RLX_ERR_INVALID_ARG;
+    if (!ffn_fused_supported(H, F)) return RLX_ERR_UNSUPPORTED;
+    RLX_CUDA_TRY(init_kernels_for_current_device());
+    FfnPre pre{(const bf16*)h, (const bf16*)wo, bo, ln1_gamma, ln1_beta};
+    return launch_ffn_fused((const bf16*)ctx, (const bf16*)w1, b1, (const bf16*)w2, b2, M, H, F, (bf16*)out, status,
+                            static_cast<cudaStream_t>(stream), nullptr, ln2_gamma, ln2_beta, ln_eps, &pre);
 }
 
 rlx_status_t rlx_pool_l2norm(const void* x, const int32_t* mask, int32_t B, int32_t S, int32_t H, float* out,

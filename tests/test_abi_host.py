@@ -44,7 +44,7 @@ def test_create_validates_shapes(lib):
     enc = binding.Encoder(**_cfg(max_batch=128))
     assert enc.kernels_per_forward(32, 128) == 3 + 5 * 6   # small batch: LayerNorm folded into the GEMMs automatically
     assert enc.kernels_per_forward(100, 128) == 3 + 7 * 6  # packing + embed + 7 per layer + pool
-    assert enc.kernels_per_forward(128, 128) == 3 + 5 * 6  # from 16384 padded tokens on: feed-forward block and second LayerNorm in one kernel
+    assert enc.kernels_per_forward(128, 128) == 3 + 3 * 6  # from 16384 padded tokens on: everything behind the attention in one kernel
     enc.close()
     for bad, status in [
         (dict(hidden=400, num_heads=10), 2),    # H % 128
@@ -62,13 +62,13 @@ def test_create_validates_shapes(lib):
 
 def test_kernel_count_follows_the_layernorm_fusion_flags(lib):
     enc = binding.Encoder(**_cfg(max_batch=256, max_seq=256))
-    assert enc.kernels_per_forward(256, 256) == 3 + 5 * 6     # default: one LayerNorm kernel, one feed-forward kernel (with the second LayerNorm)
+    assert enc.kernels_per_forward(256, 256) == 3 + 3 * 6     # default: QKV GEMM, attention, and one kernel for the rest of the layer
     enc.close()
     two = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_NO_FUSED_FFN))
     assert two.kernels_per_forward(256, 256) == 3 + 7 * 6
     two.close()
     one = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_FUSED_FFN | binding.FLAG_NO_AUTO_FOLD))
-    assert one.kernels_per_forward(8, 64) == 3 + 5 * 6        # forced at every size
+    assert one.kernels_per_forward(8, 64) == 3 + 3 * 6        # forced at every size
     one.close()
     cl = binding.Encoder(**_cfg(max_batch=256, max_seq=256, flags=binding.FLAG_CLUSTER_LN))
     assert cl.kernels_per_forward(256, 256) == 3 + 5 * 6      # folded into the GEMMs (cluster statistics)

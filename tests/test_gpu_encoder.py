@@ -330,10 +330,10 @@ def test_graph_cache_reuse_and_new_inputs(rlx):
 
 @pytest.mark.parametrize("flags", [0x1400, 0x1401], ids=["graph", "eager"])
 def test_fused_ffn_forward_against_the_two_kernel_forward(rlx, flags):
-    """RLX_FLAG_FUSED_FFN: FFN-up, GELU, FFN-down and the second LayerNorm of every layer in one kernel.  The
-    feed-forward part has the rounding points and the k order of the two-kernel form; the LayerNorm works on
-    the unrounded sums (one bf16 rounding fewer per layer), so the embeddings differ from the plain 7-kernel
-    layer's by rounding noise only (0x400 keeps LayerNorm folding out of both)."""
+    """RLX_FLAG_FUSED_FFN: everything of a layer behind the attention in one kernel.  The products have the
+    rounding points and the k order of the separate GEMMs; both LayerNorms work on unrounded sums (two bf16
+    roundings fewer per layer), so the embeddings differ from the plain 7-kernel layer's by rounding noise only
+    (0x400 keeps LayerNorm folding out of both)."""
     inp = make_inputs(CONFIGS["c2"])
     w = rlx.upload_weights(inp.params, inp.layers)
     plain, status = run_gpu(rlx, inp, weights=w, flags=0x400 | (flags & 1))
@@ -346,9 +346,8 @@ def test_fused_ffn_forward_against_the_two_kernel_forward(rlx, flags):
 
 
 def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
-    """Without a flag the one-kernel feed-forward block (with the second LayerNorm) takes over at batch*seq >=
-    16384; RLX_FLAG_NO_FUSED_FFN (0x2000) keeps the two GEMMs and the LayerNorm kernel.  Two kernels less per
-    layer, embeddings equal up to rounding noise."""
+    """Without a flag the one-kernel layer tail takes over at batch*seq >= 16384; RLX_FLAG_NO_FUSED_FFN (0x2000)
+    keeps the 7-kernel layer.  Four kernels less per layer, embeddings equal up to rounding noise."""
     inp = make_inputs(CONFIGS["c2"], batch=130, num_layers=2)
     w = rlx.upload_weights(inp.params, inp.layers)
     auto, status = run_gpu(rlx, inp, weights=w, flags=0)
@@ -362,6 +361,6 @@ def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
     assert c.batch * c.seq >= 16384
     a = rlx.Encoder.from_config(c, flags=0, max_batch=c.batch, max_seq=c.seq)
     b = rlx.Encoder.from_config(c, flags=0x2000, max_batch=c.batch, max_seq=c.seq)
-    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == 2 * c.num_layers
+    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == 4 * c.num_layers
     assert a.kernels_per_forward(127, 128) == b.kernels_per_forward(127, 128)
     a.close(); b.close()

@@ -217,6 +217,37 @@ def test_ffn_fused_matches_oracle(rlx, M, H, F):
     assert_close_bf16_out(got_ln, oracle.layernorm(ref, gamma, beta, 1e-12), extra_abs=1e-2)
 
 
+@pytest.mark.parametrize("M,H,F", [(256, 384, 256), (300, 384, 1536), (5000, 384, 1536), (40000, 384, 1536), (1000, 256, 512),
+                                   (37, 384, 128)])
+def test_layer_tail_matches_oracle(rlx, M, H, F):
+    """Out-projection + residual + LayerNorm + feed-forward block + residual + LayerNorm in one kernel against
+    the oracle's linear / layernorm / gelu.  The reference mirrors the two bf16 roundings inside (x1 and the
+    hidden activation); both LayerNorms see unrounded sums."""
+    rng = np.random.default_rng(M + H + F + 1)
+    ctx = rand_bf16(rng, (M, H))
+    h = rand_bf16(rng, (M, H))
+    wo = rand_bf16(rng, (H, H), 0.05)
+    w1 = rand_bf16(rng, (F, H), 0.05)
+    w2 = rand_bf16(rng, (H, F), 0.05)
+    bo, b2 = [(0.1 * rng.standard_normal(H)).astype(np.float32) for _ in range(2)]
+    b1 = (0.1 * rng.standard_normal(F)).astype(np.float32)
+    g1, g2 = [(1 + 0.1 * rng.standard_normal(H)).astype(np.float32) for _ in range(2)]
+    e1, e2 = [(0.1 * rng.standard_normal(H)).astype(np.float32) for _ in range(2)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = to_np64(rlx.layer_tail_bf16(bf16_dev(ctx), bf16_dev(h), bf16_dev(wo), f32_dev(bo), f32_dev(g1), f32_dev(e1),
+                                      bf16_dev(w1), f32_dev(b1), bf16_dev(w2), f32_dev(b2), f32_dev(g2), f32_dev(e2), 1e-12,
+                                      status=status))
+    assert int(status.item()) == 0
+    x1 = round_to_bf16(oracle.layernorm(oracle.linear(ctx.astype(np.float64), wo, bo) + h.astype(np.float64), g1, e1,
+                                        1e-12).astype(np.float32)).astype(np.float64)
+    g = round_to_bf16(oracle.gelu(oracle.linear(x1, w1, b1)).astype(np.float32)).astype(np.float64)
+    ref = oracle.layernorm(oracle.linear(g, w2, b2) + x1, g2, e2, 1e-12)
+    # a rounding flip of an x1 value (one bf16 ulp of |x1| ~ 1) moves the result by about that ulp
+    assert_close_bf16_out(got, ref, extra_abs=2e-2)
+    # the library's own unfused chain: same values up to those flips
+    assert np.abs(got - ref).mean() <= 2e-3
+
+
 def test_ffn_fused_layernorm_rows_with_a_large_mean(rlx):
     """Rows whose mean is 200 times their spread: the row statistics are kept as deviations from a pivot, so the
     variance does not cancel.  Zero weights make the pre-LayerNorm row exactly x + b2."""
