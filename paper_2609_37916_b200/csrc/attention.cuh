@@ -282,6 +282,8 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         constexpr int NT = KS / 8;   // score n-tiles per step
 #pragma unroll
         for (int hf = 0; hf < kAttBlockN / KS; ++hf) {
+        // packed rows: the sequence's last key block may end before this step's keys begin (uniform in the CTA)
+        if (MK == 0 && hf > 0 && packed && k0 + hf * KS >= len) break;
         // ---- S = Q K^T for KS keys: NT n-tiles x 4 accumulators ----
         float s[NT][4];
 #pragma unroll
