@@ -848,11 +848,15 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
 // RLX_FLAG_FUSED_FFN at any size, chosen by itself from 16384 padded tokens on (the number of valid tokens
 // is known only on the device), never with RLX_FLAG_NO_FUSED_FFN.
 constexpr long long kAutoFusedFfnMinTokens = 16384;
+// Sub-batches of a chunked call take the kernel choice of the whole call (its padded token count), so that
+// chunking never changes which kernels compute a row.
+thread_local long long g_whole_call_tokens = 0;
 bool ffn_fused_supported(int H, int F);
 bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S);
 bool uses_fused_ffn(const rlx_encoder_config_t& c, int B, int S) {
     if (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN | RLX_FLAG_NO_FUSED_FFN)) return false;
-    if (!(c.flags & RLX_FLAG_FUSED_FFN) && (long long)B * S < kAutoFusedFfnMinTokens) return false;
+    const long long tokens = g_whole_call_tokens > 0 ? g_whole_call_tokens : (long long)B * S;
+    if (!(c.flags & RLX_FLAG_FUSED_FFN) && tokens < kAutoFusedFfnMinTokens) return false;
     return ffn_fused_supported(c.hidden, c.ffn) && !uses_fold_ln(c, B, S);
 }
 
@@ -1167,6 +1171,10 @@ rlx_status_t enqueue_forward_any(const rlx_encoder* e, const int32_t* ids, const
                                  bool capturing, bool with_events = true) {
     if (!uses_chunks(e->cfg, B, S)) return enqueue_forward(e, ids, mask, B, S, w, out, ws, st, capturing, with_events);
     const int bc = chunk_batch(B, S);
+    struct WholeCall {
+        explicit WholeCall(long long t) { g_whole_call_tokens = t; }
+        ~WholeCall() { g_whole_call_tokens = 0; }
+    } whole((long long)B * S);
     for (int b0 = 0; b0 < B; b0 += bc) {
         const int nb = std::min(bc, B - b0);
         rlx_status_t s = enqueue_forward(e, ids + (size_t)b0 * S, mask + (size_t)b0 * S, nb, S, w,
