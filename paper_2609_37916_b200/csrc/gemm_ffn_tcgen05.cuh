@@ -121,20 +121,23 @@ struct RowCtx {
     uint32_t ln_bar;         // [4] per lane quarter
     uint32_t lead_o_empty;   // leader CTA's barrier: O has been read
     volatile int* abort_flag;
-    int r, ew, quad, half, lane;
+    int r, wslot, quad, grp, lane;   // row in the CTA; index of the warp's parameter copy; lane quarter; column group
 };
 
 // Row epilogue of a 128 x HID accumulator block:  v = O + bias + residual (the bf16 values in the X tiles),
 // optionally through LayerNorm, rounded to bf16 and written back over the residual's slots; with STORE each
 // warp then stores its 32-row slice of every 64-column tile with one TMA store (row0 = the slice's first global
 // row).  Returns false when a bounded wait ran out.
-template <int HID, bool DO_LN, bool STORE>
-__device__ __forceinline__ bool row_epilogue(const RowCtx& rc, const float* bias, const float* gamma, const float* beta, float eps,
+template <int HID, bool DO_LN, bool STORE, int GROUPS>
+__device__ __noinline__ bool row_epilogue(const RowCtx rc, const float* bias, const float* gamma, const float* beta, float eps,
                                              uint32_t ln_parity, const CUtensorMap* tmap_out, int row0) {
     const uint32_t lane_addr = rc.lane_addr, xs = rc.xs, gs = rc.gs, ln_bar = rc.ln_bar, lead_o_empty = rc.lead_o_empty;
     volatile int* abort_flag = rc.abort_flag;
-    const int r = rc.r, ew = rc.ew, quad = rc.quad, half = rc.half, lane = rc.lane;
-    constexpr int kTilesPerWarp = HID / 128;   // this warp's column half = HID/2 columns = HID/128 tiles of 64
+    const int r = rc.r, wslot = rc.wslot, quad = rc.quad, grp = rc.grp, lane = rc.lane;
+    // The columns are split over GROUPS warps per lane quarter (two with the eight epilogue warps alone, three when
+    // the producer and MMA-issuing warps, idle while rows are finished, form a third group).
+    static_assert(HID % (64 * GROUPS) == 0, "whole 64-column tiles per group");
+    constexpr int kTilesPerWarp = HID / 64 / GROUPS;
     // LN variant: the row then goes through LayerNorm before it is rounded.  A row's H values sit with two
     // threads (same lane quarter and lane, the two column halves): a first pass over O and X sums v and
     // v^2 per thread, the pair swaps its sums through shared memory (the first G buffer, idle until the
@@ -147,19 +150,20 @@ __device__ __forceinline__ bool row_epilogue(const RowCtx& rc, const float* bias
     // b2 (and gamma, beta) of the warp's column half go to a private copy in the idle G buffers first
     // (behind the 2 KB the row sums are swapped through): every thread needs every value, and broadcast
     // reads from shared memory are several times cheaper than same-address global loads.
-    constexpr int kParamVecs = DO_LN ? 3 : 1, kHalfCols = HID / 2;
-    const uint32_t par = gs + 2048 + ew * (3 * kHalfCols * 4);
-    static_assert(2048 + kEpiWarps * 3 * kHalfCols * 4 <= 2 * Cfg<HID>::G_BYTES, "parameter copies fit in the G buffers");
+    constexpr int kParamVecs = DO_LN ? 3 : 1, kHalfCols = HID / GROUPS;
+    constexpr int kScratch = GROUPS * BLOCK_M * 8;   // (mean, M2) per row and group
+    const uint32_t par = gs + kScratch + wslot * (3 * kHalfCols * 4);
+    static_assert(kScratch + 4 * GROUPS * 3 * kHalfCols * 4 <= 2 * Cfg<HID>::G_BYTES, "parameter copies fit in the G buffers");
     for (int idx = lane; idx < kParamVecs * (kHalfCols / 4); idx += 32) {
         const int a = idx / (kHalfCols / 4), w4 = idx - a * (kHalfCols / 4);
-        const float* src = (a == 0 ? bias : a == 1 ? gamma : beta) + half * kHalfCols;
+        const float* src = (a == 0 ? bias : a == 1 ? gamma : beta) + grp * kHalfCols;
         st_shared_f32x4(par + (a * kHalfCols + w4 * 4) * 4, __ldg(reinterpret_cast<const float4*>(src) + w4));
     }
     __syncwarp();
     const auto param4 = [&](int a, int col0, int i4) {   // 4 values of vector a at columns col0 + 4*i4 ..
-        return ld_shared_f32x4(par + (a * kHalfCols + (col0 - half * kHalfCols) + 4 * i4) * 4);
+        return ld_shared_f32x4(par + (a * kHalfCols + (col0 - grp * kHalfCols) + 4 * i4) * 4);
     };
-    const auto chunk_col = [&](int cidx) { return (half * kTilesPerWarp + (cidx >> 1)) * 64 + (cidx & 1) * 32; };
+    const auto chunk_col = [&](int cidx) { return (grp * kTilesPerWarp + (cidx >> 1)) * 64 + (cidx & 1) * 32; };
     float ln_a = 1.f, ln_c = 0.f;    // y = (v * ln_a + ln_c) * gamma + beta
     if constexpr (DO_LN) {
         // sums of (v - pivot) and (v - pivot)^2 with the thread's first value as the pivot: no cancellation
@@ -210,19 +214,26 @@ __device__ __forceinline__ bool row_epilogue(const RowCtx& rc, const float* bias
             unpack_f32x2(sq2, q0, q1);
             sum = a0 + a1; sq = q0 + q1;
         }
-        // this thread's half row: mean and sum of squared deviations; the halves combine pairwise
-        constexpr float kHalf = (float)(HID / 2);
-        const float my_mean = pivot + sum * (1.f / kHalf);
-        const float my_m2 = fmaxf(sq - sum * sum * (1.f / kHalf), 0.f);
-        st_shared_f32x2(gs + (uint32_t)((half * BLOCK_M + r) * 8), my_mean, my_m2);
+        // this thread's part of the row: mean and sum of squared deviations; the parts are combined in group order
+        // by every thread of the row, so that all of them normalise with the same two numbers
+        constexpr float kPart = (float)kHalfCols;
+        const float my_mean = pivot + sum * (1.f / kPart);
+        const float my_m2 = fmaxf(sq - sum * sum * (1.f / kPart), 0.f);
+        st_shared_f32x2(gs + (uint32_t)((grp * BLOCK_M + r) * 8), my_mean, my_m2);
         __syncwarp();
         if (lane == 0) mbar_arrive(ln_bar + 8 * quad);
         if (!mbar_wait(ln_bar + 8 * quad, ln_parity, abort_flag)) return false;
-        float o_mean, o_m2;
-        ld_shared_f32x2(gs + (uint32_t)(((half ^ 1) * BLOCK_M + r) * 8), o_mean, o_m2);
-        const float mean = 0.5f * (my_mean + o_mean);
-        const float dm = my_mean - o_mean;
-        const float var = (my_m2 + o_m2 + dm * dm * (0.5f * kHalf)) * (1.f / HID);
+        float mean, m2;
+        ld_shared_f32x2(gs + (uint32_t)(r * 8), mean, m2);
+#pragma unroll
+        for (int g = 1; g < GROUPS; ++g) {
+            float o_mean, o_m2;
+            ld_shared_f32x2(gs + (uint32_t)((g * BLOCK_M + r) * 8), o_mean, o_m2);
+            const float dm = o_mean - mean;
+            mean += dm * (1.f / (g + 1));                              // g parts of kPart columns so far, one more
+            m2 += o_m2 + dm * dm * (kPart * (float)g / (float)(g + 1));
+        }
+        const float var = m2 * (1.f / HID);
         ln_a = rsqrtf(var + eps);
         ln_c = -mean * ln_a;
     }
@@ -286,6 +297,12 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                          const __grid_constant__ CUtensorMap tmap_w2, const __grid_constant__ CUtensorMap tmap_out,
                          const __grid_constant__ CUtensorMap tmap_wo, const __grid_constant__ CUtensorMap tmap_h, const FfnParams p) {
     using C = Cfg<HID>;
+    // Warps that finish rows: the eight epilogue warps as two column groups.  A third group made of the warps that
+    // have nothing to issue while rows are finished (X / W1 producer and the three MMA-issuing warps: lane quarters
+    // 0, 1, 2, 3; kGroups = 3 at H = 384, every hook below is in place) was measured SLOWER (101 against 96 us per
+    // layer at 37 k rows): the passes are paced by the shared-memory pipe, not by the number of warps.
+    constexpr int kGroups = 2;
+    constexpr int kRowWarps = 4 * kGroups;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -310,11 +327,11 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         mbar_init(x_full, 1);
-        mbar_init(o_empty, 2 * kEpiWarps);
-        mbar_init(x_empty, 2 + kEpiWarps);      // both first-product warps' last commits + this CTA's epilogue warps
+        mbar_init(o_empty, 2 * kRowWarps);
+        mbar_init(x_empty, 2 + kRowWarps);      // both first-product warps' last commits + this CTA's row-epilogue warps
         mbar_init(o_full, 1);
-        for (int i = 0; i < 4; ++i) mbar_init(ln_bar + 8 * i, 2);
-        mbar_init(a_done, 1); mbar_init(h_full, 1); mbar_init(x_ready, 2 * kEpiWarps);
+        for (int i = 0; i < 4; ++i) mbar_init(ln_bar + 8 * i, kGroups);
+        mbar_init(a_done, 1); mbar_init(h_full, 1); mbar_init(x_ready, 2 * kRowWarps);
         for (int i = 0; i < 2; ++i) {
             mbar_init(w1_full + 8 * i, 1); mbar_init(w2_full + 8 * i, 1);
             mbar_init(w1_empty + 8 * i, 1); mbar_init(w2_empty + 8 * i, 1);
@@ -343,26 +360,78 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     const int pairs = gridDim.x / 2, pair0 = blockIdx.x / 2;
     const int n_chunks = p.F / kChunk;
 
+    // ---- row epilogues (the LayerNorm in front with PRE, the block's end), shared by every warp that finishes rows
+    const bool epi_warp = warp >= 2 && warp < 2 + kEpiWarps;
+    const bool helper_warp = kGroups == 3 && (warp <= 1 || warp == 2 + kEpiWarps || warp == 3 + kEpiWarps);   // lane quarters 0, 1, 2, 3
+    RowCtx rc;
+    rc.quad = warp & 3;
+    rc.lane_addr = tmem + ((uint32_t)(rc.quad * 32) << 16);
+    rc.xs = xs; rc.gs = gs; rc.ln_bar = ln_bar; rc.abort_flag = abort_flag; rc.lane = lane;
+    rc.r = rc.quad * 32 + lane;
+    rc.grp = epi_warp ? (warp - 2) >> 2 : 2;
+    rc.wslot = epi_warp ? warp - 2 : kEpiWarps + rc.quad;
+    rc.lead_o_empty = map_to_cta(o_empty, 0);
+    const uint32_t lead_x_ready = map_to_cta(x_ready, 0);
+    // x1 = LayerNorm(ctx Wo^T + bo + h) for the block's rows, written over the residual rows h in the X tiles: the
+    // A operand of the first products and the residual of the block's end, never in global memory
+    const auto front_rows = [&](uint32_t nb) -> bool {
+        if (!mbar_wait(a_done, nb & 1, abort_flag)) return false;
+        tc_fence_after();
+        if (!mbar_wait(h_full, nb & 1, abort_flag)) return false;
+        if (!row_epilogue<HID, true, false, kGroups>(rc, p.bo, p.ln1_gamma, p.ln1_beta, p.ln_eps, 0u, nullptr, 0)) return false;
+        fence_proxy_async();     // generic-proxy writes -> visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster_release_cta(lead_x_ready);
+        return true;
+    };
+    // out = [LayerNorm](O + b2 + X).  The resident X tiles serve twice more: each thread reads its residual values
+    // from them and writes the finished bf16 outputs back to the same 16-byte slots (same rows, same swizzle), and
+    // the warp then stores its 32-row slice of a 64-column tile with one TMA store -- the tile's layout in shared
+    // memory is the one the TMA load produced, so the store map has the load map's geometry.
+    const auto final_rows = [&](uint32_t nb, int blk) -> bool {
+        if (!mbar_wait(o_full, nb & 1, abort_flag)) return false;
+        tc_fence_after();
+        if (!row_epilogue<HID, LN, true, kGroups>(rc, p.b2, p.ln_gamma, p.ln_beta, p.ln_eps, PRE ? 1u : (nb & 1), &tmap_out,
+                                                  blk * kPairRows + (int)cta_rank * BLOCK_M + rc.quad * 32)) return false;
+        if (lane == 0) {
+            bulk_wait_read<0>();      // the stores have read their slices: X may be overwritten
+            mbar_arrive(x_empty);
+        }
+        __syncwarp();
+        return true;
+    };
+
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer of X and the W1 chunks (both CTAs)
-        if (lane == 0) {
+        // The whole warp runs the loop (lane 0 issues): at H = 384 it also finishes rows as lane quarter 0 of the
+        // third column group -- after the first two W1 chunks are on their way (PRE) and after the block's last one.
+        {
             bool ok = true;
             uint32_t nb = 0, cc = 0;   // blocks and chunks done so far
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                if (nb >= 1 && !(ok = mbar_wait(x_empty, (nb - 1) & 1, abort_flag))) break;
-                const uint32_t lead_x = map_to_cta(x_full, 0);
-                if (cta_rank == 0) mbar_expect_tx(x_full, 2 * C::X_BYTES);
-                const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
-                for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d_cg2(xs + kb * BLOCK_M * 128, &tmap_x, kb * BLOCK_K, xrow, lead_x);
-                for (int c = 0; c < n_chunks; ++c, ++cc) {
-                    const uint32_t st = cc & 1, use = cc >> 1;
-                    if (use >= 1 && !(ok = mbar_wait(w1_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
-                    const uint32_t lead1 = map_to_cta(w1_full + 8 * st, 0);
-                    if (cta_rank == 0) mbar_expect_tx(w1_full + 8 * st, 2 * C::W1_STAGE);
-                    for (int kb = 0; kb < C::KB1; ++kb)
-                        tma_load_2d_cg2(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128, &tmap_w1, kb * BLOCK_K,
-                                        c * kChunk + (int)cta_rank * C::W1_ROWS, lead1);
+                if (nb >= 1 && !(ok = mbar_wait_warp(x_empty, (nb - 1) & 1, abort_flag))) break;
+                if (lane == 0) {
+                    const uint32_t lead_x = map_to_cta(x_full, 0);
+                    if (cta_rank == 0) mbar_expect_tx(x_full, 2 * C::X_BYTES);
+                    const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
+                    for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d_cg2(xs + kb * BLOCK_M * 128, &tmap_x, kb * BLOCK_K, xrow, lead_x);
                 }
+                for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
+                    if (PRE && helper_warp && c == 2 && !(ok = front_rows(nb))) break;
+                    const uint32_t st = cc & 1, use = cc >> 1;
+                    if (use >= 1 && !(ok = mbar_wait_warp(w1_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
+                    if (lane == 0) {
+                        const uint32_t lead1 = map_to_cta(w1_full + 8 * st, 0);
+                        if (cta_rank == 0) mbar_expect_tx(w1_full + 8 * st, 2 * C::W1_STAGE);
+                        for (int kb = 0; kb < C::KB1; ++kb)
+                            tma_load_2d_cg2(w1s + st * C::W1_STAGE + kb * C::W1_ROWS * 128, &tmap_w1, kb * BLOCK_K,
+                                            c * kChunk + (int)cta_rank * C::W1_ROWS, lead1);
+                    }
+                    __syncwarp();
+                }
+                if (!ok) break;
+                if (PRE && helper_warp && n_chunks <= 2 && !(ok = front_rows(nb))) break;
+                if (helper_warp && !(ok = final_rows(nb, blk))) break;
             }
         }
     } else if (warp == 4 + kEpiWarps) {
@@ -410,14 +479,16 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         // a second warp: odd chunks into S buffer 1; F is a multiple of 128, so the parity of a chunk is
         // the parity of its ring slot in every block); a third warp issues the second products.  Whole-warp
         // loops, one elected lane issues.
-        if (cta_rank == 0) {
+        // In both CTAs these warps are lane quarters 1 and 3 of the third column group of the row epilogues (H = 384).
+        {
             constexpr uint32_t id1 = make_idesc(kPairRows, kChunk);
             const uint32_t st = warp == 1 ? 0u : 1u;
             bool ok = true;
             uint32_t nb = 0;
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                if (!(ok = mbar_wait_warp(PRE ? x_ready : x_full, nb & 1, abort_flag))) break;
-                for (int c = st; c < n_chunks && ok; c += 2) {
+                if (PRE && helper_warp && !(ok = front_rows(nb))) break;
+                if (cta_rank == 0 && !(ok = mbar_wait_warp(PRE ? x_ready : x_full, nb & 1, abort_flag))) break;
+                for (int c = st; cta_rank == 0 && c < n_chunks && ok; c += 2) {
                     const uint32_t use = (nb * n_chunks + c) >> 1;
                     if (!(ok = mbar_wait_warp(w1_full + 8 * st, use & 1, abort_flag))) break;
                     if (use >= 1 && !(ok = mbar_wait_warp(s_empty + 8 * st, (use - 1) & 1, abort_flag))) break;
@@ -437,16 +508,19 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                     }
                     __syncwarp();
                 }
+                if (!ok) break;
+                if (helper_warp && !(ok = final_rows(nb, blk))) break;
             }
         }
     } else if (warp == 2 + kEpiWarps) {
         // ------------------------------------------------------------ second products O += G_c W2_c^T (leader CTA)
-        if (cta_rank == 0) {
+        // In both CTAs this warp is lane quarter 2 of the third column group of the row epilogues (H = 384).
+        {
             constexpr uint32_t id2 = make_idesc(kPairRows, HID / 2);
             bool ok = true;
             uint32_t nb = 0, cc = 0, u2 = 0, oe = 0;   // blocks, chunks, W2-ring uses, completions of o_empty waited for
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-                if (PRE) {
+                if (PRE && cta_rank == 0) {
                     // the projection in front:  O = ctx Wo^T, the resident tiles as A, Wo's k-block tiles through the ring
                     if (!(ok = mbar_wait_warp(x_full, nb & 1, abort_flag))) break;
                     if (nb >= 1) {   // the previous block's result rows have been read out of O
@@ -473,7 +547,8 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                     }
                     if (!ok) break;
                 }
-                for (int c = 0; c < n_chunks && ok; ++c, ++cc, ++u2) {
+                if (PRE && helper_warp && !(ok = front_rows(nb))) break;
+                for (int c = 0; cta_rank == 0 && c < n_chunks && ok; ++c, ++cc, ++u2) {
                     const uint32_t st = cc & 1, use = cc >> 1, st2 = u2 & 1;
                     if (!(ok = mbar_wait_warp(w2_full + 8 * st2, (u2 >> 1) & 1, abort_flag))) break;
                     // first accumulation of the block overwrites O: its last readers (the previous block's epilogue, or
@@ -499,34 +574,21 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                     }
                     __syncwarp();
                 }
+                if (!ok) break;
+                if (helper_warp && !(ok = final_rows(nb, blk))) break;
             }
         }
     } else {
         // ------------------------------------------------------------ epilogue warps (both CTAs)
-        const int ew = warp - 2, quad = warp & 3, half = ew >> 2;
-        const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-        const int r = quad * 32 + lane;                      // this thread's row within the CTA's 128
+        const int ew = warp - 2, half = ew >> 2;
+        const uint32_t lane_addr = rc.lane_addr;
+        const int r = rc.r;                                  // this thread's row within the CTA's 128
         const uint32_t b1_slot = base + C::B1_OFF + ew * 128;
-        RowCtx rc;
-        rc.lane_addr = lane_addr; rc.xs = xs; rc.gs = gs; rc.ln_bar = ln_bar; rc.abort_flag = abort_flag;
-        rc.r = r; rc.ew = ew; rc.quad = quad; rc.half = half; rc.lane = lane;
-            const uint32_t lead_s_empty = map_to_cta(s_empty, 0), lead_g_full = map_to_cta(g_full, 0), lead_o_empty = map_to_cta(o_empty, 0);
-        rc.lead_o_empty = lead_o_empty;
+        const uint32_t lead_s_empty = map_to_cta(s_empty, 0), lead_g_full = map_to_cta(g_full, 0);
         bool ok = true;
         uint32_t nb = 0, cc = 0;
-        const uint32_t lead_x_ready = map_to_cta(x_ready, 0);
         for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
-            if (PRE) {
-                // x1 = LayerNorm(ctx Wo^T + bo + h) for the block's rows, written over the residual rows h in the X
-                // tiles: the A operand of the first products and the residual of the block's end, never in global memory
-                if (!(ok = mbar_wait(a_done, nb & 1, abort_flag))) break;
-                tc_fence_after();
-                if (!(ok = mbar_wait(h_full, nb & 1, abort_flag))) break;
-                if (!(ok = row_epilogue<HID, true, false>(rc, p.bo, p.ln1_gamma, p.ln1_beta, p.ln_eps, 0u, nullptr, 0))) break;
-                fence_proxy_async();     // generic-proxy writes -> visible to the tensor core's reads
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster_release_cta(lead_x_ready);
-            }
+            if (PRE && !(ok = front_rows(nb))) break;
             // Software pipeline over the chunks: the registers hold S_c when an iteration starts; the probe of
             // S_{c+1}'s barrier, the tensor-memory load of S_{c+1} and the probe of the G buffer's barrier are
             // issued between the halves of the GELU arithmetic, so their round trips (150-250 cycles each)
@@ -594,19 +656,7 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             }
             if (!ok) break;
             // ---- end of the block: out = O + b2 + X ----
-            if (!(ok = mbar_wait(o_full, nb & 1, abort_flag))) break;
-            tc_fence_after();
-            // The resident X tiles serve twice more: each thread reads its residual values from them and writes
-            // the finished bf16 outputs back to the same 16-byte slots (same rows, same swizzle), and the warp
-            // then stores its 32-row slice of a 64-column tile with one TMA store -- the tile's layout in shared
-            // memory is the one the TMA load produced, so the store map has the load map's geometry.
-            if (!(ok = row_epilogue<HID, LN, true>(rc, p.b2, p.ln_gamma, p.ln_beta, p.ln_eps, PRE ? 1u : (nb & 1), &tmap_out,
-                                                   blk * kPairRows + (int)cta_rank * BLOCK_M + quad * 32))) break;
-            if (lane == 0) {
-                bulk_wait_read<0>();      // the stores have read their slices: X may be overwritten
-                mbar_arrive(x_empty);
-            }
-            __syncwarp();
+            if (!(ok = final_rows(nb, blk))) break;
         }
     }
 
