@@ -199,3 +199,22 @@ def test_scaled_matmul_validates_on_the_host(lib):
     assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 2, 8, 64, 32, fake, fake, None, None) == 1   # residual missing
     assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 0, 8, 100, 32, fake, fake, None, None) == 2  # N % 64
     assert sm(fake, fake, fake, fmt(4, 3, 1), fake, None, 0, 8, 64, 32, None, fake, None, None) == 1   # no scratch
+
+
+def test_layer_tail_and_fused_ffn_validate_on_the_host(lib):
+    fake, odd = C.c_void_p(0x1000), C.c_void_p(0x1008)
+    eps = C.c_float(1e-12)
+    ffn = lib.rlx_ffn_fused_bf16
+    assert ffn(fake, fake, fake, fake, fake, None, None, C.c_float(0), 8, 384, 1536, None, None, None) == 1      # no output
+    assert ffn(fake, fake, fake, fake, fake, fake, None, eps, 8, 384, 1536, fake, None, None) == 1               # gamma without beta
+    assert ffn(fake, fake, fake, fake, fake, fake, fake, C.c_float(0), 8, 384, 1536, fake, None, None) == 1      # LayerNorm needs eps > 0
+    assert ffn(odd, fake, fake, fake, fake, None, None, C.c_float(0), 8, 384, 1536, fake, None, None) == 1       # misaligned x
+    assert ffn(fake, fake, fake, fake, fake, None, None, C.c_float(0), 8, 512, 2048, fake, None, None) == 2      # hidden 512: no room in tensor memory
+    assert ffn(fake, fake, fake, fake, fake, None, None, C.c_float(0), 8, 384, 1600, fake, None, None) == 2      # F % 128
+    tail = lib.rlx_layer_tail_bf16
+    args = [fake] * 12
+    assert tail(*args, eps, 8, 384, 1536, None, None, None) == 1
+    assert tail(*args, C.c_float(0), 8, 384, 1536, fake, None, None) == 1
+    assert tail(*(args[:5] + [None] + args[6:]), eps, 8, 384, 1536, fake, None, None) == 1                        # a LayerNorm vector missing
+    assert tail(*args, eps, 8, 768, 3072, fake, None, None) == 2
+    assert tail(*args, eps, 0, 384, 1536, fake, None, None) == 1
