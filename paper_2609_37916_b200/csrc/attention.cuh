@@ -74,19 +74,30 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 }
 
 constexpr int kAttBlockM = 128;  // query rows per CTA (8 warps x 16 rows)
-constexpr int kAttBlockN = 64;   // keys per shared-memory stage
-constexpr int kAttStages = 4;    // K/V ring depth (three blocks in flight ahead of the one being used)
+constexpr int kAttBlockN = 64;   // keys per shared-memory stage (default ring, see AttRing)
+constexpr int kAttStages = 4;    // K/V ring depth of the default ring (three blocks in flight ahead of the one being used)
 constexpr int kAttThreads = 256;
 constexpr int kAttMaxSeq = 512;
 
-template <int D>
+// Keys per shared-memory stage and depth of the K/V ring.  The encoder's own shape (head_dim 32, at most 512 keys,
+// no window, no rotation: the launcher's choice, kernel parameter WIDE) takes 128-key stages in a two-deep ring: a sequence is one to four stages, so half as
+// many CTA-wide barriers are crossed for the same shared memory (-5 % at 256 x 256).  Long sequences (the mask
+// kinds, rotary q/k, head_dim 64 / 128) keep 64-key stages four deep: with thousands of keys the prefetch
+// distance matters more than the barrier count (the 128 x 2 ring measured 30-50 % slower there).
+template <bool WIDE>
+struct AttRing {
+    static constexpr int BN = WIDE ? 128 : kAttBlockN;
+    static constexpr int ST = WIDE ? 2 : kAttStages;
+};
+
+template <int D, int BN = kAttBlockN, int ST = kAttStages>
 struct AttSmem {
     static constexpr int kStride = D + 8;  // +16 bytes per row: conflict-free ldmatrix
     __nv_bfloat16 q[kAttBlockM * kStride];  // Q tile; reused as the output staging tile at the end
-    __nv_bfloat16 k[kAttStages][kAttBlockN * kStride];
-    __nv_bfloat16 v[kAttStages][kAttBlockN * kStride];
+    __nv_bfloat16 k[ST][BN * kStride];
+    __nv_bfloat16 v[ST][BN * kStride];
     float bias[kAttMaxSeq];                 // padded mode: 0 for a valid key, -inf for a masked one
-    int blk_full[kAttMaxSeq / kAttBlockN];  // padded mode: 1 when all 64 keys of the block are valid
+    int blk_full[kAttMaxSeq / BN];          // padded mode: 1 when all keys of the block are valid
     int kv_end;
     int q_any;
 };
@@ -113,12 +124,13 @@ struct AttKind {
 //   padded: seq_start == nullptr.  Sequence b occupies rows b*S .. b*S+S; `mask` flags valid keys.
 //   packed: rows of sequence b are seq_start[b] .. seq_start[b]+seq_len[b], all valid (mask unused).
 template <int D, int MK = 0, bool ROPE = false, int KS = (((D == 32 && MK == 0 && !ROPE) || D == 128) ? 32 : 64),
-          int MINB = (D == 32 ? (KS == 32 ? 4 : 3) : D == 64 ? 2 : 1)>
+          int MINB = (D == 32 ? (KS == 32 ? 4 : 3) : D == 64 ? 2 : 1), bool WIDE = false>
 __global__ void __launch_bounds__(kAttThreads, MINB)
 attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __restrict__ mask,
                       const int32_t* __restrict__ seq_start, const int32_t* __restrict__ seq_len,
                       __nv_bfloat16* __restrict__ ctx, int S, int H, float scale_log2e, AttKind kind) {
-    using SM = AttSmem<D>;
+    constexpr int BN = AttRing<WIDE>::BN, ST = AttRing<WIDE>::ST;
+    using SM = AttSmem<D, BN, ST>;
     constexpr int STR = SM::kStride;
     constexpr int KT = D / 16;       // k-tiles of the QK^T product
     constexpr int ND = D / 8;        // n-tiles of the PV product
@@ -144,10 +156,10 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     int kv_end = len;
     if (!packed) {
         if (tid == 0) { sm.kv_end = 0; sm.q_any = 0; }
-        if (tid < kAttMaxSeq / kAttBlockN) sm.blk_full[tid] = 1;
+        if (tid < kAttMaxSeq / BN) sm.blk_full[tid] = 1;
         __syncthreads();
         int last = 0, any = 0;
-        const int spad = (S + kAttBlockN - 1) / kAttBlockN * kAttBlockN;
+        const int spad = (S + BN - 1) / BN * BN;
         for (int k = tid; k < spad; k += kAttThreads) {
             const bool valid = (k < S) && (__ldg(mask + row0 + k) != 0);
             sm.bias[k] = valid ? 0.f : -INFINITY;
@@ -155,7 +167,7 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 last = k + 1;
                 any |= (k >= q0 && k < q0 + kAttBlockM);
             } else {
-                sm.blk_full[k / kAttBlockN] = 0;   // benign race: every writer stores 0
+                sm.blk_full[k / BN] = 0;   // benign race: every writer stores 0
             }
         }
         if (last) atomicMax(&sm.kv_end, last);
@@ -172,11 +184,11 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
             return;
         }
     }
-    int jb0 = 0, nblk = (kv_end + kAttBlockN - 1) / kAttBlockN;   // key blocks jb0 .. nblk-1
+    int jb0 = 0, nblk = (kv_end + BN - 1) / BN;   // key blocks jb0 .. nblk-1
     if (MK) {
         const int q_hi = min(q0 + kAttBlockM, len);                // one past this CTA's last real row
-        jb0 = max(0, q0 - kind.window + 1) / kAttBlockN;
-        nblk = (q_hi + kAttBlockN - 1) / kAttBlockN;
+        jb0 = max(0, q0 - kind.window + 1) / BN;
+        nblk = (q_hi + BN - 1) / BN;
     }
 
     auto load_rows = [&](const __nv_bfloat16* base, __nv_bfloat16* dst, int first_row, int nrows) {
@@ -206,10 +218,10 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
     };
     load_qk(qbase, sm.q, q0, kAttBlockM);
 #pragma unroll
-    for (int j = 0; j < kAttStages - 1; ++j) {
+    for (int j = 0; j < ST - 1; ++j) {
         if (jb0 + j < nblk) {
-            load_qk(kbase, sm.k[j], (jb0 + j) * kAttBlockN, kAttBlockN);
-            load_rows(vbase, sm.v[j], (jb0 + j) * kAttBlockN, kAttBlockN);
+            load_qk(kbase, sm.k[j], (jb0 + j) * BN, BN);
+            load_rows(vbase, sm.v[j], (jb0 + j) * BN, BN);
         }
         cp_async_commit();
     }
@@ -247,24 +259,24 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
 
     const int r0 = q0 + warp * 16;   // first query row of this warp (index within the sequence)
     for (int j = jb0; j < nblk; ++j) {
-        const int buf = (j - jb0) % kAttStages;
-        cp_async_wait<kAttStages - 2>();   // block j (and Q) have landed
+        const int buf = (j - jb0) % ST;
+        cp_async_wait<ST - 2>();   // block j (and Q) have landed
         if (ROPE && j == jb0) {            // own copies of Q and the first key block: rotate before publishing
             rope_rows(sm.q, q0, kAttBlockM);
-            rope_rows(sm.k[buf], j * kAttBlockN, kAttBlockN);
+            rope_rows(sm.k[buf], j * BN, BN);
         }
         __syncthreads();                   // ... for every thread; and block j-1's stage is free
-        if (j + kAttStages - 1 < nblk) {
-            const int nb = (j - jb0 + kAttStages - 1) % kAttStages;
-            load_qk(kbase, sm.k[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
-            load_rows(vbase, sm.v[nb], (j + kAttStages - 1) * kAttBlockN, kAttBlockN);
+        if (j + ST - 1 < nblk) {
+            const int nb = (j - jb0 + ST - 1) % ST;
+            load_qk(kbase, sm.k[nb], (j + ST - 1) * BN, BN);
+            load_rows(vbase, sm.v[nb], (j + ST - 1) * BN, BN);
         }
         cp_async_commit();
         if (ROPE && j + 1 < nblk) {
             // block j+1 is rotated one step ahead by the threads that copied it; nobody reads it before
             // the barrier at the top of the next iteration
-            cp_async_wait<kAttStages - 2>();
-            rope_rows(sm.k[(j + 1 - jb0) % kAttStages], (j + 1) * kAttBlockN, kAttBlockN);
+            cp_async_wait<ST - 2>();
+            rope_rows(sm.k[(j + 1 - jb0) % ST], (j + 1) * BN, BN);
         }
         if (!warp_active) continue;
         if (j == jb0) {
@@ -275,13 +287,13 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 ldmatrix_x4(smem_u32(sm.q + r * STR + c), qf[kt][0], qf[kt][1], qf[kt][2], qf[kt][3]);
             }
         }
-        const int k0 = j * kAttBlockN;
-        if (MK && (k0 > r0 + 15 || k0 + kAttBlockN - 1 <= r0 - kind.window)) continue;   // nothing visible
+        const int k0 = j * BN;
+        if (MK && (k0 > r0 + 15 || k0 + BN - 1 <= r0 - kind.window)) continue;   // nothing visible
         // The online-softmax step covers KS keys (64: the whole staged block; 32: half of it, which halves
         // the score and probability registers and lets a fourth CTA fit on the SM at head_dim 32).
         constexpr int NT = KS / 8;   // score n-tiles per step
 #pragma unroll
-        for (int hf = 0; hf < kAttBlockN / KS; ++hf) {
+        for (int hf = 0; hf < BN / KS; ++hf) {
         // packed rows: the sequence's last key block may end before this step's keys begin (uniform in the CTA)
         if (MK == 0 && hf > 0 && packed && k0 + hf * KS >= len) break;
         // ---- S = Q K^T for KS keys: NT n-tiles x 4 accumulators ----
@@ -303,7 +315,7 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
         // ---- masking only where the block has an invalid key ----
         if (MK) {
             // the block needs the element test unless every key is visible to all 16 rows
-            if (k0 + kAttBlockN > len || k0 + kAttBlockN - 1 > r0 || k0 <= r0 + 15 - kind.window) {
+            if (k0 + BN > len || k0 + BN - 1 > r0 || k0 <= r0 + 15 - kind.window) {
                 const int ia = r0 + g, ib = ia + 8;   // rows of accumulators {0,1} and {2,3}
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -315,7 +327,7 @@ attention_bf16_kernel(const __nv_bfloat16* __restrict__ qkv, const int32_t* __re
                 }
             }
         } else {
-            const bool need_mask = packed ? (k0 + kAttBlockN > len) : (sm.blk_full[j] == 0);
+            const bool need_mask = packed ? (k0 + BN > len) : (sm.blk_full[j] == 0);
             if (need_mask) {
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {

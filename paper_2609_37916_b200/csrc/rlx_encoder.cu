@@ -250,10 +250,14 @@ cudaError_t init_kernels_for_current_device() {
                                   rlx::tca::Smem<64>::BYTES)) != cudaSuccess) return e;
 #define RLX_ATT_SMEM_ATTR(D, MK, ROPE)                                                                       \
     if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<D, MK, ROPE>,                                  \
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(rlx::AttSmem<D>))) != \
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize,                 \
+                                  (int)sizeof(rlx::AttSmem<D>))) != \
         cudaSuccess)                                                                                        \
         return e;
     RLX_ATT_SMEM_ATTR(32, 0, false) RLX_ATT_SMEM_ATTR(64, 0, false)
+    if ((e = cudaFuncSetAttribute(rlx::attention_bf16_kernel<32, 0, false, 32, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)sizeof(rlx::AttSmem<32, rlx::AttRing<true>::BN, rlx::AttRing<true>::ST>))) != cudaSuccess)
+        return e;
     RLX_ATT_SMEM_ATTR(32, 0, true) RLX_ATT_SMEM_ATTR(64, 0, true)
     RLX_ATT_SMEM_ATTR(32, 1, false) RLX_ATT_SMEM_ATTR(64, 1, false)
     RLX_ATT_SMEM_ATTR(32, 1, true) RLX_ATT_SMEM_ATTR(64, 1, true)
@@ -378,10 +382,15 @@ rlx_status_t launch_attention_bf16(const bf16* qkv, const int32_t* mask, const i
     const bool rope = rope_cos != nullptr;
     if (d != 32 && d != 64 && d != 128) return RLX_ERR_UNSUPPORTED;
 #define RLX_ATT_LAUNCH(D, MK, ROPE)                                                                              \
-    RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<D, MK, ROPE>, grid, rlx::kAttThreads, sizeof(rlx::AttSmem<D>), \
+    RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<D, MK, ROPE>, grid, rlx::kAttThreads,                      \
+                           sizeof(rlx::AttSmem<D>),                                                                 \
                            st, qkv, mask, seq_start, seq_len, ctx, S, H, scale_log2e, kind))
     if (d == 32) {
-        if (!positional && !rope) RLX_ATT_LAUNCH(32, 0, false);
+        if (!positional && !rope && S <= rlx::kAttMaxSeq)   // the encoder's shape: 128-key stages, two deep
+            RLX_CUDA_TRY(launch_ex(rlx::attention_bf16_kernel<32, 0, false, 32, 4, true>, grid, rlx::kAttThreads,
+                                   sizeof(rlx::AttSmem<32, rlx::AttRing<true>::BN, rlx::AttRing<true>::ST>), st, qkv, mask, seq_start,
+                                   seq_len, ctx, S, H, scale_log2e, kind));
+        else if (!positional && !rope) RLX_ATT_LAUNCH(32, 0, false);
         else if (!positional) RLX_ATT_LAUNCH(32, 0, true);
         else if (!rope) RLX_ATT_LAUNCH(32, 1, false);
         else RLX_ATT_LAUNCH(32, 1, true);
