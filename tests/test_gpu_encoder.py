@@ -364,3 +364,28 @@ def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
     assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == 4 * c.num_layers
     assert a.kernels_per_forward(127, 128) == b.kernels_per_forward(127, 128)
     a.close(); b.close()
+
+
+def test_layer_tail_forward_on_random_shapes(rlx):
+    """Random batches (1..40 sequences of 1..512 positions, empty sequences, masks with holes, random LayerNorm
+    affine, 1..3 layers) through the forced 3-kernel layer, graph / eager / unpacked: against the oracle, run
+    twice for bit-for-bit repeatability."""
+    rng = np.random.default_rng(4242)
+    for _ in range(10):
+        B = int(rng.integers(1, 40))
+        S = int(rng.choice([1, 7, 16, 33, 64, 65, 127, 128, 200, 256, 300, 512]))
+        L = int(rng.integers(1, 4))
+        lengths = rng.integers(0, S + 1, size=B)
+        lengths[rng.integers(0, B)] = S
+        inp = make_inputs(CONFIGS["c1"], batch=B, seq=S, num_layers=L, lengths=lengths,
+                          ln_affine_random=bool(rng.integers(0, 2)), mask_holes=0.2 if rng.integers(0, 3) == 0 else 0.0)
+        ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
+        w = rlx.upload_weights(inp.params, inp.layers)
+        for flags in (0x1400, 0x1401, 0x1408):
+            enc = rlx.Encoder.from_config(inp.cfg, flags=flags, max_batch=B, max_seq=S)
+            assert enc.kernels_per_forward(B, S) == (2 if flags & 8 else 3) + 3 * L
+            a, status = run_gpu(rlx, inp, weights=w, enc=enc)
+            b, _ = run_gpu(rlx, inp, weights=w, enc=enc)
+            enc.close()
+            assert status == 0 and np.array_equal(a, b), (B, S, L, hex(flags))
+            check(a, ref, inp.lengths, tight=False)
