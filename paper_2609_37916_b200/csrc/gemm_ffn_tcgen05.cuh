@@ -51,7 +51,7 @@ struct Cfg {
     static constexpr int G_BYTES = BLOCK_M * 128;                   // one k-block tile of G
     static constexpr int X_OFF = 0, W1_OFF = X_BYTES, W2_OFF = W1_OFF + 2 * W1_STAGE, G_OFF = W2_OFF + 2 * W2_STAGE;
     static constexpr int BAR_OFF = G_OFF + 2 * G_BYTES;
-    static constexpr int B1_OFF = BAR_OFF + 256;                    // per epilogue warp: the 32 bias values of its chunk half
+    static constexpr int B1_OFF = BAR_OFF + 512;                    // per epilogue warp: the 32 bias values of its chunk half
     static constexpr int SMEM_BYTES = B1_OFF + kEpiWarps * 128 + 1024;
     static constexpr int COL_S = HID;                               // S buffers behind O
     static constexpr int TMEM_COLS = 512;
@@ -309,24 +309,24 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
     unsigned char* gbase = smem_raw + (base - raw);
     const uint32_t xs = base + C::X_OFF, w1s = base + C::W1_OFF, w2s = base + C::W2_OFF, gs = base + C::G_OFF;
     const uint32_t bars = base + C::BAR_OFF;
-    // leader-side barriers that both CTAs' TMA / warps arrive on: x_full, w1_full[2], w2_full[2], s_empty[2],
+    // leader-side barriers that both CTAs' TMA / warps arrive on: x_full[6] (one per k-block tile), w1_full[2], w2_full[2], s_empty[2],
     // g_full[2], o_empty.  Per-CTA barriers (multicast commits / own warps): x_empty, w1_empty[2], w2_empty[2],
     // s_full[2], g_empty[2], o_full.
-    const uint32_t x_full = bars, w1_full = x_full + 8, w2_full = w1_full + 16, s_empty = w2_full + 16, g_full = s_empty + 16;
+    const uint32_t x_full = bars, w1_full = x_full + 48, w2_full = w1_full + 16, s_empty = w2_full + 16, g_full = s_empty + 16;
     const uint32_t o_empty = g_full + 16, x_empty = o_empty + 8, w1_empty = x_empty + 8, w2_empty = w1_empty + 16;
     const uint32_t s_full = w2_empty + 16, g_empty = s_full + 16, o_full = g_empty + 16;
     const uint32_t ln_bar = o_full + 8;   // [4] per lane quarter: the two column halves' row sums are in shared memory
     // PRE variant: a_done (per CTA: the projection's products are complete), h_full (per CTA: the residual rows have
     // landed in the X tiles), x_ready (leader: all 16 epilogue warps have written their rows of X)
     const uint32_t a_done = ln_bar + 32, h_full = a_done + 8, x_ready = h_full + 8;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 27);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gbase + C::BAR_OFF + 8 * 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = cluster_ctarank();
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
-        mbar_init(x_full, 1);
+        for (int i = 0; i < C::KB1; ++i) mbar_init(x_full + 8 * i, 1);
         mbar_init(o_empty, 2 * kRowWarps);
         mbar_init(x_empty, 2 + kRowWarps);      // both first-product warps' last commits + this CTA's row-epilogue warps
         mbar_init(o_full, 1);
@@ -411,10 +411,12 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
                 if (nb >= 1 && !(ok = mbar_wait_warp(x_empty, (nb - 1) & 1, abort_flag))) break;
                 if (lane == 0) {
+                    // one barrier per k-block tile: the projection in front starts on tile 0 while the others land
                     const uint32_t lead_x = map_to_cta(x_full, 0);
-                    if (cta_rank == 0) mbar_expect_tx(x_full, 2 * C::X_BYTES);
+                    if (cta_rank == 0)
+                        for (int kb = 0; kb < C::KB1; ++kb) mbar_expect_tx(x_full + 8 * kb, 2 * BLOCK_M * 128);
                     const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
-                    for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d_cg2(xs + kb * BLOCK_M * 128, &tmap_x, kb * BLOCK_K, xrow, lead_x);
+                    for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d_cg2(xs + kb * BLOCK_M * 128, &tmap_x, kb * BLOCK_K, xrow, lead_x + 8 * kb);
                 }
                 for (int c = 0; c < n_chunks && ok; ++c, ++cc) {
                     if (PRE && helper_warp && c == 2 && !(ok = front_rows(nb))) break;
@@ -439,15 +441,23 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
         // A thread of its own: behind the W1 loads in one thread, a W2 slot that frees late (its second
         // product waits for the epilogue warps) would hold back the next chunk's W1 tiles as well.
         // PRE variant: the same ring first carries the k-block tiles of Wo (same shape: H output rows, 64 columns
-        // of K), and this thread also reloads the X tiles with the residual rows once the projection has read
-        // them -- between its first two W2 chunks, whose slots free at about that moment anyway.
+        // of K), and this thread also reloads the X tiles with the residual rows, tile by tile: the ring slot of Wo's
+        // k-block kb is free when the products on ctx tile kb have completed, which is when that tile is dead, so
+        // the residual tile follows the wait this thread does anyway before it reuses the slot.
         if (lane == 0) {
             bool ok = true;
             uint32_t u2 = 0, nb = 0;     // uses of the ring so far
+            uint32_t blk_u0 = 0;         // ... at the start of the current block
+            int blk_row = 0;             // this CTA's first row of the current block
             const auto load_tile = [&](const CUtensorMap* tmap, int kcol) -> bool {
                 const uint32_t st = u2 & 1, use = u2 >> 1;
-                ++u2;
                 if (use >= 1 && !mbar_wait(w2_empty + 8 * st, (use - 1) & 1, abort_flag)) return false;
+                if (PRE && u2 >= blk_u0 + 2 && u2 - 2 - blk_u0 < (uint32_t)C::KB1) {   // the slot held Wo's k-block kb of this block
+                    const int kb = (int)(u2 - 2 - blk_u0);
+                    if (kb == 0) mbar_expect_tx(h_full, C::X_BYTES);
+                    tma_load_2d(xs + kb * BLOCK_M * 128, &tmap_h, kb * BLOCK_K, blk_row, h_full);
+                }
+                ++u2;
                 const uint32_t lead2 = map_to_cta(w2_full + 8 * st, 0);
                 if (cta_rank == 0) mbar_expect_tx(w2_full + 8 * st, 2 * C::W2_STAGE);
                 for (int i = 0; i < 2; ++i)   // instruction i covers output columns i*HID/2 .., this CTA feeds its half of them
@@ -456,19 +466,13 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
                 return true;
             };
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
+                blk_u0 = u2;
+                blk_row = blk * kPairRows + (int)cta_rank * BLOCK_M;
                 if (PRE) {
                     for (int kb = 0; kb < C::KB1 && ok; ++kb) ok = load_tile(&tmap_wo, kb * BLOCK_K);
                     if (!ok) break;
                 }
-                for (int c = 0; c < n_chunks && ok; ++c) {
-                    if (PRE && c == 1) {
-                        if (!(ok = mbar_wait(a_done, nb & 1, abort_flag))) break;
-                        mbar_expect_tx(h_full, C::X_BYTES);
-                        const int xrow = blk * kPairRows + (int)cta_rank * BLOCK_M;
-                        for (int kb = 0; kb < C::KB1; ++kb) tma_load_2d(xs + kb * BLOCK_M * 128, &tmap_h, kb * BLOCK_K, xrow, h_full);
-                    }
-                    ok = load_tile(&tmap_w2, c * kChunk);
-                }
+                for (int c = 0; c < n_chunks && ok; ++c) ok = load_tile(&tmap_w2, c * kChunk);
             }
         }
     } else if (warp == 1 || warp == 3 + kEpiWarps) {
@@ -487,7 +491,14 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             uint32_t nb = 0;
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
                 if (PRE && helper_warp && !(ok = front_rows(nb))) break;
-                if (cta_rank == 0 && !(ok = mbar_wait_warp(PRE ? x_ready : x_full, nb & 1, abort_flag))) break;
+                if (cta_rank == 0) {
+                    if (PRE) {
+                        ok = mbar_wait_warp(x_ready, nb & 1, abort_flag);
+                    } else {
+                        for (int kb = 0; kb < C::KB1 && ok; ++kb) ok = mbar_wait_warp(x_full + 8 * kb, nb & 1, abort_flag);
+                    }
+                    if (!ok) break;
+                }
                 for (int c = st; cta_rank == 0 && c < n_chunks && ok; c += 2) {
                     const uint32_t use = (nb * n_chunks + c) >> 1;
                     if (!(ok = mbar_wait_warp(w1_full + 8 * st, use & 1, abort_flag))) break;
@@ -522,13 +533,13 @@ ffn_fused_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gri
             for (int blk = pair0; blk < blocks && ok; blk += pairs, ++nb) {
                 if (PRE && cta_rank == 0) {
                     // the projection in front:  O = ctx Wo^T, the resident tiles as A, Wo's k-block tiles through the ring
-                    if (!(ok = mbar_wait_warp(x_full, nb & 1, abort_flag))) break;
                     if (nb >= 1) {   // the previous block's result rows have been read out of O
                         if (!(ok = mbar_wait_warp(o_empty, oe & 1, abort_flag))) break;
                         ++oe;
                     }
                     for (int kb = 0; kb < C::KB1 && ok; ++kb, ++u2) {
                         const uint32_t st2 = u2 & 1;
+                        if (!(ok = mbar_wait_warp(x_full + 8 * kb, nb & 1, abort_flag))) break;   // ctx tile kb has landed
                         if (!(ok = mbar_wait_warp(w2_full + 8 * st2, (u2 >> 1) & 1, abort_flag))) break;
                         tc_fence_after();
                         if (elect_one()) {
