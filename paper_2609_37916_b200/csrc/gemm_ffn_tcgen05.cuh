@@ -1,27 +1,38 @@
-// Feed-forward block in one kernel:  out = gelu(X W1^T + b1) W2^T + b2 + X   (X = the LayerNorm output that
-// is both the block's input and its residual; W1 [F, H], W2 [H, F]; erf GELU).  The F-wide hidden activation
-// never reaches global memory: it is produced and consumed in chunks of 64 columns.
+// The part of an encoder layer behind the attention in one kernel (Section 3.2, operator fusion), in three forms
+// (template switches LN, PRE):
+//   plain        out = gelu(X W1^T + b1) W2^T + b2 + X                        X [M, H] is input AND residual
+//   LN           out = LayerNorm(gelu(X W1^T + b1) W2^T + b2 + X)
+//   LN + PRE     X   = LayerNorm(ctx Wo^T + bo + h) first (ctx: the attention's context rows, h: the layer's input
+//                rows), then the LN form: the whole layer tail; X never reaches global memory
+// W1 [F, H], W2 [H, F], Wo [H, H]; erf GELU.  The F-wide hidden activation never reaches global memory either: it
+// is produced and consumed in chunks of 64 columns.
 //
 // A CTA pair (tcgen05 cta_group::2, M = 256) owns a block of 256 rows at a time:
-//   X block    resident in shared memory for the whole block (H/64 swizzled k-block tiles per CTA); it is the
-//              A operand of every first product and, at the end, the residual (read from shared memory)
-//   chunk c    S_c = X W1[64c .. 64c+63, :]^T            M = 256, N = 64, K = H       -> TMEM (two S buffers)
-//              G_c = bf16(gelu(S_c + b1))                 epilogue warps: TMEM -> registers -> shared memory,
-//                                                         written in the K-major 128-byte-swizzled layout the
-//                                                         tensor core reads (two G buffers of one k-block)
-//              O  += G_c W2[:, 64c .. 64c+63]^T           M = 256, N = H (two instructions of H/2), K = 64
-//   end        out = O + b2 + X  -> bf16, written back over the X tile slots the residual was read from, and
-//              stored from there with one TMA store per warp and 64-column tile (the shared memory is full,
-//              the X tiles are the only staging room and already have the store's layout)
-// Roles (per CTA): warp 0 loads X and the W1 chunks, another warp the W2 chunks (so a late W2 slot never holds
-// back W1); in the leader CTA two warps issue the first products (even / odd chunks) and a third the second
-// products -- a thread pays ~100 cycles per tcgen05.mma, and one thread for a chunk's 32 instructions paced the
-// kernel; eight epilogue warps turn S_c into G_c in a software pipeline that overlaps the barrier probes and
-// the tensor-memory load of S_{c+1} with the GELU arithmetic of S_c.  W1 / W2 chunks stream through
-// two-stage rings, each CTA loading its half of the rows.  TMEM: O (H columns) + 2 x 64 columns of S = 512
-// at H = 384.
-// Rounding points are those of the two-kernel form (G rounded to bf16 once, fp32 accumulation in the same
-// k order), so the results agree with it to the last bit wherever the accumulation order is the same.
+//   front (PRE)  the ctx rows land in the X tiles (H/64 swizzled k-block tiles per CTA, one barrier per tile);
+//                O = ctx Wo^T with Wo's k-block tiles through the W2 ring; the residual rows h are loaded over
+//                each ctx tile as soon as the products on it have completed; row epilogue: X = bf16(LayerNorm(O +
+//                bo + h)) written over h in the same swizzled slots -- the A operand of what follows
+//   X block      resident in shared memory for the whole block; the A operand of every first product and, at the
+//                end, the residual (read from shared memory)
+//   chunk c      S_c = X W1[64c .. 64c+63, :]^T            M = 256, N = 64, K = H       -> TMEM (two S buffers)
+//                G_c = bf16(gelu(S_c + b1))                 epilogue warps: TMEM -> registers -> shared memory,
+//                                                           written in the K-major 128-byte-swizzled layout the
+//                                                           tensor core reads (two G buffers of one k-block)
+//                O  += G_c W2[:, 64c .. 64c+63]^T           M = 256, N = H (two instructions of H/2), K = 64
+//   end          out = [LayerNorm](O + b2 + X) -> bf16, written back over the X tile slots the residual was read
+//                from, and stored from there with one TMA store per warp and 64-column tile (the shared memory is
+//                full; the X tiles are the only staging room and already have the store's layout)
+// Roles (per CTA, 13 warps): warp 0 loads X and the W1 chunks, another warp the W2 chunks, Wo's tiles and the
+// residual tiles (so a late W2 slot never holds back W1); in the leader CTA two warps issue the first products
+// (even / odd chunks) and a third the second products and the projection in front -- a thread pays ~100 cycles
+// per tcgen05.mma, and one thread for a chunk's 32 instructions paced the kernel; eight epilogue warps turn S_c
+// into G_c in a software pipeline that overlaps the barrier probes and the tensor-memory load of S_{c+1} with
+// the GELU arithmetic of S_c, and run the row epilogues (two passes over tensor memory for a LayerNorm: pivoted
+// row sums, then normalise).  W1 / W2 chunks stream through two-stage rings, each CTA loading its half of the
+// rows.  TMEM: O (H columns) + 2 x 64 columns of S = 512 at H = 384.
+// Rounding points of the products are those of the separate GEMMs (G and X rounded to bf16 once, fp32
+// accumulation in the same k order): without LayerNorm the result is bit for bit the two-GEMM form's.  The
+// LayerNorms work on the unrounded fp32 sums.
 // All mbarrier waits are bounded; on expiry the CTA sets the status bit and leaves.
 #pragma once
 #include <cuda.h>
