@@ -455,6 +455,9 @@ def run_ours(args):
         ms3 = [a.elapsed_time(b) for a, b in ev3]
         peaks3, kind3 = load_peaks()
         kt3, ov3 = kernel_table(run3.cfg, run3.mine.lengths, run3.names, pc3, statistics.median(ms3), peaks3)
+        for cls, mb in load_dram_traffic().get("c3", {}).items():   # ncu dram__bytes per launch (profiles/dram_traffic.md)
+            if cls in kt3:
+                kt3[cls]["traffic"] = mb * 1e6
         roofline_c3 = {"workload": workload_config("c3")["workload"], "steps": args.c3_steps, "p50_ms": statistics.median(ms3),
                        "sequences_per_s": run3.cfg.batch / (statistics.median(ms3) / 1e3), "valid_tokens": int(run3.mine.lengths.sum()),
                        "clocks": s3.summary(), "peak_source": kind3, "event_overhead_us_per_launch": ov3,
