@@ -84,7 +84,7 @@ typedef enum {
                                       memory) at every batch size, so that a layer is 3 kernels; hidden 256 or 384,
                                       F % 128 == 0; ignored together with the LayerNorm fusion flags, the bring-up
                                       GEMM, or where the folded layer is chosen.  Without this flag that form is
-                                      chosen AUTOMATICALLY for calls with batch*seq >= 16384 (the kernel works in
+                                      chosen AUTOMATICALLY for calls with batch*seq >= 32768 (the kernel works in
                                       blocks of 256 rows per CTA pair and needs about a wave of them to win) */
 #define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep out-projection, LayerNorms and the two feed-forward GEMMs as separate
                                          kernels at every batch size */

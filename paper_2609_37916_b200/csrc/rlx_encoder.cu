@@ -854,9 +854,11 @@ bool uses_fused_ln(const rlx_encoder_config_t& c, int B, int S) {
 // Everything of a layer behind the attention in one kernel (out-projection, residual, LayerNorm, FFN-up, GELU,
 // FFN-down, residual, LayerNorm): a layer is QKV GEMM, attention and this.  The kernel works in blocks of 256
 // rows, one per CTA pair, so it needs about a wave of blocks to beat the separate kernels: forced by
-// RLX_FLAG_FUSED_FFN at any size, chosen by itself from 16384 padded tokens on (the number of valid tokens
-// is known only on the device), never with RLX_FLAG_NO_FUSED_FFN.
-constexpr long long kAutoFusedFfnMinTokens = 16384;
+// RLX_FLAG_FUSED_FFN at any size, chosen by itself from 32768 padded tokens on, never with
+// RLX_FLAG_NO_FUSED_FFN.  The number of VALID tokens is known only on the device: the form pays from about 9000
+// valid rows on (8972 valid: -1 %, 37 k: -15 %) and loses up to 20 % on a heavily padded batch (20480 padded,
+// 2729 valid: 393 against 330 us), so the padded threshold is set where a half-empty batch still breaks even.
+constexpr long long kAutoFusedFfnMinTokens = 32768;
 // Sub-batches of a chunked call take the kernel choice of the whole call (its padded token count), so that
 // chunking never changes which kernels compute a row.
 thread_local long long g_whole_call_tokens = 0;

@@ -41,10 +41,11 @@ def _cfg(**kw):
 
 
 def test_create_validates_shapes(lib):
-    enc = binding.Encoder(**_cfg(max_batch=128))
+    enc = binding.Encoder(**_cfg(max_batch=256))
     assert enc.kernels_per_forward(32, 128) == 3 + 5 * 6   # small batch: LayerNorm folded into the GEMMs automatically
     assert enc.kernels_per_forward(100, 128) == 3 + 7 * 6  # packing + embed + 7 per layer + pool
-    assert enc.kernels_per_forward(128, 128) == 3 + 3 * 6  # from 16384 padded tokens on: everything behind the attention in one kernel
+    assert enc.kernels_per_forward(128, 128) == 3 + 7 * 6
+    assert enc.kernels_per_forward(256, 128) == 3 + 3 * 6  # from 32768 padded tokens on: everything behind the attention in one kernel
     enc.close()
     for bad, status in [
         (dict(hidden=400, num_heads=10), 2),    # H % 128

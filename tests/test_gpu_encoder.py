@@ -345,10 +345,10 @@ def test_fused_ffn_forward_against_the_two_kernel_forward(rlx, flags):
     check(fused, ref, inp.lengths)
 
 
-def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
-    """Without a flag the one-kernel layer tail takes over at batch*seq >= 16384; RLX_FLAG_NO_FUSED_FFN (0x2000)
+def test_fused_ffn_is_chosen_from_32768_padded_tokens_on(rlx):
+    """Without a flag the one-kernel layer tail takes over at batch*seq >= 32768; RLX_FLAG_NO_FUSED_FFN (0x2000)
     keeps the 7-kernel layer.  Four kernels less per layer, embeddings equal up to rounding noise."""
-    inp = make_inputs(CONFIGS["c2"], batch=130, num_layers=2)
+    inp = make_inputs(CONFIGS["c2"], batch=256, num_layers=2)
     w = rlx.upload_weights(inp.params, inp.layers)
     auto, status = run_gpu(rlx, inp, weights=w, flags=0)
     assert status == 0
@@ -358,11 +358,11 @@ def test_fused_ffn_is_chosen_from_16384_padded_tokens_on(rlx):
     ref = oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers)
     check(auto, ref, inp.lengths)
     c = inp.cfg
-    assert c.batch * c.seq >= 16384
+    assert c.batch * c.seq >= 32768
     a = rlx.Encoder.from_config(c, flags=0, max_batch=c.batch, max_seq=c.seq)
     b = rlx.Encoder.from_config(c, flags=0x2000, max_batch=c.batch, max_seq=c.seq)
-    assert b.kernels_per_forward(130, 128) - a.kernels_per_forward(130, 128) == 4 * c.num_layers
-    assert a.kernels_per_forward(127, 128) == b.kernels_per_forward(127, 128)
+    assert b.kernels_per_forward(256, 128) - a.kernels_per_forward(256, 128) == 4 * c.num_layers
+    assert a.kernels_per_forward(255, 128) == b.kernels_per_forward(255, 128)
     a.close(); b.close()
 
 
