@@ -88,6 +88,14 @@ typedef enum {
                                       blocks of 256 rows per CTA pair and needs about a wave of them to win) */
 #define RLX_FLAG_NO_FUSED_FFN 0x2000u /* keep out-projection, LayerNorms and the two feed-forward GEMMs as separate
                                          kernels at every batch size */
+#define RLX_FLAG_DEVICE_CHOICE 0x4000u /* captured forwards of at least 12288 padded tokens carry both forms of the layer
+                                          (3 and 7 kernels) as the bodies of an IF / ELSE graph node; the packing kernel
+                                          takes the 3-kernel form when at least 9216 tokens are valid.  Removes the guess
+                                          from the padded size (the 3-kernel form loses up to 20 % on a heavily padded
+                                          batch) for 15-20 us per forward.  Ignored with the flags that fix the form, with
+                                          RLX_FLAG_NO_GRAPH / _KERNEL_EVENTS / _CHUNKED / _NO_PACK; the result is bit for
+                                          bit that of the form taken; rlx_encoder_kernels_per_forward keeps reporting the
+                                          host rule's count */
 #define RLX_FLAG_CHUNKED 0x800u /* token-chunk scheduling: a call of more than 16384 padded tokens runs as sub-batches of
                                    about that size, one after the other through the same workspace, so that every
                                    kernel's input is still in L2 when its consumer starts.  Results are bit for bit

@@ -33,6 +33,7 @@ FLAG_NO_AUTO_FOLD = 0x400
 FLAG_CHUNKED = 0x800
 FLAG_FUSED_FFN = 0x1000
 FLAG_NO_FUSED_FFN = 0x2000
+FLAG_DEVICE_CHOICE = 0x4000
 EPI_BIAS, EPI_BIAS_GELU, EPI_BIAS_RESIDUAL = 0, 1, 2
 GEMM_TCGEN05, GEMM_SIMT, GEMM_TCGEN05_PAIR, GEMM_TCGEN05_SINGLE, GEMM_TCGEN05_RESIDENT = 0, 1, 2, 3, 4
 STATIC_WORKSPACE_BYTES = 16 << 20

@@ -310,8 +310,10 @@ struct Packing {   // device arrays written by pack_sequences_kernel; all null i
 };
 
 rlx_status_t launch_pack(const int32_t* mask, int B, int S, int32_t* seq_len, int32_t* seq_start,
-                         int32_t* pos_of_rank, unsigned int* ticket, cudaStream_t st) {
-    rlx::pack_sequences_kernel<<<B, rlx::kPackThreads, 0, st>>>(mask, B, S, seq_len, seq_start, pos_of_rank, ticket);
+                         int32_t* pos_of_rank, unsigned int* ticket, cudaStream_t st,
+                         cudaGraphConditionalHandle cond = 0, int cond_min_rows = 0) {
+    rlx::pack_sequences_kernel<<<B, rlx::kPackThreads, 0, st>>>(mask, B, S, seq_len, seq_start, pos_of_rank, ticket, cond,
+                                                                cond_min_rows);
     RLX_CUDA_TRY(cudaGetLastError());
     return RLX_OK;
 }
@@ -862,13 +864,32 @@ constexpr long long kAutoFusedFfnMinTokens = 32768;
 // Sub-batches of a chunked call take the kernel choice of the whole call (its padded token count), so that
 // chunking never changes which kernels compute a row.
 thread_local long long g_whole_call_tokens = 0;
+// Bodies of the IF / ELSE node of a captured forward are recorded with the choice forced (1: layer tail, 0: separate
+// kernels; -1: the host's rule).
+thread_local int g_force_layer_tail = -1;
+// RLX_FLAG_DEVICE_CHOICE: captured forwards from this size on carry BOTH forms of the layer behind an IF / ELSE node
+// that the packing kernel sets from the packed row count: the host knows only the padded size, and the layer tail
+// loses up to 20 % on a heavily padded batch (measured: it pays from about 9000 valid rows on).  The node costs
+// 15-20 us per forward (no programmatic launch across it), which is why the host's rule is the default.
+constexpr long long kDeviceChoiceMinTokens = 12288;   // padded tokens; below, the separate kernels always win
+constexpr int kDeviceChoiceMinRows = 9216;            // packed rows from which the layer tail is taken
 bool ffn_fused_supported(int H, int F);
 bool uses_fold_ln(const rlx_encoder_config_t& c, int B, int S);
 bool uses_fused_ffn(const rlx_encoder_config_t& c, int B, int S) {
+    if (g_force_layer_tail >= 0) return g_force_layer_tail == 1;
     if (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN | RLX_FLAG_NO_FUSED_FFN)) return false;
     const long long tokens = g_whole_call_tokens > 0 ? g_whole_call_tokens : (long long)B * S;
     if (!(c.flags & RLX_FLAG_FUSED_FFN) && tokens < kAutoFusedFfnMinTokens) return false;
     return ffn_fused_supported(c.hidden, c.ffn) && !uses_fold_ln(c, B, S);
+}
+
+bool uses_device_choice(const rlx_encoder_config_t& c, int B, int S) {
+    if (c.flags & (RLX_FLAG_GEMM_SIMT | RLX_FLAG_FUSED_LN | RLX_FLAG_CLUSTER_LN | RLX_FLAG_NO_FUSED_FFN | RLX_FLAG_FUSED_FFN |
+                   RLX_FLAG_KERNEL_EVENTS | RLX_FLAG_CHUNKED | RLX_FLAG_NO_PACK | RLX_FLAG_NO_GRAPH | RLX_FLAG_FOLD_LN))
+        return false;
+    return (c.flags & RLX_FLAG_DEVICE_CHOICE) && g_force_layer_tail < 0 && g_whole_call_tokens == 0 &&
+           (long long)B * S >= kDeviceChoiceMinTokens &&
+           ffn_fused_supported(c.hidden, c.ffn) && !uses_fold_ln(c, B, S);
 }
 
 // RLX_FLAG_CLUSTER_LN: LayerNorm folded into the out-proj / FFN-down GEMMs with cluster-wide row
@@ -922,6 +943,7 @@ struct rlx_encoder {
     int last_kernels = 0;                   // kernels of the most recent forward (for kernel_times)
     std::vector<cudaEvent_t> events;        // RLX_FLAG_KERNEL_EVENTS: one before the first kernel, one after each
     cudaStream_t side_stream = nullptr;     // side branch of the captured graph (weight prefetch)
+    cudaStream_t body_stream = nullptr;     // the two bodies of a captured forward's IF / ELSE node are recorded here
     cudaEvent_t fork_event = nullptr, join_event = nullptr, fold_event = nullptr;
     cudaStream_t capture_stream = nullptr;  // graphs are recorded here (the caller's stream may be the
                                             // legacy default stream, which cannot be captured)
@@ -945,7 +967,7 @@ void drop_graphs(rlx_encoder* e) {
 // The kernel sequence of one forward, enqueued on `st` (eagerly or under stream capture).
 rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int32_t* mask, int B, int S,
                              const rlx_encoder_weights_t* w, float* out, unsigned char* ws, cudaStream_t st,
-                             bool capturing, bool with_events = true) {
+                             bool capturing, bool with_events = true, bool body_only = false) {
     const rlx_encoder_config_t& c = e->cfg;
     const int H = c.hidden, F = c.ffn, T = B * S, h = c.num_heads, d = e->head_dim;
     const bool simt = (c.flags & RLX_FLAG_GEMM_SIMT) != 0;
@@ -983,7 +1005,7 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
     } pdl_scope(!(c.flags & RLX_FLAG_NO_PDL) && !timing);
     // side branch (captured graphs only): prefetch the Linear weights into L2 when they all fit
     bool forked = false;
-    if (capturing && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH) && !fold) {   // the fold pass reads the weights anyway
+    if (capturing && !body_only && e->side_stream && !(c.flags & RLX_FLAG_NO_PREFETCH) && !fold) {   // the fold pass reads the weights anyway
         const size_t per_layer = ((size_t)3 * H * H + (size_t)H * H + (size_t)2 * H * F) * sizeof(bf16);
         if (per_layer * c.num_layers <= ((size_t)48 << 20) && 4 * c.num_layers <= rlx::kMaxPrefetch) {
             rlx::PrefetchList pf = {};
@@ -1012,11 +1034,47 @@ rlx_status_t enqueue_forward(const rlx_encoder* e, const int32_t* ids, const int
         int32_t* seq_len = reinterpret_cast<int32_t*>(ws + a.seq_len);
         int32_t* seq_start = reinterpret_cast<int32_t*>(ws + a.seq_start);
         int32_t* pos_of_rank = reinterpret_cast<int32_t*>(ws + a.pos_of_rank);
+        pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
         // The tickets live in the status block, which the caller zeroes once before the first call; each
         // kernel leaves its own at zero again, so no memset node sits in front of the first kernel.
-        RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank,
-                            reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset), st));
-        pk.seq_len = seq_len; pk.seq_start = seq_start; pk.pos_of_rank = pos_of_rank; pk.B = B;
+        unsigned int* ticket = reinterpret_cast<unsigned int*>(ws + a.status + kTicketOffset);
+        if (capturing && !body_only && e->body_stream && uses_device_choice(c, B, S)) {
+            // Both forms of everything behind the packing kernel, as the two bodies of an IF / ELSE node whose
+            // condition that kernel sets from the packed row count.
+            cudaStreamCaptureStatus cstat;
+            cudaGraph_t gcap = nullptr;
+            const cudaGraphNode_t* deps = nullptr;
+            size_t ndeps = 0;
+            RLX_CUDA_TRY(cudaStreamGetCaptureInfo_v2(st, &cstat, nullptr, &gcap, &deps, &ndeps));
+            if (cstat != cudaStreamCaptureStatusActive || gcap == nullptr) return RLX_ERR_CUDA;
+            cudaGraphConditionalHandle cond;
+            RLX_CUDA_TRY(cudaGraphConditionalHandleCreate(&cond, gcap, 0, cudaGraphCondAssignDefault));
+            RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank, ticket, st, cond, kDeviceChoiceMinRows));
+            RLX_CUDA_TRY(cudaStreamGetCaptureInfo_v2(st, &cstat, nullptr, &gcap, &deps, &ndeps));
+            cudaGraphNodeParams np = {};
+            np.type = cudaGraphNodeTypeConditional;
+            np.conditional.handle = cond;
+            np.conditional.type = cudaGraphCondTypeIf;
+            np.conditional.size = 2;
+            cudaGraphNode_t cnode = nullptr;
+            RLX_CUDA_TRY(cudaGraphAddNode(&cnode, gcap, deps, ndeps, &np));
+            for (int body = 0; body < 2; ++body) {
+                RLX_CUDA_TRY(cudaStreamBeginCaptureToGraph(e->body_stream, np.conditional.phGraph_out[body], nullptr, nullptr, 0,
+                                                           cudaStreamCaptureModeThreadLocal));
+                g_force_layer_tail = body == 0 ? 1 : 0;
+                const rlx_status_t bs = enqueue_forward(e, ids, mask, B, S, w, out, ws, e->body_stream, true, false, true);
+                g_force_layer_tail = -1;
+                g_pdl_launch = !(c.flags & RLX_FLAG_NO_PDL) && !timing;   // the nested call's scope switched it off
+                cudaGraph_t ended = nullptr;
+                const cudaError_t ce = cudaStreamEndCapture(e->body_stream, &ended);
+                if (bs != RLX_OK) return bs;
+                RLX_CUDA_TRY(ce);
+            }
+            RLX_CUDA_TRY(cudaStreamUpdateCaptureDependencies(st, &cnode, 1, cudaStreamSetCaptureDependencies));
+            if (forked) RLX_CUDA_TRY(cudaStreamWaitEvent(st, e->join_event, 0));   // join the side branch
+            return RLX_OK;
+        }
+        if (!body_only) RLX_TRY(launch_pack(mask, B, S, seq_len, seq_start, pos_of_rank, ticket, st));
     }
     const int32_t* rows = pk.total();
     const bool fuse_ln = !fold && uses_fused_ln(c, B, S);
@@ -1314,6 +1372,7 @@ rlx_status_t forward_device(rlx_encoder* e, const int32_t* ids, const int32_t* m
     // capture once for this (batch, seq, pointer set)
     cudaGraph_t graph = nullptr;
     if (!e->capture_stream) RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking));
+    if (!e->body_stream) RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->body_stream, cudaStreamNonBlocking));
     if (!e->side_stream) {
         RLX_CUDA_TRY(cudaStreamCreateWithFlags(&e->side_stream, cudaStreamNonBlocking));
         RLX_CUDA_TRY(cudaEventCreateWithFlags(&e->fork_event, cudaEventDisableTiming));
@@ -1371,6 +1430,7 @@ void rlx_encoder_destroy(rlx_encoder_t* e) {
     drop_graphs(e);
     if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
     if (e->side_stream) cudaStreamDestroy(e->side_stream);
+    if (e->body_stream) cudaStreamDestroy(e->body_stream);
     if (e->fork_event) cudaEventDestroy(e->fork_event);
     if (e->join_event) cudaEventDestroy(e->join_event);
     if (e->fold_event) cudaEventDestroy(e->fold_event);

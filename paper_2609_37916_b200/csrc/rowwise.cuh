@@ -92,7 +92,7 @@ constexpr int kPackThreads = 128;
 __global__ void __launch_bounds__(kPackThreads)
 pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* __restrict__ seq_len,
                       int32_t* __restrict__ seq_start, int32_t* __restrict__ pos_of_rank,
-                      unsigned int* __restrict__ ticket) {
+                      unsigned int* __restrict__ ticket, cudaGraphConditionalHandle cond, int cond_min_rows) {
     __shared__ int warp_cnt[kPackThreads / 32];
     __shared__ int is_last;
     pdl_launch_dependents();
@@ -143,6 +143,9 @@ pack_sequences_kernel(const int32_t* __restrict__ mask, int B, int S, int32_t* _
         if (lane == 0) {
             seq_start[B] = carry;
             *ticket = 0;   // ready for the next launch
+            // captured forwards that carry both forms of the layer: the IF / ELSE node behind this kernel takes the
+            // one-kernel layer tail when there are enough packed rows for it to pay
+            if (cond != 0) cudaGraphSetConditional(cond, carry >= cond_min_rows ? 1u : 0u);
         }
     }
 }

@@ -389,3 +389,22 @@ def test_layer_tail_forward_on_random_shapes(rlx):
             enc.close()
             assert status == 0 and np.array_equal(a, b), (B, S, L, hex(flags))
             check(a, ref, inp.lengths, tight=False)
+
+
+def test_captured_forward_chooses_the_layer_form_on_the_device(rlx):
+    """RLX_FLAG_DEVICE_CHOICE (0x4000): from 12288 padded tokens on a captured forward carries both forms of the layer
+    behind an IF / ELSE graph node; the packing kernel takes the layer tail when at least 9216 rows are valid.  Same call, same
+    shapes, two masks: the dense batch gives bit for bit the forced layer-tail result, the sparse one the
+    separate kernels' result."""
+    B, S = 100, 128
+    for lengths, forced in ((np.full(B, S), 0x1400), (np.full(B, 30), 0x2400)):
+        inp = make_inputs(CONFIGS["c2"], batch=B, seq=S, num_layers=2, lengths=lengths)
+        w = rlx.upload_weights(inp.params, inp.layers)
+        auto, status = run_gpu(rlx, inp, weights=w, flags=0x4400)
+        assert status == 0
+        ref_path, status = run_gpu(rlx, inp, weights=w, flags=forced)
+        assert status == 0
+        assert np.array_equal(auto, ref_path), int(lengths.sum())
+        again, _ = run_gpu(rlx, inp, weights=w, flags=0x4400)
+        assert np.array_equal(auto, again)
+        check(auto, oracle.encoder_forward(inp.cfg, inp.ids, inp.mask, inp.params, inp.layers), inp.lengths)
